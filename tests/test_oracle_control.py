@@ -1,0 +1,267 @@
+"""Pins for the oracle's control logic: accept rule, ranking, jump walk, ALP, generate."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import synth
+from oracle import odb_oracle as O
+from oracle.inputs import model_from_synth
+
+f32 = lambda *a: np.array(a, dtype=np.float32)
+
+
+# ----------------------------------------------------------------------------- accept / rank
+
+def test_accept_set_rule():
+    conf = f32(.95, .2, .93, .9, .5)
+    masked = np.array([1, 1, 1, 1, 0], dtype=bool)
+    assert O.accept_set(conf, masked, 0.9).tolist() == [True, False, True, False, False]   # strict ">"
+    # nothing passes -> the single most confident masked position; ties -> lowest position
+    assert O.accept_set(f32(.3, .7, .7, .99), np.array([1, 1, 1, 0], bool), 0.9).tolist() == [False, True, False, False]
+    # unmasked positions never accepted even if confident
+    assert O.accept_set(f32(.99, .1), np.array([0, 1], bool), 0.9).tolist() == [False, True]
+    assert not O.accept_set(f32(.99, .1), np.array([0, 0], bool), 0.9).any()
+    # the compare happens in fp32: 0.9 as fp32 is not > fp32(0.9)
+    assert not (np.float32(0.9) > np.float32(0.9))
+    assert O.accept_set(f32(0.9, 0.1), np.array([1, 1], bool), 0.9).tolist() == [True, False]  # by fallback only
+
+
+def test_rank_candidates():
+    conf = f32(.5, .8, .8, .1, .7)
+    masked = np.array([1, 1, 1, 1, 0], bool)
+    assert O.rank_candidates(conf, masked, 2) == [1, 2]
+    assert O.rank_candidates(conf, masked, 4) == [1, 2, 0, 3]
+    assert O.rank_candidates(conf, np.array([0, 0, 0, 1, 0], bool), 4) == [3]
+
+
+def test_copy_subsets():
+    assert O.copy_subsets(0, 1, False) == [()]
+    assert O.copy_subsets(2, 4, False) == [(), (1,), (2,), (1, 2)]         # Section 4.2.1
+    assert O.copy_subsets(1, 4, False) == [(), (1,)]
+    assert O.copy_subsets(0, 4, False) == [()]
+    assert O.copy_subsets(4, 8, True) == [(), (1,), (2,), (1, 2), (3,), (1, 2, 3), (4,), (1, 2, 3, 4)]  # Section 4.2.2
+    assert O.copy_subsets(3, 8, True) == [(), (1,), (2,), (1, 2), (3,), (1, 2, 3)]
+
+
+# ----------------------------------------------------------------------------- jump walk
+
+def _walk(conf_rows, tok_rows, masked, subsets, rank_off, rank_tok, tau=0.9):
+    conf = np.array(conf_rows, dtype=np.float32)
+    tok = np.array(tok_rows, dtype=np.int32)
+    return O.jump_walk(conf, tok, np.array(masked, bool), subsets, rank_off, rank_tok, tau)
+
+
+S1 = [(), (1,), (2,), (1, 2)]
+
+
+def test_jump_both_hit_goes_to_copy_3():
+    # Section 4.2.1: B and D both unmasked in block 0 -> jump directly to block 3
+    masked = [1, 1, 1, 1]
+    conf = [[.95, .92, .1, .2], [0, .5, .1, .2], [.5, 0, .1, .2], [0, 0, .3, .6]]
+    tok = [[7, 8, 1, 1], [7, 8, 1, 1], [7, 8, 1, 1], [7, 8, 5, 6]]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 3] and last == 3
+    assert new == {0: 7, 1: 8, 3: 6}            # block 3's own decoding (fallback: its best position) is incorporated
+
+
+def test_jump_one_hit_then_verify_other():
+    masked = [1, 1, 1, 1]
+    # only B (rank 1) unmasked in block 0 -> block 1; there D passes -> block 3
+    conf = [[.95, .5, .1, .2], [0, .91, .1, .2], [.5, 0, .1, .2], [0, 0, .95, .6]]
+    tok = [[7, 8, 1, 1], [7, 8, 1, 1], [7, 8, 1, 1], [7, 8, 5, 6]]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 1, 3] and new == {0: 7, 1: 8, 2: 5}
+    # verification fails in block 1 -> adopt block 1's decoding
+    conf[1] = [0, .3, .6, .2]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 1] and last == 1 and new == {0: 7, 2: 1}    # block 1's own decoding (its top-1) is adopted
+    # an acceptance by the top-1 fallback verifies D just like one by threshold
+    conf[1] = [0, .6, .3, .2]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 1, 3]
+    # only D (rank 2) unmasked -> block 2
+    conf[0] = [.5, .95, .1, .2]
+    conf[2] = [.3, 0, .1, .2]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 2, 3]   # block 2's fallback accepts B's position (its top-1), which verifies B
+
+
+def test_jump_needs_token_match_and_no_hit_stays():
+    masked = [1, 1, 1, 1]
+    conf = [[.95, .5, .1, .2], [0, .5, .1, .2], [.5, 0, .1, .2], [0, 0, .3, .6]]
+    tok = [[9, 8, 1, 1], [7, 8, 1, 1], [7, 8, 1, 1], [7, 8, 5, 6]]      # block 0 now predicts 9, fill was 7
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0] and new == {0: 9}
+    # accepted position is not a candidate -> stay in block 0
+    conf[0] = [.5, .4, .1, .97]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0] and new == {3: 1}
+
+
+def test_jump_chain_union_keeps_earlier_link():
+    masked = [1, 1, 1, 1]
+    # block 0 accepts rank-1 position and position 3 (token 4); block 1 would predict 6 at position 3
+    conf = [[.95, .5, .1, .93], [0, .5, .1, .99], [0, 0, 0, 0], [0, 0, 0, 0]]
+    tok = [[7, 8, 1, 4], [7, 8, 1, 6], [0, 0, 0, 0], [0, 0, 0, 0]]
+    new, chain, last = _walk(conf, tok, masked, S1, [0, 1], [7, 8])
+    assert chain == [0, 1] and new == {0: 7, 3: 4}
+
+
+def test_jump_walk_worked_example_six_positions():
+    """Hand-worked case: tau .9, block of 6, fills match.  Block 0 accepts only r1; copy {r1}
+    then accepts r2; copy {r1,r2} accepts one more position; three tokens from one forward."""
+    masked = [0, 1, 0, 1, 1, 1]                 # p0, p2 already decoded; r1 = p1, r2 = p5
+    n = -1.0
+    conf = [[n, .92, n, .50, .20, .85],
+            [n, n, n, .60, .25, .91],
+            [n, .3, n, .1, .1, n],
+            [n, n, n, .95, .30, n]]
+    tok = [[0, 11, 0, 13, 14, 15]] * 4
+    new, chain, last = _walk(conf, tok, masked, S1, [1, 5], [11, 15])
+    assert chain == [0, 1, 3] and last == 3 and new == {1: 11, 5: 15, 3: 13}
+
+
+def test_jump_walk_stage2_lattice():
+    S2 = O.copy_subsets(4, 8, True)
+    masked = [1] * 6
+    rank_off, rank_tok = [0, 1, 2, 3], [10, 11, 12, 13]
+    tok = [[10, 11, 12, 13, 14, 15]] * 8
+    conf = np.zeros((8, 6), np.float32)
+    conf[0, [0, 1, 2]] = .95                     # ranks 1,2,3 hit in block 0 -> largest available superset {1,2,3}
+    conf[5, 3] = .95                             # there rank 4 hits -> {1,2,3,4}
+    conf[7, 4] = .5
+    new, chain, last = O.jump_walk(conf, np.array(tok, np.int32), np.array(masked, bool), S2, rank_off, rank_tok, .9)
+    assert chain == [0, 5, 7] and new == {0: 10, 1: 11, 2: 12, 3: 13, 4: 14}
+    conf[:] = 0
+    conf[0, 2] = .95                             # only rank 3 hit -> copy {3} (index 4); no further superset of {3} exists
+    conf[4, 5] = .2
+    new, chain, last = O.jump_walk(conf, np.array(tok, np.int32), np.array(masked, bool), S2, rank_off, rank_tok, .9)
+    assert chain == [0, 4] and new == {2: 12, 5: 15}
+
+
+# ----------------------------------------------------------------------------- ALP
+
+def test_alp_scan_cases():
+    eos = 5
+    conf = f32(.1, .95, .99, .4, .97)
+    assert O.alp_scan(conf, np.array([1, 2, 3, 4, 6]), 20, 10, eos, 0.9) is None          # no EOS
+    assert O.alp_scan(conf, np.array([5, 2, 3, 5, 6]), 20, 10, eos, 0.9) is None          # EOS below threshold
+    assert O.alp_scan(conf, np.array([5, 5, 5, 4, 5]), 20, 10, eos, 0.9) == 12            # earliest passing EOS, slot kept
+    assert O.alp_scan(conf, np.array([1, 2, 3, 4, 5]), 20, 10, eos, 0.9) == 15
+    assert O.alp_scan(f32(.9), np.array([5]), 20, 10, eos, 0.9) is None                   # strict ">"
+
+
+# ----------------------------------------------------------------------------- generate
+
+@pytest.fixture(scope="module")
+def tiny_model():
+    return model_from_synth(synth.TINY, seed=0)
+
+
+def test_generate_cfg1_one_token_per_iteration(tiny_model):
+    x0 = synth.sequence(0, 0, 64, 64, synth.TINY)
+    x, trace = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16))
+    assert (x[:64] == x0[:64]).all() and (x[64:] != synth.TINY.mask_id).all()
+    assert all(len(t["accepted"]) >= 1 for t in trace)                # progress every iteration
+    assert [t["kind"] for t in trace].count("refresh") == 4
+    # random weights: no confidence gets near 0.9, every iteration accepts exactly one token
+    assert len(trace) == 64 and all(len(t["accepted"]) == 1 for t in trace)
+    for t in trace:
+        (p, _), = t["accepted"]
+        assert 64 + 16 * t["block"] <= p < 64 + 16 * (t["block"] + 1)  # unmasking restricted to the block
+
+
+def test_generate_threshold_extremes(tiny_model):
+    x0 = synth.sequence(0, 0, 64, 64, synth.TINY)
+    # tau >= 1: never exceeded -> exactly one token per iteration, in descending confidence order
+    x_hi, tr_hi = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16, accept_threshold=1.0))
+    assert len(tr_hi) == 64
+    # tau < 0: everything exceeds -> a block fills in its refresh iteration: iterations == blocks
+    x_lo, tr_lo = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16, accept_threshold=-1.0))
+    assert len(tr_lo) == 4 and all(t["kind"] == "refresh" and len(t["accepted"]) == 16 for t in tr_lo)
+    # the first iteration of block 0 is the same prediction in both runs
+    cache, conf, tok = O.refresh_prefill(tiny_model, x0, 128, 64)
+    assert (x_lo[64:80] == tok[:16]).all()
+    assert tr_hi[0]["accepted"] == [(64 + int(np.argmax(conf[:16])), int(tok[np.argmax(conf[:16])]))]
+
+
+def test_jump_share_is_lossless_when_single_accepts(tiny_model):
+    """When every accept set is a single position, copy {r1} is exactly the state plain decoding
+    reaches next, so the jump walk reproduces plain decoding with fewer forwards."""
+    x0 = synth.sequence(0, 0, 64, 64, synth.TINY)
+    x1, tr1 = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16, n_copies=1))
+    x4, tr4 = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16, n_copies=4))
+    assert (x1 == x4).all()
+    assert len(tr4) < len(tr1)
+    assert [t["kind"] for t in tr4].count("refresh") == 4
+    assert max(len(t["chain"]) for t in tr4) <= 3 and max(len(t["accepted"]) for t in tr4) <= 3
+    # the order of commitment is the same sequence of (position, token) pairs
+    flat = lambda tr: [a for t in tr for a in t["accepted"]]
+    assert sorted(flat(tr1)) == sorted(flat(tr4))
+
+
+def test_generate_stage2_runs_and_respects_row_budget(tiny_model):
+    x0 = synth.sequence(0, 0, 64, 64, synth.TINY)
+    p = O.DecodeParams(block_len=16, n_copies=8)
+    x8, tr8 = O.generate(tiny_model, x0, 64, p)
+    assert (x8[64:] != synth.TINY.mask_id).all()
+    assert any(t.get("stage2") for t in tr8) and any(not t.get("stage2") for t in tr8 if t["kind"] == "step")
+    assert O.use_stage2(p, 16, 9) is False and O.use_stage2(p, 16, 10) is True          # ceil(64/7) = 10
+    assert 16 + 7 * (16 - 10) <= 4 * 16 < 16 + 7 * (16 - 9)
+    assert O.use_stage2(p, 32, 18) is False and O.use_stage2(p, 32, 19) is True
+
+
+def test_alp_truncates_and_generation_continues_shorter():
+    """A sharp 64-word model with an [EOS] direction planted deep in the response: with truncate
+    threshold 0 the first refresh must cut the response at the first predicted [EOS].  Lengths
+    never grow afterwards."""
+    shape = dataclasses.replace(synth.TINY_PEAKY, vocab=64, mask_id=63, eos_id=62)
+    m = model_from_synth(shape, seed=5)
+    x0 = synth.sequence(5, 0, 32, 64, shape)
+    # plant an [EOS] direction: the LM-head row of [EOS] points along what is particular to the
+    # final hidden state of response position 40 in the first refresh
+    hid, _, _ = O.forward_rows(m, x0.astype(np.int64), np.arange(96), None, None, np.ones((96, 96), bool),
+                               return_hidden=True)
+    n = O.bf16_round(O.rmsnorm(hid, m.final_gain, m.rms_eps))[32:]
+    lm = m.lm_head.copy()
+    lm[shape.eos_id] = O.bf16_round(30.0 * (n[40] - n.mean(0)))
+    m = dataclasses.replace(m, lm_head=lm)
+    eos = shape.eos_id
+    _, conf, tok = O.refresh_prefill(m, x0, 96, 32)
+    first = int(np.flatnonzero(tok == eos)[0])
+    assert 16 < first <= 40                                           # lands beyond the first block
+    p = O.DecodeParams(block_len=16, truncate_threshold=0.0)
+    x, tr = O.generate(m, x0, 32, p)
+    lens = [t["T"] for t in tr]
+    assert tr[0]["T"] == 32 + first + 1                               # cut at that position, slot kept
+    assert all(a >= b for a, b in zip(lens, lens[1:])) and lens[-1] < 96
+    assert len(x) == lens[-1] and (x[32:] != shape.mask_id).all()
+    last_block = (len(x) - 32 - 1) // 16
+    assert tr[-1]["block"] == last_block                              # a partial last block is still decoded
+    # a high truncate threshold leaves the length alone unless the confidence passes it
+    x_hi, tr_hi = O.generate(m, x0, 32, dataclasses.replace(p, truncate_threshold=float(conf[first]) + 1e-3), max_iters=1)
+    assert tr_hi[0]["T"] == 96 or tr_hi[0]["T"] > tr[0]["T"]
+    # ALP off: full length
+    x_off, tr_off = O.generate(m, x0, 32, dataclasses.replace(p, alp=False))
+    assert len(x_off) == 96
+    # after the cut the run is that of a session that owns only the first T' tokens: replaying
+    # block 1's refresh on the truncated sequence reproduces the traced decision
+    T1 = tr[0]["T"]
+    n0 = sum(1 for t in tr if t["block"] == 0)
+    xa = x0[:T1].astype(np.int64)
+    for t in tr[:n0]:
+        for pos, tk in t["accepted"]:
+            xa[pos] = tk
+    _, conf_a, tok_a = O.refresh_prefill(m, xa, T1, 48)
+    newL = O.alp_scan(conf_a, tok_a, 48, 32, eos, 0.0)
+    T2 = T1 if newL is None else min(T1, 32 + newL)
+    assert tr[n0]["kind"] == "refresh" and tr[n0]["block"] == 1 and tr[n0]["T"] == T2
+
+
+def test_length_schedule_lever(tiny_model):
+    x0 = synth.sequence(0, 0, 64, 64, synth.TINY)
+    sched = lambda b, L: {0: 40, 1: 24}.get(b)
+    x, tr = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16), length_schedule=sched)
+    assert len(x) == 64 + 24 and [t["T"] for t in tr if t["kind"] == "refresh"] == [104, 88]
+    assert (x[64:] != synth.TINY.mask_id).all()
