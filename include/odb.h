@@ -1,0 +1,199 @@
+/*
+ * odb.h - C ABI of the ODB-dLLM block-decoding hot path for NVIDIA B200 (sm_100a).
+ *
+ * What the library computes (paper: "Orchestrating Dual-Boundaries", arXiv 2511.21759):
+ *   - odb_refresh_prefill   : the block-boundary cache refresh, a full bidirectional forward
+ *                             that rewrites the K/V cache of every position (Sections 1, 2.1
+ *                             and 4.1: "all tokens in the response sequence are computed and
+ *                             the KV cache is updated");
+ *   - odb_block_decode_step : one decoding iteration of the current block over the main block
+ *                             and its speculative copies, attending the cached K/V of every
+ *                             token outside the block (DualCache, Section 2.1; copies and their
+ *                             block-wise mask, Section 4.2; decoded-share layout, Section 4.2.2);
+ *   - odb_unmask_accept     : the confidence-threshold accept rule (Section 3, Observation 3),
+ *                             the accept-jump walk over the copies (Section 4.2.1) and, after a
+ *                             refresh, adaptive length prediction (Section 4.1).
+ * Adaptive length prediction needs no call of its own: the [EOS] scan runs inside
+ * odb_unmask_accept(after_refresh = 1), and the host can also shorten a response with
+ * odb_session_set_gen_len, the same lever.
+ *
+ * Conventions
+ *   - Every call returns an int32 status: ODB_OK (0) or a negative ODB_ERR_* code; nothing is
+ *     printed, thrown or aborted.  odb_status_string() names a code.
+ *   - The library allocates NO large device memory.  Weights, K/V cache and workspace are
+ *     caller-owned device buffers passed as raw pointers with their byte sizes; the library
+ *     borrows them until the handle that received them is destroyed.  (Handles themselves
+ *     hold a few KB of device state: TMA descriptors are host objects; the RoPE table lives in
+ *     the caller's workspace.)
+ *   - All matrices are row-major with the reduction (input-feature) dimension contiguous,
+ *     bf16.  RMSNorm gains are fp32.
+ *   - Work is enqueued on the session's stream (a cudaStream_t passed as void*).
+ *     odb_refresh_prefill and odb_block_decode_step are asynchronous.  odb_unmask_accept
+ *     enqueues its kernel, waits for the stream and returns the per-sequence results in host
+ *     memory, because the host control loop needs them to choose the next call.
+ *   - Sessions are independent; one session is not thread-safe.
+ *   - Device-side waits (TMA/MMA barriers) are bounded: a wait that expires records
+ *     ODB_ERR_TIMEOUT in the session's device status word, the kernel finishes normally and the
+ *     next odb_unmask_accept / odb_session_status reports it.
+ */
+#ifndef ODB_H_
+#define ODB_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    ODB_OK = 0,
+    ODB_ERR_ARG = -1,       /* null pointer, bad enum, misaligned buffer */
+    ODB_ERR_SHAPE = -2,     /* unsupported model shape or size beyond the configured maxima */
+    ODB_ERR_WORKSPACE = -3, /* caller buffer too small */
+    ODB_ERR_STATE = -4,     /* call not valid in the session's current state */
+    ODB_ERR_CUDA = -5,      /* a CUDA runtime/driver call failed (odb_last_cuda_error) */
+    ODB_ERR_TIMEOUT = -6    /* a bounded device-side wait expired */
+};
+
+#define ODB_MAX_COPIES 8
+#define ODB_MAX_RANKS 4
+#define ODB_MAX_CHAIN 5
+
+/* Model shape (the paper names LLaDA-Instruct / LLaDA-1.5 but states no internals; this is the
+ * LLaDA-style pre-norm block: RMSNorm, MHA with rotate-half RoPE, SwiGLU, untied LM head).
+ * Requirements: d_model == n_heads*head_dim; head_dim in {64,128}; d_model, d_ffn multiples of
+ * 16; vocab >= 2. */
+typedef struct odb_config {
+    int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+    int32_t mask_id, eos_id;
+    float rope_theta, rms_eps;
+    int32_t max_batch;  /* sequences per session */
+    int32_t max_seq;    /* prompt + response positions per sequence */
+    int32_t max_block;  /* block length upper bound (<= 64) */
+    int32_t max_copies; /* 1, 4 or 8 */
+    int32_t with_lm_head; /* 0: single-layer microbench without LM head (no conf/tok outputs) */
+} odb_config;
+
+/* Device pointers to the weights; per-layer arrays are HOST arrays of n_layers device pointers.
+ * wqkv = [Wq; Wk; Wv] stacked on the output dimension, wgu = [Wgate; Wup] likewise. */
+typedef struct odb_weights {
+    const void* embed;          /* bf16 [vocab][d_model] */
+    const void* lm_head;        /* bf16 [vocab][d_model], NULL iff with_lm_head == 0 */
+    const float* final_norm;    /* fp32 [d_model] */
+    const float* const* norm1;  /* fp32 [d_model] per layer */
+    const void* const* wqkv;    /* bf16 [3*d_model][d_model] per layer */
+    const void* const* wo;      /* bf16 [d_model][d_model] per layer */
+    const float* const* norm2;  /* fp32 [d_model] per layer */
+    const void* const* wgu;     /* bf16 [2*d_ffn][d_model] per layer */
+    const void* const* wd;      /* bf16 [d_model][d_ffn] per layer */
+} odb_weights;
+
+typedef struct odb_decode_params {
+    int32_t block_len;          /* tokens per block (paper: 32) */
+    int32_t n_copies;           /* 1 plain; 4 accept-jump (Section 4.2.1); 8 adds decoded-share (4.2.2) */
+    float accept_threshold;     /* strict ">" */
+    float truncate_threshold;   /* adaptive length prediction, strict ">" */
+    int32_t stage2_min_decoded; /* decoded tokens in the block from which the 8-copy layout is used;
+                                   -1 = ceil(4*block/7), where it fits the row budget of 4 full copies */
+    int32_t alp;                /* 1: scan for [EOS] after a refresh and truncate */
+} odb_decode_params;
+
+/* Per-sequence result of odb_unmask_accept (host memory, valid on return). */
+typedef struct odb_result {
+    int32_t masks_left;    /* masked positions remaining in the current block */
+    int32_t n_accepted;    /* tokens committed by this call */
+    int32_t chain_len;     /* copies visited by the jump walk (>= 1) */
+    int32_t chain[ODB_MAX_CHAIN];
+    int32_t gen_len;       /* response length after this call (ALP may have shortened it) */
+    int32_t block_start;   /* absolute position of the current block */
+    int32_t block_end;
+    int32_t accepted_pos[64]; /* first n_accepted entries: absolute positions, ascending link order */
+    int32_t accepted_tok[64];
+} odb_result;
+
+typedef struct odb_model odb_model;
+typedef struct odb_session odb_session;
+
+const char* odb_status_string(int32_t status);
+/* Text of the last CUDA error seen by this thread's library calls ("" if none). */
+const char* odb_last_cuda_error(void);
+
+/* Validates the shape, builds TMA descriptors for the weight matrices.  The weight buffers must
+ * stay valid and unchanged while the model lives.  *out is set only on ODB_OK. */
+int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model** out);
+int32_t odb_model_destroy(odb_model* m);
+
+/* Bytes of the K/V cache: bf16 [max_batch][n_layers][2][n_heads][max_seq][head_dim]. */
+size_t odb_kv_bytes(const odb_config* cfg);
+/* Bytes of scratch the session needs for activations, split-K partials, logits, RoPE table,
+ * row tables and control state, for the maxima in cfg. */
+size_t odb_workspace_bytes(const odb_config* cfg);
+
+/* kv and workspace are device buffers, 256-byte aligned, of at least odb_kv_bytes /
+ * odb_workspace_bytes; stream is a cudaStream_t (NULL = default stream).  The call initialises
+ * the workspace (RoPE table, state) on the stream and waits for it. */
+int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* workspace, size_t ws_bytes,
+                           void* stream, odb_session** out);
+int32_t odb_session_destroy(odb_session* s);
+
+/* Sequence `seq` := ids_host[0 .. prompt_len+gen_len): the prompt followed by the response
+ * allocation (normally all mask_id; already-decoded tokens are allowed, which is how a session
+ * is resumed).  Resets the sequence to block 0.  Synchronous. */
+int32_t odb_session_set_sequence(odb_session* s, int32_t seq, const int32_t* ids_host,
+                                 int32_t prompt_len, int32_t gen_len);
+/* Shortens the response of `seq` to new_gen_len tokens (never grows; must keep at least one
+ * position of the current block).  Valid between a refresh and the accept that follows it. */
+int32_t odb_session_set_gen_len(odb_session* s, int32_t seq, int32_t new_gen_len);
+/* Copies the sequence's ids (prompt + current response length) to ids_host[0..cap); *len gets
+ * the count.  Synchronous. */
+int32_t odb_session_get_tokens(odb_session* s, int32_t seq, int32_t* ids_host, int32_t cap, int32_t* len);
+/* Marks a sequence inactive (finished) / active; inactive sequences take no part in later calls. */
+int32_t odb_session_set_active(odb_session* s, int32_t seq, int32_t active);
+/* Reads and clears the device status word (ODB_OK or ODB_ERR_TIMEOUT).  Synchronous. */
+int32_t odb_session_status(odb_session* s);
+
+/* Refresh prefill for every active sequence at the start of its block `block_index[seq]`
+ * (host array [max_batch]; a negative entry leaves that sequence out of this refresh; entries
+ * of inactive sequences are ignored; p supplies block_len): full forward over positions
+ * [0, T), K/V of every position and layer written to the cache, confidence and greedy token of
+ * response rows [block_start, T) left on the device for odb_unmask_accept.  Asynchronous. */
+int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const int32_t* block_index);
+
+/* One decoding iteration of the current block of every active sequence, over the copies chosen
+ * by the previous odb_unmask_accept.  Sequences whose block has no masked position left take no
+ * part.  Leaves confidence and greedy token per copy and block position on the device.
+ * Requires a preceding refresh + accept for the block.  Asynchronous. */
+int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p);
+
+/* Applies the accept rule and the jump walk to the outputs of the preceding refresh
+ * (after_refresh = 1: copy 0 only, preceded by the [EOS] scan / truncation when p->alp) or
+ * step (after_refresh = 0), commits tokens, ranks the next speculative candidates.
+ * results: host array [max_batch].  Waits for the stream. */
+int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t after_refresh,
+                          odb_result* results);
+
+/* ---- test / measurement entry points --------------------------------------------------- */
+
+/* Copies a device buffer of the last forward to the host.  which: 0 logits fp32 [rows][vocab];
+ * 1 conf fp32 [rows]; 2 tok int32 [rows]; 3 residual stream fp32 [rows][d_model]; 4 q, 5 k,
+ * 6 v bf16 [rows][d_model] of the LAST layer; 7 attention output bf16 [rows][d_model];
+ * 8 row tokens int32 [rows]; 9 row positions int32 [rows]; 10 row copy ids int32 [rows].
+ * *rows gets the row count of that buffer.  Synchronous. */
+int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap_bytes, int32_t* rows);
+
+/* out[M][N] (fp32, device) = x[M][K] (bf16, device) * w[N][K]^T (bf16, device) with the
+ * weight-streaming tcgen05 GEMM, K split k_splits ways and reduced in fixed order.  scratch:
+ * device buffer of >= k_splits*M*N*4 + 512 bytes.  k_splits = 0 picks the library's heuristic.
+ * Runs on `stream` and waits for it; returns ODB_ERR_TIMEOUT if a device-side wait expired. */
+int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, size_t scratch_bytes,
+                       int32_t M, int32_t N, int32_t K, int32_t k_splits, void* stream);
+
+/* Algorithmic bytes one odb_block_decode_step must move for `rows` query rows and `keys`
+ * visible cached positions per sequence (weights once + K/V once); used by the benchmark. */
+double odb_step_algorithmic_bytes(const odb_config* cfg, int32_t keys);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ODB_H_ */

@@ -309,6 +309,22 @@ def accept_set(conf: np.ndarray, masked: np.ndarray, tau: float) -> np.ndarray:
     return acc
 
 
+def decision_margin(conf: np.ndarray, masked: np.ndarray, tau: float, k_ranks: int = 0) -> float:
+    """How close the decisions taken on this row of confidences are to flipping: the smallest
+    relative gap among (a) any masked confidence and the threshold, (b) the top two masked
+    confidences when the top-1 fallback decides, (c) neighbours in the candidate ranking.
+    Diagnostic only (used to tell a near-tie from a real disagreement); decides nothing."""
+    c = np.sort(conf[masked].astype(np.float64))[::-1]
+    if len(c) == 0:
+        return np.inf
+    m = float(np.min(np.abs(c - tau) / max(abs(tau), 1e-30)))
+    if not (c > tau).any() and len(c) > 1:
+        m = min(m, float((c[0] - c[1]) / max(c[0], 1e-30)))
+    for i in range(min(k_ranks + 1, len(c)) - 1):
+        m = min(m, float((c[i] - c[i + 1]) / max(c[i], 1e-30)))
+    return m
+
+
 def rank_candidates(conf: np.ndarray, masked: np.ndarray, k: int) -> list:
     """Speculative candidates (Section 4.2): the k most confident still-masked positions
     (all of them are below the accept threshold), descending, ties to the lower position."""
@@ -429,7 +445,7 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             x[s + i] = tok_r[i]
         trace.append({"kind": "refresh", "block": b, "T": T,
                       "accepted": [(int(s + i), int(tok_r[i])) for i in np.flatnonzero(acc)],
-                      "chain": [0]})
+                      "chain": [0], "margin": decision_margin(conf_r[:B], masked, tau, k_ranks + 1)})
         last_conf, last_tok = conf_r[:B], tok_r[:B]
         while (x[s:e] == model.mask_id).any():
             if max_iters is not None and len(trace) >= max_iters:
@@ -445,9 +461,10 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             new, chain, last = jump_walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
             for i, t in new.items():
                 x[s + i] = t
+            margin = min(decision_margin(conf[c], masked & (conf[c] >= 0), tau, k_ranks + 1) for c in chain)
             trace.append({"kind": "step", "block": b, "T": T, "stage2": st2,
                           "accepted": sorted((int(s + i), int(t)) for i, t in new.items()),
-                          "chain": [int(c) for c in chain]})
+                          "chain": [int(c) for c in chain], "margin": margin})
             last_conf, last_tok = conf[last], tok[last]
         b += 1
     return x.astype(np.int32), trace

@@ -1,0 +1,305 @@
+// Control kernels: row tables of a refresh / a block step, and the unmask/accept kernel
+// (threshold accept rule, accept-jump walk over the block copies, adaptive length prediction,
+// choice of the next speculative candidates).  A few hundred scalars per sequence: one small
+// block per sequence, the sequential parts on thread 0.
+#include "odb_internal.cuh"
+
+namespace odb {
+
+namespace {
+
+struct BlockIndexParam {
+    int32_t block_index[64];
+    int32_t block_len;
+};
+
+// Rows of a refresh: every position of every active sequence, in sequence order.
+__global__ void build_refresh_rows_kernel(ControlBuffers c, int batch, BlockIndexParam bp) {
+    const int seq = blockIdx.x;
+    SeqState* st = c.state + seq;
+    if (!st->active || bp.block_index[seq] < 0) {
+        if (threadIdx.x == 0) st->in_fwd = 0;
+        return;
+    }
+    __shared__ int row0, lm0, tile0;
+    if (threadIdx.x == 0) {
+        int r = 0, l = 0, t = 0;
+        for (int j = 0; j < seq; ++j) {
+            const SeqState* o = c.state + j;
+            if (!o->active || bp.block_index[j] < 0) continue;
+            const int sj = o->P + bp.block_index[j] * bp.block_len;
+            r += o->T;
+            l += o->T - sj;
+            t += (o->T + 63) / 64;
+        }
+        row0 = r; lm0 = l; tile0 = t;
+        const int s = st->P + bp.block_index[seq] * bp.block_len;
+        st->in_fwd = 1;
+        st->block_idx = bp.block_index[seq];
+        st->s = s;
+        st->e = min(s + bp.block_len, st->T);
+        st->row0 = r;
+        st->n_rows = st->T;
+        st->lm_row0 = l;
+        st->lm_s = s;
+        st->lm_n = st->T - s;
+        st->n_ranks = 0;
+        st->n_copies = 1;
+        st->copy_mask[0] = 0;
+        st->stage2 = 0;
+    }
+    __syncthreads();
+    const int T = st->T;
+    const int s = st->P + bp.block_index[seq] * bp.block_len;
+    const int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
+    for (int p = threadIdx.x; p < T; p += blockDim.x) {
+        const int row = row0 + p;
+        c.row_tok[row] = x[p];
+        c.row_pos[row] = p;
+        c.row_seq[row] = seq;
+        c.row_copy[row] = 0;
+        c.row_flags[row] = 0;
+        if (p >= s) c.lm_rows[lm0 + (p - s)] = row;
+    }
+    for (int j = threadIdx.x; j < (T + 63) / 64; j += blockDim.x) {
+        QTile q;
+        q.q_row0 = row0 + 64 * j;
+        q.nq = min(64, T - 64 * j);
+        q.seq = seq;
+        q.cA = 0; q.cB0 = 0; q.cB1 = 0;
+        q.f0 = row0; q.n0 = T;
+        q.f1 = 0; q.n1 = 0;
+        c.tiles[tile0 + j] = q;
+    }
+}
+
+// Rows of a block step (Section 4.2; decoded-share layout: Section 4.2.2, caption of Fig. 8):
+// copy 0 holds the whole block; a speculative copy holds the whole block (stage 1) or only the
+// positions still masked in the committed state (stage 2).  Position ids are the true positions.
+__device__ int step_rows_of(const SeqState* st) {
+    const int B = st->e - st->s;
+    return st->stage2 ? B + (st->n_copies - 1) * st->n_masked : st->n_copies * B;
+}
+
+__global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id) {
+    const int seq = blockIdx.x;
+    SeqState* st = c.state + seq;
+    if (threadIdx.x != 0) return;
+    if (!st->active || st->n_masked <= 0) {
+        st->in_fwd = 0;
+        return;
+    }
+    st->in_fwd = 1;
+    int row = 0, tile = 0;
+    for (int j = 0; j < seq; ++j) {
+        const SeqState* o = c.state + j;
+        if (!o->active || o->n_masked <= 0) continue;
+        row += step_rows_of(o);
+        tile += o->n_copies;
+    }
+    const int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
+    const int s = st->s, e = st->e;
+    st->row0 = row;
+    for (int cp = 0; cp < st->n_copies; ++cp) {
+        st->copy_row0[cp] = row;
+        for (int p = s; p < e; ++p) {
+            const bool decoded = x[p] != mask_id;
+            if (st->stage2 && cp > 0 && decoded) continue;
+            int tok = x[p];
+            for (int r = 0; r < st->n_ranks; ++r)
+                if (((st->copy_mask[cp] >> r) & 1) && st->rank_off[r] == p - s) tok = st->rank_tok[r];
+            c.row_tok[row] = tok;
+            c.row_pos[row] = p;
+            c.row_seq[row] = seq;
+            c.row_copy[row] = cp;
+            c.row_flags[row] = decoded ? kRowDecoded : 0;
+            c.lm_rows[row] = row;
+            ++row;
+        }
+        st->copy_nrows[cp] = row - st->copy_row0[cp];
+        QTile q;
+        q.q_row0 = st->copy_row0[cp];
+        q.nq = st->copy_nrows[cp];
+        q.seq = seq;
+        q.cA = s; q.cB0 = e; q.cB1 = st->T;
+        q.f0 = q.q_row0; q.n0 = q.nq;
+        const bool shared = st->stage2 && cp > 0;
+        q.f1 = shared ? st->copy_row0[0] : 0;
+        q.n1 = shared ? st->copy_nrows[0] : 0;
+        c.tiles[tile + cp] = q;
+    }
+    st->n_rows = row - st->row0;
+    st->lm_row0 = st->row0;
+}
+
+// Accept rule (Section 3, Observation 3): every masked position whose confidence exceeds tau
+// (strict); if none, the single most confident one (lowest position on a tie).
+__device__ int accept_set(const float* conf, const bool* masked, int B, float tau, bool* acc) {
+    int n = 0, best = -1;
+    for (int i = 0; i < B; ++i) {
+        acc[i] = masked[i] && conf[i] > tau;
+        n += acc[i];
+        if (masked[i] && (best < 0 || conf[i] > conf[best])) best = i;
+    }
+    if (n == 0 && best >= 0) { acc[best] = true; n = 1; }
+    return n;
+}
+
+__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id) {
+    const int seq = blockIdx.x;
+    SeqState* st = c.state + seq;
+    odb_result* res = c.results + seq;
+    if (!st->active || !st->in_fwd) {
+        if (threadIdx.x == 0) {
+            res->masks_left = st->active ? st->n_masked : 0;
+            res->n_accepted = 0;
+            res->chain_len = 0;
+            res->gen_len = st->T - st->P;
+            res->block_start = st->s;
+            res->block_end = st->e;
+        }
+        return;
+    }
+    __shared__ float conf[ODB_MAX_COPIES][kMaxBlock];
+    __shared__ int tok[ODB_MAX_COPIES][kMaxBlock];
+    if (threadIdx.x != 0) return;
+
+    int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
+    const int s = st->s;
+    int n_copies = 1;
+    if (after_refresh) {
+        // adaptive length prediction (Section 4.1): first [EOS] of the whole predicted response
+        // whose confidence exceeds the truncate threshold cuts the response there (slot kept)
+        if (p.alp) {
+            for (int q = s; q < st->T; ++q) {
+                const int r = st->lm_row0 + (q - st->lm_s);
+                if (c.tok[r] == eos_id && c.conf[r] > p.truncate_threshold) { st->T = q + 1; break; }
+            }
+        }
+        st->e = min(s + p.block_len, st->T);
+        for (int i = 0; i < st->e - s; ++i) {
+            const int r = st->lm_row0 + (s + i - st->lm_s);
+            conf[0][i] = c.conf[r];
+            tok[0][i] = c.tok[r];
+        }
+    } else {
+        n_copies = st->n_copies;
+        for (int cp = 0; cp < n_copies; ++cp) {
+            for (int i = 0; i < kMaxBlock; ++i) { conf[cp][i] = -1.f; tok[cp][i] = -1; }
+            for (int r = st->copy_row0[cp]; r < st->copy_row0[cp] + st->copy_nrows[cp]; ++r) {
+                const int i = c.row_pos[r] - s;
+                conf[cp][i] = c.conf[r];
+                tok[cp][i] = c.tok[r];
+            }
+        }
+    }
+    const int B = st->e - s;
+    bool masked0[kMaxBlock], masked[kMaxBlock], acc[kMaxBlock], taken[kMaxBlock];
+    for (int i = 0; i < B; ++i) { masked0[i] = x[s + i] == mask_id; taken[i] = false; }
+
+    // accept-jump walk (Section 4.2.1): start in the main block; a candidate is hit if its
+    // position was accepted with the token it had been filled with; jump to the largest copy
+    // whose extra candidates are all hit; the accepted sets along the chain are committed,
+    // an earlier link winning at a shared position
+    int cur = 0, chain_len = 0, n_acc = 0;
+    while (true) {
+        res->chain[chain_len < ODB_MAX_CHAIN ? chain_len : ODB_MAX_CHAIN - 1] = cur;
+        ++chain_len;
+        const int X = after_refresh ? 0 : st->copy_mask[cur];
+        bool any = false;
+        for (int i = 0; i < B; ++i) masked[i] = masked0[i];
+        for (int r = 0; r < st->n_ranks; ++r)
+            if ((X >> r) & 1) masked[st->rank_off[r]] = false;
+        for (int i = 0; i < B; ++i) any |= masked[i];
+        if (!any) break;
+        accept_set(conf[cur], masked, B, p.accept_threshold, acc);
+        for (int i = 0; i < B; ++i) {
+            if (acc[i] && !taken[i]) {
+                taken[i] = true;
+                x[s + i] = tok[cur][i];
+                if (n_acc < 64) { res->accepted_pos[n_acc] = s + i; res->accepted_tok[n_acc] = tok[cur][i]; }
+                ++n_acc;
+            }
+        }
+        if (after_refresh) break;
+        int hit = 0;
+        for (int r = 0; r < st->n_ranks; ++r) {
+            const int o = st->rank_off[r];
+            if (!((X >> r) & 1) && acc[o] && tok[cur][o] == st->rank_tok[r]) hit |= 1 << r;
+        }
+        int best = -1;
+        for (int cp = 0; cp < n_copies; ++cp) {
+            const int Y = st->copy_mask[cp];
+            if ((Y & X) != X || Y == X || ((Y & ~X) & ~hit)) continue;
+            if (best < 0 || __popc(Y) > __popc(st->copy_mask[best]) ||
+                (__popc(Y) == __popc(st->copy_mask[best]) && Y < st->copy_mask[best]))
+                best = cp;
+        }
+        if (best < 0) break;
+        cur = best;
+    }
+
+    // state after the walk; next candidates: the most confident still-masked positions of the
+    // adopted copy (Section 4.2), ties to the lower position
+    int n_masked = 0;
+    for (int i = 0; i < B; ++i) {
+        masked[i] = masked0[i] && !taken[i];
+        n_masked += masked[i];
+    }
+    const int k_ranks = p.n_copies >= 8 ? 4 : p.n_copies >= 4 ? 2 : 0;
+    int n_ranks = 0;
+    for (int r = 0; r < k_ranks; ++r) {
+        int best = -1;
+        for (int i = 0; i < B; ++i)
+            if (masked[i] && (best < 0 || conf[cur][i] > conf[cur][best])) best = i;
+        if (best < 0) break;
+        masked[best] = false;
+        st->rank_off[n_ranks] = best;
+        st->rank_tok[n_ranks] = tok[cur][best];
+        ++n_ranks;
+    }
+    st->n_ranks = n_ranks;
+    st->n_masked = n_masked;
+    // stage switch (Section 4.2.2 gives no number): decoded-share once eight copies fit the row
+    // budget of four full copies, B + 7 (B - n_dec) <= 4 B
+    const int thr = p.stage2_min_decoded >= 0 ? p.stage2_min_decoded : (4 * B + 6) / 7;
+    const int stage2 = (p.n_copies >= 8 && (B - n_masked) >= thr) ? 1 : 0;
+    const int want = p.n_copies >= 8 ? (stage2 ? 8 : 4) : p.n_copies >= 4 ? 4 : 1;
+    const int all_masks[ODB_MAX_COPIES] = {0, 1, 2, 3, 4, 7, 8, 15};
+    int nc = 0;
+    for (int i = 0; i < want; ++i)
+        if ((all_masks[i] >> n_ranks) == 0) st->copy_mask[nc++] = all_masks[i];
+    st->n_copies = nc;
+    st->stage2 = stage2;
+
+    res->masks_left = n_masked;
+    res->n_accepted = n_acc;
+    res->chain_len = chain_len;
+    res->gen_len = st->T - st->P;
+    res->block_start = s;
+    res->block_end = st->e;
+}
+
+}  // namespace
+
+cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st) {
+    build_step_rows_kernel<<<batch, 32, 0, st>>>(c, batch, mask_id);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
+                          int mask_id, int eos_id, cudaStream_t st) {
+    accept_kernel<<<batch, 32, 0, st>>>(c, p, after_refresh, mask_id, eos_id);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index,
+                                           int block_len, cudaStream_t st) {
+    BlockIndexParam bp;
+    for (int i = 0; i < 64; ++i) bp.block_index[i] = i < batch ? block_index[i] : 0;
+    bp.block_len = block_len;
+    build_refresh_rows_kernel<<<batch, 256, 0, st>>>(c, batch, bp);
+    return cudaGetLastError();
+}
+
+}  // namespace odb

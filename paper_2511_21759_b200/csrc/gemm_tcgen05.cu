@@ -1,0 +1,367 @@
+// Weight-streaming GEMM for sm_100a: TMA -> shared memory -> tcgen05.mma -> TMEM -> registers.
+//
+// Computes, for every K split s,   partial[s][m][n] = sum_{k in split s} x[m][k] * w[n][k]
+// with x the bf16 activations [M][K] (few rows: block_len * copies in a decode step; all
+// positions in a refresh) and w a bf16 weight matrix [N][K].  The 128-row side of the tensor
+// core tile is given to the WEIGHTS (they are the large, streamed operand) and the activation
+// rows ride on the MMA's N dimension (32..256), so a 32-row decode step wastes no tensor-core
+// rows and every weight byte is fetched from HBM exactly once.
+//
+// One CTA = one 128 x BN output tile over one K range.  Warp 0 lane 0 issues TMA loads into a
+// ring of shared-memory stages, warp 1 lane 0 issues the MMAs (accumulator in TMEM) and frees
+// stages through tcgen05.commit, warps 2..5 read the accumulator back (tcgen05.ld) and store
+// fp32 partials.  Splits are reduced later in a fixed order by the consumer kernel, so results
+// are run-to-run identical.  Every mbarrier wait is bounded: on expiry the CTA records
+// ODB_ERR_TIMEOUT, stops issuing work, releases its TMEM and exits.
+#include "odb_internal.cuh"
+
+namespace odb {
+
+namespace {
+
+constexpr int kBM = 128;          // weight rows per tile (MMA M)
+constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
+constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
+constexpr int kThreads = 192;
+constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s at the boost clock
+
+constexpr uint64_t kEvictFirst = 0x12F0000000000000ull;   // L2 policy: streamed once (weights)
+constexpr uint64_t kEvictLast = 0x14F0000000000000ull;    // L2 policy: re-read by every CTA (activations)
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the CTA has been aborted or the limit expired.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* cta_abort, int* status) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity)) {
+        if (*cta_abort) return false;
+        if (clock64() - t0 > kWaitLimitCycles) {
+            *cta_abort = 1;
+            atomicExch(status, ODB_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tmap, uint64_t* bar, int c0, int c1,
+                                            uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(hint)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor: K-major operand, rows of 128 bytes, 128-byte swizzle,
+// 8-row groups 1024 bytes apart.
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);   // start address / 16
+    d |= static_cast<uint64_t>(1) << 16;                   // leading byte offset (unused with swizzle)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;           // stride byte offset between 8-row groups
+    d |= static_cast<uint64_t>(1) << 46;                   // descriptor version of this architecture
+    d |= static_cast<uint64_t>(2) << 61;                   // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, tile M x N.
+__host__ __device__ constexpr uint32_t make_instr_desc(int m, int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+           (static_cast<uint32_t>(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]),
+          "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]),
+          "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]),
+          "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+struct alignas(8) GemmShared {
+    uint64_t full[16];
+    uint64_t empty[16];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    int abort;
+};
+
+// BN: activation rows per tile (MMA N): 32, 64, 128 or 256.
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+            float* __restrict__ partial, int M, int N, int nkb_total, int nkb_per_split, int stages, int* status) {
+    extern __shared__ __align__(1024) uint8_t smem_raw[];
+    constexpr uint32_t kABytes = kBM * kBK * 2;
+    constexpr uint32_t kBBytes = BN * kBK * 2;
+    constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+
+    uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + static_cast<size_t>(stages) * kStageBytes);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int n0 = blockIdx.x * kBM;
+    const int m0 = blockIdx.y * BN;
+    const int split = blockIdx.z;
+    const int kb0 = split * nkb_per_split;
+    int nkb = nkb_total - kb0;
+    if (nkb > nkb_per_split) nkb = nkb_per_split;
+    volatile int* cta_abort = &sh->abort;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < stages; ++i) {
+            mbar_init(&sh->full[i], 1);
+            mbar_init(&sh->empty[i], 1);
+        }
+        mbar_init(&sh->acc_full, 1);
+        sh->abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 0 && lane == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_w)) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_x)) : "memory");
+    }
+    if (warp == 1) {   // whole warp: allocate the accumulator's TMEM columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                     "r"(kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = sh->tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- TMA producer ----
+            int issued = 0;
+            for (int i = 0; i < nkb; ++i) {
+                const int st = i % stages;
+                const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+                if (!mbar_wait(&sh->empty[st], ph ^ 1u, cta_abort, status)) break;
+                uint8_t* a_dst = tiles + static_cast<size_t>(st) * kStageBytes;
+                uint8_t* b_dst = a_dst + kABytes;
+                mbar_expect_tx(&sh->full[st], kStageBytes);
+                tma_load_2d(a_dst, &tmap_w, &sh->full[st], (kb0 + i) * kBK, n0, kEvictFirst);
+                tma_load_2d(b_dst, &tmap_x, &sh->full[st], (kb0 + i) * kBK, m0, kEvictLast);
+                issued = i + 1;
+            }
+            if (*cta_abort) {
+                // aborted: let the copies still in flight land before the CTA's shared memory goes away
+                const int first = issued > stages ? issued - stages : 0;
+                for (int i = first; i < issued; ++i) {
+                    const long long t0 = clock64();
+                    while (!mbar_try_wait(&sh->full[i % stages], static_cast<uint32_t>(i / stages) & 1u) &&
+                           clock64() - t0 < kWaitLimitCycles / 8) {
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer ----
+            constexpr uint32_t idesc = make_instr_desc(kBM, BN);
+            bool ok = true;
+            for (int i = 0; i < nkb && ok; ++i) {
+                const int st = i % stages;
+                const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
+                ok = mbar_wait(&sh->full[st], ph, cta_abort, status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t a_addr = smem_u32(tiles + static_cast<size_t>(st) * kStageBytes);
+                const uint32_t b_addr = a_addr + kABytes;
+#pragma unroll
+                for (int k = 0; k < kBK / kUmmaK; ++k) {
+                    umma_bf16(tmem_acc, make_smem_desc(a_addr + k * kUmmaK * 2), make_smem_desc(b_addr + k * kUmmaK * 2),
+                              idesc, (i > 0 || k > 0) ? 1u : 0u);
+                }
+                umma_commit(&sh->empty[st]);   // frees the stage once these MMAs have read it
+            }
+            if (ok) umma_commit(&sh->acc_full);
+        }
+    } else {
+        // ---- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 ----
+        const int q = warp & 3;
+        const int n = n0 + q * 32 + lane;
+        if (mbar_wait(&sh->acc_full, 0, cta_abort, status)) {
+            tc_fence_after();
+            float* out = partial + static_cast<size_t>(split) * M * N;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (n < N) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + c * 32 + j;
+                        if (m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
+                    }
+                }
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
+    }
+}
+
+__global__ void reduce_partials_kernel(const float* __restrict__ partial, int splits, size_t stride,
+                                       float* __restrict__ out, size_t n) {
+    const size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    float acc = partial[i];
+    for (int s = 1; s < splits; ++s) acc += partial[s * stride + i];
+    out[i] = acc;
+}
+
+// ---- tensor maps -----------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    }
+    return fn;
+}
+
+// bf16 [rows][K] row-major, box = 64 K-elements x box_rows rows, 128-byte swizzle, zero fill.
+cudaError_t make_tmap_2d(CUtensorMap* out, const void* base, int rows, int K, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return cudaErrorNotSupported;
+    cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(rows)};
+    cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+int pick_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
+
+template <int BN>
+cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st) {
+    const int nkb_total = (a.K + kBK - 1) / kBK;
+    const int nkb_per_split = (nkb_total + a.splits - 1) / a.splits;
+    const uint32_t stage_bytes = kBM * kBK * 2 + BN * kBK * 2;
+    // two CTAs per SM for the narrow tiles (hides each CTA's prologue and drain), one for 256
+    const uint32_t budget = BN <= 64 ? 100 * 1024 : BN == 128 ? 196 * 1024 : 200 * 1024;
+    int stages = static_cast<int>(budget / stage_bytes);
+    if (stages > 16) stages = 16;
+    if (stages > nkb_per_split) stages = nkb_per_split < 2 ? 2 : nkb_per_split;
+    const size_t smem = static_cast<size_t>(stages) * stage_bytes + sizeof(GemmShared) + 1024;
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    dim3 grid((a.N + kBM - 1) / kBM, (a.M + BN - 1) / BN, a.splits);
+    gemm_kernel<BN><<<grid, kThreads, smem, st>>>(a.tmap_w, tmx, a.partial, a.M, a.N, nkb_total, nkb_per_split, stages,
+                                                  a.status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { return make_tmap_2d(out, w, N, K, kBM); }
+
+int gemm_pick_splits(int M, int N, int K) {
+    const int bn = pick_bn(M);
+    const int tiles = ((N + kBM - 1) / kBM) * ((M + bn - 1) / bn);
+    const int nkb = (K + kBK - 1) / kBK;
+    int splits = (2 * 148 + tiles - 1) / tiles;
+    if (splits > nkb / 4) splits = nkb / 4;
+    if (splits > 16) splits = 16;
+    if (splits < 1) splits = 1;
+    // no empty split: ceil(nkb/splits) * (splits-1) < nkb
+    while (splits > 1 && ((nkb + splits - 1) / splits) * (splits - 1) >= nkb) --splits;
+    return splits;
+}
+
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
+    const int bn = pick_bn(a.M);
+    CUtensorMap tmx;
+    cudaError_t e = make_tmap_2d(&tmx, a.x, a.M, a.K, bn);
+    if (e != cudaSuccess) return e;
+    switch (bn) {
+        case 32: return launch_bn<32>(a, tmx, st);
+        case 64: return launch_bn<64>(a, tmx, st);
+        case 128: return launch_bn<128>(a, tmx, st);
+        default: return launch_bn<256>(a, tmx, st);
+    }
+}
+
+cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,
+                                   cudaStream_t st) {
+    reduce_partials_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, splits, stride, out, n);
+    return cudaGetLastError();
+}
+
+}  // namespace odb

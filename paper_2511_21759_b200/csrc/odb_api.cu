@@ -1,0 +1,567 @@
+// C ABI of the library: handles, argument validation, workspace carve-up and the host-side
+// orchestration of one forward (refresh prefill or block decode step) over the kernels.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+#include <string>
+#include <vector>
+
+#include "odb_internal.cuh"
+
+using namespace odb;
+
+namespace {
+
+thread_local std::string g_cuda_error;
+
+int32_t cuda_fail(cudaError_t e) {
+    g_cuda_error = cudaGetErrorString(e);
+    return ODB_ERR_CUDA;
+}
+
+#define ODB_CUDA(call)                                   \
+    do {                                                 \
+        cudaError_t e__ = (call);                        \
+        if (e__ != cudaSuccess) return cuda_fail(e__);   \
+    } while (0)
+
+size_t align_up(size_t v, size_t a = 256) { return (v + a - 1) / a * a; }
+
+int32_t check_config(const odb_config* c) {
+    if (!c) return ODB_ERR_ARG;
+    if (c->n_layers < 1 || c->d_model < 16 || c->n_heads < 1 || c->vocab < 2) return ODB_ERR_SHAPE;
+    if (c->head_dim != 64 && c->head_dim != 128) return ODB_ERR_SHAPE;
+    if (c->d_model != c->n_heads * c->head_dim) return ODB_ERR_SHAPE;
+    if (c->d_model % 16 || c->d_ffn % 16 || c->d_ffn < 16) return ODB_ERR_SHAPE;
+    if (c->max_batch < 1 || c->max_batch > 64 || c->max_seq < 2) return ODB_ERR_SHAPE;
+    if (c->max_block < 1 || c->max_block > kMaxBlock) return ODB_ERR_SHAPE;
+    if (c->max_copies != 1 && c->max_copies != 4 && c->max_copies != 8) return ODB_ERR_SHAPE;
+    if (c->mask_id < 0 || c->mask_id >= c->vocab || c->eos_id < 0 || c->eos_id >= c->vocab) return ODB_ERR_ARG;
+    return ODB_OK;
+}
+
+// Carve-up of the caller's workspace.  Offsets only; shared by odb_workspace_bytes and
+// odb_session_create so that both always agree.
+struct Layout {
+    size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
+    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf;
+    size_t h, a, q, k, v, o, g, partial, logits, conf, tok, part_o, part_ml;
+    size_t total;
+};
+
+Layout make_layout(const odb_config& c) {
+    Layout L{};
+    const size_t step_rows = static_cast<size_t>(c.max_copies) * c.max_block;
+    const size_t per_seq = step_rows > static_cast<size_t>(c.max_seq) ? step_rows : static_cast<size_t>(c.max_seq);
+    L.rows = per_seq * c.max_batch;
+    L.lm_chunk = L.rows < 2048 ? L.rows : 2048;
+    const size_t refresh_tiles = static_cast<size_t>(c.max_batch) * ((c.max_seq + 63) / 64);
+    const size_t step_tiles = static_cast<size_t>(c.max_batch) * c.max_copies;
+    L.tiles = refresh_tiles > step_tiles ? refresh_tiles : step_tiles;
+    L.partial_rows = L.rows > 4096 ? L.rows : 4096;
+    L.attn_rows = L.rows > 2048 ? L.rows : 2048;
+    const size_t d = c.d_model, F = c.d_ffn;
+    const size_t nmax = 3 * d > 2 * F ? 3 * d : 2 * F;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+    L.rope = take(static_cast<size_t>(c.max_seq) * (c.head_dim / 2) * sizeof(float2));
+    L.state = take(sizeof(SeqState) * c.max_batch);
+    L.results = take(sizeof(odb_result) * c.max_batch);
+    L.status = take(sizeof(int));
+    L.x = take(sizeof(int32_t) * c.max_batch * c.max_seq);
+    L.row_tok = take(4 * L.rows);
+    L.row_pos = take(4 * L.rows);
+    L.row_seq = take(4 * L.rows);
+    L.row_copy = take(4 * L.rows);
+    L.row_flags = take(4 * L.rows);
+    L.lm_rows = take(4 * L.rows);
+    L.tile_buf = take(sizeof(QTile) * L.tiles);
+    L.h = take(4 * L.rows * d);
+    L.a = take(2 * L.rows * d);
+    L.q = take(2 * L.rows * d);
+    L.k = take(2 * L.rows * d);
+    L.v = take(2 * L.rows * d);
+    L.o = take(2 * L.rows * d);
+    L.g = take(2 * L.rows * F);
+    L.partial = take(4 * L.partial_rows * nmax);
+    L.logits = take(c.with_lm_head ? 4 * L.lm_chunk * c.vocab : 256);
+    L.conf = take(4 * L.rows);
+    L.tok = take(4 * L.rows);
+    L.part_o = take(4 * L.attn_rows * d);
+    L.part_ml = take(4 * L.attn_rows * c.n_heads * 2);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+struct odb_model {
+    odb_config cfg;
+    const __nv_bfloat16* embed;
+    const float* final_norm;
+    std::vector<const float*> norm1, norm2;
+    std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_d;
+    CUtensorMap tm_lm;
+};
+
+struct odb_session {
+    odb_model* m;
+    cudaStream_t st;
+    uint8_t* ws;
+    __nv_bfloat16* kv;
+    Layout L;
+    ControlBuffers cb;
+    std::vector<SeqState> mirror;
+    SeqState* pinned_state;
+    odb_result* pinned_results;
+    int* pinned_status;
+    int phase;            // 0 idle, 1 refresh enqueued, 2 accepted, 3 step enqueued
+    int last_rows, last_lm_rows;
+    template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
+};
+
+extern "C" {
+
+const char* odb_status_string(int32_t s) {
+    switch (s) {
+        case ODB_OK: return "ok";
+        case ODB_ERR_ARG: return "invalid argument";
+        case ODB_ERR_SHAPE: return "unsupported shape";
+        case ODB_ERR_WORKSPACE: return "buffer too small";
+        case ODB_ERR_STATE: return "call not valid in this state";
+        case ODB_ERR_CUDA: return "CUDA error";
+        case ODB_ERR_TIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+const char* odb_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model** out) {
+    int32_t rc = check_config(cfg);
+    if (rc != ODB_OK) return rc;
+    if (!w || !out || !w->embed || !w->final_norm || !w->norm1 || !w->norm2 || !w->wqkv || !w->wo || !w->wgu || !w->wd)
+        return ODB_ERR_ARG;
+    if ((cfg->with_lm_head != 0) != (w->lm_head != nullptr)) return ODB_ERR_ARG;
+    odb_model* m = new (std::nothrow) odb_model();
+    if (!m) return ODB_ERR_ARG;
+    m->cfg = *cfg;
+    m->embed = static_cast<const __nv_bfloat16*>(w->embed);
+    m->final_norm = w->final_norm;
+    const int d = cfg->d_model, F = cfg->d_ffn, nl = cfg->n_layers;
+    m->tm_qkv.resize(nl); m->tm_o.resize(nl); m->tm_gu.resize(nl); m->tm_d.resize(nl);
+    cudaError_t e = cudaSuccess;
+    for (int l = 0; l < nl && e == cudaSuccess; ++l) {
+        if (!w->norm1[l] || !w->norm2[l] || !w->wqkv[l] || !w->wo[l] || !w->wgu[l] || !w->wd[l]) {
+            delete m;
+            return ODB_ERR_ARG;
+        }
+        m->norm1.push_back(w->norm1[l]);
+        m->norm2.push_back(w->norm2[l]);
+        e = make_weight_tmap(&m->tm_qkv[l], w->wqkv[l], 3 * d, d);
+        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_o[l], w->wo[l], d, d);
+        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_gu[l], w->wgu[l], 2 * F, d);
+        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_d[l], w->wd[l], d, F);
+    }
+    if (e == cudaSuccess && cfg->with_lm_head) e = make_weight_tmap(&m->tm_lm, w->lm_head, cfg->vocab, d);
+    if (e != cudaSuccess) {
+        delete m;
+        return cuda_fail(e);
+    }
+    *out = m;
+    return ODB_OK;
+}
+
+int32_t odb_model_destroy(odb_model* m) {
+    delete m;
+    return ODB_OK;
+}
+
+size_t odb_kv_bytes(const odb_config* c) {
+    if (check_config(c) != ODB_OK) return 0;
+    return static_cast<size_t>(c->max_batch) * c->n_layers * 2 * c->n_heads * c->max_seq * c->head_dim * 2;
+}
+
+size_t odb_workspace_bytes(const odb_config* c) {
+    if (check_config(c) != ODB_OK) return 0;
+    return make_layout(*c).total;
+}
+
+int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* workspace, size_t ws_bytes, void* stream,
+                           odb_session** out) {
+    if (!m || !kv || !workspace || !out) return ODB_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(kv) | reinterpret_cast<uintptr_t>(workspace)) & 255) return ODB_ERR_ARG;
+    const odb_config& c = m->cfg;
+    const Layout L = make_layout(c);
+    if (kv_bytes < odb_kv_bytes(&c) || ws_bytes < L.total) return ODB_ERR_WORKSPACE;
+    odb_session* s = new (std::nothrow) odb_session();
+    if (!s) return ODB_ERR_ARG;
+    s->m = m;
+    s->st = static_cast<cudaStream_t>(stream);
+    s->ws = static_cast<uint8_t*>(workspace);
+    s->kv = static_cast<__nv_bfloat16*>(kv);
+    s->L = L;
+    s->phase = 0;
+    s->last_rows = s->last_lm_rows = 0;
+    s->mirror.assign(c.max_batch, SeqState{});
+    s->pinned_state = nullptr;
+    s->pinned_results = nullptr;
+    s->pinned_status = nullptr;
+    cudaError_t e = cudaMallocHost(&s->pinned_state, sizeof(SeqState) * c.max_batch);
+    if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_results, sizeof(odb_result) * c.max_batch);
+    if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_status, sizeof(int));
+    // RoPE table: angle(pos, i) = pos * theta^(-2i/hd), evaluated in double, stored as fp32 (cos, sin)
+    std::vector<float2> rope(static_cast<size_t>(c.max_seq) * (c.head_dim / 2));
+    for (int i = 0; i < c.head_dim / 2; ++i) {
+        const double inv = pow(static_cast<double>(c.rope_theta), -2.0 * i / c.head_dim);
+        for (int p = 0; p < c.max_seq; ++p) {
+            const double ang = p * inv;
+            rope[static_cast<size_t>(p) * (c.head_dim / 2) + i] = make_float2(static_cast<float>(cos(ang)),
+                                                                              static_cast<float>(sin(ang)));
+        }
+    }
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(s->ws + L.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s->st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->ws + L.state, 0, L.x - L.state, s->st);   // state, results, status
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s->st);
+    if (e != cudaSuccess) {
+        odb_session_destroy(s);
+        return cuda_fail(e);
+    }
+    ControlBuffers& cb = s->cb;
+    cb.state = s->at<SeqState>(L.state);
+    cb.x = s->at<int32_t>(L.x);
+    cb.max_seq = c.max_seq;
+    cb.row_tok = s->at<int32_t>(L.row_tok);
+    cb.row_pos = s->at<int32_t>(L.row_pos);
+    cb.row_seq = s->at<int32_t>(L.row_seq);
+    cb.row_copy = s->at<int32_t>(L.row_copy);
+    cb.row_flags = s->at<int32_t>(L.row_flags);
+    cb.lm_rows = s->at<int32_t>(L.lm_rows);
+    cb.tiles = s->at<QTile>(L.tile_buf);
+    cb.conf = s->at<float>(L.conf);
+    cb.tok = s->at<int32_t>(L.tok);
+    cb.results = s->at<odb_result>(L.results);
+    *out = s;
+    return ODB_OK;
+}
+
+int32_t odb_session_destroy(odb_session* s) {
+    if (!s) return ODB_OK;
+    if (s->pinned_state) cudaFreeHost(s->pinned_state);
+    if (s->pinned_results) cudaFreeHost(s->pinned_results);
+    if (s->pinned_status) cudaFreeHost(s->pinned_status);
+    delete s;
+    return ODB_OK;
+}
+
+static int32_t push_state(odb_session* s, int seq) {
+    ODB_CUDA(cudaMemcpyAsync(s->cb.state + seq, &s->mirror[seq], sizeof(SeqState), cudaMemcpyHostToDevice, s->st));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    return ODB_OK;
+}
+
+int32_t odb_session_set_sequence(odb_session* s, int32_t seq, const int32_t* ids, int32_t prompt_len, int32_t gen_len) {
+    if (!s || !ids) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (seq < 0 || seq >= c.max_batch || prompt_len < 0 || gen_len < 1) return ODB_ERR_ARG;
+    if (prompt_len + gen_len > c.max_seq) return ODB_ERR_SHAPE;
+    for (int i = 0; i < prompt_len + gen_len; ++i)
+        if (ids[i] < 0 || ids[i] >= c.vocab) return ODB_ERR_ARG;
+    ODB_CUDA(cudaMemcpyAsync(s->cb.x + static_cast<size_t>(seq) * c.max_seq, ids, sizeof(int32_t) * (prompt_len + gen_len),
+                             cudaMemcpyHostToDevice, s->st));
+    SeqState st{};
+    st.active = 1;
+    st.P = prompt_len;
+    st.T = prompt_len + gen_len;
+    st.n_copies = 1;
+    s->mirror[seq] = st;
+    s->phase = 0;
+    return push_state(s, seq);
+}
+
+int32_t odb_session_set_gen_len(odb_session* s, int32_t seq, int32_t new_gen_len) {
+    if (!s) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (seq < 0 || seq >= c.max_batch) return ODB_ERR_ARG;
+    if (s->phase != 1) return ODB_ERR_STATE;      // only between a refresh and its accept
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    // the refresh's row-table kernel has set the block; fetch it
+    ODB_CUDA(cudaMemcpy(&s->mirror[seq], s->cb.state + seq, sizeof(SeqState), cudaMemcpyDeviceToHost));
+    SeqState& st = s->mirror[seq];
+    if (!st.active) return ODB_ERR_STATE;
+    if (new_gen_len > st.T - st.P) return ODB_ERR_ARG;                 // never grows
+    if (st.P + new_gen_len <= st.s) return ODB_ERR_ARG;                // keeps a position of the block
+    st.T = st.P + new_gen_len;
+    if (st.e > st.T) st.e = st.T;
+    return push_state(s, seq);
+}
+
+int32_t odb_session_get_tokens(odb_session* s, int32_t seq, int32_t* ids, int32_t cap, int32_t* len) {
+    if (!s || !ids || !len) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (seq < 0 || seq >= c.max_batch) return ODB_ERR_ARG;
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    ODB_CUDA(cudaMemcpy(&s->mirror[seq], s->cb.state + seq, sizeof(SeqState), cudaMemcpyDeviceToHost));
+    const int T = s->mirror[seq].T;
+    if (cap < T) return ODB_ERR_WORKSPACE;
+    ODB_CUDA(cudaMemcpy(ids, s->cb.x + static_cast<size_t>(seq) * c.max_seq, sizeof(int32_t) * T, cudaMemcpyDeviceToHost));
+    *len = T;
+    return ODB_OK;
+}
+
+int32_t odb_session_set_active(odb_session* s, int32_t seq, int32_t active) {
+    if (!s) return ODB_ERR_ARG;
+    if (seq < 0 || seq >= s->m->cfg.max_batch) return ODB_ERR_ARG;
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    ODB_CUDA(cudaMemcpy(&s->mirror[seq], s->cb.state + seq, sizeof(SeqState), cudaMemcpyDeviceToHost));
+    s->mirror[seq].active = active ? 1 : 0;
+    return push_state(s, seq);
+}
+
+int32_t odb_session_status(odb_session* s) {
+    if (!s) return ODB_ERR_ARG;
+    int* dev = s->at<int>(s->L.status);
+    ODB_CUDA(cudaMemcpyAsync(s->pinned_status, dev, sizeof(int), cudaMemcpyDeviceToHost, s->st));
+    ODB_CUDA(cudaMemsetAsync(dev, 0, sizeof(int), s->st));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    return *s->pinned_status;
+}
+
+}  // extern "C"
+
+namespace {
+
+// One forward over the M rows of the row table already built on the device.
+int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) {
+    const odb_model* m = s->m;
+    const odb_config& c = m->cfg;
+    const Layout& L = s->L;
+    cudaStream_t st = s->st;
+    const int d = c.d_model, F = c.d_ffn, H = c.n_heads, hd = c.head_dim;
+    float* h = s->at<float>(L.h);
+    __nv_bfloat16* a = s->at<__nv_bfloat16>(L.a);
+    __nv_bfloat16* q = s->at<__nv_bfloat16>(L.q);
+    __nv_bfloat16* k = s->at<__nv_bfloat16>(L.k);
+    __nv_bfloat16* v = s->at<__nv_bfloat16>(L.v);
+    __nv_bfloat16* o = s->at<__nv_bfloat16>(L.o);
+    __nv_bfloat16* g = s->at<__nv_bfloat16>(L.g);
+    float* partial = s->at<float>(L.partial);
+    int* status = s->at<int>(L.status);
+    const size_t nmax = 3 * static_cast<size_t>(d) > 2 * static_cast<size_t>(F) ? 3 * static_cast<size_t>(d)
+                                                                                : 2 * static_cast<size_t>(F);
+    auto gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, float* out, int rows, int N, int K, int* splits) {
+        GemmArgs ga;
+        ga.tmap_w = tw;
+        ga.x = x;
+        ga.partial = out;
+        ga.M = rows; ga.N = N; ga.K = K;
+        int sp = *splits > 0 ? *splits : gemm_pick_splits(rows, N, K);
+        const size_t cap = L.partial_rows * nmax / (static_cast<size_t>(rows) * N);
+        if (static_cast<size_t>(sp) > cap) sp = static_cast<int>(cap < 1 ? 1 : cap);
+        ga.splits = sp;
+        ga.status = status;
+        *splits = sp;
+        return launch_gemm(ga, st);
+    };
+
+    ODB_CUDA(launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
+    const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
+    int res_splits = 0;
+    size_t res_stride = 0;
+    int ks = (2 * 148 + n_tiles * H - 1) / (n_tiles * H);
+    if (ks > 8) ks = 8;
+    if (static_cast<size_t>(ks) * M > L.attn_rows) ks = static_cast<int>(L.attn_rows / M);
+    if (ks < 1) ks = 1;
+    for (int l = 0; l < c.n_layers; ++l) {
+        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, nullptr, M, d, c.rms_eps, st));
+        int sp = 0;
+        ODB_CUDA(gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
+        QkvRopeArgs qa;
+        qa.partial = partial; qa.splits = sp; qa.pstride = static_cast<size_t>(M) * 3 * d;
+        qa.rope = s->at<float2>(L.rope);
+        qa.row_pos = s->cb.row_pos; qa.row_seq = s->cb.row_seq;
+        qa.q = q; qa.k = k; qa.v = v;
+        qa.cache = write_cache ? s->kv : nullptr;
+        qa.layer = l; qa.n_layers = c.n_layers; qa.H = H; qa.hd = hd; qa.max_seq = c.max_seq; qa.M = M;
+        ODB_CUDA(launch_qkv_rope(qa, st));
+        AttnArgs aa;
+        aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
+        aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
+        aa.part_o = s->at<float>(L.part_o); aa.part_ml = s->at<float>(L.part_ml);
+        aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = ks;
+        ODB_CUDA(launch_attention(aa, st));
+        sp = 0;
+        ODB_CUDA(gemm(m->tm_o[l], o, partial, M, d, d, &sp));
+        ODB_CUDA(launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps, st));
+        sp = 0;
+        ODB_CUDA(gemm(m->tm_gu[l], a, partial, M, 2 * F, d, &sp));
+        ODB_CUDA(launch_swiglu(partial, sp, static_cast<size_t>(M) * 2 * F, g, M, F, st));
+        sp = 0;
+        ODB_CUDA(gemm(m->tm_d[l], g, partial, M, d, F, &sp));
+        res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
+    }
+    if (!c.with_lm_head) {
+        // fold the last projection into the residual stream (the normalised copy is not used)
+        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, nullptr, M, d, c.rms_eps, st));
+        return ODB_OK;
+    }
+    float* logits = s->at<float>(L.logits);
+    for (int r0 = 0; r0 < n_lm; r0 += static_cast<int>(L.lm_chunk)) {
+        const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
+        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps, st));
+        int sp = 1;
+        ODB_CUDA(gemm(m->tm_lm, a, logits, rows, c.vocab, d, &sp));
+        ODB_CUDA(launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0, st));
+    }
+    return ODB_OK;
+}
+
+int32_t pull_state(odb_session* s) {
+    const int nb = s->m->cfg.max_batch;
+    ODB_CUDA(cudaMemcpyAsync(s->pinned_state, s->cb.state, sizeof(SeqState) * nb, cudaMemcpyDeviceToHost, s->st));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    for (int i = 0; i < nb; ++i) s->mirror[i] = s->pinned_state[i];
+    return ODB_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const int32_t* block_index) {
+    if (!s || !p || !block_index) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
+    if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;   // an accept is pending
+    int M = 0, n_lm = 0, n_tiles = 0;
+    for (int i = 0; i < c.max_batch; ++i) {
+        const SeqState& st = s->mirror[i];
+        if (!st.active || block_index[i] < 0) continue;
+        const int bs = st.P + block_index[i] * p->block_len;
+        if (bs >= st.T) return ODB_ERR_ARG;
+        M += st.T;
+        n_lm += st.T - bs;
+        n_tiles += (st.T + 63) / 64;
+    }
+    if (M == 0) return ODB_ERR_STATE;
+    ODB_CUDA(launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
+    int32_t rc = forward(s, M, c.with_lm_head ? n_lm : 0, n_tiles, true);
+    if (rc != ODB_OK) return rc;
+    s->last_rows = M;
+    s->last_lm_rows = n_lm;
+    s->phase = 1;
+    return ODB_OK;
+}
+
+int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
+    if (!s || !p) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (s->phase != 2) return ODB_ERR_STATE;
+    int M = 0, n_tiles = 0;
+    for (int i = 0; i < c.max_batch; ++i) {
+        const SeqState& st = s->mirror[i];
+        if (!st.active || st.n_masked <= 0) continue;
+        const int B = st.e - st.s;
+        M += st.stage2 ? B + (st.n_copies - 1) * st.n_masked : st.n_copies * B;
+        n_tiles += st.n_copies;
+    }
+    if (M == 0) return ODB_ERR_STATE;
+    if (static_cast<size_t>(M) > s->L.rows) return ODB_ERR_SHAPE;
+    ODB_CUDA(launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
+    int32_t rc = forward(s, M, c.with_lm_head ? M : 0, n_tiles, false);
+    if (rc != ODB_OK) return rc;
+    s->last_rows = M;
+    s->last_lm_rows = M;
+    s->phase = 3;
+    return ODB_OK;
+}
+
+int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t after_refresh, odb_result* results) {
+    if (!s || !p || !results) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (!c.with_lm_head) return ODB_ERR_STATE;
+    if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
+    if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
+    if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
+    if (s->phase != (after_refresh ? 1 : 3)) return ODB_ERR_STATE;
+    ODB_CUDA(launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id, s->st));
+    ODB_CUDA(cudaMemcpyAsync(s->pinned_results, s->cb.results, sizeof(odb_result) * c.max_batch, cudaMemcpyDeviceToHost, s->st));
+    int* dev_status = s->at<int>(s->L.status);
+    ODB_CUDA(cudaMemcpyAsync(s->pinned_status, dev_status, sizeof(int), cudaMemcpyDeviceToHost, s->st));
+    int32_t rc = pull_state(s);
+    if (rc != ODB_OK) return rc;
+    memcpy(results, s->pinned_results, sizeof(odb_result) * c.max_batch);
+    s->phase = 2;
+    if (*s->pinned_status != 0) {
+        cudaMemsetAsync(dev_status, 0, sizeof(int), s->st);
+        return *s->pinned_status;
+    }
+    return ODB_OK;
+}
+
+int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap, int32_t* rows) {
+    if (!s || !host || !rows) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    const Layout& L = s->L;
+    const size_t M = s->last_rows, nlm = s->last_lm_rows, d = c.d_model;
+    size_t off = 0, bytes = 0, n = M;
+    switch (which) {
+        case 0: off = L.logits; n = nlm < L.lm_chunk ? nlm : L.lm_chunk; bytes = 4 * n * c.vocab; break;
+        case 1: off = L.conf; n = nlm; bytes = 4 * n; break;
+        case 2: off = L.tok; n = nlm; bytes = 4 * n; break;
+        case 3: off = L.h; bytes = 4 * M * d; break;
+        case 4: off = L.q; bytes = 2 * M * d; break;
+        case 5: off = L.k; bytes = 2 * M * d; break;
+        case 6: off = L.v; bytes = 2 * M * d; break;
+        case 7: off = L.o; bytes = 2 * M * d; break;
+        case 8: off = L.row_tok; bytes = 4 * M; break;
+        case 9: off = L.row_pos; bytes = 4 * M; break;
+        case 10: off = L.row_copy; bytes = 4 * M; break;
+        default: return ODB_ERR_ARG;
+    }
+    if (which == 0 && !c.with_lm_head) return ODB_ERR_STATE;
+    if (cap < bytes) return ODB_ERR_WORKSPACE;
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    ODB_CUDA(cudaMemcpy(host, s->ws + off, bytes, cudaMemcpyDeviceToHost));
+    *rows = static_cast<int32_t>(n);
+    return ODB_OK;
+}
+
+int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, size_t scratch_bytes, int32_t M,
+                       int32_t N, int32_t K, int32_t k_splits, void* stream) {
+    if (!x || !w || !out || !scratch) return ODB_ERR_ARG;
+    if (M < 1 || N < 1 || K < 8 || K % 8) return ODB_ERR_SHAPE;
+    int splits = k_splits > 0 ? k_splits : gemm_pick_splits(M, N, K);
+    const int nkb = (K + 63) / 64;
+    if (splits > nkb) splits = nkb;
+    while (splits > 1 && ((nkb + splits - 1) / splits) * (splits - 1) >= nkb) --splits;
+    const size_t part_bytes = align_up(static_cast<size_t>(splits) * M * N * 4);
+    if (scratch_bytes < part_bytes + 256) return ODB_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* status = reinterpret_cast<int*>(static_cast<uint8_t*>(scratch) + part_bytes);   // behind the partials
+    ODB_CUDA(cudaMemsetAsync(status, 0, sizeof(int), st));
+    GemmArgs ga;
+    ODB_CUDA(make_weight_tmap(&ga.tmap_w, w, N, K));
+    ga.x = x;
+    ga.partial = static_cast<float*>(scratch);
+    ga.M = M; ga.N = N; ga.K = K;
+    ga.splits = splits;
+    ga.status = status;
+    ODB_CUDA(launch_gemm(ga, st));
+    ODB_CUDA(launch_reduce_partials(ga.partial, splits, static_cast<size_t>(M) * N, out, static_cast<size_t>(M) * N, st));
+    int host_status = 0;
+    ODB_CUDA(cudaMemcpyAsync(&host_status, status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    ODB_CUDA(cudaStreamSynchronize(st));
+    return host_status;
+}
+
+double odb_step_algorithmic_bytes(const odb_config* c, int32_t keys) {
+    if (check_config(c) != ODB_OK) return 0.0;
+    const double d = c->d_model, F = c->d_ffn;
+    const double per_layer = (3 * d * d + d * d + 2 * F * d + d * F) * 2.0 + 2.0 * keys * d * 2.0;
+    return c->n_layers * per_layer + (c->with_lm_head ? 2.0 * c->vocab * d : 0.0);
+}
+
+}  // extern "C"

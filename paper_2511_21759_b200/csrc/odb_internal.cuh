@@ -1,0 +1,128 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/odb.h"
+
+namespace odb {
+
+// ---------------------------------------------------------------------------------------
+// session-wide device state
+// ---------------------------------------------------------------------------------------
+
+constexpr int kMaxBlock = 64;
+
+// Per-sequence control state, resident on the device and mirrored on the host after every
+// odb_unmask_accept.  Positions are absolute (prompt position 0 first).
+struct SeqState {
+    int32_t active;
+    int32_t in_fwd;               // took part in the forward last built (refresh or step)
+    int32_t P, T;                 // prompt length, current total length (prompt + response)
+    int32_t block_idx, s, e;      // current block [s, e)
+    int32_t n_masked;             // masked positions left in [s, e)
+    // speculative candidates for the next step (Section 4.2): offsets inside the block and the
+    // tokens they would be filled with, most confident first
+    int32_t n_ranks;
+    int32_t rank_off[ODB_MAX_RANKS];
+    int32_t rank_tok[ODB_MAX_RANKS];
+    // copies of the next step: bit r-1 of copy_mask[c] set <=> copy c fills rank r
+    int32_t n_copies;
+    int32_t copy_mask[ODB_MAX_COPIES];
+    int32_t stage2;               // decoded-share layout (Section 4.2.2) for the next step
+    // row table placement of the step last built
+    int32_t row0, n_rows;
+    int32_t copy_row0[ODB_MAX_COPIES];
+    int32_t copy_nrows[ODB_MAX_COPIES];
+    // placement of the last refresh's outputs: conf/tok of position p at lm_row0 + (p - lm_s)
+    int32_t lm_row0, lm_s, lm_n;
+};
+
+// One attention work item: up to 64 query rows that share one key set.
+// Keys, in order: cached positions [0, cA) and [cB0, cB1) of sequence `seq`, then the fresh
+// rows [f0, f0 + n0) (all visible), then the fresh rows [f1, f1 + n1) of which only those
+// flagged kRowDecoded are visible (decoded tokens of copy 0 shared with a speculative copy).
+struct QTile {
+    int32_t q_row0, nq;
+    int32_t seq;
+    int32_t cA, cB0, cB1;
+    int32_t f0, n0;
+    int32_t f1, n1;
+};
+
+constexpr int kRowDecoded = 1;   // row_flags bit: the row's position is decoded in the committed state
+
+// ---------------------------------------------------------------------------------------
+// kernel launchers (each enqueues on `st`; returns cudaError_t of the launch)
+// ---------------------------------------------------------------------------------------
+
+struct TmaEncoder;   // wraps the driver's tensor-map encode entry point
+
+// Weight-streaming GEMM: partial[s][M][N] (fp32) = x[M][K_s] * w[N][K_s]^T for each K split s.
+struct GemmArgs {
+    CUtensorMap tmap_w;    // bf16 [N][K], box 64 x 128, 128B swizzle
+    const void* x;         // bf16 [M][K] device
+    float* partial;        // fp32 [splits][M][N]
+    int M, N, K;
+    int splits;
+    int* status;           // device status word
+};
+int gemm_pick_splits(int M, int N, int K);
+cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K);
+cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
+cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,
+                                   cudaStream_t st);
+
+cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d,
+                         cudaStream_t st);
+// h[row] += sum_s partial[s][row] (if partial), out[i] = bf16(rmsnorm(h[map ? map[i] : i]) * gain)
+cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
+                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps,
+                           cudaStream_t st);
+struct QkvRopeArgs {
+    const float* partial; int splits; size_t pstride;      // [splits][M][3d]
+    const float2* rope;                                    // [max_seq][hd/2] (cos, sin)
+    const int32_t* row_pos; const int32_t* row_seq;
+    __nv_bfloat16 *q, *k, *v;                              // [M][d]
+    __nv_bfloat16* cache;                                  // NULL: do not write the cache
+    int layer, n_layers, H, hd, max_seq, M;
+};
+cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
+cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
+                          cudaStream_t st);
+cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
+                              cudaStream_t st);
+
+struct AttnArgs {
+    const QTile* tiles; int n_tiles;
+    const __nv_bfloat16 *q, *k, *v;       // fresh rows [M][H*hd]
+    const __nv_bfloat16* cache;           // [batch][L][2][H][max_seq][hd]
+    const int32_t* row_flags;
+    __nv_bfloat16* o;                     // [M][H*hd]
+    float* part_o; float* part_ml;        // split workspaces [ks][M][H][hd], [ks][M][H][2]
+    int layer, n_layers, H, hd, max_seq, M, ksplit;
+};
+cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
+
+// control kernels (control.cu)
+struct ControlBuffers {
+    SeqState* state;          // [batch]
+    int32_t* x;               // [batch][max_seq] token ids
+    int32_t max_seq;
+    int32_t* row_tok; int32_t* row_pos; int32_t* row_seq; int32_t* row_copy; int32_t* row_flags;
+    int32_t* lm_rows;         // rows whose logits are needed
+    QTile* tiles;
+    const float* conf; const int32_t* tok;   // outputs of the last forward, per logit row
+    odb_result* results;      // [batch] device copy
+};
+// block_index[seq] < 0: the sequence takes no part in this refresh
+cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index, int block_len,
+                                      cudaStream_t st);
+cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st);
+cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
+                          int mask_id, int eos_id, cudaStream_t st);
+
+}  // namespace odb
