@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the block-decoding hot path (one line of JSON on stdout).
+
+A "step" is one block cycle of the generation: refresh prefill + accept, then block decode
+steps + accepts until the block is full, for the workload named in `config.workload`
+(default: the 32-layer 8B-shaped model, batch 1, prompt 512, response 256, block 32).  The
+headline value is generated tokens per second over the timed steps.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+--impl reference times the CPU oracle (as it stands) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "gen tokens/s (8B-shaped, bs1, block 32); decode-step % of HBM roofline"
+UNIT = "tokens/s"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": p["hbm_gbs"], "bf16_tflops": p["bf16_tflops"],
+                "bf16_tflops_sustained": p.get("bf16_tflops_sustained", p["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([c.strip() for c in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except subprocess.TimeoutExpired:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], 0.0, set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx = max(mx, float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": mx or None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ----------------------------------------------------------------------------- CPU oracle arm
+
+def oracle_sample(wl, budget_layers=2):
+    """Times the oracle, as it stands, on a bounded sample of the workload: one refresh and one
+    block decode step of the first `budget_layers` layers (fp32), plus the LM head of the step
+    rows; layer time is scaled to the full depth.  Returns tokens/s of a block cycle so estimated
+    and a description of the sample."""
+    import synth
+    from oracle import odb_oracle as O
+    from oracle.inputs import model_from_synth
+    shape = wl.shape
+    nl = min(budget_layers, shape.n_layers)
+    T, P, Bk = wl.prompt_len + wl.gen_len, wl.prompt_len, wl.block_len
+    small = shape.with_layers(nl)
+    om = model_from_synth(small, seed=0, dtype=np.float32, with_lm_head=False)
+    for l in range(nl):
+        om.layer(l)                                   # weight synthesis is input preparation, not timed
+    x0 = synth.sequence(0, 0, P, wl.gen_len, shape).astype(np.int64)
+    t0 = time.perf_counter()
+    cache, _, _ = O.refresh_prefill(om, x0, T, P, dtype=np.float32)
+    t_refresh_layers = time.perf_counter() - t0
+    subsets = O.copy_subsets(2, wl.n_copies, False)
+    rank_pos, rank_tok = [P, P + 1][:2 if wl.n_copies > 1 else 0], [1, 2][:2 if wl.n_copies > 1 else 0]
+    t0 = time.perf_counter()
+    hid, _, _ = O.block_decode_step(om, cache, x0, T, P, P + Bk, subsets, rank_pos, rank_tok, False, dtype=np.float32)
+    t_step_layers = time.perf_counter() - t0
+    t_lm_step = t_lm_refresh = 0.0
+    if wl.with_lm_head:
+        lm = synth.bf16_bits_to_f32(synth.lm_head_bits(shape, 0))
+        n = O.bf16_round(O.rmsnorm(hid.astype(np.float32), np.ones(shape.d_model, np.float32), shape.rms_eps))
+        t0 = time.perf_counter()
+        O.confidence(n @ lm.T, shape.mask_id)
+        t_lm_step = time.perf_counter() - t0
+        t_lm_refresh = t_lm_step * (wl.gen_len / max(len(n), 1))
+    scale = shape.n_layers / nl
+    t_refresh = t_refresh_layers * scale + t_lm_refresh
+    t_step = t_step_layers * scale + t_lm_step
+    # random weights: one token per iteration, so a block of Bk tokens = 1 refresh + (Bk - 1) steps
+    t_block = t_refresh + (Bk - 1) * t_step
+    cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
+    return {"tokens_per_s": Bk / t_block, "t_step_s": t_step, "t_refresh_s": t_refresh, "cores": cores,
+            "sample": f"{nl} of {shape.n_layers} layers of one refresh (T={T}) and one block step (M={len(subsets) * Bk}) "
+                      f"in fp32 + LM head of the step rows, layer time scaled x{scale:g}; block cycle = 1 refresh + {Bk - 1} steps"}
+
+
+def run_reference(args, wl):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    for i in range(args.warmup + args.steps):
+        r = oracle_sample(wl)
+        if i >= args.warmup:
+            vals.append(r)
+    v = float(np.mean([r["tokens_per_s"] for r in vals]))
+    ms = float(np.mean([wl.block_len / r["tokens_per_s"] for r in vals])) * 1e3
+    line = {"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic", "config": config_of(wl),
+            "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
+                             "sample": vals[-1]["sample"]},
+            "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def config_of(wl):
+    return {"workload": wl.name, "batch": wl.batch, "prompt_len": wl.prompt_len, "gen_len": wl.gen_len,
+            "block_len": wl.block_len, "n_copies": wl.n_copies, "layers": wl.shape.n_layers,
+            "d_model": wl.shape.d_model, "vocab": wl.shape.vocab,
+            "l2": "weights streamed per forward (15 GB) exceed L2 (126 MB); no flush needed",
+            "step": "one block cycle: refresh prefill + accept, then block decode steps + accepts until the block is full"}
+
+
+# ----------------------------------------------------------------------------- CUDA arm
+
+def run_cuda(args, wl):
+    import torch
+    import synth
+    from paper_2511_21759_b200 import engine as E
+    import __graft_entry__ as G
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        G.build()
+    if dist:
+        dist.barrier()
+    peaks = load_peaks()
+    shape = wl.shape
+    T = wl.prompt_len + wl.gen_len
+    gm = E.Model.from_synth(shape, seed=0, device=f"cuda:{local}", with_lm_head=wl.with_lm_head, max_batch=wl.batch,
+                            max_seq=T, max_block=wl.block_len, max_copies=max(wl.n_copies, 1))
+    sess = E.Session(gm)
+    params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies, accept_threshold=wl.accept_threshold,
+                            truncate_threshold=wl.truncate_threshold)
+    n_blocks = wl.gen_len // wl.block_len
+    seqs = [synth.sequence(0, rank * wl.batch + i, wl.prompt_len, wl.gen_len, shape) for i in range(wl.batch)]
+    pinned = [torch.from_numpy(s.copy()).pin_memory() for s in seqs]
+
+    state = {"block": 0}
+
+    def reset():
+        for i in range(wl.batch):
+            sess.set_sequence(i, pinned[i].numpy(), wl.prompt_len)
+        state["block"] = 0
+
+    def block_cycle(e2e=False):
+        """refresh + accept, then steps + accepts until the block is full; returns (tokens, iterations)."""
+        if state["block"] >= n_blocks:
+            reset()
+        if e2e:   # inputs come from the host every step, the result goes back to the host
+            toks = [sess.get_tokens(i) for i in range(wl.batch)] if state["block"] else [p.numpy() for p in pinned]
+            blk = state["block"]
+            for i in range(wl.batch):
+                sess.set_sequence(i, toks[i], wl.prompt_len)
+            state["block"] = blk
+        b = state["block"]
+        sess.refresh_prefill(params, [b] * wl.batch)
+        res = sess.unmask_accept(params, True)
+        toks, iters = sum(res[i].n_accepted for i in range(wl.batch)), 1
+        while any(res[i].masks_left > 0 for i in range(wl.batch)):
+            sess.block_decode_step(params)
+            res = sess.unmask_accept(params, False)
+            toks += sum(res[i].n_accepted for i in range(wl.batch))
+            iters += 1
+        state["block"] += 1
+        if e2e:
+            for i in range(wl.batch):
+                sess.get_tokens(i)
+        return toks, iters
+
+    def timed(n, e2e=False):
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record(sess.stream)
+        toks = iters = 0
+        for _ in range(n):
+            t, it = block_cycle(e2e)
+            toks += t; iters += it
+        ev1.record(sess.stream)
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1)
+        if dist:
+            t_ = torch.tensor([ms], device="cuda")
+            dist.all_reduce(t_, op=dist.ReduceOp.MAX)
+            ms = float(t_.item())
+            if dist:
+                dist.barrier()
+        return ms, toks, iters
+
+    reset()
+    timed(args.warmup)
+    sess.profile_read()
+    with ClockSampler(local) as clocks:
+        ms, toks, iters = timed(args.steps)
+    _, launches = sess.profile_read()
+    clk = clocks.summary()
+    value = world * toks / (ms * 1e-3)
+
+    # end to end: same steps, sequence pushed from pinned host memory and read back every step
+    timed(1, e2e=True)
+    ms_e, toks_e, _ = timed(args.steps, e2e=True)
+    e2e_value = world * toks_e / (ms_e * 1e-3)
+
+    # per-kind device time of decode steps and refreshes, measured live with event pairs
+    sess.profile(True)
+    if state["block"] >= n_blocks:
+        reset()
+    sess.refresh_prefill(params, [state["block"]] * wl.batch)
+    res = sess.unmask_accept(params, True)
+    ms_refresh, n_refresh = sess.profile_read()
+    n_prof = 0
+    while any(res[i].masks_left > 0 for i in range(wl.batch)) and n_prof < 16:
+        sess.block_decode_step(params)
+        res = sess.unmask_accept(params, False)
+        n_prof += 1
+    ms_step, n_step = sess.profile_read()
+    sess.profile(False)
+    # whole decode step (enqueue to completion), events on the session's stream, profiling off
+    state["block"] = n_blocks
+    reset()
+    sess.refresh_prefill(params, [0] * wl.batch)
+    res = sess.unmask_accept(params, True)
+    step_ms = []
+    for _ in range(12):
+        if not any(res[i].masks_left > 0 for i in range(wl.batch)):
+            break
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(sess.stream)
+        sess.block_decode_step(params)
+        b_.record(sess.stream)
+        res = sess.unmask_accept(params, False)
+        step_ms.append(a.elapsed_time(b_))
+    state["block"] = n_blocks
+
+    keys = T - wl.block_len                                   # cached positions outside the block
+    step_bytes = gm.step_algorithmic_bytes(keys) * 1.0
+    d, F, V, nl = shape.d_model, shape.d_ffn, shape.vocab, shape.n_layers
+    gemm_bytes = nl * (3 * d * d + d * d + 2 * F * d + d * F) * 2 + (V * d * 2 if wl.with_lm_head else 0)
+    gemm_launches = max(n_step["gemm"], 1)
+    gemm_ms = ms_step["gemm"] / max(n_prof, 1)                # per decode step
+    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else None
+    step_med = float(np.median(step_ms)) if step_ms else None
+    roofline = {"bound": "hbm", "kernel": "gemm_kernel<32> (tcgen05 weight-streaming GEMM), all launches of one decode step",
+                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
+                "traffic": None, "bytes_per_step": gemm_bytes, "launches_per_step": gemm_launches / max(n_prof, 1),
+                "ms_per_step": gemm_ms,
+                "decode_step": {"ms": step_med, "algorithmic_bytes": step_bytes,
+                                "achieved_gbs": step_bytes / (step_med * 1e-3) / 1e9 if step_med else None,
+                                "frac_of_measured": step_bytes / (step_med * 1e-3) / 1e9 / peaks["hbm_gbs"] if step_med else None,
+                                "frac_of_nominal_8tbs": step_bytes / (step_med * 1e-3) / 1e9 / 8000.0 if step_med else None,
+                                "ms_by_kind": {k: v / max(n_prof, 1) for k, v in ms_step.items()}},
+                "refresh": {"ms_by_kind": ms_refresh, "T": T}}
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic", "config": config_of(wl),
+            "tokens_per_step": toks / args.steps, "iterations_per_step": iters / args.steps,
+            "clocks": clk,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * T * wl.batch,
+                    "d2h_bytes_per_step": 4 * T * wl.batch},
+            "gpu_launches": int(sum(launches.values())),
+            "roofline": roofline}
+    if rank == 0:
+        if world == 1 and not args.no_cpu_baseline:
+            r = oracle_sample(wl)
+            line["cpu_baseline"] = {"value": r["tokens_per_s"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
+                                    "sample": r["sample"], "t_step_s": r["t_step_s"], "t_refresh_s": r["t_refresh_s"]}
+        print(json.dumps(line))
+    sess.close()
+    gm.close()
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="cfg3_8b_c1")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    import synth
+    wl = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_cuda(args, wl)
+
+
+if __name__ == "__main__":
+    main()

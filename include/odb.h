@@ -56,6 +56,16 @@ enum {
     ODB_ERR_TIMEOUT = -6    /* a bounded device-side wait expired */
 };
 
+/* kernel kinds of the launch accounting (odb_session_profile_read) */
+enum {
+    ODB_KIND_GEMM = 0,        /* tcgen05 weight-streaming GEMMs (QKV, O, gate/up, down, LM head) */
+    ODB_KIND_ATTENTION = 1,   /* block-query attention (+ its split merge) */
+    ODB_KIND_ELEMENTWISE = 2, /* embedding, RMSNorm, RoPE/cache scatter, SwiGLU */
+    ODB_KIND_CONFIDENCE = 3,  /* vocab-wide max / sum / argmax */
+    ODB_KIND_CONTROL = 4,     /* row tables, accept / jump / ALP */
+    ODB_PROFILE_KINDS = 5
+};
+
 #define ODB_MAX_COPIES 8
 #define ODB_MAX_RANKS 4
 #define ODB_MAX_CHAIN 5
@@ -188,6 +198,15 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap_byt
  * Runs on `stream` and waits for it; returns ODB_ERR_TIMEOUT if a device-side wait expired. */
 int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, size_t scratch_bytes,
                        int32_t M, int32_t N, int32_t K, int32_t k_splits, void* stream);
+
+/* Launch accounting.  odb_session_profile(s, 1) waits for the stream, clears the counters and
+ * from then on brackets every kernel launch of the session with a CUDA event pair (this
+ * serialises nothing but costs two event records per launch; leave it off when timing whole
+ * steps).  odb_session_profile_read waits for the stream, returns per kind the launches counted
+ * since the last read and (profiling on) the summed device time in ms, and clears both.
+ * Launches are counted whether profiling is on or off. */
+int32_t odb_session_profile(odb_session* s, int32_t enable);
+int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* launches_by_kind);
 
 /* Algorithmic bytes one odb_block_decode_step must move for `rows` query rows and `keys`
  * visible cached positions per sequence (weights once + K/V once); used by the benchmark. */

@@ -7,7 +7,7 @@
 // grid = (tiles, heads, key splits); each CTA streams its share of the keys in tiles of 64
 // through shared memory with 16-byte cp.async loads (double buffered, XOR-swizzled rows) and
 // runs an online-softmax on mma.sync m16n8k16 bf16 tiles (fp32 scores, statistics and output
-// accumulator; probabilities rounded to bf16 for the P.V product).  With more than one key
+// accumulator; probabilities enter the P.V product as a two-term bf16 sum).  With more than one key
 // split the unnormalised partial outputs and (max, sum) pairs are merged in split order by a
 // second kernel, so the result does not depend on scheduling.
 #include "odb_internal.cuh"
@@ -204,20 +204,29 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
                 o_acc[i][2 * r + 1] *= corr;
             }
         }
-        // O += P V
+        // O += P V.  P is fed to the tensor core as a sum of two bf16 terms (value rounded to bf16
+        // plus the rounded remainder), so the product carries ~16 significant bits of P instead of
+        // 8: with near-uniform attention the output is a small average of large terms and a bare
+        // bf16 P would cost a full bf16 step of the result.
 #pragma unroll
         for (int kk = 0; kk < 4; ++kk) {
-            uint32_t pa[4];
-            pa[0] = pack_bf16(s[2 * kk][0], s[2 * kk][1]);
-            pa[1] = pack_bf16(s[2 * kk][2], s[2 * kk][3]);
-            pa[2] = pack_bf16(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-            pa[3] = pack_bf16(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            uint32_t pa[4], pl[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const float x0 = s[2 * kk + (u >> 1)][(u & 1) * 2], x1 = s[2 * kk + (u >> 1)][(u & 1) * 2 + 1];
+                const __nv_bfloat162 hi = __floats2bfloat162_rn(x0, x1);
+                const float2 hf = __bfloat1622float2(hi);
+                pa[u] = *reinterpret_cast<const uint32_t*>(&hi);
+                pl[u] = pack_bf16(x0 - hf.x, x1 - hf.y);
+            }
 #pragma unroll
             for (int dp = 0; dp < HD / 16; ++dp) {
                 uint32_t vb[4];
                 ldmatrix_x4_trans(vb, vbase + swz<HD>(kk * 16 + r8 + (j & 1) * 8, dp * 2 + (j >> 1)));
                 mma_bf16(o_acc[2 * dp], pa, vb[0], vb[1]);
                 mma_bf16(o_acc[2 * dp + 1], pa, vb[2], vb[3]);
+                mma_bf16(o_acc[2 * dp], pl, vb[0], vb[1]);
+                mma_bf16(o_acc[2 * dp + 1], pl, vb[2], vb[3]);
             }
         }
     }

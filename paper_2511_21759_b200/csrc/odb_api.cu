@@ -118,6 +118,13 @@ struct odb_session {
     int* pinned_status;
     int phase;            // 0 idle, 1 refresh enqueued, 2 accepted, 3 step enqueued
     int last_rows, last_lm_rows;
+    // launch accounting: kernels launched per kind since the last read; with profiling on, a CUDA
+    // event pair brackets every launch so that per-kind device time can be summed afterwards
+    long long launches[ODB_PROFILE_KINDS];
+    bool profiling;
+    std::vector<cudaEvent_t> ev;        // pairs (start, stop)
+    std::vector<int> ev_kind;
+    size_t ev_used;
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
 
@@ -204,6 +211,9 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->L = L;
     s->phase = 0;
     s->last_rows = s->last_lm_rows = 0;
+    memset(s->launches, 0, sizeof(s->launches));
+    s->profiling = false;
+    s->ev_used = 0;
     s->mirror.assign(c.max_batch, SeqState{});
     s->pinned_state = nullptr;
     s->pinned_results = nullptr;
@@ -252,6 +262,7 @@ int32_t odb_session_destroy(odb_session* s) {
     if (s->pinned_state) cudaFreeHost(s->pinned_state);
     if (s->pinned_results) cudaFreeHost(s->pinned_results);
     if (s->pinned_status) cudaFreeHost(s->pinned_status);
+    for (cudaEvent_t e : s->ev) cudaEventDestroy(e);
     delete s;
     return ODB_OK;
 }
@@ -333,6 +344,31 @@ int32_t odb_session_status(odb_session* s) {
 
 namespace {
 
+// Brackets one kernel launch: counts it and, when profiling, records an event pair around it.
+struct LaunchScope {
+    odb_session* s;
+    bool timed;
+    size_t slot;
+    LaunchScope(odb_session* s_, int kind) : s(s_), timed(false), slot(0) {
+        ++s->launches[kind];
+        if (!s->profiling) return;
+        if (s->ev_used + 2 > s->ev.size()) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) return;
+            s->ev.push_back(a);
+            s->ev.push_back(b);
+            s->ev_kind.push_back(kind);
+        }
+        slot = s->ev_used;
+        s->ev_kind[slot / 2] = kind;
+        s->ev_used += 2;
+        timed = cudaEventRecord(s->ev[slot], s->st) == cudaSuccess;
+    }
+    ~LaunchScope() {
+        if (timed) cudaEventRecord(s->ev[slot + 1], s->st);
+    }
+};
+
 // One forward over the M rows of the row table already built on the device.
 int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) {
     const odb_model* m = s->m;
@@ -366,7 +402,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         return launch_gemm(ga, st);
     };
 
-    ODB_CUDA(launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
+#define ODB_LAUNCH(kind, call)          \
+    do {                                \
+        LaunchScope scope__(s, kind);   \
+        ODB_CUDA(call);                 \
+    } while (0)
+    ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
     const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
     int res_splits = 0;
     size_t res_stride = 0;
@@ -375,9 +416,9 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
     if (static_cast<size_t>(ks) * M > L.attn_rows) ks = static_cast<int>(L.attn_rows / M);
     if (ks < 1) ks = 1;
     for (int l = 0; l < c.n_layers; ++l) {
-        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, nullptr, M, d, c.rms_eps, st));
         int sp = 0;
-        ODB_CUDA(gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
         QkvRopeArgs qa;
         qa.partial = partial; qa.splits = sp; qa.pstride = static_cast<size_t>(M) * 3 * d;
         qa.rope = s->at<float2>(L.rope);
@@ -385,35 +426,36 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         qa.q = q; qa.k = k; qa.v = v;
         qa.cache = write_cache ? s->kv : nullptr;
         qa.layer = l; qa.n_layers = c.n_layers; qa.H = H; qa.hd = hd; qa.max_seq = c.max_seq; qa.M = M;
-        ODB_CUDA(launch_qkv_rope(qa, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_qkv_rope(qa, st));
         AttnArgs aa;
         aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
         aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
         aa.part_o = s->at<float>(L.part_o); aa.part_ml = s->at<float>(L.part_ml);
         aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = ks;
-        ODB_CUDA(launch_attention(aa, st));
+        ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention(aa, st));
+        if (ks > 1) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
         sp = 0;
-        ODB_CUDA(gemm(m->tm_o[l], o, partial, M, d, d, &sp));
-        ODB_CUDA(launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps, st));
         sp = 0;
-        ODB_CUDA(gemm(m->tm_gu[l], a, partial, M, 2 * F, d, &sp));
-        ODB_CUDA(launch_swiglu(partial, sp, static_cast<size_t>(M) * 2 * F, g, M, F, st));
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_gu[l], a, partial, M, 2 * F, d, &sp));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_swiglu(partial, sp, static_cast<size_t>(M) * 2 * F, g, M, F, st));
         sp = 0;
-        ODB_CUDA(gemm(m->tm_d[l], g, partial, M, d, F, &sp));
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, &sp));
         res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
     }
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
-        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, nullptr, M, d, c.rms_eps, st));
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
     for (int r0 = 0; r0 < n_lm; r0 += static_cast<int>(L.lm_chunk)) {
         const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
-        ODB_CUDA(launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps, st));
         int sp = 1;
-        ODB_CUDA(gemm(m->tm_lm, a, logits, rows, c.vocab, d, &sp));
-        ODB_CUDA(launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0, st));
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, logits, rows, c.vocab, d, &sp));
+        ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0, st));
     }
     return ODB_OK;
 }
@@ -446,7 +488,7 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
         n_tiles += (st.T + 63) / 64;
     }
     if (M == 0) return ODB_ERR_STATE;
-    ODB_CUDA(launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
+    ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
     int32_t rc = forward(s, M, c.with_lm_head ? n_lm : 0, n_tiles, true);
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
@@ -469,7 +511,7 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
     }
     if (M == 0) return ODB_ERR_STATE;
     if (static_cast<size_t>(M) > s->L.rows) return ODB_ERR_SHAPE;
-    ODB_CUDA(launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
+    ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
     int32_t rc = forward(s, M, c.with_lm_head ? M : 0, n_tiles, false);
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
@@ -486,7 +528,7 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
     if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != (after_refresh ? 1 : 3)) return ODB_ERR_STATE;
-    ODB_CUDA(launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id, s->st));
+    ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id, s->st));
     ODB_CUDA(cudaMemcpyAsync(s->pinned_results, s->cb.results, sizeof(odb_result) * c.max_batch, cudaMemcpyDeviceToHost, s->st));
     int* dev_status = s->at<int>(s->L.status);
     ODB_CUDA(cudaMemcpyAsync(s->pinned_status, dev_status, sizeof(int), cudaMemcpyDeviceToHost, s->st));
@@ -555,6 +597,31 @@ int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, 
     ODB_CUDA(cudaMemcpyAsync(&host_status, status, sizeof(int), cudaMemcpyDeviceToHost, st));
     ODB_CUDA(cudaStreamSynchronize(st));
     return host_status;
+}
+
+int32_t odb_session_profile(odb_session* s, int32_t enable) {
+    if (!s) return ODB_ERR_ARG;
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    s->profiling = enable != 0;
+    s->ev_used = 0;
+    memset(s->launches, 0, sizeof(s->launches));
+    return ODB_OK;
+}
+
+int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* launches_by_kind) {
+    if (!s || !ms_by_kind || !launches_by_kind) return ODB_ERR_ARG;
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    for (int k = 0; k < ODB_PROFILE_KINDS; ++k) {
+        ms_by_kind[k] = 0.0;
+        launches_by_kind[k] = s->launches[k];
+        s->launches[k] = 0;
+    }
+    for (size_t i = 0; i + 1 < s->ev_used; i += 2) {
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, s->ev[i], s->ev[i + 1]) == cudaSuccess) ms_by_kind[s->ev_kind[i / 2]] += ms;
+    }
+    s->ev_used = 0;
+    return ODB_OK;
 }
 
 double odb_step_algorithmic_bytes(const odb_config* c, int32_t keys) {

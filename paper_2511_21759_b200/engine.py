@@ -150,6 +150,16 @@ class Session:
                 "odb_unmask_accept")
         return self._results
 
+    def profile(self, enable: bool):
+        B.check(B.lib().odb_session_profile(self.handle, 1 if enable else 0), "odb_session_profile")
+
+    def profile_read(self):
+        """({kind: ms}, {kind: launches}) since the last read."""
+        ms = (C.c_double * len(B.KINDS))()
+        n = (C.c_int64 * len(B.KINDS))()
+        B.check(B.lib().odb_session_profile_read(self.handle, ms, n), "odb_session_profile_read")
+        return dict(zip(B.KINDS, list(ms))), dict(zip(B.KINDS, list(n)))
+
     _READ = {"logits": (0, np.float32), "conf": (1, np.float32), "tok": (2, np.int32), "hidden": (3, np.float32),
              "q": (4, np.uint16), "k": (5, np.uint16), "v": (6, np.uint16), "o": (7, np.uint16),
              "row_tok": (8, np.int32), "row_pos": (9, np.int32), "row_copy": (10, np.int32)}

@@ -46,3 +46,138 @@ def compare_traces(gpu_trace, oracle_trace, seq=0, near_tie=1e-3):
     if len(gpu_trace) != len(oracle_trace):
         return n, {"iter": n, "gpu": None, "oracle": None, "margin": np.inf, "near_tie": False}
     return n, None
+
+
+def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, check_logits=True, max_iters=None,
+                      seq=0):
+    """Lock-step parity harness for one sequence.
+
+    Every iteration both sides start from the same state.  (1) Numerics: the GPU's logits /
+    confidences / greedy tokens are compared with the oracle's for that state.  (2) Control: the
+    oracle's accept rule, jump walk, ranking and row-table code are run on the GPU's OWN fp32
+    confidences and tokens and must reproduce the GPU's decision, chain and next row table bit
+    for bit (same inputs, same precision => identical integers).  (3) Bit-exact tokens: the
+    decision the oracle takes from ITS confidences is compared too; where it differs, the
+    oracle's decision margin must be below the confidence error measured in that iteration (a
+    near-tie); these are counted and returned, never hidden.  The GPU's decision then advances
+    both sides.  Returns a stats dict."""
+    shape_mask, eos = om.mask_id, om.eos_id
+    Bk, tau = op.block_len, op.accept_threshold
+    k_ranks = {1: 0, 4: 2, 8: 4}[op.n_copies]
+    x = np.array(x0, dtype=np.int64)
+    T = len(x)
+    st = {"iters": 0, "refreshes": 0, "steps": 0, "tokens": 0, "oracle_decision_diff": 0, "near_ties": [],
+          "worst_logit": 0.0, "worst_conf": 0.0, "tok_diff": 0}
+
+    def numerics(g_conf, g_tok, g_logits, o_conf, o_tok, o_logits):
+        rel = np.abs(g_conf.astype(np.float64) - o_conf) / np.maximum(o_conf, 1e-30)
+        st["worst_conf"] = max(st["worst_conf"], float(rel.max()))
+        if g_logits is not None:
+            ok, worst = logits_close(g_logits, o_logits, tol)
+            st["worst_logit"] = max(st["worst_logit"], worst)
+            assert ok, f"logits off by {worst:.2f} x bound at iteration {st['iters']}"
+            l32 = o_logits.astype(np.float32).astype(np.float64)
+            l32[:, shape_mask] = -np.inf
+            top2 = np.partition(l32, -2, axis=1)[:, -2:]
+            gap = np.abs(top2[:, 1] - top2[:, 0])
+            err = np.abs(g_logits - o_logits).max(axis=1)
+            diff = g_tok != o_tok
+            assert not (diff & (gap > 2 * err)).any(), "greedy token differs beyond the logit error"
+            st["tok_diff"] += int(diff.sum())
+        return float(rel.max())
+
+    def res_tuple(r):
+        return (sorted((r.accepted_pos[j], r.accepted_tok[j]) for j in range(r.n_accepted)),
+                [r.chain[j] for j in range(r.chain_len)])
+
+    b = 0
+    while True:
+        s = P + b * Bk
+        if s >= T or (max_iters is not None and st["iters"] >= max_iters):
+            break
+        sess.refresh_prefill(gp, b)
+        g_conf, g_tok = sess.debug_read("conf"), sess.debug_read("tok")
+        g_logits = sess.debug_read("logits") if check_logits else None
+        out = O.refresh_prefill(om, x, T, s, return_logits=True)
+        cache, o_conf, o_tok, o_logits = out
+        assert len(g_conf) == T - s
+        cerr = numerics(g_conf, g_tok, g_logits, o_conf, o_tok, o_logits)
+        newL = O.alp_scan(g_conf, g_tok, s, P, eos, op.truncate_threshold) if op.alp else None
+        newL_o = O.alp_scan(o_conf, o_tok, s, P, eos, op.truncate_threshold) if op.alp else None
+        if schedule is not None:
+            cand = schedule(b, T - P)
+            if cand is not None and s - P < cand < T - P:
+                sess.set_gen_len(seq, cand)
+                newL = cand if newL is None else min(newL, cand)
+                newL_o = cand if newL_o is None else min(newL_o, cand)
+        res = sess.unmask_accept(gp, True)[seq]
+        if newL is not None and P + newL < T:
+            T = P + newL
+            x = x[:T]
+        assert res.gen_len == T - P, (res.gen_len, T - P)
+        e = min(s + Bk, T)
+        B = e - s
+        assert (res.block_start, res.block_end) == (s, e)
+        masked = x[s:e] == shape_mask
+        acc = O.accept_set(g_conf[:B], masked, tau)
+        want = [(int(s + i), int(g_tok[i])) for i in np.flatnonzero(acc)]
+        assert res_tuple(res) == (want, [0]), (res_tuple(res), want)
+        acc_o = O.accept_set(o_conf[:B], masked, tau)
+        want_o = [(int(s + i), int(o_tok[i])) for i in np.flatnonzero(acc_o)]
+        if want_o != want or newL_o != newL:
+            margin = O.decision_margin(o_conf[:B], masked, tau, 0)
+            st["oracle_decision_diff"] += 1
+            st["near_ties"].append((st["iters"], "refresh", margin, cerr))
+        for p_, t_ in want:
+            x[p_] = t_
+        st["iters"] += 1; st["refreshes"] += 1; st["tokens"] += len(want)
+        assert res.masks_left == int((x[s:e] == shape_mask).sum())
+        last_conf, last_tok = g_conf[:B], g_tok[:B]
+        while (x[s:e] == shape_mask).any():
+            if max_iters is not None and st["iters"] >= max_iters:
+                break
+            masked = x[s:e] == shape_mask
+            ranks = O.rank_candidates(last_conf, masked, k_ranks)
+            rank_pos = [s + i for i in ranks]
+            rank_tok = [int(last_tok[i]) for i in ranks]
+            st2 = O.use_stage2(op, B, int((~masked).sum()))
+            subsets = O.copy_subsets(len(ranks), 4 if (op.n_copies == 8 and not st2) else op.n_copies, st2)
+            o_c, o_t, o_logits, r_copy, r_pos = O.block_decode_step(om, cache, x, T, s, e, subsets, rank_pos,
+                                                                    rank_tok, st2, return_logits=True)
+            _, _, r_tok = O.build_rows(x, s, e, shape_mask, subsets, rank_pos, rank_tok, st2)
+            sess.block_decode_step(gp)
+            assert np.array_equal(sess.debug_read("row_pos"), r_pos), "row positions"
+            assert np.array_equal(sess.debug_read("row_copy"), r_copy), "row copies"
+            assert np.array_equal(sess.debug_read("row_tok"), r_tok), "row tokens (ranking / fills)"
+            g_cr, g_tr = sess.debug_read("conf"), sess.debug_read("tok")
+            g_logits = sess.debug_read("logits") if check_logits else None
+            cerr = numerics(g_cr, g_tr, g_logits, o_c[r_copy, r_pos - s], o_t[r_copy, r_pos - s], o_logits)
+            C = len(subsets)
+            g_c = np.full((C, B), -1.0, dtype=np.float32)
+            g_t = np.full((C, B), -1, dtype=np.int32)
+            g_c[r_copy, r_pos - s] = g_cr
+            g_t[r_copy, r_pos - s] = g_tr
+            res = sess.unmask_accept(gp, False)[seq]
+            new, chain, last = O.jump_walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
+            want = sorted((int(s + i), int(t)) for i, t in new.items())
+            assert res_tuple(res) == (want, [int(c) for c in chain]), (res_tuple(res), want, chain)
+            new_o, chain_o, last_o = O.jump_walk(o_c, o_t, masked, subsets, ranks, rank_tok, tau)
+            if new_o != new or chain_o != chain:
+                margin = min(O.decision_margin(o_c[c], masked & (o_c[c] >= 0), tau, 0) for c in chain_o)
+                st["oracle_decision_diff"] += 1
+                st["near_ties"].append((st["iters"], "step", margin, cerr))
+            for p_, t_ in want:
+                x[p_] = t_
+            st["iters"] += 1; st["steps"] += 1; st["tokens"] += len(want)
+            assert res.masks_left == int((x[s:e] == shape_mask).sum())
+            last_conf, last_tok = g_c[last], g_t[last]
+        b += 1
+    st["tokens_final"] = x.astype(np.int32)
+    return st
+
+
+def assert_near_ties_only(st, floor=1e-3):
+    """Every iteration where the oracle would have decided differently must be a near-tie: its
+    decision margin no larger than four times the confidence error measured there (floor 1e-3)."""
+    for it, kind, margin, cerr in st["near_ties"]:
+        assert margin <= max(floor, 4 * cerr), f"iteration {it} ({kind}): margin {margin:.3e}, conf error {cerr:.3e}"

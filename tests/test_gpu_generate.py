@@ -14,7 +14,7 @@ import pytest
 import synth
 from oracle import odb_oracle as O
 from oracle.inputs import model_from_synth
-from gpu_common import engine, requires_gpu, compare_traces
+from gpu_common import engine, requires_gpu, compare_traces, lockstep_generate, assert_near_ties_only
 
 NEAR_TIE = 1e-3
 
@@ -56,6 +56,33 @@ def _assert_parity(gtok, gtrace, otok, otrace):
 @pytest.mark.parametrize("wl", ["cfg1_tiny", "cfg1_tiny_c4", "peaky_c1", "peaky_c4", "peaky_c8"])
 def test_generate_matches_oracle(wl):
     _assert_parity(*_run_both(wl))
+
+
+@requires_gpu
+@pytest.mark.parametrize("wl_name,tol", [("cfg1_tiny", 2e-2), ("cfg1_tiny_c4", 2e-2), ("peaky_c1", 4e-2),
+                                         ("peaky_c4", 4e-2), ("peaky_c8", 4e-2)])
+def test_lockstep_generate(wl_name, tol):
+    """Whole generation in lock step: numerics every iteration, control bit-exact on the GPU's own
+    confidences, oracle-side decisions equal except at measured near-ties.  The sharp-logit model
+    amplifies bf16 rounding (the oracle's own fp32 and fp64 runs differ by 0.8 of the 2e-2 bound
+    there), hence its wider logit tolerance."""
+    E = engine()
+    wl = synth.WORKLOADS[wl_name]
+    om = model_from_synth(wl.shape, seed=0)
+    gm = E.Model.from_synth(wl.shape, seed=0, max_batch=1, max_seq=wl.prompt_len + wl.gen_len,
+                            max_block=wl.block_len, max_copies=8)
+    sess = E.Session(gm)
+    x0 = synth.sequence(0, 0, wl.prompt_len, wl.gen_len, wl.shape)
+    sess.set_sequence(0, x0, wl.prompt_len)
+    kw = dict(block_len=wl.block_len, n_copies=wl.n_copies)
+    st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=tol)
+    assert sess.status() == 0
+    assert np.array_equal(sess.get_tokens(0), st["tokens_final"])
+    assert (st["tokens_final"][wl.prompt_len:] != wl.shape.mask_id).all() and st["tokens"] == wl.gen_len
+    assert_near_ties_only(st)
+    print(f"\n{wl_name}: {st['iters']} iterations ({st['refreshes']} refreshes), worst logit {st['worst_logit']:.2f} x bound, "
+          f"worst conf rel err {st['worst_conf']:.2e}, oracle-side decision diffs {st['oracle_decision_diff']}")
+    sess.close(); gm.close()
 
 
 @requires_gpu
