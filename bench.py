@@ -331,6 +331,71 @@ def run_cuda(args, wl):
         dist.destroy_process_group()
 
 
+def run_layer_microbench(args, wl):
+    """Single-layer block-decode-step microbenchmark (model without LM head): one refresh fills the
+    cache, then every timed iteration is one odb_block_decode_step over block 0 with the workload's
+    number of copies.  L2 is flushed (256 MB written) before every iteration; each iteration is
+    timed on its own with CUDA events on the session's stream."""
+    import torch
+    import __graft_entry__ as G
+    from paper_2511_21759_b200 import engine as E
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    G.build()
+    peaks = load_peaks()
+    shape, T = wl.shape, wl.prompt_len + wl.gen_len
+    import synth
+    gm = E.Model.from_synth(shape, seed=0, with_lm_head=False, max_batch=1, max_seq=T, max_block=wl.block_len,
+                            max_copies=max(wl.n_copies, 1))
+    sess = E.Session(gm)
+    params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies)
+    sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape), wl.prompt_len)
+    sess.refresh_prefill(params, 0)
+    sess.unmask_accept(params, True)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    times = []
+    with ClockSampler(0) as clocks:
+        for i in range(args.warmup + args.steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(sess.stream)
+            sess.block_decode_step(params)
+            b.record(sess.stream)
+            sess.unmask_accept(params, False)
+            if i >= args.warmup:
+                times.append(a.elapsed_time(b))
+    _, launches = sess.profile_read()
+    sess.profile(True)
+    for _ in range(8):
+        flush.zero_()
+        sess.block_decode_step(params)
+        sess.unmask_accept(params, False)
+    ms_kind, n_kind = sess.profile_read()
+    sess.profile(False)
+    ms = float(np.median(times))
+    keys = T - wl.block_len
+    step_bytes = gm.step_algorithmic_bytes(keys)
+    d, F = shape.d_model, shape.d_ffn
+    gemm_bytes = (3 * d * d + d * d + 2 * F * d + d * F) * 2
+    gemm_ms = ms_kind["gemm"] / 8
+    line = {"metric": "single-layer block decode step latency", "value": ms * 1e3, "unit": "us", "n_gpus": 1,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": False, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": dict(config_of(wl), l2="flushed before every iteration (256 MB written)",
+                           step="one odb_block_decode_step of the single layer"),
+            "clocks": clocks.summary(), "gpu_launches": int(sum(launches.values())),
+            "roofline": {"bound": "hbm", "kernel": "whole layer step (4 GEMMs + attention + elementwise)",
+                         "achieved": step_bytes / (ms * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                         "frac": step_bytes / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                         "traffic": None, "algorithmic_bytes": step_bytes,
+                         "gemm": {"ms": gemm_ms, "achieved_gbs": gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms else None},
+                         "ms_by_kind": {k: v / 8 for k, v in ms_kind.items()},
+                         "p10_ms": float(np.percentile(times, 10)), "p90_ms": float(np.percentile(times, 90))}}
+    print(json.dumps(line))
+    sess.close()
+    gm.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -344,6 +409,8 @@ def main():
     wl = synth.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, wl)
+    elif not wl.with_lm_head:
+        run_layer_microbench(args, wl)
     else:
         run_cuda(args, wl)
 

@@ -179,7 +179,10 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p);
 /* Applies the accept rule and the jump walk to the outputs of the preceding refresh
  * (after_refresh = 1: copy 0 only, preceded by the [EOS] scan / truncation when p->alp) or
  * step (after_refresh = 0), commits tokens, ranks the next speculative candidates.
- * results: host array [max_batch].  Waits for the stream. */
+ * results: host array [max_batch].  Waits for the stream.
+ * With a model built without LM head (layer microbenchmark) there are no confidences: the call
+ * commits nothing and only lays out the copies of the next step (speculative fills: the first
+ * masked positions with token id 0), so masks_left never decreases. */
 int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t after_refresh,
                           odb_result* results);
 

@@ -70,6 +70,8 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
     uint8_t* sV = sK + 2 * kTileBytes;               // [2][64][HD]
     uint8_t* sValid = sV + 2 * kTileBytes;           // [2][64]
 
+    pdl_launch_dependents();
+    pdl_wait();
     const QTile t = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
     const int z = blockIdx.z;
@@ -264,6 +266,8 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
 // grid (M, H), block HD: merge the key splits in split order.
 __global__ void attention_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                          __nv_bfloat16* __restrict__ o, int M, int H, int hd, int ksplit) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
     float mmax = -INFINITY;
     for (int z = 0; z < ksplit; ++z)
@@ -291,11 +295,10 @@ cudaError_t launch_hd(const AttnArgs& a, cudaStream_t st) {
         attr_done = true;
     }
     dim3 grid(a.n_tiles, a.H, a.ksplit);
-    attention_kernel<HD><<<grid, kAttnThreads, smem, st>>>(a);
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_kernel(attention_kernel<HD>, grid, dim3(kAttnThreads), smem, st, a);
     if (e != cudaSuccess || a.ksplit == 1) return e;
-    attention_combine_kernel<<<dim3(a.M, a.H), HD, 0, st>>>(a.part_o, a.part_ml, a.o, a.M, a.H, HD, a.ksplit);
-    return cudaGetLastError();
+    return launch_kernel(attention_combine_kernel, dim3(a.M, a.H), dim3(HD), 0, st, static_cast<const float*>(a.part_o),
+                         static_cast<const float*>(a.part_ml), a.o, a.M, a.H, HD, a.ksplit);
 }
 
 }  // namespace

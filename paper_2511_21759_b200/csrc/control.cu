@@ -145,7 +145,8 @@ __device__ int accept_set(const float* conf, const bool* masked, int B, float ta
     return n;
 }
 
-__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id) {
+__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id,
+                              int dry) {
     const int seq = blockIdx.x;
     SeqState* st = c.state + seq;
     odb_result* res = c.results + seq;
@@ -167,6 +168,39 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
     int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
     const int s = st->s;
     int n_copies = 1;
+    if (dry) {
+        // model without LM head (layer microbenchmark): there is nothing to decide on, so commit
+        // nothing and lay out the next step as if no position had been accepted; the speculative
+        // fills are the first masked positions with token id 0
+        if (after_refresh) st->e = min(s + p.block_len, st->T);
+        const int B = st->e - s;
+        int n_masked = 0, n_ranks = 0;
+        const int k_ranks = p.n_copies >= 8 ? 4 : p.n_copies >= 4 ? 2 : 0;
+        for (int i = 0; i < B; ++i) {
+            if (x[s + i] != mask_id) continue;
+            if (n_ranks < k_ranks) { st->rank_off[n_ranks] = i; st->rank_tok[n_ranks] = 0; ++n_ranks; }
+            ++n_masked;
+        }
+        st->n_ranks = n_ranks;
+        st->n_masked = n_masked;
+        const int thr = p.stage2_min_decoded >= 0 ? p.stage2_min_decoded : (4 * B + 6) / 7;
+        const int stage2 = (p.n_copies >= 8 && (B - n_masked) >= thr) ? 1 : 0;
+        const int want = p.n_copies >= 8 ? (stage2 ? 8 : 4) : p.n_copies >= 4 ? 4 : 1;
+        const int all_masks[ODB_MAX_COPIES] = {0, 1, 2, 3, 4, 7, 8, 15};
+        int nc = 0;
+        for (int i = 0; i < want; ++i)
+            if ((all_masks[i] >> n_ranks) == 0) st->copy_mask[nc++] = all_masks[i];
+        st->n_copies = nc;
+        st->stage2 = stage2;
+        res->masks_left = n_masked;
+        res->n_accepted = 0;
+        res->chain_len = 1;
+        res->chain[0] = 0;
+        res->gen_len = st->T - st->P;
+        res->block_start = s;
+        res->block_end = st->e;
+        return;
+    }
     if (after_refresh) {
         // adaptive length prediction (Section 4.1): first [EOS] of the whole predicted response
         // whose confidence exceeds the truncate threshold cuts the response there (slot kept)
@@ -288,8 +322,8 @@ cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_
 }
 
 cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
-                          int mask_id, int eos_id, cudaStream_t st) {
-    accept_kernel<<<batch, 32, 0, st>>>(c, p, after_refresh, mask_id, eos_id);
+                          int mask_id, int eos_id, int dry, cudaStream_t st) {
+    accept_kernel<<<batch, 32, 0, st>>>(c, p, after_refresh, mask_id, eos_id, dry);
     return cudaGetLastError();
 }
 

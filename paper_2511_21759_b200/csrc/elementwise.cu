@@ -27,6 +27,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 
 __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ row_tok,
                              float* __restrict__ h, int d) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int row = blockIdx.x;
     const __nv_bfloat16* src = embed + static_cast<size_t>(row_tok[row]) * d;
     float* dst = h + static_cast<size_t>(row) * d;
@@ -37,34 +39,57 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
 }
 
 // One block per output row.  y = x / sqrt(mean(x^2) + eps) * gain, x = residual stream row
-// (after adding the split-K partials of the preceding projection in split order).
-__global__ void rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial, int splits, size_t pstride,
-                               const float* __restrict__ gain, __nv_bfloat16* __restrict__ out,
-                               const int32_t* __restrict__ row_map, int d, float eps) {
+// (after adding the split-K partials of the preceding projection in split order).  float4
+// accesses; a thread keeps its (up to two) vectors in registers between the two passes.
+__global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
+                                                       int splits, size_t pstride, const float* __restrict__ gain,
+                                                       __nv_bfloat16* __restrict__ out,
+                                                       const int32_t* __restrict__ row_map, int d, float eps) {
     __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int orow = blockIdx.x;
     const int row = row_map ? row_map[orow] : orow;
     float* hr = h + static_cast<size_t>(row) * d;
+    const int nvec = d >> 2, stride = blockDim.x;
+    float4 keep[2];
     float ss = 0.f;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) {
-        float v = hr[i];
+    int slot = 0;
+    for (int i = threadIdx.x; i < nvec; i += stride, ++slot) {
+        float4 v = reinterpret_cast<const float4*>(hr)[i];
         if (partial) {
-            const float* p = partial + static_cast<size_t>(row) * d + i;
-            for (int s = 0; s < splits; ++s) v += p[s * pstride];
-            hr[i] = v;
+            const float4* p = reinterpret_cast<const float4*>(partial + static_cast<size_t>(row) * d) + i;
+            for (int s = 0; s < splits; ++s) {
+                const float4 t = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + s * pstride);
+                v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+            }
+            reinterpret_cast<float4*>(hr)[i] = v;
         }
-        ss += v * v;
+        if (slot < 2) keep[slot] = v;
+        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
     const float total = block_sum(ss, red);
     const float inv = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
     __nv_bfloat16* o = out + static_cast<size_t>(orow) * d;
-    for (int i = threadIdx.x; i < d; i += blockDim.x) o[i] = __float2bfloat16_rn(hr[i] * inv * gain[i]);
+    slot = 0;
+    for (int i = threadIdx.x; i < nvec; i += stride, ++slot) {
+        const float4 v = slot < 2 ? keep[slot] : reinterpret_cast<const float4*>(hr)[i];
+        const float4 g = reinterpret_cast<const float4*>(gain)[i];
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv * g.x, v.y * inv * g.y);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv * g.z, v.w * inv * g.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+        reinterpret_cast<uint2*>(o)[i] = pk;
+    }
 }
 
-// One block per row.  Sums the QKV partials, rotates q and k (rotate-half pairing: element i
+// grid (rows, pair chunks), one thread per rotation pair.  Sums the QKV partials, rotates q and k (rotate-half pairing: element i
 // pairs with i + hd/2; angle = pos * theta^(-2i/hd), table precomputed), rounds to bf16 and
 // writes the row-major fresh q/k/v; in a refresh also the K/V cache [seq][layer][k|v][head][pos][hd].
 __global__ void qkv_rope_kernel(QkvRopeArgs a) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int row = blockIdx.x;
     const int d = a.H * a.hd, half = a.hd / 2;
     const int pos = a.row_pos[row];
@@ -78,7 +103,7 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
         ck = a.cache + (static_cast<size_t>(seq) * a.n_layers + a.layer) * 2 * per_kv;
         cv = ck + per_kv;
     }
-    for (int t = threadIdx.x; t < d / 2; t += blockDim.x) {
+    for (int t = blockIdx.y * blockDim.x + threadIdx.x; t < d / 2; t += gridDim.y * blockDim.x) {
         const int head = t / half, i = t % half;
         const int e0 = head * a.hd + i, e1 = e0 + half;
         float q0 = 0.f, q1 = 0.f, k0 = 0.f, k1 = 0.f, v0 = 0.f, v1 = 0.f;
@@ -109,6 +134,8 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
 // g[m][f] = bf16( silu(gate) * up ), gate = sum_s partial[s][m][f], up = sum_s partial[s][m][F + f]
 __global__ void swiglu_kernel(const float* __restrict__ partial, int splits, size_t pstride,
                               __nv_bfloat16* __restrict__ g, int M, int F) {
+    pdl_launch_dependents();
+    pdl_wait();
     const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (idx >= static_cast<size_t>(M) * F) return;
     const int m = static_cast<int>(idx / F), f = static_cast<int>(idx % F);
@@ -122,72 +149,121 @@ __global__ void swiglu_kernel(const float* __restrict__ partial, int splits, siz
     g[idx] = __float2bfloat16_rn(act * up);
 }
 
-// One block per row of logits: greedy token (lowest id on ties, [MASK] excluded) and its
-// softmax probability conf = 1 / sum_j exp(l_j - l_max).
-__global__ void confidence_kernel(const float* __restrict__ logits, int V, int mask_id, float* __restrict__ conf,
-                                  int32_t* __restrict__ tok) {
-    __shared__ float red_v[32];
-    __shared__ int red_i[32];
-    __shared__ float red[32];
-    const float* l = logits + static_cast<size_t>(blockIdx.x) * V;
-    float best = -INFINITY;
-    int besti = 0x7fffffff;
-    for (int i = threadIdx.x; i < V; i += blockDim.x) {
-        const float v = (i == mask_id) ? -INFINITY : l[i];
-        if (v > best) { best = v; besti = i; }
+// Greedy token (lowest id on ties, [MASK] excluded) and its softmax probability
+// conf = 1 / sum_j exp(l_j - l_max) per row of logits.  Phase 1: grid (rows, chunks), every block
+// makes one online pass (running max / rescaled sum / argmax) over its slice of the vocabulary
+// and writes a (max, sum, argmax) triple; phase 2 merges a row's triples in chunk order.
+struct ConfPartial {
+    float m, s;
+    int idx;
+};
+
+__device__ __forceinline__ void conf_merge(float& m, float& s, int& idx, float om, float os, int oi) {
+    if (om == -INFINITY) return;                       // the other side saw nothing
+    if (m == -INFINITY) { m = om; s = os; idx = oi; return; }
+    if (om > m) {
+        s = s * expf(m - om) + os;
+        m = om;
+        idx = oi;
+    } else {
+        s += os * expf(om - m);
+        if (om == m && oi < idx) idx = oi;
     }
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+}
+
+__global__ void __launch_bounds__(256) confidence_partial_kernel(const float* __restrict__ logits, int V, int mask_id,
+                                                                 int chunk, ConfPartial* __restrict__ part) {
+    __shared__ float sm[8], ss[8];
+    __shared__ int si[8];
+    pdl_launch_dependents();
+    pdl_wait();
+    const float* l = logits + static_cast<size_t>(blockIdx.x) * V;
+    const int lo = blockIdx.y * chunk, hi = min(V, lo + chunk);
+    float m = -INFINITY, s = 0.f;
+    int idx = 0x7fffffff;
+    for (int i = lo + threadIdx.x; i < hi; i += blockDim.x) {
+        const float v = l[i];
+        if (i == mask_id) continue;
+        if (v > m) {
+            s = s * expf(m - v) + 1.0f;                 // first element: s = 0 * exp(-inf) + 1
+            m = v;
+            idx = i;
+        } else {
+            s += expf(v - m);
+        }
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
-        const float ov = __shfl_xor_sync(0xffffffffu, best, o);
-        const int oi = __shfl_xor_sync(0xffffffffu, besti, o);
-        if (ov > best || (ov == best && oi < besti)) { best = ov; besti = oi; }
+        const float om = __shfl_xor_sync(0xffffffffu, m, o);
+        const float os = __shfl_xor_sync(0xffffffffu, s, o);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, o);
+        conf_merge(m, s, idx, om, os, oi);
     }
-    if (lane == 0) { red_v[warp] = best; red_i[warp] = besti; }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { sm[warp] = m; ss[warp] = s; si[warp] = idx; }
     __syncthreads();
-    best = red_v[0]; besti = red_i[0];
-    for (int w = 1; w < nw; ++w)
-        if (red_v[w] > best || (red_v[w] == best && red_i[w] < besti)) { best = red_v[w]; besti = red_i[w]; }
-    float sum = 0.f;
-    for (int i = threadIdx.x; i < V; i += blockDim.x)
-        if (i != mask_id) sum += expf(l[i] - best);
-    const float total = block_sum(sum, red);
     if (threadIdx.x == 0) {
-        conf[blockIdx.x] = 1.0f / total;
-        tok[blockIdx.x] = besti;
+        for (int w = 1; w < (blockDim.x >> 5); ++w) conf_merge(m, s, idx, sm[w], ss[w], si[w]);
+        ConfPartial p;
+        p.m = m; p.s = s; p.idx = idx;
+        part[static_cast<size_t>(blockIdx.x) * gridDim.y + blockIdx.y] = p;
     }
+}
+
+__global__ void confidence_final_kernel(const ConfPartial* __restrict__ part, int chunks, int rows,
+                                        float* __restrict__ conf, int32_t* __restrict__ tok) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;
+    if (row >= rows) return;
+    const ConfPartial* p = part + static_cast<size_t>(row) * chunks;
+    float m = p[0].m, s = p[0].s;
+    int idx = p[0].idx;
+    for (int c = 1; c < chunks; ++c) conf_merge(m, s, idx, p[c].m, p[c].s, p[c].idx);
+    conf[row] = 1.0f / s;
+    tok[row] = idx;
 }
 
 }  // namespace
 
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d, cudaStream_t st) {
-    embed_kernel<<<M, 256, 0, st>>>(embed, row_tok, h, d);
-    return cudaGetLastError();
+    return launch_kernel(embed_kernel, dim3(M), dim3(256), 0, st, embed, row_tok, h, d);
 }
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
                            __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps,
                            cudaStream_t st) {
-    rmsnorm_kernel<<<rows_out, 256, 0, st>>>(h, partial, splits, pstride, gain, out, row_map, d, eps);
-    return cudaGetLastError();
+    int threads = ((d / 4 + 31) / 32) * 32;
+    if (threads > 1024) threads = 1024;
+    return launch_kernel(rmsnorm_kernel, dim3(rows_out), dim3(threads), 0, st, h, partial, splits, pstride, gain, out, row_map,
+                         d, eps);
 }
 
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
-    qkv_rope_kernel<<<a.M, 256, 0, st>>>(a);
-    return cudaGetLastError();
+    const int pairs = a.H * a.hd / 2;
+    return launch_kernel(qkv_rope_kernel, dim3(a.M, (pairs + 255) / 256), dim3(256), 0, st, a);
 }
 
 cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
                           cudaStream_t st) {
     const size_t n = static_cast<size_t>(M) * F;
-    swiglu_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, st>>>(partial, splits, pstride, g, M, F);
-    return cudaGetLastError();
+    return launch_kernel(swiglu_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, partial, splits, pstride,
+                         g, M, F);
 }
 
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
-                              cudaStream_t st) {
-    confidence_kernel<<<rows, 1024, 0, st>>>(logits, V, mask_id, conf, tok);
-    return cudaGetLastError();
+                              void* scratch, cudaStream_t st) {
+    // enough blocks to fill the machine; a chunk is a multiple of 256 so that threads stay coalesced
+    int chunks = (4 * 148 + rows - 1) / rows;
+    if (chunks > kConfMaxChunks) chunks = kConfMaxChunks;
+    int chunk = ((V + chunks - 1) / chunks + 255) / 256 * 256;
+    chunks = (V + chunk - 1) / chunk;
+    ConfPartial* part = static_cast<ConfPartial*>(scratch);
+    cudaError_t e = launch_kernel(confidence_partial_kernel, dim3(rows, chunks), dim3(256), 0, st, logits, V, mask_id, chunk,
+                                  part);
+    if (e != cudaSuccess) return e;
+    return launch_kernel(confidence_final_kernel, dim3((rows + 127) / 128), dim3(128), 0, st,
+                         static_cast<const ConfPartial*>(part), chunks, rows, conf, tok);
 }
 
 }  // namespace odb

@@ -13,6 +13,8 @@
 // fp32 partials.  Splits are reduced later in a fixed order by the consumer kernel, so results
 // are run-to-run identical.  Every mbarrier wait is bounded: on expiry the CTA records
 // ODB_ERR_TIMEOUT, stops issuing work, releases its TMEM and exits.
+#include <stdlib.h>
+
 #include "odb_internal.cuh"
 
 namespace odb {
@@ -139,7 +141,8 @@ struct alignas(8) GemmShared {
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-            float* __restrict__ partial, int M, int N, int nkb_total, int nkb_per_split, int stages, int* status) {
+            float* __restrict__ partial, int M, int N, int nkb_total, int nkb_per_split, int stages, int l2_prefetch,
+            int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
     constexpr uint32_t kBBytes = BN * kBK * 2;
@@ -159,6 +162,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     if (nkb > nkb_per_split) nkb = nkb_per_split;
     volatile int* cta_abort = &sh->abort;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         for (int i = 0; i < stages; ++i) {
             mbar_init(&sh->full[i], 1);
@@ -174,6 +178,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
         asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_x)) : "memory");
     }
     if (warp == 1) {   // whole warp: allocate the accumulator's TMEM columns
+        __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
                      "r"(kTmemCols)
                      : "memory");
@@ -187,8 +192,29 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     if (warp == 0) {
         if (lane == 0) {
             // ---- TMA producer ----
-            int issued = 0;
-            for (int i = 0; i < nkb; ++i) {
+            // The weights do not depend on the preceding kernel: fill the ring with weight tiles
+            // first, then wait for the predecessor and fetch the activation tiles.
+            const int pre = nkb < stages ? nkb : stages;
+            for (int i = 0; i < pre; ++i) {
+                mbar_expect_tx(&sh->full[i], kStageBytes);
+                tma_load_2d(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], (kb0 + i) * kBK, n0,
+                            kEvictFirst);
+            }
+            // and ask L2 for the weight tiles that follow, so that HBM keeps streaming while the
+            // predecessor (a short elementwise kernel) is still running
+            int pf = nkb - pre;
+            if (pf > l2_prefetch) pf = l2_prefetch;
+            for (int i = pre; i < pre + pf; ++i)
+                asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(
+                                 reinterpret_cast<uint64_t>(&tmap_w)),
+                             "r"((kb0 + i) * kBK), "r"(n0)
+                             : "memory");
+            pdl_wait();
+            for (int i = 0; i < pre; ++i)
+                tma_load_2d(tiles + static_cast<size_t>(i) * kStageBytes + kABytes, &tmap_x, &sh->full[i], (kb0 + i) * kBK,
+                            m0, kEvictLast);
+            int issued = pre;
+            for (int i = pre; i < nkb; ++i) {
                 const int st = i % stages;
                 const uint32_t ph = static_cast<uint32_t>(i / stages) & 1u;
                 if (!mbar_wait(&sh->empty[st], ph ^ 1u, cta_abort, status)) break;
@@ -236,6 +262,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
         // ---- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 ----
         const int q = warp & 3;
         const int n = n0 + q * 32 + lane;
+        pdl_wait();   // the previous reader of `partial` has finished
         if (mbar_wait(&sh->acc_full, 0, cta_abort, status)) {
             tc_fence_after();
             float* out = partial + static_cast<size_t>(split) * M * N;
@@ -254,9 +281,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             }
         }
     }
+    pdl_wait();   // every thread: keeps completion of the launch chain transitive
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
+        __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
     }
@@ -323,20 +352,45 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
         attr_done = true;
     }
     dim3 grid((a.N + kBM - 1) / kBM, (a.M + BN - 1) / BN, a.splits);
-    gemm_kernel<BN><<<grid, kThreads, smem, st>>>(a.tmap_w, tmx, a.partial, a.M, a.N, nkb_total, nkb_per_split, stages,
-                                                  a.status);
-    return cudaGetLastError();
+    static int l2_prefetch = -1;
+    if (l2_prefetch < 0) {
+        const char* e = getenv("ODB_GEMM_L2_PREFETCH");
+        l2_prefetch = e ? atoi(e) : 0;   // measured: prefetching into L2 slows the step down
+    }
+    return launch_kernel(gemm_kernel<BN>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.M, a.N, nkb_total,
+                         nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
 }
 
 }  // namespace
 
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { return make_tmap_2d(out, w, N, K, kBM); }
 
+bool pdl_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = getenv("ODB_PDL");
+        v = (e && e[0] == '0') ? 0 : 1;
+    }
+    return v != 0;
+}
+
+static int target_ctas() {
+    static int v = 0;
+    if (!v) {
+        const char* e = getenv("ODB_GEMM_TARGET_CTAS");
+        v = e ? atoi(e) : 2 * 148;
+        if (v < 1) v = 2 * 148;
+    }
+    return v;
+}
+
 int gemm_pick_splits(int M, int N, int K) {
     const int bn = pick_bn(M);
     const int tiles = ((N + kBM - 1) / kBM) * ((M + bn - 1) / bn);
     const int nkb = (K + kBK - 1) / kBK;
-    int splits = (2 * 148 + tiles - 1) / tiles;
+    // all work units must be resident at once (two CTA slots per SM) and equal in size: a
+    // second, partly filled wave would double the kernel's time
+    int splits = target_ctas() / tiles;
     if (splits > nkb / 4) splits = nkb / 4;
     if (splits > 16) splits = 16;
     if (splits < 1) splits = 1;

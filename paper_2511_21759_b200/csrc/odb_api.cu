@@ -46,7 +46,7 @@ int32_t check_config(const odb_config* c) {
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
     size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf;
-    size_t h, a, q, k, v, o, g, partial, logits, conf, tok, part_o, part_ml;
+    size_t h, a, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
     size_t total;
 };
 
@@ -88,6 +88,7 @@ Layout make_layout(const odb_config& c) {
     L.logits = take(c.with_lm_head ? 4 * L.lm_chunk * c.vocab : 256);
     L.conf = take(4 * L.rows);
     L.tok = take(4 * L.rows);
+    L.conf_part = take(12 * L.lm_chunk * kConfMaxChunks);
     L.part_o = take(4 * L.attn_rows * d);
     L.part_ml = take(4 * L.attn_rows * c.n_heads * 2);
     L.total = off;
@@ -455,7 +456,8 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps, st));
         int sp = 1;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, logits, rows, c.vocab, d, &sp));
-        ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0, st));
+        ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0,
+                                                             s->ws + L.conf_part, st));
     }
     return ODB_OK;
 }
@@ -523,12 +525,12 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
 int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t after_refresh, odb_result* results) {
     if (!s || !p || !results) return ODB_ERR_ARG;
     const odb_config& c = s->m->cfg;
-    if (!c.with_lm_head) return ODB_ERR_STATE;
     if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
     if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != (after_refresh ? 1 : 3)) return ODB_ERR_STATE;
-    ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id, s->st));
+    ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id,
+                                           c.with_lm_head ? 0 : 1, s->st));
     ODB_CUDA(cudaMemcpyAsync(s->pinned_results, s->cb.results, sizeof(odb_result) * c.max_batch, cudaMemcpyDeviceToHost, s->st));
     int* dev_status = s->at<int>(s->L.status);
     ODB_CUDA(cudaMemcpyAsync(s->pinned_status, dev_status, sizeof(int), cudaMemcpyDeviceToHost, s->st));

@@ -8,7 +8,40 @@
 
 #include "../../include/odb.h"
 
+#include <utility>
+
 namespace odb {
+
+// ---------------------------------------------------------------------------------------
+// programmatic dependent launch: every kernel of a forward lets its successor start early
+// (launch_dependents at entry) and waits for its predecessor's results (wait) only where it
+// first needs them, so prologues, tensor-map fetches and weight prefetches overlap the
+// predecessor's tail.  Every such kernel executes pdl_wait() before it exits, which keeps the
+// completion order of the chain transitive.
+// ---------------------------------------------------------------------------------------
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
+bool pdl_enabled();   // ODB_PDL=0 in the environment turns the launch attribute off
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                          Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ---------------------------------------------------------------------------------------
 // session-wide device state
@@ -93,8 +126,10 @@ struct QkvRopeArgs {
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
 cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
                           cudaStream_t st);
+// scratch: rows * kConfMaxChunks * 12 bytes of per-chunk (max, sum, argmax) triples
+constexpr int kConfMaxChunks = 64;
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
-                              cudaStream_t st);
+                              void* scratch, cudaStream_t st);
 
 struct AttnArgs {
     const QTile* tiles; int n_tiles;
@@ -122,7 +157,8 @@ struct ControlBuffers {
 cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index, int block_len,
                                       cudaStream_t st);
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st);
+// dry: model without LM head; commits nothing, only lays out the next step
 cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
-                          int mask_id, int eos_id, cudaStream_t st);
+                          int mask_id, int eos_id, int dry, cudaStream_t st);
 
 }  // namespace odb
