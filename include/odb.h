@@ -86,17 +86,21 @@ typedef struct odb_config {
 } odb_config;
 
 /* Device pointers to the weights; per-layer arrays are HOST arrays of n_layers device pointers.
- * wqkv = [Wq; Wk; Wv] stacked on the output dimension, wgu = [Wgate; Wup] likewise. */
+ * wqkv = [Wq; Wk; Wv] stacked on the output dimension, wgu = [Wgate; Wup] likewise.
+ * Every projection matrix (wqkv, wo, wgu, wd, lm_head) is given in the library's PACKED layout,
+ * produced from the row-major [out][in] matrix by odb_pack_weight: tiles of 128 output rows x 64
+ * input columns, each tile 16 KB contiguous, tiles ordered [out_tile][in_block], zero padded to
+ * whole tiles.  The embedding table stays row-major. */
 typedef struct odb_weights {
     const void* embed;          /* bf16 [vocab][d_model] */
-    const void* lm_head;        /* bf16 [vocab][d_model], NULL iff with_lm_head == 0 */
+    const void* lm_head;        /* packed bf16 [vocab][d_model], NULL iff with_lm_head == 0 */
     const float* final_norm;    /* fp32 [d_model] */
     const float* const* norm1;  /* fp32 [d_model] per layer */
-    const void* const* wqkv;    /* bf16 [3*d_model][d_model] per layer */
-    const void* const* wo;      /* bf16 [d_model][d_model] per layer */
+    const void* const* wqkv;    /* packed bf16 [3*d_model][d_model] per layer */
+    const void* const* wo;      /* packed bf16 [d_model][d_model] per layer */
     const float* const* norm2;  /* fp32 [d_model] per layer */
-    const void* const* wgu;     /* bf16 [2*d_ffn][d_model] per layer */
-    const void* const* wd;      /* bf16 [d_model][d_ffn] per layer */
+    const void* const* wgu;     /* packed bf16 [2*d_ffn][d_model] per layer */
+    const void* const* wd;      /* packed bf16 [d_model][d_ffn] per layer */
 } odb_weights;
 
 typedef struct odb_decode_params {
@@ -128,6 +132,12 @@ typedef struct odb_session odb_session;
 const char* odb_status_string(int32_t status);
 /* Text of the last CUDA error seen by this thread's library calls ("" if none). */
 const char* odb_last_cuda_error(void);
+
+/* Bytes of the packed form of a row-major bf16 matrix [N][K] (K a multiple of 8); 0 if invalid. */
+size_t odb_packed_weight_bytes(int32_t N, int32_t K);
+/* dst (packed, odb_packed_weight_bytes(N, K) bytes, device) <- src (row-major bf16 [N][K], device).
+ * Both 16-byte aligned.  A pure permutation with zero padding; asynchronous on `stream`. */
+int32_t odb_pack_weight(const void* src, void* dst, int32_t N, int32_t K, void* stream);
 
 /* Validates the shape, builds TMA descriptors for the weight matrices.  The weight buffers must
  * stay valid and unchanged while the model lives.  *out is set only on ODB_OK. */
@@ -195,7 +205,7 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
  * *rows gets the row count of that buffer.  Synchronous. */
 int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap_bytes, int32_t* rows);
 
-/* out[M][N] (fp32, device) = x[M][K] (bf16, device) * w[N][K]^T (bf16, device) with the
+/* out[M][N] (fp32, device) = x[M][K] (bf16, device) * w[N][K]^T (PACKED bf16, device) with the
  * weight-streaming tcgen05 GEMM, K split k_splits ways and reduced in fixed order.  scratch:
  * device buffer of >= k_splits*M*N*4 + 512 bytes.  k_splits = 0 picks the library's heuristic.
  * Runs on `stream` and waits for it; returns ODB_ERR_TIMEOUT if a device-side wait expired. */

@@ -7,6 +7,11 @@
 // rows ride on the MMA's N dimension (32..256), so a 32-row decode step wastes no tensor-core
 // rows and every weight byte is fetched from HBM exactly once.
 //
+// Weights are stored PACKED: tile (n-tile of 128 rows, k-block of 64 columns) is one contiguous
+// 16 KB chunk, tiles of a row of tiles consecutive in k.  A CTA therefore reads one sequential
+// stream of whole DRAM pages; with the plain row-major layout each TMA box gathers 128 separate
+// 128-byte pieces 2K bytes apart and HBM delivers little more than half its bandwidth (measured).
+//
 // One CTA = one 128 x BN output tile over one K range.  Warp 0 lane 0 issues TMA loads into a
 // ring of shared-memory stages, warp 1 lane 0 issues the MMAs (accumulator in TMEM) and frees
 // stages through tcgen05.commit, warps 2..5 read the accumulator back (tcgen05.ld) and store
@@ -76,6 +81,15 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tmap, 
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
         " [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(smem_u32(dst)),
         "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "l"(hint)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* tmap, uint64_t* bar, int c0, int c1, int c2,
+                                            uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5}], [%2], %6;" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "l"(hint)
         : "memory");
 }
 
@@ -161,6 +175,8 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     int nkb = nkb_total - kb0;
     if (nkb > nkb_per_split) nkb = nkb_per_split;
     volatile int* cta_abort = &sh->abort;
+    // packed weights: tile (n-tile, k-block) is the contiguous 16 KB chunk number n_tile * nkb_total + k_block
+    const int wtile0 = blockIdx.x * nkb_total + kb0;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -197,7 +213,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             const int pre = nkb < stages ? nkb : stages;
             for (int i = 0; i < pre; ++i) {
                 mbar_expect_tx(&sh->full[i], kStageBytes);
-                tma_load_2d(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], (kb0 + i) * kBK, n0,
+                tma_load_3d(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], 0, 0, wtile0 + i,
                             kEvictFirst);
             }
             // and ask L2 for the weight tiles that follow, so that HBM keeps streaming while the
@@ -205,9 +221,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             int pf = nkb - pre;
             if (pf > l2_prefetch) pf = l2_prefetch;
             for (int i = pre; i < pre + pf; ++i)
-                asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(
+                asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];" ::"l"(
                                  reinterpret_cast<uint64_t>(&tmap_w)),
-                             "r"((kb0 + i) * kBK), "r"(n0)
+                             "r"(0), "r"(0), "r"(wtile0 + i)
                              : "memory");
             pdl_wait();
             for (int i = 0; i < pre; ++i)
@@ -221,7 +237,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 uint8_t* a_dst = tiles + static_cast<size_t>(st) * kStageBytes;
                 uint8_t* b_dst = a_dst + kABytes;
                 mbar_expect_tx(&sh->full[st], kStageBytes);
-                tma_load_2d(a_dst, &tmap_w, &sh->full[st], (kb0 + i) * kBK, n0, kEvictFirst);
+                tma_load_3d(a_dst, &tmap_w, &sh->full[st], 0, 0, wtile0 + i, kEvictFirst);
                 tma_load_2d(b_dst, &tmap_x, &sh->full[st], (kb0 + i) * kBK, m0, kEvictLast);
                 issued = i + 1;
             }
@@ -332,6 +348,38 @@ cudaError_t make_tmap_2d(CUtensorMap* out, const void* base, int rows, int K, in
     return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
 }
 
+// Packed weight [n_tiles * k_blocks][128][64] bf16: one tile = 16 KB contiguous, rows of 128 bytes.
+cudaError_t make_tmap_packed(CUtensorMap* out, const void* base, int N, int K) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return cudaErrorNotSupported;
+    const cuuint64_t ntiles = static_cast<cuuint64_t>((N + kBM - 1) / kBM) * ((K + kBK - 1) / kBK);
+    cuuint64_t dims[3] = {static_cast<cuuint64_t>(kBK), static_cast<cuuint64_t>(kBM), ntiles};
+    cuuint64_t strides[2] = {static_cast<cuuint64_t>(kBK) * 2, static_cast<cuuint64_t>(kBK) * kBM * 2};
+    cuuint32_t box[3] = {static_cast<cuuint32_t>(kBK), static_cast<cuuint32_t>(kBM), 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+// dst[((tn * KB + kb) * 128 + r) * 64 + c] = src[(tn * 128 + r) * K + kb * 64 + c], zero beyond N or K
+__global__ void pack_weight_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int N, int K,
+                                   int KB) {
+    const size_t chunk = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;   // 8 elements (16 bytes) each
+    const size_t total = static_cast<size_t>((N + kBM - 1) / kBM) * KB * kBM * (kBK / 8);
+    if (chunk >= total) return;
+    const int c8 = static_cast<int>(chunk % (kBK / 8));
+    const int r = static_cast<int>((chunk / (kBK / 8)) % kBM);
+    const size_t tile = chunk / (kBK / 8) / kBM;
+    const int kb = static_cast<int>(tile % KB);
+    const int tn = static_cast<int>(tile / KB);
+    const int n = tn * kBM + r, k = kb * kBK + c8 * 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (n < N && k < K) v = *reinterpret_cast<const uint4*>(src + static_cast<size_t>(n) * K + k);   // K % 8 == 0
+    reinterpret_cast<uint4*>(dst)[chunk] = v;
+}
+
 int pick_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
 
 template <int BN>
@@ -363,7 +411,19 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
 
 }  // namespace
 
-cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { return make_tmap_2d(out, w, N, K, kBM); }
+cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { return make_tmap_packed(out, w, N, K); }
+
+size_t packed_weight_bytes(int N, int K) {
+    return static_cast<size_t>((N + kBM - 1) / kBM) * ((K + kBK - 1) / kBK) * kBM * kBK * 2;
+}
+
+cudaError_t launch_pack_weight(const void* src, void* dst, int N, int K, cudaStream_t st) {
+    const int KB = (K + kBK - 1) / kBK;
+    const size_t chunks = packed_weight_bytes(N, K) / 16;
+    pack_weight_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(dst), N, K, KB);
+    return cudaGetLastError();
+}
 
 bool pdl_enabled() {
     static int v = -1;

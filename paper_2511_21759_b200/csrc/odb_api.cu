@@ -146,6 +146,19 @@ const char* odb_status_string(int32_t s) {
 
 const char* odb_last_cuda_error(void) { return g_cuda_error.c_str(); }
 
+size_t odb_packed_weight_bytes(int32_t N, int32_t K) {
+    if (N < 1 || K < 8 || K % 8) return 0;
+    return packed_weight_bytes(N, K);
+}
+
+int32_t odb_pack_weight(const void* src, void* dst, int32_t N, int32_t K, void* stream) {
+    if (!src || !dst) return ODB_ERR_ARG;
+    if (N < 1 || K < 8 || K % 8) return ODB_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) return ODB_ERR_ARG;
+    ODB_CUDA(launch_pack_weight(src, dst, N, K, static_cast<cudaStream_t>(stream)));
+    return ODB_OK;
+}
+
 int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model** out) {
     int32_t rc = check_config(cfg);
     if (rc != ODB_OK) return rc;

@@ -96,7 +96,7 @@ struct TmaEncoder;   // wraps the driver's tensor-map encode entry point
 
 // Weight-streaming GEMM: partial[s][M][N] (fp32) = x[M][K_s] * w[N][K_s]^T for each K split s.
 struct GemmArgs {
-    CUtensorMap tmap_w;    // bf16 [N][K], box 64 x 128, 128B swizzle
+    CUtensorMap tmap_w;    // packed bf16 weight tiles [n_tile * k_blocks][128][64], 128B swizzle
     const void* x;         // bf16 [M][K] device
     float* partial;        // fp32 [splits][M][N]
     int M, N, K;
@@ -104,7 +104,9 @@ struct GemmArgs {
     int* status;           // device status word
 };
 int gemm_pick_splits(int M, int N, int K);
-cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K);
+cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
+size_t packed_weight_bytes(int N, int K);
+cudaError_t launch_pack_weight(const void* src_row_major, void* dst_packed, int N, int K, cudaStream_t st);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,
                                    cudaStream_t st);

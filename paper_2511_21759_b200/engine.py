@@ -26,6 +26,16 @@ def bits_to_device(bits: np.ndarray, device) -> torch.Tensor:
     return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).to(device).view(torch.bfloat16)
 
 
+def pack_weight(w: torch.Tensor) -> torch.Tensor:
+    """Row-major bf16 [N][K] on the device -> the library's packed tile layout (odb_pack_weight)."""
+    N, K = w.shape
+    w = w.contiguous()
+    out = torch.empty(B.lib().odb_packed_weight_bytes(N, K) // 2, dtype=torch.bfloat16, device=w.device)
+    st = torch.cuda.current_stream(w.device)
+    B.check(B.lib().odb_pack_weight(w.data_ptr(), out.data_ptr(), N, K, C.c_void_p(st.cuda_stream)), "odb_pack_weight")
+    return out
+
+
 @dataclasses.dataclass
 class DecodeParams:
     block_len: int
@@ -62,22 +72,24 @@ class Model:
         B.check(B.lib().odb_model_create(C.byref(self.cfg), C.byref(w), C.byref(self.handle)), "odb_model_create")
 
     @classmethod
-    def from_synth(cls, shape, seed=0, device="cuda", *, with_lm_head=True, **kw) -> "Model":
-        """Uploads the seeded synthetic weights of `shape` (data marshalling only)."""
+    def from_synth(cls, shape, seed=0, device="cuda", *, with_lm_head=True, lm_head_bits=None, **kw) -> "Model":
+        """Uploads the seeded synthetic weights of `shape` (data marshalling only).  lm_head_bits
+        (bf16 bit patterns [V][d]) replaces the generated LM head when given."""
         import synth
         d = shape.d_model
         ones = lambda: torch.ones(d, dtype=torch.float32, device=device)
         t = {"embed": bits_to_device(synth.embed_bits(shape, seed), device),
-             "lm_head": bits_to_device(synth.lm_head_bits(shape, seed), device) if with_lm_head else None,
+             "lm_head": pack_weight(bits_to_device(lm_head_bits if lm_head_bits is not None
+                                                   else synth.lm_head_bits(shape, seed), device)) if with_lm_head else None,
              "final_norm": ones(), "norm1": [], "wqkv": [], "wo": [], "norm2": [], "wgu": [], "wd": []}
         for l in range(shape.n_layers):
             w = synth.layer_bits(shape, l, seed)
             t["norm1"].append(ones())
             t["norm2"].append(ones())
-            t["wqkv"].append(bits_to_device(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0), device))
-            t["wo"].append(bits_to_device(w["wo"], device))
-            t["wgu"].append(bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device))
-            t["wd"].append(bits_to_device(w["wd"], device))
+            t["wqkv"].append(pack_weight(bits_to_device(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0), device)))
+            t["wo"].append(pack_weight(bits_to_device(w["wo"], device)))
+            t["wgu"].append(pack_weight(bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device)))
+            t["wd"].append(pack_weight(bits_to_device(w["wd"], device)))
         return cls(shape, t, with_lm_head=with_lm_head, **kw)
 
     def close(self):
@@ -179,9 +191,11 @@ class Session:
 
 
 def debug_gemm(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Tensor:
-    """out[M][N] fp32 = x[M][K] @ w[N][K]^T through the library's tcgen05 GEMM."""
+    """out[M][N] fp32 = x[M][K] @ w[N][K]^T through the library's tcgen05 GEMM (w row-major here; it is
+    packed with odb_pack_weight first)."""
     M, K = x.shape
     N = w.shape[0]
+    w = pack_weight(w)
     out = torch.empty(M, N, dtype=torch.float32, device=x.device)
     scratch = torch.empty(max(k_splits, 16) * M * N * 4 + 1024, dtype=torch.uint8, device=x.device)
     st = torch.cuda.current_stream(x.device)

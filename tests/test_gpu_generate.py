@@ -19,15 +19,13 @@ from gpu_common import engine, requires_gpu, compare_traces, lockstep_generate, 
 NEAR_TIE = 1e-3
 
 
-def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=None, om=None, tensors_patch=None):
+def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=None, om=None, lm_head_bits=None):
     E = engine()
     wl = synth.WORKLOADS[wl_name]
     shape = shape or wl.shape
     om = om or model_from_synth(shape, seed=seed)
     gm = E.Model.from_synth(shape, seed=seed, max_batch=1, max_seq=wl.prompt_len + wl.gen_len,
-                            max_block=wl.block_len, max_copies=8)
-    if tensors_patch:
-        tensors_patch(gm)
+                            max_block=wl.block_len, max_copies=8, lm_head_bits=lm_head_bits)
     sess = E.Session(gm)
     x0 = x0 if x0 is not None else synth.sequence(seed, 0, wl.prompt_len, wl.gen_len, shape)
     sess.set_sequence(0, x0, wl.prompt_len)
@@ -107,13 +105,12 @@ def test_generate_alp_truncates():
     lm = om.lm_head.copy()
     lm[shape.eos_id] = row
     om = dataclasses.replace(om, lm_head=lm)
-    import torch
-    def patch(gm):
-        gm.t["lm_head"][shape.eos_id] = torch.from_numpy(row.astype(np.float32)).to("cuda").to(torch.bfloat16)
+    bits = synth.lm_head_bits(shape, 5)
+    bits[shape.eos_id] = (row.astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)   # row is bf16-exact
     wl = dataclasses.replace(synth.WORKLOADS["peaky_c1"], prompt_len=32, gen_len=64)
     synth.WORKLOADS["_alp"] = wl
     try:
-        gtok, gtrace, otok, otrace = _run_both("_alp", seed=5, shape=shape, x0=x0, om=om, tensors_patch=patch,
+        gtok, gtrace, otok, otrace = _run_both("_alp", seed=5, shape=shape, x0=x0, om=om, lm_head_bits=bits,
                                                params_kw=dict(truncate_threshold=0.0))
     finally:
         del synth.WORKLOADS["_alp"]
