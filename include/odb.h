@@ -90,7 +90,9 @@ typedef struct odb_config {
  * Every projection matrix (wqkv, wo, wgu, wd, lm_head) is given in the library's PACKED layout,
  * produced from the row-major [out][in] matrix by odb_pack_weight: tiles of 128 output rows x 64
  * input columns, each tile 16 KB contiguous, tiles ordered [out_tile][in_block], zero padded to
- * whole tiles.  The embedding table stays row-major. */
+ * whole tiles.  wgu uses the gate/up variant (odb_pack_gate_up): tile t holds gate rows
+ * [64t, 64t+64) followed by up rows [64t, 64t+64), so that the GEMM epilogue can form
+ * silu(gate) * up inside one tile.  The embedding table stays row-major. */
 typedef struct odb_weights {
     const void* embed;          /* bf16 [vocab][d_model] */
     const void* lm_head;        /* packed bf16 [vocab][d_model], NULL iff with_lm_head == 0 */
@@ -99,7 +101,7 @@ typedef struct odb_weights {
     const void* const* wqkv;    /* packed bf16 [3*d_model][d_model] per layer */
     const void* const* wo;      /* packed bf16 [d_model][d_model] per layer */
     const float* const* norm2;  /* fp32 [d_model] per layer */
-    const void* const* wgu;     /* packed bf16 [2*d_ffn][d_model] per layer */
+    const void* const* wgu;     /* gate/up-packed bf16 [2*d_ffn][d_model] per layer */
     const void* const* wd;      /* packed bf16 [d_model][d_ffn] per layer */
 } odb_weights;
 
@@ -138,6 +140,10 @@ size_t odb_packed_weight_bytes(int32_t N, int32_t K);
 /* dst (packed, odb_packed_weight_bytes(N, K) bytes, device) <- src (row-major bf16 [N][K], device).
  * Both 16-byte aligned.  A pure permutation with zero padding; asynchronous on `stream`. */
 int32_t odb_pack_weight(const void* src, void* dst, int32_t N, int32_t K, void* stream);
+
+/* Gate/up variant: src is row-major bf16 [2F][K], gate rows first then up rows. */
+size_t odb_packed_gate_up_bytes(int32_t F, int32_t K);
+int32_t odb_pack_gate_up(const void* src, void* dst, int32_t F, int32_t K, void* stream);
 
 /* Validates the shape, builds TMA descriptors for the weight matrices.  The weight buffers must
  * stay valid and unchanged while the model lives.  *out is set only on ODB_OK. */

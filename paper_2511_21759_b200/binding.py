@@ -57,6 +57,8 @@ SIGNATURES = {
     "odb_last_cuda_error": (C.c_char_p, []),
     "odb_packed_weight_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
     "odb_pack_weight": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
+    "odb_packed_gate_up_bytes": (C.c_size_t, [C.c_int32, C.c_int32]),
+    "odb_pack_gate_up": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p]),
     "odb_model_create": (C.c_int32, [C.POINTER(odb_config), C.POINTER(odb_weights), C.POINTER(C.c_void_p)]),
     "odb_model_destroy": (C.c_int32, [C.c_void_p]),
     "odb_kv_bytes": (C.c_size_t, [C.POINTER(odb_config)]),

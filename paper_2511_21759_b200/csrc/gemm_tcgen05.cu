@@ -152,11 +152,15 @@ struct alignas(8) GemmShared {
 };
 
 // BN: activation rows per tile (MMA N): 32, 64, 128 or 256.
-template <int BN>
+// SWIGLU: the weight is the gate/up matrix packed with gate and up rows interleaved in groups of
+// 64 (tile t = gate rows [64t, 64t+64) then up rows [64t, 64t+64)); the epilogue pairs TMEM lane r
+// (gate) with lane r + 64 (up) through shared memory and stores bf16(silu(gate) * up) to
+// g[m][64 t + r]; N is then the FFN width F and there is no K split.
+template <int BN, bool SWIGLU>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-            float* __restrict__ partial, int M, int N, int nkb_total, int nkb_per_split, int stages, int l2_prefetch,
-            int* status) {
+            float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, int M, int N, int nkb_total,
+            int nkb_per_split, int stages, int l2_prefetch, int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
     constexpr uint32_t kBBytes = BN * kBK * 2;
@@ -277,23 +281,54 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     } else {
         // ---- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 ----
         const int q = warp & 3;
-        const int n = n0 + q * 32 + lane;
-        pdl_wait();   // the previous reader of `partial` has finished
-        if (mbar_wait(&sh->acc_full, 0, cta_abort, status)) {
-            tc_fence_after();
-            float* out = partial + static_cast<size_t>(split) * M * N;
+        pdl_wait();   // the previous reader of the output buffer has finished
+        const bool ok = mbar_wait(&sh->acc_full, 0, cta_abort, status);
+        if (ok) tc_fence_after();
+        if constexpr (!SWIGLU) {
+            const int n = n0 + q * 32 + lane;
+            if (ok) {
+                float* out = partial + static_cast<size_t>(split) * M * N;
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (n < N) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + c * 32 + j;
+                            if (m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
+                        }
+                    }
+                }
+            }
+        } else {
+            // all MMAs have completed, so the stage ring is free: use it to hand the up values over.
+            // Every epilogue warp executes every barrier, whether or not its wait succeeded.
+            float* xch = reinterpret_cast<float*>(tiles);           // [64][33]
+            const int f = blockIdx.x * 64 + (q & 1) * 32 + lane;       // FFN feature of this lane's pair
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
-                tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
-                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (n < N) {
+                if (ok) {
+                    tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                }
+                if (ok && q >= 2) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) xch[((q & 1) * 32 + lane) * 33 + j] = __uint_as_float(v[j]);
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (ok && q < 2 && f < N) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + c * 32 + j;
-                        if (m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
+                        const float gate = __uint_as_float(v[j]);
+                        const float up = xch[((q & 1) * 32 + lane) * 33 + j];
+                        if (m < M) act_out[static_cast<size_t>(m) * N + f] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
                     }
                 }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
             }
         }
     }
@@ -380,9 +415,27 @@ __global__ void pack_weight_kernel(const __nv_bfloat16* __restrict__ src, __nv_b
     reinterpret_cast<uint4*>(dst)[chunk] = v;
 }
 
+// Gate/up variant: src is [2F][K] = gate rows then up rows; packed tile t holds gate rows
+// [64t, 64t+64) in its rows 0..63 and up rows [64t, 64t+64) in its rows 64..127.
+__global__ void pack_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __nv_bfloat16* __restrict__ dst, int F, int K,
+                                    int KB) {
+    const size_t chunk = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const size_t total = static_cast<size_t>((F + 63) / 64) * KB * kBM * (kBK / 8);
+    if (chunk >= total) return;
+    const int c8 = static_cast<int>(chunk % (kBK / 8));
+    const int r = static_cast<int>((chunk / (kBK / 8)) % kBM);
+    const size_t tile = chunk / (kBK / 8) / kBM;
+    const int kb = static_cast<int>(tile % KB);
+    const int t = static_cast<int>(tile / KB);
+    const int f = t * 64 + (r & 63), k = kb * kBK + c8 * 8;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (f < F && k < K) v = *reinterpret_cast<const uint4*>(src + (static_cast<size_t>(r < 64 ? 0 : F) + f) * K + k);
+    reinterpret_cast<uint4*>(dst)[chunk] = v;
+}
+
 int pick_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
 
-template <int BN>
+template <int BN, bool SWIGLU>
 cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st) {
     const int nkb_total = (a.K + kBK - 1) / kBK;
     const int nkb_per_split = (nkb_total + a.splits - 1) / a.splits;
@@ -395,18 +448,19 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
     const size_t smem = static_cast<size_t>(stages) * stage_bytes + sizeof(GemmShared) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN, SWIGLU>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    dim3 grid((a.N + kBM - 1) / kBM, (a.M + BN - 1) / BN, a.splits);
+    // SWIGLU: N is the FFN width and a weight tile holds 64 gate + 64 up rows
+    dim3 grid(SWIGLU ? (a.N + 63) / 64 : (a.N + kBM - 1) / kBM, (a.M + BN - 1) / BN, a.splits);
     static int l2_prefetch = -1;
     if (l2_prefetch < 0) {
         const char* e = getenv("ODB_GEMM_L2_PREFETCH");
         l2_prefetch = e ? atoi(e) : 0;   // measured: prefetching into L2 slows the step down
     }
-    return launch_kernel(gemm_kernel<BN>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.M, a.N, nkb_total,
-                         nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
+    return launch_kernel(gemm_kernel<BN, SWIGLU>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out, a.M,
+                         a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
 }
 
 }  // namespace
@@ -415,6 +469,22 @@ cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { re
 
 size_t packed_weight_bytes(int N, int K) {
     return static_cast<size_t>((N + kBM - 1) / kBM) * ((K + kBK - 1) / kBK) * kBM * kBK * 2;
+}
+
+size_t packed_gate_up_bytes(int F, int K) {
+    return static_cast<size_t>((F + 63) / 64) * ((K + kBK - 1) / kBK) * kBM * kBK * 2;
+}
+
+cudaError_t make_gate_up_tmap(CUtensorMap* out, const void* w, int F, int K) {
+    return make_tmap_packed(out, w, ((F + 63) / 64) * kBM, K);
+}
+
+cudaError_t launch_pack_gate_up(const void* src, void* dst, int F, int K, cudaStream_t st) {
+    const int KB = (K + kBK - 1) / kBK;
+    const size_t chunks = packed_gate_up_bytes(F, K) / 16;
+    pack_gate_up_kernel<<<static_cast<unsigned>((chunks + 255) / 256), 256, 0, st>>>(
+        static_cast<const __nv_bfloat16*>(src), static_cast<__nv_bfloat16*>(dst), F, K, KB);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_pack_weight(const void* src, void* dst, int N, int K, cudaStream_t st) {
@@ -464,11 +534,20 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
     CUtensorMap tmx;
     cudaError_t e = make_tmap_2d(&tmx, a.x, a.M, a.K, bn);
     if (e != cudaSuccess) return e;
+    if (a.act_out) {
+        if (a.splits != 1) return cudaErrorInvalidValue;
+        switch (bn) {
+            case 32: return launch_bn<32, true>(a, tmx, st);
+            case 64: return launch_bn<64, true>(a, tmx, st);
+            case 128: return launch_bn<128, true>(a, tmx, st);
+            default: return launch_bn<256, true>(a, tmx, st);
+        }
+    }
     switch (bn) {
-        case 32: return launch_bn<32>(a, tmx, st);
-        case 64: return launch_bn<64>(a, tmx, st);
-        case 128: return launch_bn<128>(a, tmx, st);
-        default: return launch_bn<256>(a, tmx, st);
+        case 32: return launch_bn<32, false>(a, tmx, st);
+        case 64: return launch_bn<64, false>(a, tmx, st);
+        case 128: return launch_bn<128, false>(a, tmx, st);
+        default: return launch_bn<256, false>(a, tmx, st);
     }
 }
 

@@ -159,6 +159,19 @@ int32_t odb_pack_weight(const void* src, void* dst, int32_t N, int32_t K, void* 
     return ODB_OK;
 }
 
+size_t odb_packed_gate_up_bytes(int32_t F, int32_t K) {
+    if (F < 1 || K < 8 || K % 8) return 0;
+    return packed_gate_up_bytes(F, K);
+}
+
+int32_t odb_pack_gate_up(const void* src, void* dst, int32_t F, int32_t K, void* stream) {
+    if (!src || !dst) return ODB_ERR_ARG;
+    if (F < 1 || K < 8 || K % 8) return ODB_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst)) & 15) return ODB_ERR_ARG;
+    ODB_CUDA(launch_pack_gate_up(src, dst, F, K, static_cast<cudaStream_t>(stream)));
+    return ODB_OK;
+}
+
 int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model** out) {
     int32_t rc = check_config(cfg);
     if (rc != ODB_OK) return rc;
@@ -182,7 +195,7 @@ int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model*
         m->norm2.push_back(w->norm2[l]);
         e = make_weight_tmap(&m->tm_qkv[l], w->wqkv[l], 3 * d, d);
         if (e == cudaSuccess) e = make_weight_tmap(&m->tm_o[l], w->wo[l], d, d);
-        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_gu[l], w->wgu[l], 2 * F, d);
+        if (e == cudaSuccess) e = make_gate_up_tmap(&m->tm_gu[l], w->wgu[l], F, d);
         if (e == cudaSuccess) e = make_weight_tmap(&m->tm_d[l], w->wd[l], d, F);
     }
     if (e == cudaSuccess && cfg->with_lm_head) e = make_weight_tmap(&m->tm_lm, w->lm_head, cfg->vocab, d);
@@ -406,6 +419,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         ga.tmap_w = tw;
         ga.x = x;
         ga.partial = out;
+        ga.act_out = nullptr;
         ga.M = rows; ga.N = N; ga.K = K;
         int sp = *splits > 0 ? *splits : gemm_pick_splits(rows, N, K);
         const size_t cap = L.partial_rows * nmax / (static_cast<size_t>(rows) * N);
@@ -451,9 +465,17 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps, st));
-        sp = 0;
-        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_gu[l], a, partial, M, 2 * F, d, &sp));
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_swiglu(partial, sp, static_cast<size_t>(M) * 2 * F, g, M, F, st));
+        {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
+            GemmArgs ga;
+            ga.tmap_w = m->tm_gu[l];
+            ga.x = a;
+            ga.partial = nullptr;
+            ga.act_out = g;
+            ga.M = M; ga.N = F; ga.K = d;
+            ga.splits = 1;
+            ga.status = status;
+            ODB_LAUNCH(ODB_KIND_GEMM, launch_gemm(ga, st));
+        }
         sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, &sp));
         res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
@@ -602,6 +624,7 @@ int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, 
     GemmArgs ga;
     ODB_CUDA(make_weight_tmap(&ga.tmap_w, w, N, K));
     ga.x = x;
+    ga.act_out = nullptr;
     ga.partial = static_cast<float*>(scratch);
     ga.M = M; ga.N = N; ga.K = K;
     ga.splits = splits;

@@ -99,6 +99,7 @@ struct GemmArgs {
     CUtensorMap tmap_w;    // packed bf16 weight tiles [n_tile * k_blocks][128][64], 128B swizzle
     const void* x;         // bf16 [M][K] device
     float* partial;        // fp32 [splits][M][N]
+    __nv_bfloat16* act_out; // non-null: gate/up GEMM with the SwiGLU epilogue, writes bf16 [M][N = F]; splits == 1
     int M, N, K;
     int splits;
     int* status;           // device status word
@@ -106,6 +107,9 @@ struct GemmArgs {
 int gemm_pick_splits(int M, int N, int K);
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
 size_t packed_weight_bytes(int N, int K);
+size_t packed_gate_up_bytes(int F, int K);
+cudaError_t make_gate_up_tmap(CUtensorMap* out, const void* w_packed, int F, int K);
+cudaError_t launch_pack_gate_up(const void* src_gate_then_up, void* dst_packed, int F, int K, cudaStream_t st);
 cudaError_t launch_pack_weight(const void* src_row_major, void* dst_packed, int N, int K, cudaStream_t st);
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,

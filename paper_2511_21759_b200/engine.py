@@ -36,6 +36,17 @@ def pack_weight(w: torch.Tensor) -> torch.Tensor:
     return out
 
 
+def pack_gate_up(w: torch.Tensor) -> torch.Tensor:
+    """Row-major bf16 [2F][K] (gate rows, then up rows) -> the gate/up packed layout (odb_pack_gate_up)."""
+    F2, K = w.shape
+    w = w.contiguous()
+    out = torch.empty(B.lib().odb_packed_gate_up_bytes(F2 // 2, K) // 2, dtype=torch.bfloat16, device=w.device)
+    st = torch.cuda.current_stream(w.device)
+    B.check(B.lib().odb_pack_gate_up(w.data_ptr(), out.data_ptr(), F2 // 2, K, C.c_void_p(st.cuda_stream)),
+            "odb_pack_gate_up")
+    return out
+
+
 @dataclasses.dataclass
 class DecodeParams:
     block_len: int
@@ -88,7 +99,7 @@ class Model:
             t["norm2"].append(ones())
             t["wqkv"].append(pack_weight(bits_to_device(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0), device)))
             t["wo"].append(pack_weight(bits_to_device(w["wo"], device)))
-            t["wgu"].append(pack_weight(bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device)))
+            t["wgu"].append(pack_gate_up(bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device)))
             t["wd"].append(pack_weight(bits_to_device(w["wd"], device)))
         return cls(shape, t, with_lm_head=with_lm_head, **kw)
 
