@@ -72,6 +72,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
 
     pdl_launch_dependents();
     pdl_wait();
+    l2_prefetch_slice(a.pf, (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x * gridDim.y * gridDim.z);
     const QTile t = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
     const int z = blockIdx.z;

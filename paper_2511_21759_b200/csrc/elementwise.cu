@@ -44,10 +44,12 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
 __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
                                                        int splits, size_t pstride, const float* __restrict__ gain,
                                                        __nv_bfloat16* __restrict__ out,
-                                                       const int32_t* __restrict__ row_map, int d, float eps) {
+                                                       const int32_t* __restrict__ row_map, int d, float eps,
+                                                       L2Prefetch pf) {
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
+    l2_prefetch_slice(pf, blockIdx.x, gridDim.x);
     const int orow = blockIdx.x;
     const int row = row_map ? row_map[orow] : orow;
     float* hr = h + static_cast<size_t>(row) * d;
@@ -90,6 +92,7 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, co
 __global__ void qkv_rope_kernel(QkvRopeArgs a) {
     pdl_launch_dependents();
     pdl_wait();
+    l2_prefetch_slice(a.pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
     const int row = blockIdx.x;
     const int d = a.H * a.hd, half = a.hd / 2;
     const int pos = a.row_pos[row];
@@ -231,12 +234,12 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 }
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps,
+                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps, L2Prefetch pf,
                            cudaStream_t st) {
     int threads = ((d / 4 + 31) / 32) * 32;
     if (threads > 1024) threads = 1024;
     return launch_kernel(rmsnorm_kernel, dim3(rows_out), dim3(threads), 0, st, h, partial, splits, pstride, gain, out, row_map,
-                         d, eps);
+                         d, eps, pf);
 }
 
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {

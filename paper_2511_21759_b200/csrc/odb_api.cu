@@ -1,6 +1,7 @@
 // C ABI of the library: handles, argument validation, workspace carve-up and the host-side
 // orchestration of one forward (refresh prefill or block decode step) over the kernels.
 #include <math.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <new>
@@ -104,6 +105,8 @@ struct odb_model {
     std::vector<const float*> norm1, norm2;
     std::vector<CUtensorMap> tm_qkv, tm_o, tm_gu, tm_d;
     CUtensorMap tm_lm;
+    std::vector<const void*> p_qkv, p_o, p_gu;   // packed weight buffers (for L2 prefetch hints)
+    const void* p_lm;
 };
 
 struct odb_session {
@@ -183,6 +186,7 @@ int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model*
     m->cfg = *cfg;
     m->embed = static_cast<const __nv_bfloat16*>(w->embed);
     m->final_norm = w->final_norm;
+    m->p_lm = w->lm_head;
     const int d = cfg->d_model, F = cfg->d_ffn, nl = cfg->n_layers;
     m->tm_qkv.resize(nl); m->tm_o.resize(nl); m->tm_gu.resize(nl); m->tm_d.resize(nl);
     cudaError_t e = cudaSuccess;
@@ -193,6 +197,9 @@ int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model*
         }
         m->norm1.push_back(w->norm1[l]);
         m->norm2.push_back(w->norm2[l]);
+        m->p_qkv.push_back(w->wqkv[l]);
+        m->p_o.push_back(w->wo[l]);
+        m->p_gu.push_back(w->wgu[l]);
         e = make_weight_tmap(&m->tm_qkv[l], w->wqkv[l], 3 * d, d);
         if (e == cudaSuccess) e = make_weight_tmap(&m->tm_o[l], w->wo[l], d, d);
         if (e == cudaSuccess) e = make_gate_up_tmap(&m->tm_gu[l], w->wgu[l], F, d);
@@ -443,8 +450,24 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
     if (ks > 8) ks = 8;
     if (static_cast<size_t>(ks) * M > L.attn_rows) ks = static_cast<int>(L.attn_rows / M);
     if (ks < 1) ks = 1;
+    // L2 prefetch hints (decode steps only): while a short kernel runs between two GEMMs, HBM is
+    // idle; the kernel asks L2 for the head of the next GEMM's weights.  Sizes in bytes.
+    static const long long pf_mb = getenv("ODB_L2_PREFETCH_MB") ? atoll(getenv("ODB_L2_PREFETCH_MB")) : 8;   // measured: 8 MB helps, 24 MB and more lengthen the hinting kernel
+    const bool hint = !write_cache && pdl_enabled() && pf_mb > 0;
+    const unsigned long long pf_bytes = static_cast<unsigned long long>(pf_mb) << 20;
+    auto hint_of = [&](const void* base, size_t total, size_t offset) {
+        L2Prefetch pf{nullptr, 0};
+        if (hint && offset < total) {
+            pf.ptr = static_cast<const char*>(base) + offset;
+            pf.bytes = total - offset < pf_bytes ? total - offset : pf_bytes;
+        }
+        return pf;
+    };
+    const size_t qkv_bytes = packed_weight_bytes(3 * d, d), o_bytes = packed_weight_bytes(d, d),
+                 gu_bytes = packed_gate_up_bytes(F, d);
     for (int l = 0; l < c.n_layers; ++l) {
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, nullptr, M, d, c.rms_eps,
+                                                        hint_of(m->p_qkv[l], qkv_bytes, 0), st));
         int sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
         QkvRopeArgs qa;
@@ -454,17 +477,20 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         qa.q = q; qa.k = k; qa.v = v;
         qa.cache = write_cache ? s->kv : nullptr;
         qa.layer = l; qa.n_layers = c.n_layers; qa.H = H; qa.hd = hd; qa.max_seq = c.max_seq; qa.M = M;
+        qa.pf = hint_of(m->p_o[l], o_bytes, 0);
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_qkv_rope(qa, st));
         AttnArgs aa;
         aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
         aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
         aa.part_o = s->at<float>(L.part_o); aa.part_ml = s->at<float>(L.part_ml);
         aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = ks;
+        aa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
         ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention(aa, st));
         if (ks > 1) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
         sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, nullptr, M, d, c.rms_eps,
+                                                        hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
         {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
             GemmArgs ga;
             ga.tmap_w = m->tm_gu[l];
@@ -482,13 +508,15 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
     }
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, nullptr, M, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, nullptr, M, d, c.rms_eps,
+                                                        L2Prefetch{nullptr, 0}, st));
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
     for (int r0 = 0; r0 < n_lm; r0 += static_cast<int>(L.lm_chunk)) {
         const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, s->cb.lm_rows + r0, rows, d, c.rms_eps,
+                                                        hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
         int sp = 1;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, logits, rows, c.vocab, d, &sp));
         ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0,

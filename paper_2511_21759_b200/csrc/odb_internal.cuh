@@ -27,6 +27,29 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 
 bool pdl_enabled();   // ODB_PDL=0 in the environment turns the launch attribute off
 
+// A byte range of the NEXT GEMM's packed weights that a short kernel asks L2 to fetch while it
+// runs: HBM would otherwise sit idle between two weight-streaming GEMMs.  Fire and forget.
+struct L2Prefetch {
+    const void* ptr;
+    unsigned long long bytes;
+};
+
+#ifdef __CUDACC__
+// Block `cta` of `n_ctas` requests its share of the range in 32 KB bulk prefetches (thread 0).
+__device__ __forceinline__ void l2_prefetch_slice(const L2Prefetch& pf, int cta, int n_ctas) {
+    if (pf.bytes == 0 || threadIdx.x != 0) return;
+    constexpr unsigned long long kChunk = 32768;
+    const unsigned long long n_chunks = (pf.bytes + kChunk - 1) / kChunk;
+    for (unsigned long long c = cta; c < n_chunks; c += n_ctas) {
+        const unsigned long long off = c * kChunk;
+        const unsigned sz = static_cast<unsigned>((pf.bytes - off < kChunk ? pf.bytes - off : kChunk) & ~15ull);
+        if (sz)
+            asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(static_cast<const char*>(pf.ptr) + off), "r"(sz)
+                         : "memory");
+    }
+}
+#endif
+
 template <typename... KArgs, typename... Args>
 cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                           Args&&... args) {
@@ -119,7 +142,7 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
                          cudaStream_t st);
 // h[row] += sum_s partial[s][row] (if partial), out[i] = bf16(rmsnorm(h[map ? map[i] : i]) * gain)
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps,
+                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps, L2Prefetch pf,
                            cudaStream_t st);
 struct QkvRopeArgs {
     const float* partial; int splits; size_t pstride;      // [splits][M][3d]
@@ -128,6 +151,7 @@ struct QkvRopeArgs {
     __nv_bfloat16 *q, *k, *v;                              // [M][d]
     __nv_bfloat16* cache;                                  // NULL: do not write the cache
     int layer, n_layers, H, hd, max_seq, M;
+    L2Prefetch pf;
 };
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
 cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
@@ -145,6 +169,7 @@ struct AttnArgs {
     __nv_bfloat16* o;                     // [M][H*hd]
     float* part_o; float* part_ml;        // split workspaces [ks][M][H][hd], [ks][M][H][2]
     int layer, n_layers, H, hd, max_seq, M, ksplit;
+    L2Prefetch pf;
 };
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
 
