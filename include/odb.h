@@ -218,6 +218,32 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap_byt
 int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, size_t scratch_bytes,
                        int32_t M, int32_t N, int32_t K, int32_t k_splits, void* stream);
 
+/* The same GEMM as odb_debug_gemm, for callers that may not allocate device memory.  (The paper
+ * has no counterpart to this call; it exists for integration only.)
+ *
+ * Who needs it: code that runs after the process has handed every remaining byte of device memory
+ * to a pool of its own (a serving engine that sized its K/V cache to fill the GPU), a plug-in inside
+ * a host application that owns the device allocator, or a latency-critical path that cannot accept
+ * the implicit device synchronisation and the late failure modes of cudaMalloc.  Such a caller still
+ * passes x, w_packed and out, but has no buffer to lend for the split-K partial sums, so this entry
+ * point keeps them in a fixed array that is part of the library's device image:
+ * ODB_STATIC_SCRATCH_BYTES of partial sums plus a 256-byte status slot.  Every GPU that loads the
+ * library holds that array from load until the process exits.
+ *
+ * Limit: k_splits * M * N * 4 bytes must fit ODB_STATIC_SCRATCH_BYTES (k_splits after the library's
+ * heuristic when 0 is passed), otherwise ODB_ERR_WORKSPACE is returned and nothing is launched.
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ * The first call on a device looks up the array's device address (with that device current); make
+ * that first call before any stream capture begins.
+ * All calls on a device share the one array: two calls whose kernels overlap on the GPU (different
+ * streams, or different host threads) race on it; serialise them.  The array keeps the previous
+ * call's contents; the call itself clears the one word that has to start at zero.
+ * Otherwise identical to odb_debug_gemm: out[M][N] fp32 = x[M][K] bf16 * w[N][K]^T (packed bf16);
+ * runs on `stream`, waits for it, returns ODB_OK or ODB_ERR_TIMEOUT / ODB_ERR_CUDA. */
+#define ODB_STATIC_SCRATCH_BYTES (8u << 20)
+int32_t odb_gemm_static_scratch(const void* x, const void* w_packed, float* out, int32_t M, int32_t N, int32_t K,
+                                int32_t k_splits, void* stream);
+
 /* Launch accounting.  odb_session_profile(s, 1) waits for the stream, clears the counters and
  * from then on brackets every kernel launch of the session with a CUDA event pair (this
  * serialises nothing but costs two event records per launch; leave it off when timing whole

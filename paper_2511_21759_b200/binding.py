@@ -15,6 +15,7 @@ LIB_PATH = os.path.join(HERE, "libodb.so")
 
 ODB_OK, ODB_ERR_ARG, ODB_ERR_SHAPE, ODB_ERR_WORKSPACE, ODB_ERR_STATE, ODB_ERR_CUDA, ODB_ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
 ODB_MAX_COPIES, ODB_MAX_RANKS, ODB_MAX_CHAIN = 8, 4, 5
+ODB_STATIC_SCRATCH_BYTES = 8 << 20
 KINDS = ("gemm", "attention", "elementwise", "confidence", "control")
 
 
@@ -77,6 +78,8 @@ SIGNATURES = {
     "odb_debug_read": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_int32)]),
     "odb_debug_gemm": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_int32, C.c_void_p]),
+    "odb_gemm_static_scratch": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                            C.c_void_p]),
     "odb_session_profile": (C.c_int32, [C.c_void_p, C.c_int32]),
     "odb_session_profile_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "odb_step_algorithmic_bytes": (C.c_double, [C.POINTER(odb_config), C.c_int32]),

@@ -215,6 +215,20 @@ def debug_gemm(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Ten
     return out
 
 
+def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Tensor:
+    """Same product as debug_gemm through odb_gemm_static_scratch: the library keeps the split-K
+    partial sums in its own fixed device array, so the call itself allocates nothing (the tensors
+    created here are the caller's inputs and output)."""
+    M, K = x.shape
+    N = w.shape[0]
+    w = pack_weight(w)
+    out = torch.empty(M, N, dtype=torch.float32, device=x.device)
+    st = torch.cuda.current_stream(x.device)
+    B.check(B.lib().odb_gemm_static_scratch(x.data_ptr(), w.data_ptr(), out.data_ptr(), M, N, K, k_splits,
+                                            C.c_void_p(st.cuda_stream)), "odb_gemm_static_scratch")
+    return out
+
+
 def generate(sess: Session, params: DecodeParams, *,
              length_schedule: Optional[Callable[[int, int, int], Optional[int]]] = None,
              max_iters: Optional[int] = None):
