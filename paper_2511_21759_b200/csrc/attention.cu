@@ -130,7 +130,10 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
         }
     };
 
+    // the first two tiles are requested at once; later ones one iteration ahead
     if (t0 < t1) load_tile(t0, 0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (t0 + 1 < t1) load_tile(t0 + 1, 1);
     asm volatile("cp.async.commit_group;" ::: "memory");
 
     float o_acc[HD / 8][4];
@@ -143,11 +146,10 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
 
     for (int tile = t0; tile < t1; ++tile) {
         const int buf = (tile - t0) & 1;
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        __syncthreads();                                   // tile `tile` landed; everyone is done with buf^1
-        if (tile + 1 < t1) load_tile(tile + 1, buf ^ 1);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        if (!warp_active) continue;
+        if (tile + 1 < t1) asm volatile("cp.async.wait_group 1;" ::: "memory");
+        else asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();                                   // tile `tile` has landed
+        if (warp_active) {
 
         const uint32_t kbase = smem_u32(sK + buf * kTileBytes);
         const uint32_t vbase = smem_u32(sV + buf * kTileBytes);
@@ -232,6 +234,12 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
                 mma_bf16(o_acc[2 * dp + 1], pl, vb[2], vb[3]);
             }
         }
+        }   // warp_active
+        if (tile + 2 < t1) {
+            __syncthreads();                               // everyone is done with this buffer
+            load_tile(tile + 2, buf);
+            asm volatile("cp.async.commit_group;" ::: "memory");
+        }
     }
     asm volatile("cp.async.wait_group 0;" ::: "memory");
     if (!warp_active) return;
@@ -264,25 +272,41 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
     }
 }
 
-// grid (M, H), block HD: merge the key splits in split order.
+// grid (M, H), block HD / 4: merge the key splits in split order.  The (max, sum) pairs of all
+// splits are read first, then the partial outputs as float4 in groups of four independent loads.
 __global__ void attention_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                          __nv_bfloat16* __restrict__ o, int M, int H, int hd, int ksplit) {
     pdl_launch_dependents();
     pdl_wait();
-    const int row = blockIdx.x, head = blockIdx.y, i = threadIdx.x;
+    const int row = blockIdx.x, head = blockIdx.y, d4 = threadIdx.x * 4;
+    const size_t zs = static_cast<size_t>(M) * H, base = static_cast<size_t>(row) * H + head;
+    constexpr int kMaxSplit = 8;                         // the launcher never uses more
+    float2 ml[kMaxSplit];
+#pragma unroll
+    for (int z = 0; z < kMaxSplit; ++z)
+        if (z < ksplit) ml[z] = *reinterpret_cast<const float2*>(part_ml + (z * zs + base) * 2);
+    float4 v[kMaxSplit];
+#pragma unroll
+    for (int z = 0; z < kMaxSplit; ++z)
+        if (z < ksplit) v[z] = *reinterpret_cast<const float4*>(part_o + (z * zs + base) * hd + d4);
     float mmax = -INFINITY;
-    for (int z = 0; z < ksplit; ++z)
-        mmax = fmaxf(mmax, part_ml[((static_cast<size_t>(z) * M + row) * H + head) * 2]);
-    float L = 0.f, acc = 0.f;
-    for (int z = 0; z < ksplit; ++z) {
-        const size_t pr = (static_cast<size_t>(z) * M + row) * H + head;
-        const float m = part_ml[pr * 2], l = part_ml[pr * 2 + 1];
-        if (l <= 0.f) continue;
-        const float w = exp2f(m - mmax);
-        L += l * w;
-        acc += part_o[pr * hd + i] * w;
+#pragma unroll
+    for (int z = 0; z < kMaxSplit; ++z)
+        if (z < ksplit && ml[z].y > 0.f) mmax = fmaxf(mmax, ml[z].x);
+    float L = 0.f;
+    float4 acc = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int z = 0; z < kMaxSplit; ++z) {
+        if (z < ksplit && ml[z].y > 0.f) {
+            const float wt = exp2f(ml[z].x - mmax);
+            L += ml[z].y * wt;
+            acc.x += v[z].x * wt; acc.y += v[z].y * wt; acc.z += v[z].z * wt; acc.w += v[z].w * wt;
+        }
     }
-    o[(static_cast<size_t>(row) * H + head) * hd + i] = __float2bfloat16_rn(L > 0.f ? acc / L : 0.f);
+    const float inv = L > 0.f ? 1.0f / L : 0.f;
+    __nv_bfloat16* op = o + base * hd + d4;
+    *reinterpret_cast<__nv_bfloat162*>(op) = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    *reinterpret_cast<__nv_bfloat162*>(op + 2) = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
 }
 
 template <int HD>
@@ -296,9 +320,10 @@ cudaError_t launch_hd(const AttnArgs& a, cudaStream_t st) {
         attr_done = true;
     }
     dim3 grid(a.n_tiles, a.H, a.ksplit);
+    if (a.ksplit > 8) return cudaErrorInvalidValue;
     cudaError_t e = launch_kernel(attention_kernel<HD>, grid, dim3(kAttnThreads), smem, st, a);
     if (e != cudaSuccess || a.ksplit == 1) return e;
-    return launch_kernel(attention_combine_kernel, dim3(a.M, a.H), dim3(HD), 0, st, static_cast<const float*>(a.part_o),
+    return launch_kernel(attention_combine_kernel, dim3(a.M, a.H), dim3(HD / 4), 0, st, static_cast<const float*>(a.part_o),
                          static_cast<const float*>(a.part_ml), a.o, a.M, a.H, HD, a.ksplit);
 }
 

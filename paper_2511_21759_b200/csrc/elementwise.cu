@@ -60,10 +60,17 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, co
     for (int i = threadIdx.x; i < nvec; i += stride, ++slot) {
         float4 v = reinterpret_cast<const float4*>(hr)[i];
         if (partial) {
-            const float4* p = reinterpret_cast<const float4*>(partial + static_cast<size_t>(row) * d) + i;
-            for (int s = 0; s < splits; ++s) {
-                const float4 t = *reinterpret_cast<const float4*>(reinterpret_cast<const float*>(p) + s * pstride);
-                v.x += t.x; v.y += t.y; v.z += t.z; v.w += t.w;
+            // split order is fixed; groups of four loads are issued together (uniform guard) so the
+            // reduction costs one memory round trip per group instead of one per split
+            const float* p = partial + static_cast<size_t>(row) * d + 4 * i;
+            for (int sb = 0; sb < splits; sb += 4) {
+                float4 t[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (sb + u < splits) t[u] = *reinterpret_cast<const float4*>(p + static_cast<size_t>(sb + u) * pstride);
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    if (sb + u < splits) { v.x += t[u].x; v.y += t[u].y; v.z += t[u].z; v.w += t[u].w; }
             }
             reinterpret_cast<float4*>(hr)[i] = v;
         }
@@ -110,11 +117,23 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
         const int head = t / half, i = t % half;
         const int e0 = head * a.hd + i, e1 = e0 + half;
         float q0 = 0.f, q1 = 0.f, k0 = 0.f, k1 = 0.f, v0 = 0.f, v1 = 0.f;
-        for (int s = 0; s < a.splits; ++s) {
-            const float* p = p0 + s * a.pstride;
-            q0 += p[e0]; q1 += p[e1];
-            k0 += p[d + e0]; k1 += p[d + e1];
-            v0 += p[2 * d + e0]; v1 += p[2 * d + e1];
+        for (int sb = 0; sb < a.splits; sb += 4) {
+            float t[4][6];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (sb + u < a.splits) {
+                    const float* p = p0 + static_cast<size_t>(sb + u) * a.pstride;
+                    t[u][0] = p[e0]; t[u][1] = p[e1];
+                    t[u][2] = p[d + e0]; t[u][3] = p[d + e1];
+                    t[u][4] = p[2 * d + e0]; t[u][5] = p[2 * d + e1];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (sb + u < a.splits) {
+                    q0 += t[u][0]; q1 += t[u][1]; k0 += t[u][2]; k1 += t[u][3]; v0 += t[u][4]; v1 += t[u][5];
+                }
+            }
         }
         const float2 cs = rope[i];
         const __nv_bfloat16 rq0 = __float2bfloat16_rn(q0 * cs.x - q1 * cs.y);
