@@ -440,8 +440,8 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
     const int nkb_total = (a.K + kBK - 1) / kBK;
     const int nkb_per_split = (nkb_total + a.splits - 1) / a.splits;
     const uint32_t stage_bytes = kBM * kBK * 2 + BN * kBK * 2;
-    // two CTAs per SM for the narrow tiles (hides each CTA's prologue and drain), one for 256
-    const uint32_t budget = BN <= 64 ? 100 * 1024 : BN == 128 ? 196 * 1024 : 200 * 1024;
+    // two CTAs per SM up to 128 activation rows (hides each CTA's prologue and drain), one for 256
+    const uint32_t budget = BN <= 128 ? 100 * 1024 : 200 * 1024;
     int stages = static_cast<int>(budget / stage_bytes);
     if (stages > 16) stages = 16;
     if (stages > nkb_per_split) stages = nkb_per_split < 2 ? 2 : nkb_per_split;
@@ -520,7 +520,7 @@ int gemm_pick_splits(int M, int N, int K) {
     const int nkb = (K + kBK - 1) / kBK;
     // all work units must be resident at once (two CTA slots per SM) and equal in size: a
     // second, partly filled wave would double the kernel's time
-    int splits = target_ctas() / tiles;
+    int splits = (bn <= 128 ? target_ctas() : target_ctas() / 2) / tiles;
     if (splits > nkb / 4) splits = nkb / 4;
     if (splits > 16) splits = 16;
     if (splits < 1) splits = 1;

@@ -446,7 +446,9 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
     const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
     int res_splits = 0;
     size_t res_stride = 0;
+    static const int ks_env = getenv("ODB_ATTN_KS") ? atoi(getenv("ODB_ATTN_KS")) : 0;
     int ks = (2 * 148 + n_tiles * H - 1) / (n_tiles * H);
+    if (ks_env > 0 && !write_cache) ks = ks_env;
     if (ks > 8) ks = 8;
     if (static_cast<size_t>(ks) * M > L.attn_rows) ks = static_cast<int>(L.attn_rows / M);
     if (ks < 1) ks = 1;
