@@ -520,7 +520,18 @@ int gemm_pick_splits(int M, int N, int K) {
     const int nkb = (K + kBK - 1) / kBK;
     // all work units must be resident at once (two CTA slots per SM) and equal in size: a
     // second, partly filled wave would double the kernel's time
-    int splits = (bn <= 128 ? target_ctas() : target_ctas() / 2) / tiles;
+    if (bn > 128) {
+        // compute-bound tiles, one CTA per SM: pick the K split that minimises the makespan
+        // ceil(tiles * s / SMs) / s (a 96-tile GEMM on 148 SMs would leave a third of them idle)
+        int best = 1;
+        double best_t = 1e30;
+        for (int sp = 1; sp <= 8 && sp * 8 <= nkb; ++sp) {
+            const double t = static_cast<double>((tiles * sp + 147) / 148) / sp;
+            if (t < best_t - 1e-9) { best_t = t; best = sp; }
+        }
+        return best;
+    }
+    int splits = target_ctas() / tiles;
     if (splits > nkb / 4) splits = nkb / 4;
     if (splits > 16) splits = 16;
     if (splits < 1) splits = 1;

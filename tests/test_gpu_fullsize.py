@@ -1,0 +1,85 @@
+"""Full-size parity: the 32-layer 8B-shaped model in the configuration bench.py times (batch 1,
+prompt 512, response 256, block 32), one refresh prefill and the decode step that follows it,
+against the oracle run in float32 on the host cores.
+
+Every logit of the 256 response rows of the refresh and of the 32 block rows of the step is
+compared (the oracle can afford one refresh and one step at this size; it takes about two minutes).
+Decisions are checked the lock-step way: the oracle's accept rule on the GPU's own confidences must
+give the GPU's accepted set; a differing oracle-side decision must be a measured near-tie.
+"""
+import numpy as np
+import pytest
+
+import synth
+from oracle import odb_oracle as O
+from oracle.inputs import model_from_synth
+from gpu_common import engine, requires_gpu, logits_close
+
+
+@requires_gpu
+def test_cfg3_refresh_and_first_step_match_oracle():
+    E = engine()
+    wl = synth.WORKLOADS["cfg3_8b_c1"]
+    shape, P, L, Bk = wl.shape, wl.prompt_len, wl.gen_len, wl.block_len
+    T = P + L
+    x0 = synth.sequence(0, 0, P, L, shape)
+
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=T, max_block=Bk, max_copies=1)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    gp = E.DecodeParams(block_len=Bk, n_copies=1)
+    sess.refresh_prefill(gp, 0)
+    g_logits = sess.debug_read("logits")
+    g_conf, g_tok = sess.debug_read("conf"), sess.debug_read("tok")
+    res = sess.unmask_accept(gp, True)[0]
+    g_acc = sorted((res.accepted_pos[j], res.accepted_tok[j]) for j in range(res.n_accepted))
+    sess.block_decode_step(gp)
+    s_logits = sess.debug_read("logits")
+    s_conf, s_tok = sess.debug_read("conf"), sess.debug_read("tok")
+    res2 = sess.unmask_accept(gp, False)[0]
+    s_acc = sorted((res2.accepted_pos[j], res2.accepted_tok[j]) for j in range(res2.n_accepted))
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    del gm
+
+    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
+    assert g_logits.shape == o_logits.shape == (L, shape.vocab)
+    ok, worst_r = logits_close(g_logits, o_logits)
+    assert ok, f"refresh logits off by {worst_r:.2f} x the 2e-2 bound"
+    cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
+    # control on the GPU's own numbers: bit exact
+    masked = np.ones(Bk, dtype=bool)
+    acc = O.accept_set(g_conf[:Bk], masked, wl.accept_threshold)
+    assert g_acc == [(int(P + i), int(g_tok[i])) for i in np.flatnonzero(acc)]
+    acc_o = O.accept_set(o_conf[:Bk], masked, wl.accept_threshold)
+    if not np.array_equal(acc, acc_o):
+        margin = O.decision_margin(o_conf[:Bk], masked, wl.accept_threshold, 0)
+        assert margin <= max(1e-3, 4 * cerr), (margin, cerr)
+    # greedy tokens equal wherever the oracle's top-2 logit gap exceeds the logit error
+    l32 = o_logits.copy()
+    l32[:, shape.mask_id] = -np.inf
+    top2 = np.partition(l32, -2, axis=1)[:, -2:]
+    gap = np.abs(top2[:, 1] - top2[:, 0])
+    err = np.abs(g_logits - o_logits).max(axis=1)
+    assert not ((g_tok != o_tok) & (gap > 2 * err)).any()
+
+    # the step, from the state the GPU is in (its own accepted token)
+    x = x0.astype(np.int64).copy()
+    for p_, t_ in g_acc:
+        x[p_] = t_
+    o_c, o_t, os_logits, r_copy, r_pos = O.block_decode_step(om, cache, x, T, P, P + Bk, [()], [], [], False,
+                                                             dtype=np.float32, return_logits=True)
+    ok, worst_s = logits_close(s_logits, os_logits)
+    assert ok, f"step logits off by {worst_s:.2f} x the 2e-2 bound"
+    masked = x[P:P + Bk] == shape.mask_id
+    acc = O.accept_set(s_conf, masked, wl.accept_threshold)
+    assert s_acc == [(int(P + i), int(s_tok[i])) for i in np.flatnonzero(acc)]
+    cerr_s = float((np.abs(s_conf - o_c[0]) / o_c[0]).max())
+    acc_o = O.accept_set(o_c[0], masked, wl.accept_threshold)
+    if not np.array_equal(acc, acc_o):
+        margin = O.decision_margin(o_c[0], masked, wl.accept_threshold, 0)
+        assert margin <= max(1e-3, 4 * cerr_s), (margin, cerr_s)
+    print(f"\ncfg3 full size: refresh logits {worst_r:.2f} x bound, step logits {worst_s:.2f} x bound, "
+          f"conf rel err {cerr:.2e} / {cerr_s:.2e}, greedy tokens differing: "
+          f"{int((g_tok != o_tok).sum())} of {L} (refresh), {int((s_tok != o_t[0]).sum())} of {Bk} (step)")
