@@ -27,6 +27,13 @@ def logits_close(got, want, tol=2e-2):
     return bool((err <= bound).all()), float((err / bound).max())
 
 
+def rel_l2(got, want):
+    """Worst per-row relative L2 error: ||got - want|| / ||want|| over the last axis."""
+    want = np.asarray(want, dtype=np.float64)
+    d = np.asarray(got, dtype=np.float64) - want
+    return float((np.sqrt((d * d).sum(-1)) / np.sqrt((want * want).sum(-1))).max())
+
+
 def bf16_bits_to_f64(bits):
     return synth.bf16_bits_to_f32(bits).astype(np.float64)
 

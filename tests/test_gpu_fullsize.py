@@ -3,7 +3,18 @@ prompt 512, response 256, block 32), one refresh prefill and the decode step tha
 against the oracle run in float32 on the host cores.
 
 Every logit of the 256 response rows of the refresh and of the 32 block rows of the step is
-compared (the oracle can afford one refresh and one step at this size; it takes about two minutes).
+compared (the oracle can afford one refresh and one step at this size; it takes about a minute).
+
+Tolerance at this size.  Each bf16 rounding turns an upstream relative difference delta into
+rounding flips of one bf16 step (2^-8) with probability ~delta / 2^-8, i.e. into an rms difference
+of ~sqrt(delta * 2^-8): after three or four rounding points ANY two evaluation orders differ by a
+fraction of a bf16 step in every activation, however close they started (the oracle's own float32
+and float64 runs do: 0.19 % rms in the residual stream after ONE 8B-shaped layer).  The logits of
+two correct implementations therefore differ by a few 1e-3 of their RMS per element, and the largest
+of 3.2e7 such differences sits 5-6 sigma out.  The 2e-2 figure is therefore applied to the per-row
+relative L2 error, and the element-wise check uses 6 x the small-model bound; on the 32-layer model
+the oracle's float32 and float64 runs differ from each other by about as much as the kernels differ
+from either (measured: 3.6 x vs 3.5 x the small-model bound at 16 layers).
 Decisions are checked the lock-step way: the oracle's accept rule on the GPU's own confidences must
 give the GPU's accepted set; a differing oracle-side decision must be a measured near-tie.
 """
@@ -13,7 +24,7 @@ import pytest
 import synth
 from oracle import odb_oracle as O
 from oracle.inputs import model_from_synth
-from gpu_common import engine, requires_gpu, logits_close
+from gpu_common import engine, requires_gpu, logits_close, rel_l2
 
 
 @requires_gpu
@@ -45,8 +56,11 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
     cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
     assert g_logits.shape == o_logits.shape == (L, shape.vocab)
-    ok, worst_r = logits_close(g_logits, o_logits)
-    assert ok, f"refresh logits off by {worst_r:.2f} x the 2e-2 bound"
+    l2_r = rel_l2(g_logits, o_logits)
+    assert l2_r <= 2e-2, f"refresh logits: per-row relative L2 error {l2_r:.3e}"
+    ok, worst_r = logits_close(g_logits, o_logits, 6 * 2e-2)
+    worst_r *= 6
+    assert ok, f"refresh logits off by {worst_r:.2f} x the small-model bound"
     cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
     # control on the GPU's own numbers: bit exact
     masked = np.ones(Bk, dtype=bool)
@@ -70,8 +84,11 @@ def test_cfg3_refresh_and_first_step_match_oracle():
         x[p_] = t_
     o_c, o_t, os_logits, r_copy, r_pos = O.block_decode_step(om, cache, x, T, P, P + Bk, [()], [], [], False,
                                                              dtype=np.float32, return_logits=True)
-    ok, worst_s = logits_close(s_logits, os_logits)
-    assert ok, f"step logits off by {worst_s:.2f} x the 2e-2 bound"
+    l2_s = rel_l2(s_logits, os_logits)
+    assert l2_s <= 2e-2, f"step logits: per-row relative L2 error {l2_s:.3e}"
+    ok, worst_s = logits_close(s_logits, os_logits, 6 * 2e-2)
+    worst_s *= 6
+    assert ok, f"step logits off by {worst_s:.2f} x the small-model bound"
     masked = x[P:P + Bk] == shape.mask_id
     acc = O.accept_set(s_conf, masked, wl.accept_threshold)
     assert s_acc == [(int(P + i), int(s_tok[i])) for i in np.flatnonzero(acc)]
@@ -80,6 +97,7 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     if not np.array_equal(acc, acc_o):
         margin = O.decision_margin(o_c[0], masked, wl.accept_threshold, 0)
         assert margin <= max(1e-3, 4 * cerr_s), (margin, cerr_s)
-    print(f"\ncfg3 full size: refresh logits {worst_r:.2f} x bound, step logits {worst_s:.2f} x bound, "
+    print(f"\ncfg3 full size: per-row rel. L2 error {l2_r:.2e} (refresh) {l2_s:.2e} (step); "
+          f"element-wise {worst_r:.2f} x / {worst_s:.2f} x the small-model bound; "
           f"conf rel err {cerr:.2e} / {cerr_s:.2e}, greedy tokens differing: "
           f"{int((g_tok != o_tok).sum())} of {L} (refresh), {int((s_tok != o_t[0]).sum())} of {Bk} (step)")
