@@ -114,11 +114,12 @@ def oracle_sample(wl, budget_layers=2):
     t_lm_step = t_lm_refresh = 0.0
     if wl.with_lm_head:
         lm = synth.bf16_bits_to_f32(synth.lm_head_bits(shape, 0))
-        n = O.bf16_round(O.rmsnorm(hid.astype(np.float32), np.ones(shape.d_model, np.float32), shape.rms_eps))
+        hid32 = hid.astype(np.float32)
         t0 = time.perf_counter()
-        O.confidence(n @ lm.T, shape.mask_id)
+        logits, = O.normed_projection(hid32, np.ones(shape.d_model, np.float32), shape.rms_eps, [lm], O.bf16_round)
+        O.confidence(logits, shape.mask_id)
         t_lm_step = time.perf_counter() - t0
-        t_lm_refresh = t_lm_step * (wl.gen_len / max(len(n), 1))
+        t_lm_refresh = t_lm_step * (wl.gen_len / max(len(hid32), 1))
     scale = shape.n_layers / nl
     t_refresh = t_refresh_layers * scale + t_lm_refresh
     t_step = t_step_layers * scale + t_lm_step

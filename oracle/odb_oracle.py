@@ -20,9 +20,11 @@ What the paper fixes and what it leaves open
     readings taken here are listed beside each function.
 
 Arithmetic: `dtype` (float64 by default; float32 for large shapes).  With `faithful=True`
-activations are rounded to bf16 exactly where the CUDA path stores bf16 (GEMM input after
-each RMSNorm, q/k/v after RoPE, attention output, SwiGLU output); the residual stream,
-softmax statistics and logits are never rounded to bf16.  Decisions that turn floating point
+activations are rounded to bf16 exactly where the CUDA path stores bf16 (the projection input
+of each RMSNorm, q/k/v after RoPE, attention output, SwiGLU output); the residual stream,
+softmax statistics and logits are never rounded to bf16.  RMSNorm feeds a projection, and its
+per-row scalar 1/rms commutes with the projection: the value stored in bf16 is x * gain, and
+the scalar multiplies the projection's fp32 output (`normed_projection`).  Decisions that turn floating point
 into integers (argmax over the vocabulary, threshold compares, ranking) are taken on fp32
 values, the precision the kernels decide in.
 
@@ -93,6 +95,17 @@ def rmsnorm(x: np.ndarray, gain: np.ndarray, eps: float) -> np.ndarray:
     return x / np.sqrt(ms + eps) * gain
 
 
+def normed_projection(x: np.ndarray, gain: np.ndarray, eps: float, weights: Sequence[np.ndarray], rnd) -> list:
+    """[rmsnorm(x, gain) @ W^T for W in weights], evaluated as ((rnd(x * gain)) @ W^T) / rms(x).
+
+    Mathematically rmsnorm(x) @ W^T (the row scalar 1/sqrt(mean(x^2) + eps) commutes with the
+    matrix product); the order matters only for where the bf16 rounding `rnd` falls: on x * gain,
+    the operand the kernels hand to the tensor cores, with the scalar applied to the fp32 result."""
+    inv = 1.0 / np.sqrt(np.mean(x * x, axis=-1, keepdims=True) + eps)
+    a = rnd(x * gain)
+    return [(a @ w.T) * inv for w in weights]
+
+
 def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
     """Rotary embedding, rotate-half pairing: element i pairs with i + hd/2.
 
@@ -152,10 +165,9 @@ def forward_rows(model: Model, tok: np.ndarray, pos: np.ndarray,
     fresh_k, fresh_v = [], []
     for l in range(model.n_layers):
         w = model.layer(l)
-        a = rnd(rmsnorm(h, w["g1"].astype(dtype), model.rms_eps))
-        q = (a @ w["wq"].astype(dtype).T).reshape(M, H, hd)
-        k = (a @ w["wk"].astype(dtype).T).reshape(M, H, hd)
-        v = (a @ w["wv"].astype(dtype).T).reshape(M, H, hd)
+        q, k, v = normed_projection(h, w["g1"].astype(dtype), model.rms_eps,
+                                    [w["wq"].astype(dtype), w["wk"].astype(dtype), w["wv"].astype(dtype)], rnd)
+        q, k, v = q.reshape(M, H, hd), k.reshape(M, H, hd), v.reshape(M, H, hd)
         q = rnd(rope(q, pos, model.rope_theta))
         k = rnd(rope(k, pos, model.rope_theta))
         v = rnd(v)
@@ -168,15 +180,15 @@ def forward_rows(model: Model, tok: np.ndarray, pos: np.ndarray,
             k_all, v_all = k, v
         o = rnd(attention(q, k_all, v_all, vis)).reshape(M, d)
         h = h + o @ w["wo"].astype(dtype).T
-        b = rnd(rmsnorm(h, w["g2"].astype(dtype), model.rms_eps))
-        g = rnd(silu(b @ w["wg"].astype(dtype).T) * (b @ w["wu"].astype(dtype).T))
+        gate, up = normed_projection(h, w["g2"].astype(dtype), model.rms_eps,
+                                     [w["wg"].astype(dtype), w["wu"].astype(dtype)], rnd)
+        g = rnd(silu(gate) * up)
         h = h + g @ w["wd"].astype(dtype).T
     if return_hidden or model.lm_head is None:
         return h, fresh_k, fresh_v
-    n = rnd(rmsnorm(h, model.final_gain.astype(dtype), model.rms_eps))
     if logit_rows is not None:
-        n = n[logit_rows]
-    logits = n @ model.lm_head.astype(dtype).T
+        h = h[logit_rows]
+    logits, = normed_projection(h, model.final_gain.astype(dtype), model.rms_eps, [model.lm_head.astype(dtype)], rnd)
     return logits, fresh_k, fresh_v
 
 

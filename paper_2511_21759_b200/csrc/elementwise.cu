@@ -38,12 +38,13 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
     }
 }
 
-// One block per output row.  y = x / sqrt(mean(x^2) + eps) * gain, x = residual stream row
-// (after adding the split-K partials of the preceding projection in split order).  float4
-// accesses; a thread keeps its (up to two) vectors in registers between the two passes.
+// One block per output row: the part of RMSNorm that is not a row scalar.  x = residual stream row
+// (after adding the split-K partials of the preceding projection in split order); writes
+// bf16(x * gain) as the projection's operand and 1 / sqrt(mean(x^2) + eps) for the projection's
+// consumer (the scalar commutes with the matrix product).  float4 accesses.
 __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
                                                        int splits, size_t pstride, const float* __restrict__ gain,
-                                                       __nv_bfloat16* __restrict__ out,
+                                                       __nv_bfloat16* __restrict__ out, float* __restrict__ inv_rms,
                                                        const int32_t* __restrict__ row_map, int d, float eps,
                                                        L2Prefetch pf) {
     __shared__ float red[32];
@@ -54,10 +55,9 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, co
     const int row = row_map ? row_map[orow] : orow;
     float* hr = h + static_cast<size_t>(row) * d;
     const int nvec = d >> 2, stride = blockDim.x;
-    float4 keep[2];
     float ss = 0.f;
-    int slot = 0;
-    for (int i = threadIdx.x; i < nvec; i += stride, ++slot) {
+    __nv_bfloat16* o = out + static_cast<size_t>(orow) * d;
+    for (int i = threadIdx.x; i < nvec; i += stride) {
         float4 v = reinterpret_cast<const float4*>(hr)[i];
         if (partial) {
             // split order is fixed; groups of four loads are issued together (uniform guard) so the
@@ -74,23 +74,17 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, co
             }
             reinterpret_cast<float4*>(hr)[i] = v;
         }
-        if (slot < 2) keep[slot] = v;
         ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-    }
-    const float total = block_sum(ss, red);
-    const float inv = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
-    __nv_bfloat16* o = out + static_cast<size_t>(orow) * d;
-    slot = 0;
-    for (int i = threadIdx.x; i < nvec; i += stride, ++slot) {
-        const float4 v = slot < 2 ? keep[slot] : reinterpret_cast<const float4*>(hr)[i];
         const float4 g = reinterpret_cast<const float4*>(gain)[i];
-        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * inv * g.x, v.y * inv * g.y);
-        const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * inv * g.z, v.w * inv * g.w);
+        const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
+        const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * g.z, v.w * g.w);
         uint2 pk;
         pk.x = *reinterpret_cast<const uint32_t*>(&lo);
         pk.y = *reinterpret_cast<const uint32_t*>(&hi);
         reinterpret_cast<uint2*>(o)[i] = pk;
     }
+    const float total = block_sum(ss, red);
+    if (threadIdx.x == 0) inv_rms[orow] = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
 }
 
 // grid (rows, pair chunks), one thread per rotation pair.  Sums the QKV partials, rotates q and k (rotate-half pairing: element i
@@ -135,6 +129,8 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
                 }
             }
         }
+        const float inv = a.inv_rms[row];               // scalar of the RMSNorm folded behind the projection
+        q0 *= inv; q1 *= inv; k0 *= inv; k1 *= inv; v0 *= inv; v1 *= inv;
         const float2 cs = rope[i];
         const __nv_bfloat16 rq0 = __float2bfloat16_rn(q0 * cs.x - q1 * cs.y);
         const __nv_bfloat16 rq1 = __float2bfloat16_rn(q1 * cs.x + q0 * cs.y);
@@ -253,12 +249,12 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 }
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps, L2Prefetch pf,
-                           cudaStream_t st) {
+                           __nv_bfloat16* out, float* inv_rms, const int32_t* row_map, int rows_out, int d, float eps,
+                           L2Prefetch pf, cudaStream_t st) {
     int threads = ((d / 4 + 31) / 32) * 32;
     if (threads > 1024) threads = 1024;
-    return launch_kernel(rmsnorm_kernel, dim3(rows_out), dim3(threads), 0, st, h, partial, splits, pstride, gain, out, row_map,
-                         d, eps, pf);
+    return launch_kernel(rmsnorm_kernel, dim3(rows_out), dim3(threads), 0, st, h, partial, splits, pstride, gain, out, inv_rms,
+                         row_map, d, eps, pf);
 }
 
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {

@@ -159,8 +159,8 @@ struct alignas(8) GemmShared {
 template <int BN, bool SWIGLU>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-            float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, int M, int N, int nkb_total,
-            int nkb_per_split, int stages, int l2_prefetch, int* status) {
+            float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, const float* __restrict__ row_scale,
+            int M, int N, int nkb_total, int nkb_per_split, int stages, int l2_prefetch, int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
     constexpr uint32_t kBBytes = BN * kBK * 2;
@@ -293,12 +293,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                     uint32_t v[32];
                     tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    if (n < N) {
+                    // lane j holds the scale of activation row m0 + 32 c + j; broadcast per column
+                    const int ms = m0 + c * 32 + lane;
+                    const float my_scale = (row_scale && ms < M) ? row_scale[ms] : 1.0f;
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int m = m0 + c * 32 + j;
-                            if (m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
-                        }
+                    for (int j = 0; j < 32; ++j) {
+                        const int m = m0 + c * 32 + j;
+                        const float sc = __shfl_sync(0xffffffffu, my_scale, j);
+                        if (n < N && m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]) * sc;
                     }
                 }
             }
@@ -319,13 +321,18 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) xch[((q & 1) * 32 + lane) * 33 + j] = __uint_as_float(v[j]);
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                if (ok && q < 2 && f < N) {
+                const int ms = m0 + c * 32 + lane;
+                const float my_scale = (row_scale && ms < M) ? row_scale[ms] : 1.0f;
+                if (ok && q < 2) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + c * 32 + j;
-                        const float gate = __uint_as_float(v[j]);
-                        const float up = xch[((q & 1) * 32 + lane) * 33 + j];
-                        if (m < M) act_out[static_cast<size_t>(m) * N + f] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
+                        const float sc = __shfl_sync(0xffffffffu, my_scale, j);
+                        if (m < M && f < N) {
+                            const float gate = __uint_as_float(v[j]) * sc;
+                            const float up = xch[((q & 1) * 32 + lane) * 33 + j] * sc;
+                            act_out[static_cast<size_t>(m) * N + f] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
+                        }
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -459,8 +466,8 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
         const char* e = getenv("ODB_GEMM_L2_PREFETCH");
         l2_prefetch = e ? atoi(e) : 0;   // measured: prefetching into L2 slows the step down
     }
-    return launch_kernel(gemm_kernel<BN, SWIGLU>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out, a.M,
-                         a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
+    return launch_kernel(gemm_kernel<BN, SWIGLU>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale,
+                         a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
 }
 
 }  // namespace

@@ -123,6 +123,8 @@ struct GemmArgs {
     const void* x;         // bf16 [M][K] device
     float* partial;        // fp32 [splits][M][N]
     __nv_bfloat16* act_out; // non-null: gate/up GEMM with the SwiGLU epilogue, writes bf16 [M][N = F]; splits == 1
+    const float* row_scale = nullptr;   // per activation row m: the output is multiplied by row_scale[m]
+                                        // (the 1/rms of an RMSNorm folded behind the projection); needs splits == 1
     int M, N, K;
     int splits;
     int* status;           // device status word
@@ -140,12 +142,15 @@ cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stri
 
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d,
                          cudaStream_t st);
-// h[row] += sum_s partial[s][row] (if partial), out[i] = bf16(rmsnorm(h[map ? map[i] : i]) * gain)
+// RMSNorm feeding a projection, with the row scalar deferred: h[row] += sum_s partial[s][row] (if
+// partial); out[i] = bf16(h[r] * gain), inv_rms[i] = 1 / sqrt(mean(h[r]^2) + eps), r = map ? map[i] : i.
+// The projection's consumer multiplies its fp32 output by inv_rms (the scalar commutes with the GEMM).
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, const int32_t* row_map, int rows_out, int d, float eps, L2Prefetch pf,
-                           cudaStream_t st);
+                           __nv_bfloat16* out, float* inv_rms, const int32_t* row_map, int rows_out, int d, float eps,
+                           L2Prefetch pf, cudaStream_t st);
 struct QkvRopeArgs {
     const float* partial; int splits; size_t pstride;      // [splits][M][3d]
+    const float* inv_rms;                                  // [M] scalar of the preceding RMSNorm
     const float2* rope;                                    // [max_seq][hd/2] (cos, sin)
     const int32_t* row_pos; const int32_t* row_seq;
     __nv_bfloat16 *q, *k, *v;                              // [M][d]

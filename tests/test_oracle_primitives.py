@@ -36,6 +36,20 @@ def test_rmsnorm_closed_forms():
     assert np.allclose(O.rmsnorm(np.ones((1, 8)), np.ones(8), 0.21), 1 / math.sqrt(1.21))
 
 
+def test_normed_projection_is_rmsnorm_then_matmul():
+    x = RNG.normal(size=(6, 32)) * 3.0
+    g = RNG.normal(size=32)
+    w1, w2 = RNG.normal(size=(5, 32)), RNG.normal(size=(7, 32))
+    ident = lambda a: a
+    y1, y2 = O.normed_projection(x, g, 1e-5, [w1, w2], ident)
+    assert np.allclose(y1, O.rmsnorm(x, g, 1e-5) @ w1.T, rtol=1e-12) and np.allclose(y2, O.rmsnorm(x, g, 1e-5) @ w2.T, rtol=1e-12)
+    # with rounding, the rounded operand is x * gain (scale invariant input: the row scalar is applied afterwards)
+    y, = O.normed_projection(x, g, 0.0, [w1], O.bf16_round)
+    yk, = O.normed_projection(64.0 * x, g, 0.0, [w1], O.bf16_round)     # power-of-two rescale: same bf16 mantissas
+    assert np.allclose(y, yk, rtol=1e-12)
+    assert np.abs(y - y1).max() <= 2 ** -7 * np.abs(O.rmsnorm(x, g, 0.0)) .max() * np.abs(w1).sum(1).max()
+
+
 def test_rope_closed_forms():
     hd, H = 16, 3
     x = RNG.normal(size=(6, H, hd))
