@@ -86,6 +86,21 @@ def test_lockstep_generate(wl_name, tol):
 
 
 @requires_gpu
+def test_lockstep_with_cluster_residual_epilogue():
+    """The optional decode-step path that closes the residual branches inside the GEMM (thread-block
+    clusters, split-K reduced through distributed shared memory) is selected by an environment
+    variable read once per process, so it is exercised in a child process."""
+    import os, subprocess, sys
+    engine()
+    code = ("import sys; sys.path.insert(0, 'tests'); import test_gpu_generate as t; "
+            "t.test_lockstep_generate('peaky_c4', 4e-2); t.test_lockstep_generate('cfg1_tiny', 2e-2)")
+    env = dict(os.environ, ODB_CLUSTER_EPILOGUE="1")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+
+
+@requires_gpu
 def test_generate_with_length_schedule():
     sched = lambda b, L: {0: 40, 1: 24}.get(b)
     gtok, gtrace, otok, otrace = _run_both("peaky_c4", schedule=sched)
