@@ -577,7 +577,15 @@ __global__ void pack_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __nv_
     reinterpret_cast<uint4*>(dst)[chunk] = v;
 }
 
-int pick_bn(int M) { return M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256; }
+int pick_bn(int M) {
+    static int max_bn = 0;
+    if (!max_bn) {
+        const char* e = getenv("ODB_GEMM_MAX_BN");
+        max_bn = e ? atoi(e) : 128;   // 128-row tiles run two CTAs per SM: one's epilogue overlaps the other's main loop
+    }
+    const int bn = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
+    return bn < max_bn ? bn : max_bn;
+}
 
 template <int BN, int EPI>
 cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st) {
@@ -711,16 +719,12 @@ int gemm_pick_splits(int M, int N, int K) {
     const int nkb = (K + kBK - 1) / kBK;
     // all work units must be resident at once (two CTA slots per SM) and equal in size: a
     // second, partly filled wave would double the kernel's time
-    if (bn > 128) {
-        // compute-bound tiles, one CTA per SM: pick the K split that minimises the makespan
-        // ceil(tiles * s / SMs) / s (a 96-tile GEMM on 148 SMs would leave a third of them idle)
-        int best = 1;
-        double best_t = 1e30;
-        for (int sp = 1; sp <= 8 && sp * 8 <= nkb; ++sp) {
-            const double t = static_cast<double>((tiles * sp + 147) / 148) / sp;
-            if (t < best_t - 1e-9) { best_t = t; best = sp; }
-        }
-        return best;
+    if (M > 128) {
+        // many rows (refresh): compute bound, and every K split costs M x N fp32 partials written and
+        // read back, so split only when the tiles alone cannot occupy the SMs
+        int sp = tiles >= 148 ? 1 : 148 / tiles;
+        if (sp > nkb / 8) sp = nkb / 8;
+        return sp < 1 ? 1 : sp;
     }
     int splits = target_ctas() / tiles;
     if (splits > nkb / 4) splits = nkb / 4;
