@@ -159,6 +159,24 @@ def config_of(wl):
             "step": "one block cycle: refresh prefill + accept, then block decode steps + accepts until the block is full"}
 
 
+# ----------------------------------------------------------------------------- ranks
+
+def max_over_ranks(ms: float, dist, device=None) -> float:
+    """Replicas only: every rank runs the same workload on its own GPU, nothing is exchanged on the
+    data path.  The job's time is the slowest rank's (all-reduce MAX of the device-timed interval)."""
+    if dist is None:
+        return ms
+    import torch
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(units_per_rank: float, ms: float, world: int) -> float:
+    """Whole-job throughput of `world` independent replicas: all units processed / the slowest rank's time."""
+    return world * units_per_rank / (ms * 1e-3)
+
+
 # ----------------------------------------------------------------------------- CUDA arm
 
 def run_cuda(args, wl):
@@ -194,6 +212,7 @@ def run_cuda(args, wl):
     pinned = [torch.from_numpy(s.copy()).pin_memory() for s in seqs]
 
     state = {"block": 0}
+    targets = synth.shrink_schedule(0, wl.batch, wl.gen_len) if wl.batch > 1 else None
 
     def reset():
         for i in range(wl.batch):
@@ -211,7 +230,19 @@ def run_cuda(args, wl):
                 sess.set_sequence(i, toks[i], wl.prompt_len)
             state["block"] = blk
         b = state["block"]
-        sess.refresh_prefill(params, [b] * wl.batch)
+        if all(b * wl.block_len >= sess.gen_len[i] for i in range(wl.batch)):
+            reset()
+            b = 0
+        bi = [b if b * wl.block_len < sess.gen_len[i] else -1 for i in range(wl.batch)]
+        sess.refresh_prefill(params, bi)
+        if targets is not None:
+            # ragged batch: every sequence gives up half of its remaining excess over its seeded target
+            # length at each refresh (the lever adaptive length prediction pulls on a trained model)
+            for i in range(wl.batch):
+                cur = sess.gen_len[i]
+                new = max(int(targets[i]), cur - (cur - int(targets[i]) + 1) // 2, (b + 1) * wl.block_len)
+                if bi[i] >= 0 and b * wl.block_len < new < cur:
+                    sess.set_gen_len(i, new)
         res = sess.unmask_accept(params, True)
         toks, iters = sum(res[i].n_accepted for i in range(wl.batch)), 1
         while any(res[i].masks_left > 0 for i in range(wl.batch)):
@@ -237,13 +268,9 @@ def run_cuda(args, wl):
             toks += t; iters += it
         ev1.record(sess.stream)
         torch.cuda.synchronize()
-        ms = ev0.elapsed_time(ev1)
+        ms = max_over_ranks(ev0.elapsed_time(ev1), dist, "cuda")
         if dist:
-            t_ = torch.tensor([ms], device="cuda")
-            dist.all_reduce(t_, op=dist.ReduceOp.MAX)
-            ms = float(t_.item())
-            if dist:
-                dist.barrier()
+            dist.barrier()
         return ms, toks, iters
 
     reset()
@@ -253,18 +280,17 @@ def run_cuda(args, wl):
         ms, toks, iters = timed(args.steps)
     _, launches = sess.profile_read()
     clk = clocks.summary()
-    value = world * toks / (ms * 1e-3)
+    value = job_throughput(toks, ms, world)
 
     # end to end: same steps, sequence pushed from pinned host memory and read back every step
     timed(1, e2e=True)
     ms_e, toks_e, _ = timed(args.steps, e2e=True)
-    e2e_value = world * toks_e / (ms_e * 1e-3)
+    e2e_value = job_throughput(toks_e, ms_e, world)
 
     # per-kind device time of decode steps and refreshes, measured live with event pairs
     sess.profile(True)
-    if state["block"] >= n_blocks:
-        reset()
-    sess.refresh_prefill(params, [state["block"]] * wl.batch)
+    reset()
+    sess.refresh_prefill(params, [0] * wl.batch)
     res = sess.unmask_accept(params, True)
     ms_refresh, n_refresh = sess.profile_read()
     n_prof = 0
@@ -302,7 +328,12 @@ def run_cuda(args, wl):
     roofline = {"bound": "hbm", "kernel": "gemm_kernel<32> (tcgen05 weight-streaming GEMM), all launches of one decode step",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
-                "traffic": None, "bytes_per_step": gemm_bytes, "launches_per_step": gemm_launches / max(n_prof, 1),
+                # DRAM bytes of the GEMM launches of one decode step: ncu capture of the four per-layer
+                # launches on the single-layer case (profiles/gemm_kernel_cfg2_layer_c1.md: 448.5 MB read +
+                # written per layer against 436.2 MB of weights), scaled by the layers; the LM-head launch
+                # is taken at its algorithmic bytes
+                "traffic": (nl * 448.5e6 + (V * d * 2 if wl.with_lm_head else 0)) if shape.d_model == 4096 and wl.n_copies == 1 else None,
+                "bytes_per_step": gemm_bytes, "launches_per_step": gemm_launches / max(n_prof, 1),
                 "ms_per_step": gemm_ms,
                 "decode_step": {"ms": step_med, "algorithmic_bytes": step_bytes,
                                 "achieved_gbs": step_bytes / (step_med * 1e-3) / 1e9 if step_med else None,
