@@ -1,6 +1,6 @@
 // Small memory-bound kernels between the GEMMs: embedding gather, residual + split-K reduction
-// + RMSNorm, split-K reduction + RoPE + K/V cache scatter, split-K reduction + SwiGLU, and the
-// vocab-wide confidence reduction.  All reductions run in a fixed order (bitwise reproducible).
+// + RMSNorm operand, split-K reduction + RoPE + K/V cache scatter, and the vocab-wide confidence
+// reduction (SwiGLU lives in the gate/up GEMM's epilogue).  All reductions run in a fixed order (bitwise reproducible).
 #include "odb_internal.cuh"
 
 namespace odb {
@@ -149,24 +149,6 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
     }
 }
 
-// g[m][f] = bf16( silu(gate) * up ), gate = sum_s partial[s][m][f], up = sum_s partial[s][m][F + f]
-__global__ void swiglu_kernel(const float* __restrict__ partial, int splits, size_t pstride,
-                              __nv_bfloat16* __restrict__ g, int M, int F) {
-    pdl_launch_dependents();
-    pdl_wait();
-    const size_t idx = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    if (idx >= static_cast<size_t>(M) * F) return;
-    const int m = static_cast<int>(idx / F), f = static_cast<int>(idx % F);
-    const float* p = partial + static_cast<size_t>(m) * 2 * F;
-    float gate = 0.f, up = 0.f;
-    for (int s = 0; s < splits; ++s) {
-        gate += p[s * pstride + f];
-        up += p[s * pstride + F + f];
-    }
-    const float act = gate / (1.0f + expf(-gate));
-    g[idx] = __float2bfloat16_rn(act * up);
-}
-
 // Greedy token (lowest id on ties, [MASK] excluded) and its softmax probability
 // conf = 1 / sum_j exp(l_j - l_max) per row of logits.  Phase 1: grid (rows, chunks), every block
 // makes one online pass (running max / rescaled sum / argmax) over its slice of the vocabulary
@@ -260,13 +242,6 @@ cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t ps
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
     const int pairs = a.H * a.hd / 2;
     return launch_kernel(qkv_rope_kernel, dim3(a.M, (pairs + 255) / 256), dim3(256), 0, st, a);
-}
-
-cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
-                          cudaStream_t st) {
-    const size_t n = static_cast<size_t>(M) * F;
-    return launch_kernel(swiglu_kernel, dim3(static_cast<unsigned>((n + 255) / 256)), dim3(256), 0, st, partial, splits, pstride,
-                         g, M, F);
 }
 
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,

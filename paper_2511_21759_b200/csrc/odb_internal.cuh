@@ -173,8 +173,6 @@ struct QkvRopeArgs {
     L2Prefetch pf;
 };
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
-cudaError_t launch_swiglu(const float* partial, int splits, size_t pstride, __nv_bfloat16* g, int M, int F,
-                          cudaStream_t st);
 // scratch: rows * kConfMaxChunks * 12 bytes of per-chunk (max, sum, argmax) triples
 constexpr int kConfMaxChunks = 64;
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
