@@ -204,7 +204,15 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
 
 /* ---- test / measurement entry points --------------------------------------------------- */
 
-/* Copies a device buffer of the last forward to the host.  which: 0 logits fp32 [rows][vocab];
+/* Test mode.  By default the LM-head GEMM never writes logits: its epilogue reduces each 128-entry
+ * vocabulary tile to (max, sum of exp, argmax) per row and a small kernel merges the tiles.  With the
+ * dump enabled the LM head writes fp32 logits to the workspace (readable with odb_debug_read 0) and a
+ * separate reduction produces confidence and token; greedy tokens are identical in both modes,
+ * confidences agree to fp32 rounding of a differently ordered sum. */
+int32_t odb_debug_set_logit_dump(odb_session* s, int32_t enable);
+
+/* Copies a device buffer of the last forward to the host.  which: 0 logits fp32 [rows][vocab]
+ * (needs the logit dump);
  * 1 conf fp32 [rows]; 2 tok int32 [rows]; 3 residual stream fp32 [rows][d_model]; 4 q, 5 k,
  * 6 v bf16 [rows][d_model] of the LAST layer; 7 attention output bf16 [rows][d_model];
  * 8 row tokens int32 [rows]; 9 row positions int32 [rows]; 10 row copy ids int32 [rows].

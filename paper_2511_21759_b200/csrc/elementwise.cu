@@ -153,24 +153,6 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
 // conf = 1 / sum_j exp(l_j - l_max) per row of logits.  Phase 1: grid (rows, chunks), every block
 // makes one online pass (running max / rescaled sum / argmax) over its slice of the vocabulary
 // and writes a (max, sum, argmax) triple; phase 2 merges a row's triples in chunk order.
-struct ConfPartial {
-    float m, s;
-    int idx;
-};
-
-__device__ __forceinline__ void conf_merge(float& m, float& s, int& idx, float om, float os, int oi) {
-    if (om == -INFINITY) return;                       // the other side saw nothing
-    if (m == -INFINITY) { m = om; s = os; idx = oi; return; }
-    if (om > m) {
-        s = s * expf(m - om) + os;
-        m = om;
-        idx = oi;
-    } else {
-        s += os * expf(om - m);
-        if (om == m && oi < idx) idx = oi;
-    }
-}
-
 __global__ void __launch_bounds__(256) confidence_partial_kernel(const float* __restrict__ logits, int V, int mask_id,
                                                                  int chunk, ConfPartial* __restrict__ part) {
     __shared__ float sm[8], ss[8];
@@ -210,18 +192,29 @@ __global__ void __launch_bounds__(256) confidence_partial_kernel(const float* __
     }
 }
 
-__global__ void confidence_final_kernel(const ConfPartial* __restrict__ part, int chunks, int rows,
-                                        float* __restrict__ conf, int32_t* __restrict__ tok) {
+// One warp per row: lane l merges triples l, l + 32, ... in ascending order, then the lanes are
+// merged by a fixed shuffle tree (an earlier lane's triple is always the left operand).
+__global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial* __restrict__ part, int chunks, int rows,
+                                                              float* __restrict__ conf, int32_t* __restrict__ tok) {
     pdl_launch_dependents();
     pdl_wait();
-    const int row = blockIdx.x * blockDim.x + threadIdx.x;
-    if (row >= rows) return;
+    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (row >= rows) return;                            // whole warps leave together
     const ConfPartial* p = part + static_cast<size_t>(row) * chunks;
-    float m = p[0].m, s = p[0].s;
-    int idx = p[0].idx;
-    for (int c = 1; c < chunks; ++c) conf_merge(m, s, idx, p[c].m, p[c].s, p[c].idx);
-    conf[row] = 1.0f / s;
-    tok[row] = idx;
+    float m = -INFINITY, s = 0.f;
+    int idx = 0x7fffffff;
+    for (int c = lane; c < chunks; c += 32) conf_merge(m, s, idx, p[c].m, p[c].s, p[c].idx);
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const float om = __shfl_down_sync(0xffffffffu, m, o);
+        const float os = __shfl_down_sync(0xffffffffu, s, o);
+        const int oi = __shfl_down_sync(0xffffffffu, idx, o);
+        if (lane + o < 32) conf_merge(m, s, idx, om, os, oi);
+    }
+    if (lane == 0) {
+        conf[row] = 1.0f / s;
+        tok[row] = idx;
+    }
 }
 
 }  // namespace
@@ -244,6 +237,11 @@ cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
     return launch_kernel(qkv_rope_kernel, dim3(a.M, (pairs + 255) / 256), dim3(256), 0, st, a);
 }
 
+cudaError_t launch_confidence_final(const ConfPartial* part, int chunks, int rows, float* conf, int32_t* tok,
+                                    cudaStream_t st) {
+    return launch_kernel(confidence_final_kernel, dim3((rows + 3) / 4), dim3(128), 0, st, part, chunks, rows, conf, tok);
+}
+
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
                               void* scratch, cudaStream_t st) {
     // enough blocks to fill the machine; a chunk is a multiple of 256 so that threads stay coalesced
@@ -255,8 +253,7 @@ cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id,
     cudaError_t e = launch_kernel(confidence_partial_kernel, dim3(rows, chunks), dim3(256), 0, st, logits, V, mask_id, chunk,
                                   part);
     if (e != cudaSuccess) return e;
-    return launch_kernel(confidence_final_kernel, dim3((rows + 127) / 128), dim3(128), 0, st,
-                         static_cast<const ConfPartial*>(part), chunks, rows, conf, tok);
+    return launch_confidence_final(part, chunks, rows, conf, tok, st);
 }
 
 }  // namespace odb

@@ -163,7 +163,7 @@ struct alignas(8) GemmShared {
 // projection bf16(h * gain), and this slice's contribution to sum(h^2) per activation row.  The CTA
 // that arrives last at the grid's counter turns the per-slice sums into 1/rms per row (fixed order).
 // No partial sums go through HBM and no RMSNorm kernel is needed after this GEMM.
-constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_RESIDUAL = 2;
+constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_RESIDUAL = 2, EPI_CONF = 3;
 
 __device__ __forceinline__ uint32_t dsmem_addr(const void* p, uint32_t cta_rank) {
     uint32_t r;
@@ -185,7 +185,8 @@ template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
             float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, const float* __restrict__ row_scale,
-            ResidualEpilogue re, int M, int N, int nkb_total, int nkb_per_split, int stages, int l2_prefetch,
+            ResidualEpilogue re, ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
+            int l2_prefetch,
             int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
@@ -329,6 +330,58 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                         if (n < N && m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]) * sc;
                     }
                 }
+            }
+        } else if constexpr (EPI == EPI_CONF) {
+            // LM head fused with the confidence reduction: the logits of this tile (128 vocabulary
+            // entries x BN rows) never leave the SM.  They are transposed through shared memory so that
+            // four threads scan one row's 128 logits (32 each, ascending ids, online max / sum of exp /
+            // argmax); the four are merged in id order and one (max, sum, argmax) triple per (row, tile)
+            // is stored.  The RMSNorm scalar of the row is applied first; [MASK] and padding are skipped.
+            float* xch = reinterpret_cast<float*>(tiles);           // [32 rows][129]
+            const int t = threadIdx.x - 64;                            // 0..127
+            const int n_tiles = gridDim.x;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                uint32_t v[32];
+                if (ok) {
+                    tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
+                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                }
+#pragma unroll
+                for (int j = 0; j < 32; ++j) xch[j * 129 + q * 32 + lane] = ok ? __uint_as_float(v[j]) : 0.f;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int m_l = t >> 2, part = t & 3;
+                const int m = m0 + c * 32 + m_l;
+                const float sc = (row_scale && m < M) ? row_scale[m] : 1.0f;
+                float mx = -INFINITY, sum = 0.f;
+                int idx = 0x7fffffff;
+#pragma unroll 8
+                for (int i = 0; i < 32; ++i) {
+                    const int n = n0 + part * 32 + i;
+                    const float l = xch[m_l * 129 + part * 32 + i] * sc;
+                    if (n < N && n != ce.mask_id) {
+                        if (l > mx) {
+                            sum = sum * expf(mx - l) + 1.0f;            // first element: 0 * exp(-inf) + 1
+                            mx = l;
+                            idx = n;
+                        } else {
+                            sum += expf(l - mx);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int o = 1; o < 4; o <<= 1) {
+                    const float om = __shfl_down_sync(0xffffffffu, mx, o, 4);
+                    const float os = __shfl_down_sync(0xffffffffu, sum, o, 4);
+                    const int oi = __shfl_down_sync(0xffffffffu, idx, o, 4);
+                    if (part + o < 4) conf_merge(mx, sum, idx, om, os, oi);
+                }
+                if (ok && part == 0 && m < M) {
+                    ConfPartial p;
+                    p.m = mx; p.s = sum; p.idx = idx;
+                    ce.part[static_cast<size_t>(m) * n_tiles + blockIdx.x] = p;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
             }
         } else if constexpr (EPI == EPI_RESIDUAL) {
             // park the accumulator tile in shared memory as acc[m][n] (n contiguous): the ring is free
@@ -633,11 +686,11 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
         attr[1].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = pdl_enabled() ? 2 : 1;
-        return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.residual, a.M,
-                                  a.N, nkb_total, nkb_per_split, stages, 0, a.status);
+        return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.residual, a.conf,
+                                  a.M, a.N, nkb_total, nkb_per_split, stages, 0, a.status);
     } else {
         return launch_kernel(gemm_kernel<BN, EPI>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
-                             a.row_scale, a.residual, a.M, a.N, nkb_total, nkb_per_split, stages,
+                             a.row_scale, a.residual, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
                              pdl_enabled() ? l2_prefetch : 0, a.status);
     }
 }
@@ -748,6 +801,10 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
     if (a.act_out) {
         if (a.splits != 1) return cudaErrorInvalidValue;
         return launch_epi<EPI_SWIGLU>(a, tmx, bn, st);
+    }
+    if (a.conf.part) {
+        if (a.splits != 1) return cudaErrorInvalidValue;
+        return launch_epi<EPI_CONF>(a, tmx, bn, st);
     }
     return launch_epi<EPI_PARTIAL>(a, tmx, bn, st);
 }

@@ -92,7 +92,10 @@ Layout make_layout(const odb_config& c) {
     L.logits = take(c.with_lm_head ? 4 * L.lm_chunk * c.vocab : 256);
     L.conf = take(4 * L.rows);
     L.tok = take(4 * L.rows);
-    L.conf_part = take(12 * L.lm_chunk * kConfMaxChunks);
+    {
+        const size_t lm_tiles = (static_cast<size_t>(c.vocab) + 127) / 128;
+        L.conf_part = take(12 * L.lm_chunk * (lm_tiles > static_cast<size_t>(kConfMaxChunks) ? lm_tiles : kConfMaxChunks));
+    }
     L.part_o = take(4 * L.attn_rows * d);
     L.part_ml = take(4 * L.attn_rows * c.n_heads * 2);
     L.total = off;
@@ -125,6 +128,7 @@ struct odb_session {
     int* pinned_status;
     int phase;            // 0 idle, 1 refresh enqueued, 2 accepted, 3 step enqueued
     int last_rows, last_lm_rows;
+    bool dump_logits;     // test mode: the LM head writes fp32 logits (odb_debug_read 0) instead of fusing the reduction
     // launch accounting: kernels launched per kind since the last read; with profiling on, a CUDA
     // event pair brackets every launch so that per-kind device time can be summed afterwards
     long long launches[ODB_PROFILE_KINDS];
@@ -248,6 +252,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->L = L;
     s->phase = 0;
     s->last_rows = s->last_lm_rows = 0;
+    s->dump_logits = false;
     memset(s->launches, 0, sizeof(s->launches));
     s->profiling = false;
     s->ev_used = 0;
@@ -578,10 +583,29 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
             ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
                                                             rows, d, c.rms_eps, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
         }
-        int sp = 1;
-        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, &sp, scale));
-        ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0, s->at<int32_t>(L.tok) + r0,
-                                                             s->ws + L.conf_part, st));
+        if (s->dump_logits) {
+            int sp = 1;
+            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, &sp, scale));
+            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0,
+                                                                 s->at<int32_t>(L.tok) + r0, s->ws + L.conf_part, st));
+        } else {
+            // LM head fused with the confidence reduction: per (row, vocabulary tile) statistics instead
+            // of logits, merged per row in tile order
+            GemmArgs ga;
+            ga.tmap_w = m->tm_lm;
+            ga.x = x;
+            ga.partial = nullptr;
+            ga.act_out = nullptr;
+            ga.row_scale = scale;
+            ga.conf.part = reinterpret_cast<ConfPartial*>(s->ws + L.conf_part);
+            ga.conf.mask_id = c.mask_id;
+            ga.M = rows; ga.N = c.vocab; ga.K = d;
+            ga.splits = 1;
+            ga.status = status;
+            ODB_LAUNCH(ODB_KIND_GEMM, launch_gemm(ga, st));
+            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence_final(ga.conf.part, (c.vocab + 127) / 128, rows, s->at<float>(L.conf) + r0,
+                                                                       s->at<int32_t>(L.tok) + r0, st));
+        }
     }
     return ODB_OK;
 }
@@ -689,11 +713,17 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap, in
         case 10: off = L.row_copy; bytes = 4 * M; break;
         default: return ODB_ERR_ARG;
     }
-    if (which == 0 && !c.with_lm_head) return ODB_ERR_STATE;
+    if (which == 0 && (!c.with_lm_head || !s->dump_logits)) return ODB_ERR_STATE;
     if (cap < bytes) return ODB_ERR_WORKSPACE;
     ODB_CUDA(cudaStreamSynchronize(s->st));
     ODB_CUDA(cudaMemcpy(host, s->ws + off, bytes, cudaMemcpyDeviceToHost));
     *rows = static_cast<int32_t>(n);
+    return ODB_OK;
+}
+
+int32_t odb_debug_set_logit_dump(odb_session* s, int32_t enable) {
+    if (!s) return ODB_ERR_ARG;
+    s->dump_logits = enable != 0;
     return ODB_OK;
 }
 

@@ -129,12 +129,42 @@ struct ResidualEpilogue {
     float eps = 0.f;
 };
 
+// Softmax statistics of a slice of one row of logits: running max, sum of exp(l - max), argmax
+// (lowest id on ties; [MASK] excluded by the producer).  Merged in a fixed order.
+struct ConfPartial {
+    float m, s;
+    int idx;
+};
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void conf_merge(float& m, float& s, int& idx, float om, float os, int oi) {
+    if (om == -INFINITY) return;                       // the other side saw nothing
+    if (m == -INFINITY) { m = om; s = os; idx = oi; return; }
+    if (om > m) {
+        s = s * expf(m - om) + os;
+        m = om;
+        idx = oi;
+    } else {
+        s += os * expf(om - m);
+        if (om == m && oi < idx) idx = oi;
+    }
+}
+#endif
+
+// Epilogue of the LM-head projection: instead of logits, the softmax statistics of each 128-feature
+// tile per activation row; see EPI_CONF in gemm_tcgen05.cu.  part non-null selects it.
+struct ConfEpilogue {
+    ConfPartial* part = nullptr;   // [M][n_tiles]
+    int mask_id = -1;              // feature excluded from the statistics
+};
+
 // Weight-streaming GEMM: partial[s][M][N] (fp32) = x[M][K_s] * w[N][K_s]^T for each K split s.
 struct GemmArgs {
     CUtensorMap tmap_w;    // packed bf16 weight tiles [n_tile * k_blocks][128][64], 128B swizzle
     const void* x;         // bf16 [M][K] device
     float* partial;        // fp32 [splits][M][N]
     __nv_bfloat16* act_out; // non-null: gate/up GEMM with the SwiGLU epilogue, writes bf16 [M][N = F]; splits == 1
+    ConfEpilogue conf;                  // conf.part non-null: LM head fused with the confidence statistics, splits == 1
     ResidualEpilogue residual;          // residual.h non-null: cluster split-K with the fused residual epilogue
     const float* row_scale = nullptr;   // per activation row m: the output is multiplied by row_scale[m]
                                         // (the 1/rms of an RMSNorm folded behind the projection); needs splits == 1
@@ -173,6 +203,9 @@ struct QkvRopeArgs {
     L2Prefetch pf;
 };
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
+cudaError_t launch_confidence_final(const ConfPartial* part, int chunks, int rows, float* conf, int32_t* tok,
+                                    cudaStream_t st);
+
 // scratch: rows * kConfMaxChunks * 12 bytes of per-chunk (max, sum, argmax) triples
 constexpr int kConfMaxChunks = 64;
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,

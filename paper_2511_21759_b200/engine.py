@@ -173,6 +173,10 @@ class Session:
                 "odb_unmask_accept")
         return self._results
 
+    def set_logit_dump(self, enable: bool):
+        """Test mode: the LM head writes fp32 logits (debug_read("logits")) instead of fusing the reduction."""
+        B.check(B.lib().odb_debug_set_logit_dump(self.handle, 1 if enable else 0), "odb_debug_set_logit_dump")
+
     def profile(self, enable: bool):
         B.check(B.lib().odb_session_profile(self.handle, 1 if enable else 0), "odb_session_profile")
 

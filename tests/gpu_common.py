@@ -68,6 +68,7 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
     oracle's decision margin must be below the confidence error measured in that iteration (a
     near-tie); these are counted and returned, never hidden.  The GPU's decision then advances
     both sides.  Returns a stats dict."""
+    sess.set_logit_dump(check_logits)                   # logits are only materialised in the test mode
     shape_mask, eos = om.mask_id, om.eos_id
     Bk, tau = op.block_len, op.accept_threshold
     k_ranks = {1: 0, 4: 2, 8: 4}[op.n_copies]

@@ -18,6 +18,7 @@ def _setup(shape, P, L, *, max_copies=8, seed=0, with_lm_head=True, block=16):
     sess = E.Session(gm)
     x0 = synth.sequence(seed, 0, P, L, shape)
     sess.set_sequence(0, x0, P)
+    sess.set_logit_dump(True)
     return E, om, gm, sess, x0
 
 
@@ -71,3 +72,29 @@ def test_one_layer_intermediates():
     h = sess.debug_read("hidden")
     assert np.abs(h - hid).max() <= 2e-2 * np.sqrt((hid * hid).mean())
     sess.close(); gm.close()
+
+
+@requires_gpu
+def test_fused_lm_head_confidence_equals_logit_dump():
+    """The product path never writes logits: the LM-head GEMM's epilogue reduces every vocabulary tile
+    to (max, sum of exp, argmax).  Same state, both modes: identical greedy tokens, confidences equal to
+    fp32 rounding of a differently ordered sum; the logits buffer is refused when not dumped."""
+    from paper_2511_21759_b200 import binding as B
+    for shape in (synth.TINY, synth.TINY_PEAKY):
+        P, L = 64, 64
+        E, om, gm, sess, x0 = _setup(shape, P, L)
+        p = E.DecodeParams(block_len=16)
+        sess.set_logit_dump(True)
+        sess.refresh_prefill(p, 0)
+        conf_d, tok_d = sess.debug_read("conf"), sess.debug_read("tok")
+        sess.unmask_accept(p, True)
+        sess.set_sequence(0, x0, P)
+        sess.set_logit_dump(False)
+        sess.refresh_prefill(p, 0)
+        conf_f, tok_f = sess.debug_read("conf"), sess.debug_read("tok")
+        with pytest.raises(B.OdbError) as e:
+            sess.debug_read("logits")
+        assert e.value.status == B.ODB_ERR_STATE
+        assert np.array_equal(tok_d, tok_f)
+        assert np.allclose(conf_d, conf_f, rtol=2e-6, atol=0)
+        sess.close(); gm.close()

@@ -38,6 +38,7 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=T, max_block=Bk, max_copies=1)
     sess = E.Session(gm)
     sess.set_sequence(0, x0, P)
+    sess.set_logit_dump(True)
     gp = E.DecodeParams(block_len=Bk, n_copies=1)
     sess.refresh_prefill(gp, 0)
     g_logits = sess.debug_read("logits")

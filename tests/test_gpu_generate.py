@@ -59,9 +59,11 @@ def test_generate_matches_oracle(wl):
 
 
 @requires_gpu
-@pytest.mark.parametrize("wl_name,tol", [("cfg1_tiny", 2e-2), ("cfg1_tiny_c4", 2e-2), ("peaky_c1", 4e-2),
-                                         ("peaky_c4", 4e-2), ("peaky_c8", 4e-2)])
-def test_lockstep_generate(wl_name, tol):
+@pytest.mark.parametrize("wl_name,tol,fused", [("cfg1_tiny", 2e-2, False), ("cfg1_tiny_c4", 2e-2, False),
+                                               ("peaky_c1", 4e-2, False), ("peaky_c4", 4e-2, False),
+                                               ("peaky_c8", 4e-2, False), ("cfg1_tiny_c4", 2e-2, True),
+                                               ("peaky_c8", 4e-2, True)])
+def test_lockstep_generate(wl_name, tol, fused):
     """Whole generation in lock step: numerics every iteration, control bit-exact on the GPU's own
     confidences, oracle-side decisions equal except at measured near-ties.  The sharp-logit model
     amplifies bf16 rounding (the oracle's own fp32 and fp64 runs differ by 0.8 of the 2e-2 bound
@@ -75,7 +77,10 @@ def test_lockstep_generate(wl_name, tol):
     x0 = synth.sequence(0, 0, wl.prompt_len, wl.gen_len, wl.shape)
     sess.set_sequence(0, x0, wl.prompt_len)
     kw = dict(block_len=wl.block_len, n_copies=wl.n_copies)
-    st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=tol)
+    # fused: the product path (LM head fused with the confidence reduction, no logits); otherwise the
+    # test mode that also materialises the logits for the element-wise comparison
+    st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=tol,
+                           check_logits=not fused)
     assert sess.status() == 0
     assert np.array_equal(sess.get_tokens(0), st["tokens_final"])
     assert (st["tokens_final"][wl.prompt_len:] != wl.shape.mask_id).all() and st["tokens"] == wl.gen_len
@@ -93,7 +98,7 @@ def test_lockstep_with_cluster_residual_epilogue():
     import os, subprocess, sys
     engine()
     code = ("import sys; sys.path.insert(0, 'tests'); import test_gpu_generate as t; "
-            "t.test_lockstep_generate('peaky_c4', 4e-2); t.test_lockstep_generate('cfg1_tiny', 2e-2)")
+            "t.test_lockstep_generate('peaky_c4', 4e-2, False); t.test_lockstep_generate('cfg1_tiny', 2e-2, False)")
     env = dict(os.environ, ODB_CLUSTER_EPILOGUE="1")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=600)
