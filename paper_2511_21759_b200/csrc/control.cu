@@ -81,6 +81,22 @@ __device__ int step_rows_of(const SeqState* st) {
     return st->stage2 ? B + (st->n_copies - 1) * st->n_masked : st->n_copies * B;
 }
 
+// Number of StepTiles of a sequence's next step: copies packed in order into items of <= 8 slabs.
+__host__ __device__ int step_tiles_of_counts(int n_copies, int rows_copy0, int rows_other) {
+    int tiles = 0, slabs = 0;
+    for (int cp = 0; cp < n_copies; ++cp) {
+        const int need = ((cp == 0 ? rows_copy0 : rows_other) + 15) / 16;
+        if (slabs == 0 || slabs + need > 8) { ++tiles; slabs = 0; }
+        slabs += need;
+    }
+    return tiles;
+}
+
+__device__ int step_tiles_of(const SeqState* st) {
+    const int B = st->e - st->s;
+    return step_tiles_of_counts(st->n_copies, B, st->stage2 ? st->n_masked : B);
+}
+
 __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id) {
     const int seq = blockIdx.x;
     SeqState* st = c.state + seq;
@@ -130,6 +146,46 @@ __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id)
     }
     st->n_rows = row - st->row0;
     st->lm_row0 = st->row0;
+    // attention work items that share the cached K/V among copies: copies are packed, in order, into
+    // items of at most 8 slabs of 16 rows (the host counts them with the same rule, step_tiles_of)
+    int stile = 0;
+    for (int j = 0; j < seq; ++j) {
+        const SeqState* o = c.state + j;
+        if (!o->active || o->n_masked <= 0) continue;
+        stile += step_tiles_of(o);
+    }
+    StepTile cur;
+    int have = 0;
+    auto add_src = [&](int cp) {
+        for (int i = 0; i < cur.n_src; ++i)
+            if (cur.src_copy[i] == cp) return;
+        cur.src_copy[cur.n_src] = cp;
+        cur.src_row0[cur.n_src] = st->copy_row0[cp];
+        cur.src_n[cur.n_src] = st->copy_nrows[cp];
+        ++cur.n_src;
+    };
+    auto flush = [&]() {
+        if (st->stage2) add_src(0);   // copy 0's decoded rows are visible to every speculative copy
+        c.step_tiles[stile++] = cur;
+        have = 0;
+    };
+    for (int cp = 0; cp < st->n_copies; ++cp) {
+        const int slabs = (st->copy_nrows[cp] + 15) / 16;
+        if (have && cur.n_slabs + slabs > 8) flush();
+        if (!have) {
+            cur.seq = seq; cur.cA = s; cur.cB0 = e; cur.cB1 = st->T;
+            cur.n_slabs = 0; cur.n_src = 0; cur.stage2 = st->stage2;
+            have = 1;
+        }
+        for (int k = 0; k < slabs; ++k) {
+            cur.slab_copy[cur.n_slabs] = cp;
+            cur.slab_row0[cur.n_slabs] = st->copy_row0[cp] + 16 * k;
+            cur.slab_n[cur.n_slabs] = min(16, st->copy_nrows[cp] - 16 * k);
+            ++cur.n_slabs;
+        }
+        add_src(cp);
+    }
+    if (have) flush();
 }
 
 // Accept rule (Section 3, Observation 3): every masked position whose confidence exceeds tau
@@ -315,6 +371,10 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
 }
 
 }  // namespace
+
+int step_tiles_host(int n_copies, int rows_copy0, int rows_other) {
+    return step_tiles_of_counts(n_copies, rows_copy0, rows_other);
+}
 
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st) {
     build_step_rows_kernel<<<batch, 32, 0, st>>>(c, batch, mask_id);

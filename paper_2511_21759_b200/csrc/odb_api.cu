@@ -46,7 +46,7 @@ int32_t check_config(const odb_config* c) {
 // odb_session_create so that both always agree.
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
-    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf;
+    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, step_tile_buf;
     size_t h, a, inv, sumsq, counter, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
     size_t total;
 };
@@ -78,6 +78,7 @@ Layout make_layout(const odb_config& c) {
     L.row_flags = take(4 * L.rows);
     L.lm_rows = take(4 * L.rows);
     L.tile_buf = take(sizeof(QTile) * L.tiles);
+    L.step_tile_buf = take(sizeof(StepTile) * static_cast<size_t>(c.max_batch) * c.max_copies);
     L.h = take(4 * L.rows * d);
     L.a = take(2 * L.rows * d);
     L.inv = take(4 * L.rows);
@@ -293,6 +294,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     cb.row_flags = s->at<int32_t>(L.row_flags);
     cb.lm_rows = s->at<int32_t>(L.lm_rows);
     cb.tiles = s->at<QTile>(L.tile_buf);
+    cb.step_tiles = s->at<StepTile>(L.step_tile_buf);
     cb.conf = s->at<float>(L.conf);
     cb.tok = s->at<int32_t>(L.tok);
     cb.results = s->at<odb_result>(L.results);
@@ -413,7 +415,7 @@ struct LaunchScope {
 };
 
 // One forward over the M rows of the row table already built on the device.
-int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) {
+int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0) {
     const odb_model* m = s->m;
     const odb_config& c = m->cfg;
     const Layout& L = s->L;
@@ -524,6 +526,22 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         qa.layer = l; qa.n_layers = c.n_layers; qa.H = H; qa.hd = hd; qa.max_seq = c.max_seq; qa.M = M;
         qa.pf = hint_of(m->p_o[l], o_bytes, 0);
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_qkv_rope(qa, st));
+        if (n_step_tiles > 0) {
+            // several copies: one work item serves all copies of a block, cached K/V loaded once
+            StepAttnArgs sa;
+            sa.tiles = s->cb.step_tiles; sa.n_tiles = n_step_tiles;
+            sa.q = q; sa.k = k; sa.v = v; sa.cache = s->kv; sa.row_flags = s->cb.row_flags; sa.o = o;
+            sa.part_o = s->at<float>(L.part_o); sa.part_ml = s->at<float>(L.part_ml);
+            sa.layer = l; sa.n_layers = c.n_layers; sa.H = H; sa.hd = hd; sa.max_seq = c.max_seq; sa.M = M;
+            int sks = (2 * 148 + n_step_tiles * H - 1) / (n_step_tiles * H) + 1;
+            if (sks > 8) sks = 8;
+            if (static_cast<size_t>(sks) * M > L.attn_rows) sks = static_cast<int>(L.attn_rows / M);
+            if (sks < 2) sks = 2;
+            sa.ksplit = sks;
+            sa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
+            ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
+            ++s->launches[ODB_KIND_ATTENTION];
+        } else {
         AttnArgs aa;
         aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
         aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
@@ -532,6 +550,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache) 
         aa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
         ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention(aa, st));
         if (ks > 1) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
+        }
         if (cs_o) {
             ODB_LAUNCH(ODB_KIND_GEMM, residual_gemm(m->tm_o[l], o, d, cs_o, m->norm2[l]));
         } else {
@@ -651,18 +670,22 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
     if (!s || !p) return ODB_ERR_ARG;
     const odb_config& c = s->m->cfg;
     if (s->phase != 2) return ODB_ERR_STATE;
-    int M = 0, n_tiles = 0;
+    int M = 0, n_tiles = 0, n_step_tiles = 0;
+    bool multi = false;
     for (int i = 0; i < c.max_batch; ++i) {
         const SeqState& st = s->mirror[i];
         if (!st.active || st.n_masked <= 0) continue;
         const int B = st.e - st.s;
         M += st.stage2 ? B + (st.n_copies - 1) * st.n_masked : st.n_copies * B;
         n_tiles += st.n_copies;
+        if (st.n_copies > 1) multi = true;
+        n_step_tiles += step_tiles_host(st.n_copies, B, st.stage2 ? st.n_masked : B);
     }
+    if (!multi || static_cast<size_t>(2) * M > s->L.attn_rows) n_step_tiles = 0;   // plain kernel for single copies
     if (M == 0) return ODB_ERR_STATE;
     if (static_cast<size_t>(M) > s->L.rows) return ODB_ERR_SHAPE;
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
-    int32_t rc = forward(s, M, c.with_lm_head ? M : 0, n_tiles, false);
+    int32_t rc = forward(s, M, c.with_lm_head ? M : 0, n_tiles, false, n_step_tiles);
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
     s->last_lm_rows = M;

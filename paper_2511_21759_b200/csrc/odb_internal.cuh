@@ -109,6 +109,21 @@ struct QTile {
     int32_t f1, n1;
 };
 
+// A decode-step attention work item: up to 8 slabs of 16 query rows, each slab inside one block copy
+// of one sequence, all sharing the sequence's cached keys (positions [0, cA) and [cB0, cB1)) - the
+// cached K/V tiles are loaded once for every copy in the item.  Fresh keys: the rows of the copies
+// listed in src_*; a slab of copy c sees source copy c (all rows) and, in the decoded-share layout,
+// source copy 0 (only rows flagged kRowDecoded).
+struct StepTile {
+    int32_t seq;
+    int32_t cA, cB0, cB1;
+    int32_t n_slabs;
+    int32_t slab_copy[8], slab_row0[8], slab_n[8];   // copy id, first global row, valid rows (<= 16)
+    int32_t n_src;
+    int32_t src_copy[ODB_MAX_COPIES], src_row0[ODB_MAX_COPIES], src_n[ODB_MAX_COPIES];
+    int32_t stage2;
+};
+
 constexpr int kRowDecoded = 1;   // row_flags bit: the row's position is decoded in the committed state
 
 // ---------------------------------------------------------------------------------------
@@ -223,6 +238,19 @@ struct AttnArgs {
 };
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
 
+// Decode-step attention over StepTiles (copies of a block share the cached K/V loads).
+struct StepAttnArgs {
+    const StepTile* tiles; int n_tiles;
+    const __nv_bfloat16 *q, *k, *v;       // fresh rows [M][H*hd]
+    const __nv_bfloat16* cache;
+    const int32_t* row_flags;
+    __nv_bfloat16* o;
+    float* part_o; float* part_ml;        // split workspaces, merged by attention_combine
+    int layer, n_layers, H, hd, max_seq, M, ksplit;   // ksplit >= 2: the last split handles the fresh keys
+    L2Prefetch pf;
+};
+cudaError_t launch_step_attention(const StepAttnArgs& a, cudaStream_t st);
+
 // control kernels (control.cu)
 struct ControlBuffers {
     SeqState* state;          // [batch]
@@ -231,6 +259,7 @@ struct ControlBuffers {
     int32_t* row_tok; int32_t* row_pos; int32_t* row_seq; int32_t* row_copy; int32_t* row_flags;
     int32_t* lm_rows;         // rows whose logits are needed
     QTile* tiles;
+    StepTile* step_tiles;     // decode steps with more than one copy
     const float* conf; const int32_t* tok;   // outputs of the last forward, per logit row
     odb_result* results;      // [batch] device copy
 };
@@ -238,6 +267,7 @@ struct ControlBuffers {
 cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index, int block_len,
                                       cudaStream_t st);
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st);
+int step_tiles_host(int n_copies, int rows_copy0, int rows_other);   // StepTiles of one sequence's step
 // dry: model without LM head; commits nothing, only lays out the next step
 cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
                           int mask_id, int eos_id, int dry, cudaStream_t st);
