@@ -203,7 +203,7 @@ def run_cuda(args, wl):
     shape = wl.shape
     T = wl.prompt_len + wl.gen_len
     gm = E.Model.from_synth(shape, seed=0, device=f"cuda:{local}", with_lm_head=wl.with_lm_head, max_batch=wl.batch,
-                            max_seq=T, max_block=wl.block_len, max_copies=max(wl.n_copies, 1))
+                            max_seq=T, max_block=wl.block_len, max_copies=4 if args.modes else max(wl.n_copies, 1))
     sess = E.Session(gm)
     params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies, accept_threshold=wl.accept_threshold,
                             truncate_threshold=wl.truncate_threshold)
@@ -325,7 +325,9 @@ def run_cuda(args, wl):
     gemm_ms = ms_step["gemm"] / max(n_prof, 1)                # per decode step
     achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else None
     step_med = float(np.median(step_ms)) if step_ms else None
-    roofline = {"bound": "hbm", "kernel": "gemm_kernel<32> (tcgen05 weight-streaming GEMM), all launches of one decode step",
+    rows = wl.batch * wl.block_len * wl.n_copies
+    bn = 32 if rows <= 32 else 64 if rows <= 64 else 128
+    roofline = {"bound": "hbm", "kernel": f"gemm_kernel<{bn}, *> (tcgen05 weight-streaming GEMM), all launches of one decode step",
                 "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                 "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
                 # DRAM bytes of the GEMM launches of one decode step: ncu capture of the four per-layer
@@ -350,6 +352,27 @@ def run_cuda(args, wl):
                     "d2h_bytes_per_step": 4 * T * wl.batch},
             "gpu_launches": int(sum(launches.values())),
             "roofline": roofline}
+    if args.modes and world == 1 and wl.batch == 1:
+        # the three systems of the paper's tables on this workload's shapes, whole response each:
+        # cache-less baseline, DualCache block decoding, and the full method (speed relative to the first two)
+        modes = {}
+        for mode in ("vanilla", "fast_dllm", "odb"):
+            mp, cache_blocks = E.mode_settings(mode, wl.block_len, n_copies=4, accept_threshold=wl.accept_threshold)
+            reset()
+            torch.cuda.synchronize()
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0.record(sess.stream)
+            _, mtrace = E.generate(sess, mp, cache_blocks=cache_blocks)
+            m1.record(sess.stream)
+            torch.cuda.synchronize()
+            sess.set_active(0, True)
+            cnt = E.trace_counters(mtrace)
+            mms = m0.elapsed_time(m1)
+            modes[mode] = dict(cnt, ms=mms, tokens_per_s=cnt["tokens"] / (mms * 1e-3))
+        for mode in modes:
+            modes[mode]["speed_vs_vanilla"] = modes[mode]["tokens_per_s"] / modes["vanilla"]["tokens_per_s"]
+            modes[mode]["speed_vs_fast_dllm"] = modes[mode]["tokens_per_s"] / modes["fast_dllm"]["tokens_per_s"]
+        line["modes"] = modes
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             r = oracle_sample(wl)
@@ -436,6 +459,8 @@ def main():
     ap.add_argument("--workload", default="cfg3_8b_c1")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--modes", action="store_true",
+                    help="also run the whole response as cache-less baseline / DualCache block decoding / full method")
     args = ap.parse_args()
     import synth
     wl = synth.WORKLOADS[args.workload]

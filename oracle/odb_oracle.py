@@ -422,13 +422,16 @@ def use_stage2(params: DecodeParams, B: int, n_decoded: int) -> bool:
 
 def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, faithful=True,
              dtype=np.float64, length_schedule: Optional[Callable[[int, int], Optional[int]]] = None,
-             max_iters: Optional[int] = None):
+             max_iters: Optional[int] = None, cache_blocks: bool = True):
     """Whole-response generation: per block a refresh (itself a decoding iteration restricted
     to the block), adaptive length prediction, then block steps until the block is full.
 
     x0: prompt ids followed by [MASK]s.  `length_schedule(block_index, gen_len)` may return a
     shorter response length at a refresh (same lever as ALP; drives the ragged batch
-    workload).  Returns (tokens [P + final length], trace list of per-iteration dicts).
+    workload).  cache_blocks=False is the cache-less baseline of Section 1 (bidirectional
+    attention without a KV cache: every iteration re-executes the whole prefill), i.e. every
+    iteration of a block is a refresh and no block step is ever taken.
+    Returns (tokens [P + final length], trace list of per-iteration dicts).
     """
     x = np.array(x0, dtype=np.int64)
     T = len(x)
@@ -459,6 +462,10 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
                       "accepted": [(int(s + i), int(tok_r[i])) for i in np.flatnonzero(acc)],
                       "chain": [0], "margin": decision_margin(conf_r[:B], masked, tau, k_ranks + 1)})
         last_conf, last_tok = conf_r[:B], tok_r[:B]
+        if not cache_blocks:
+            if not (x[s:e] == model.mask_id).any():
+                b += 1
+            continue
         while (x[s:e] == model.mask_id).any():
             if max_iters is not None and len(trace) >= max_iters:
                 break
@@ -480,3 +487,30 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             last_conf, last_tok = conf[last], tok[last]
         b += 1
     return x.astype(np.int32), trace
+
+
+# The three systems the paper compares (Tables 2 and 3), as settings of `generate`:
+# the cache-less dLLM baseline (one token per full forward: no confidence passes a threshold of 1),
+# Fast-dLLM (DualCache block decoding with threshold acceptance, fixed length, no speculation),
+# and the paper's method (adaptive length prediction + jump-share speculation).
+def mode_settings(mode: str, block_len: int, n_copies: int = 4, accept_threshold: float = 0.9):
+    """Returns (DecodeParams, cache_blocks) for "vanilla", "fast_dllm" or "odb"."""
+    if mode == "vanilla":
+        return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=1.0, alp=False), False
+    if mode == "fast_dllm":
+        return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=accept_threshold, alp=False), True
+    if mode == "odb":
+        return DecodeParams(block_len=block_len, n_copies=n_copies, accept_threshold=accept_threshold, alp=True), True
+    raise ValueError(mode)
+
+
+def trace_counters(trace) -> dict:
+    """Counters of Section 5.3: NFE = forward passes (refreshes and block steps alike); Eff_NFE =
+    effective state changes of the unmasking sequence = links of the jump chains (equal to NFE
+    without speculation); tokens = positions committed."""
+    nfe = len(trace)
+    eff = sum(len(t["chain"]) for t in trace)
+    tokens = sum(len(t["accepted"]) for t in trace)
+    return {"nfe": nfe, "eff_nfe": eff, "tokens": tokens, "refreshes": sum(t["kind"] == "refresh" for t in trace),
+            "tokens_per_nfe": tokens / nfe if nfe else 0.0}
+

@@ -533,7 +533,10 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             sa.q = q; sa.k = k; sa.v = v; sa.cache = s->kv; sa.row_flags = s->cb.row_flags; sa.o = o;
             sa.part_o = s->at<float>(L.part_o); sa.part_ml = s->at<float>(L.part_ml);
             sa.layer = l; sa.n_layers = c.n_layers; sa.H = H; sa.hd = hd; sa.max_seq = c.max_seq; sa.M = M;
-            int sks = (2 * 148 + n_step_tiles * H - 1) / (n_step_tiles * H) + 1;
+            // one work item per SM at most (measured on 4 copies of a 32-token block, 32 heads: 4 key splits
+            // beat 3, 6 and 8: every split writes and re-reads a full fp32 output tile)
+            int sks = 148 / (n_step_tiles * H);
+            if (ks_env > 0) sks = ks_env;
             if (sks > 8) sks = 8;
             if (static_cast<size_t>(sks) * M > L.attn_rows) sks = static_cast<int>(L.attn_rows / M);
             if (sks < 2) sks = 2;

@@ -235,7 +235,7 @@ def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> 
 
 def generate(sess: Session, params: DecodeParams, *,
              length_schedule: Optional[Callable[[int, int, int], Optional[int]]] = None,
-             max_iters: Optional[int] = None):
+             max_iters: Optional[int] = None, cache_blocks: bool = True):
     """Runs every sequence set on the session to completion.
 
     Per iteration: the sequences standing at a block boundary are refreshed and accepted
@@ -243,7 +243,9 @@ def generate(sess: Session, params: DecodeParams, *,
     step and its accept.  length_schedule(seq, block_index, gen_len) may return a shorter
     response length, applied between the refresh and its accept (the lever adaptive length
     prediction also pulls).  Returns ({seq: tokens}, trace); trace is a list of per-call dicts
-    {"kind", "seqs": {seq: {"accepted", "chain", "masks_left", "gen_len", "block"}}}."""
+    {"kind", "seqs": {seq: {"accepted", "chain", "masks_left", "gen_len", "block"}}}.
+    cache_blocks=False is the cache-less baseline (Section 1): every iteration of a block is a
+    refresh prefill and no block step is taken."""
     seqs = sorted(sess.gen_len)
     block = {i: 0 for i in seqs}
     need_refresh = {i: True for i in seqs}
@@ -285,7 +287,7 @@ def generate(sess: Session, params: DecodeParams, *,
             touched = todo
         for i in touched:
             sess.gen_len[i] = res[i].gen_len
-            need_refresh[i] = False
+            need_refresh[i] = not cache_blocks
             if res[i].masks_left == 0:
                 block[i] += 1
                 if block[i] * params.block_len >= sess.gen_len[i]:
@@ -294,3 +296,28 @@ def generate(sess: Session, params: DecodeParams, *,
                 else:
                     need_refresh[i] = True
     return {i: sess.get_tokens(i) for i in seqs}, trace
+
+
+def mode_settings(mode: str, block_len: int, n_copies: int = 4, accept_threshold: float = 0.9):
+    """(DecodeParams, cache_blocks) of the three systems of Tables 2 and 3: "vanilla" (no cache, one
+    token per full forward), "fast_dllm" (DualCache block decoding, threshold acceptance, fixed
+    length) and "odb" (adaptive length prediction + jump-share speculation)."""
+    if mode == "vanilla":
+        return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=1.0, alp=False), False
+    if mode == "fast_dllm":
+        return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=accept_threshold, alp=False), True
+    if mode == "odb":
+        return DecodeParams(block_len=block_len, n_copies=n_copies, accept_threshold=accept_threshold, alp=True), True
+    raise ValueError(mode)
+
+
+def trace_counters(trace, seq: int = 0) -> dict:
+    """Section 5.3's counters for one sequence of a `generate` trace: NFE (forward passes), Eff_NFE
+    (links of the jump chains = effective state changes), committed tokens."""
+    recs = [t for t in trace if seq in t["seqs"]]
+    nfe = len(recs)
+    eff = sum(len(t["seqs"][seq]["chain"]) for t in recs)
+    tokens = sum(len(t["seqs"][seq]["accepted"]) for t in recs)
+    return {"nfe": nfe, "eff_nfe": eff, "tokens": tokens, "refreshes": sum(t["kind"] == "refresh" for t in recs),
+            "tokens_per_nfe": tokens / nfe if nfe else 0.0}
+

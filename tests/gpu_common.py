@@ -56,7 +56,7 @@ def compare_traces(gpu_trace, oracle_trace, seq=0, near_tie=1e-3):
 
 
 def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, check_logits=True, max_iters=None,
-                      seq=0):
+                      seq=0, cache_blocks=True):
     """Lock-step parity harness for one sequence.
 
     Every iteration both sides start from the same state.  (1) Numerics: the GPU's logits /
@@ -67,7 +67,8 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
     decision the oracle takes from ITS confidences is compared too; where it differs, the
     oracle's decision margin must be below the confidence error measured in that iteration (a
     near-tie); these are counted and returned, never hidden.  The GPU's decision then advances
-    both sides.  Returns a stats dict."""
+    both sides.  cache_blocks=False runs the cache-less baseline (every iteration a refresh).
+    Returns a stats dict."""
     sess.set_logit_dump(check_logits)                   # logits are only materialised in the test mode
     shape_mask, eos = om.mask_id, om.eos_id
     Bk, tau = op.block_len, op.accept_threshold
@@ -141,6 +142,10 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
         st["iters"] += 1; st["refreshes"] += 1; st["tokens"] += len(want)
         assert res.masks_left == int((x[s:e] == shape_mask).sum())
         last_conf, last_tok = g_conf[:B], g_tok[:B]
+        if not cache_blocks:                            # cache-less baseline: the next iteration is a refresh again
+            if not (x[s:e] == shape_mask).any():
+                b += 1
+            continue
         while (x[s:e] == shape_mask).any():
             if max_iters is not None and st["iters"] >= max_iters:
                 break

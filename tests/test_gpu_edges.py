@@ -1,0 +1,73 @@
+"""Edge cases of the decoding iteration through the C ABI, each in lock step with the oracle: ragged
+tails (response not a multiple of the block, prompt not a multiple of any tile), the degenerate
+shapes (no prompt, a one-position block, a one-position response), and the largest sizes the
+library accepts (block 64 with 8 copies = 512 query rows; a 2048-position sequence)."""
+import numpy as np
+import pytest
+
+import synth
+from oracle import odb_oracle as O
+from oracle.inputs import model_from_synth
+from gpu_common import engine, requires_gpu, lockstep_generate, assert_near_ties_only
+
+CASES = [
+    # name              shape        P    L   block copies  max_iters
+    ("ragged_tail",     "TINY",      37,  41, 16,   4,      None),   # last block has 9 positions; odd prompt
+    ("ragged_peaky_c8", "TINY_PEAKY", 51, 45, 16,   8,      None),   # last block 13, stage-2 copies on a short block
+    ("no_prompt",       "TINY",      0,   32, 16,   4,      None),   # the first refresh has no prefix at all
+    ("block_of_one",    "TINY",      20,  5,  1,    1,      None),   # every iteration is a refresh
+    ("response_of_one", "TINY",      33,  1,  16,   4,      None),   # one masked position in total
+    ("block_3_c4",      "TINY_PEAKY", 17, 10, 3,    4,      None),   # fewer masked positions than candidate ranks
+    ("block64_c8",      "TINY_PEAKY", 64, 128, 64,  8,      None),   # 512 query rows per step: the largest step
+    ("long_2048",       "TINY",      1984, 64, 32,  4,      12),     # the longest sequence: 16 key splits in the step
+]
+
+
+@requires_gpu
+@pytest.mark.parametrize("name,shape_name,P,L,Bk,copies,max_iters", CASES, ids=[c[0] for c in CASES])
+def test_edge_case_in_lockstep(name, shape_name, P, L, Bk, copies, max_iters):
+    E = engine()
+    shape = getattr(synth, shape_name)
+    om = model_from_synth(shape, seed=3)
+    gm = E.Model.from_synth(shape, seed=3, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=8)
+    sess = E.Session(gm)
+    x0 = synth.sequence(3, 0, P, L, shape)
+    sess.set_sequence(0, x0, P)
+    kw = dict(block_len=Bk, n_copies=copies)
+    tol = 4e-2 if shape_name == "TINY_PEAKY" else 2e-2
+    st = lockstep_generate(E, sess, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=tol,
+                           max_iters=max_iters)
+    assert sess.status() == 0
+    assert_near_ties_only(st)
+    if max_iters is None:
+        assert np.array_equal(sess.get_tokens(0), st["tokens_final"])
+        assert (st["tokens_final"][P:] != shape.mask_id).all() and st["tokens"] == L
+        assert st["refreshes"] == -(-L // Bk)
+    else:
+        assert st["iters"] == max_iters and st["tokens"] >= max_iters
+    print(f"\n{name}: {st['iters']} iterations ({st['refreshes']} refreshes), worst logit {st['worst_logit']:.2f} x bound, "
+          f"oracle-side decision diffs {st['oracle_decision_diff']}")
+    sess.close(); gm.close()
+
+
+@requires_gpu
+def test_fully_decoded_block_is_a_state_error_not_a_launch():
+    """A step on a block with no masked position left has no rows: the call reports the state error
+    and launches nothing (the degenerate empty input)."""
+    E = engine()
+    shape = synth.TINY
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=24, max_block=1, max_copies=1)
+    sess = E.Session(gm)
+    sess.set_sequence(0, synth.sequence(0, 0, 20, 4, shape), 20)
+    gp = E.DecodeParams(block_len=1, n_copies=1)
+    sess.refresh_prefill(gp, 0)
+    res = sess.unmask_accept(gp, True)[0]
+    assert res.n_accepted == 1 and res.masks_left == 0        # top-1 fallback filled the only position
+    from paper_2511_21759_b200 import binding as B
+    with pytest.raises(B.OdbError) as err:
+        sess.block_decode_step(gp)
+    assert err.value.status == B.ODB_ERR_STATE
+    assert sess.status() == 0
+    sess.refresh_prefill(gp, 1)                                # the session is still usable
+    assert sess.unmask_accept(gp, True)[0].n_accepted == 1
+    sess.close(); gm.close()

@@ -106,6 +106,52 @@ def test_lockstep_with_cluster_residual_epilogue():
 
 
 @requires_gpu
+@pytest.mark.parametrize("mode", ["vanilla", "fast_dllm", "odb"])
+def test_baseline_modes_in_lockstep(mode):
+    """The three systems the paper's tables compare, as settings of the same calls: the cache-less
+    baseline (every iteration a refresh prefill, one token each), DualCache block decoding without
+    speculation or length prediction, and the full method."""
+    E = engine()
+    shape = synth.TINY_PEAKY
+    P, L, Bk = 40, 24, 8
+    om = model_from_synth(shape, seed=2)
+    gm = E.Model.from_synth(shape, seed=2, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=8)
+    sess = E.Session(gm)
+    x0 = synth.sequence(2, 0, P, L, shape)
+    sess.set_sequence(0, x0, P)
+    gp, cache_g = E.mode_settings(mode, Bk)
+    op, cache_o = O.mode_settings(mode, Bk)
+    assert cache_g == cache_o and dataclasses.asdict(op) == {k: getattr(gp, k) for k in dataclasses.asdict(op)}
+    st = lockstep_generate(E, sess, om, x0, P, gp, op, tol=4e-2, cache_blocks=cache_g)
+    assert sess.status() == 0
+    assert_near_ties_only(st)
+    assert np.array_equal(sess.get_tokens(0), st["tokens_final"])
+    if mode == "vanilla":
+        assert st["iters"] == st["refreshes"] == L and st["steps"] == 0
+    else:
+        assert st["refreshes"] == L // Bk and st["iters"] <= L
+    sess.close(); gm.close()
+
+
+@requires_gpu
+def test_trace_counters_match_the_oracle_definition():
+    E = engine()
+    wl = synth.WORKLOADS["peaky_c4"]
+    gm = E.Model.from_synth(wl.shape, seed=0, max_batch=1, max_seq=wl.prompt_len + wl.gen_len, max_block=wl.block_len,
+                            max_copies=8)
+    sess = E.Session(gm)
+    sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, wl.shape), wl.prompt_len)
+    gp, cache_blocks = E.mode_settings("odb", wl.block_len)
+    _, gtrace = E.generate(sess, gp, cache_blocks=cache_blocks)
+    c = E.trace_counters(gtrace)
+    # the same counters from the oracle's function on the GPU's trace, re-shaped to the oracle's records
+    as_oracle = [{"kind": t["kind"], "accepted": t["seqs"][0]["accepted"], "chain": t["seqs"][0]["chain"]} for t in gtrace]
+    assert c == O.trace_counters(as_oracle)
+    assert c["tokens"] == wl.gen_len and c["eff_nfe"] >= c["nfe"] and c["refreshes"] == wl.gen_len // wl.block_len
+    sess.close(); gm.close()
+
+
+@requires_gpu
 def test_generate_with_length_schedule():
     sched = lambda b, L: {0: 40, 1: 24}.get(b)
     gtok, gtrace, otok, otrace = _run_both("peaky_c4", schedule=sched)

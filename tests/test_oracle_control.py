@@ -265,3 +265,64 @@ def test_length_schedule_lever(tiny_model):
     x, tr = O.generate(tiny_model, x0, 64, O.DecodeParams(block_len=16), length_schedule=sched)
     assert len(x) == 64 + 24 and [t["T"] for t in tr if t["kind"] == "refresh"] == [104, 88]
     assert (x[64:] != synth.TINY.mask_id).all()
+
+
+# ---- baseline modes and counters (Tables 2 and 3; Section 5.3) ----------------------------------
+
+def test_cacheless_baseline_is_one_refresh_per_token():
+    shape = synth.TINY
+    om = model_from_synth(shape, seed=0)
+    P, L, Bk = 24, 12, 4
+    x0 = synth.sequence(0, 0, P, L, shape)
+    params, cache_blocks = O.mode_settings("vanilla", Bk)
+    assert not cache_blocks and params.n_copies == 1 and not params.alp
+    x, trace = O.generate(om, x0, P, params, cache_blocks=cache_blocks)
+    c = O.trace_counters(trace)
+    # no confidence exceeds 1, so the fallback commits exactly one token per full forward
+    assert c == {"nfe": L, "eff_nfe": L, "tokens": L, "refreshes": L, "tokens_per_nfe": 1.0}
+    assert all(t["kind"] == "refresh" and len(t["accepted"]) == 1 for t in trace)
+    assert [t["block"] for t in trace] == [i // Bk for i in range(L)]          # blocks in order, Bk iterations each
+    assert (x[P:] != shape.mask_id).all()
+    # every iteration sees the exact current state: each committed token is the argmax of an uncached
+    # forward over the sequence as it stood, at the most confident masked position of the block
+    xs = x0.astype(np.int64).copy()
+    for t in trace:
+        s = P + t["block"] * Bk
+        _, conf, tok = O.refresh_prefill(om, xs, len(xs), s)
+        masked = xs[s:s + Bk] == shape.mask_id
+        i = int(np.argmax(np.where(masked, conf[:Bk], -1.0)))
+        assert t["accepted"] == [(s + i, int(tok[i]))]
+        xs[s + i] = tok[i]
+
+
+def test_block_of_one_makes_cached_and_cacheless_decoding_identical():
+    # with one position per block every iteration is a refresh in both systems
+    shape = synth.TINY
+    om = model_from_synth(shape, seed=1)
+    P, L = 16, 6
+    x0 = synth.sequence(1, 0, P, L, shape)
+    p = O.DecodeParams(block_len=1, n_copies=1, alp=False)
+    xa, ta = O.generate(om, x0, P, p, cache_blocks=True)
+    xb, tb = O.generate(om, x0, P, p, cache_blocks=False)
+    assert np.array_equal(xa, xb)
+    assert [(t["kind"], t["accepted"]) for t in ta] == [(t["kind"], t["accepted"]) for t in tb]
+
+
+def test_counters_of_the_three_systems():
+    shape = synth.TINY_PEAKY
+    om = model_from_synth(shape, seed=0)
+    wl = synth.WORKLOADS["peaky_c4"]
+    x0 = synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape)
+    out = {}
+    for mode in ("vanilla", "fast_dllm", "odb"):
+        params, cache_blocks = O.mode_settings(mode, wl.block_len)
+        x, trace = O.generate(om, x0, wl.prompt_len, params, cache_blocks=cache_blocks)
+        out[mode] = (x, O.trace_counters(trace))
+    L, nb = wl.gen_len, wl.gen_len // wl.block_len
+    assert out["vanilla"][1]["nfe"] == L and out["vanilla"][1]["refreshes"] == L
+    f, o = out["fast_dllm"][1], out["odb"][1]
+    assert f["refreshes"] == nb and f["eff_nfe"] == f["nfe"] <= L              # no speculation: one state change per pass
+    assert o["refreshes"] <= nb and o["nfe"] <= f["nfe"]                       # jumps only ever save passes
+    assert o["eff_nfe"] >= o["nfe"]                                            # several state changes in one pass
+    assert f["tokens"] == L and o["tokens"] == len(out["odb"][0]) - wl.prompt_len
+
