@@ -71,8 +71,10 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
     uint8_t* sValid = sV + 2 * kTileBytes;           // [2][64]
 
     pdl_launch_dependents();
-    pdl_wait();
-    l2_prefetch_slice(a.pf, (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x * gridDim.y * gridDim.z);
+    // a.early (decode steps): the tile table and the K/V cache were complete before this launch chain
+    // began, so cached key tiles are requested before waiting for the predecessor (the kernel that
+    // writes q and the fresh k/v); otherwise nothing is touched before the wait
+    if (!a.early) pdl_wait();
     const QTile t = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
     const int z = blockIdx.z;
@@ -90,14 +92,6 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
     const __nv_bfloat16* ck = a.cache + (static_cast<size_t>(t.seq) * a.n_layers + a.layer) * 2 * per_kv +
                               static_cast<size_t>(head) * a.max_seq * HD;
     const __nv_bfloat16* cv = ck + per_kv;
-
-    // ---- Q tile ----
-    for (int c = threadIdx.x; c < kTileQ * CH; c += kAttnThreads) {
-        const int r = c / CH, ch = c % CH;
-        const bool ok = r < t.nq;
-        const __nv_bfloat16* src = ok ? a.q + static_cast<size_t>(t.q_row0 + r) * d + head * HD + ch * 8 : a.q;
-        cp_async16(sQ + swz<HD>(r, ch), src, ok);
-    }
 
     auto load_tile = [&](int tile, int buf) {
         for (int c = threadIdx.x; c < kTileK * CH; c += kAttnThreads) {
@@ -130,10 +124,30 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnArgs a) {
         }
     };
 
-    // the first two tiles are requested at once; later ones one iteration ahead
-    if (t0 < t1) load_tile(t0, 0);
+    // The first two tiles are requested at once, later ones one iteration ahead.  Four cp.async groups:
+    // the two tiles if they hold cached keys only (before the wait), then Q with whatever is left of
+    // tile t0, then what is left of tile t0 + 1.
+    bool pre0 = false, pre1 = false;
+    if (a.early) {
+        pre0 = t0 < t1 && (t0 + 1) * kTileK <= nA + nB;
+        pre1 = t0 + 1 < t1 && (t0 + 2) * kTileK <= nA + nB;
+        if (pre0) load_tile(t0, 0);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (pre1) load_tile(t0 + 1, 1);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        pdl_wait();
+    }
+    l2_prefetch_slice(a.pf, (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x * gridDim.y * gridDim.z);
+    // ---- Q tile ----
+    for (int c = threadIdx.x; c < kTileQ * CH; c += kAttnThreads) {
+        const int r = c / CH, ch = c % CH;
+        const bool ok = r < t.nq;
+        const __nv_bfloat16* src = ok ? a.q + static_cast<size_t>(t.q_row0 + r) * d + head * HD + ch * 8 : a.q;
+        cp_async16(sQ + swz<HD>(r, ch), src, ok);
+    }
+    if (t0 < t1 && !pre0) load_tile(t0, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    if (t0 + 1 < t1) load_tile(t0 + 1, 1);
+    if (t0 + 1 < t1 && !pre1) load_tile(t0 + 1, 1);
     asm volatile("cp.async.commit_group;" ::: "memory");
 
     float o_acc[HD / 8][4];
@@ -294,8 +308,8 @@ __global__ void __launch_bounds__(256) step_attention_kernel(StepAttnArgs a) {
     uint8_t* sValid = sV + 2 * kTileBytes;           // [2][64]: 0 invalid, 1 valid, 2 valid and decoded
 
     pdl_launch_dependents();
-    pdl_wait();
-    l2_prefetch_slice(a.pf, (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x * gridDim.y * gridDim.z);
+    // the tile table and the K/V cache were complete before this step's launch chain began: the splits
+    // that stream cached keys request their first two tiles before waiting for the predecessor
     const StepTile& t = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
     const int z = blockIdx.z, ks = gridDim.z;
@@ -313,14 +327,6 @@ __global__ void __launch_bounds__(256) step_attention_kernel(StepAttnArgs a) {
                               static_cast<size_t>(head) * a.max_seq * HD;
     const __nv_bfloat16* cv = ck + per_kv;
 
-    // ---- Q: slab w holds the rows slab_row0[w] .. + slab_n[w] ----
-    for (int c = threadIdx.x; c < 128 * CH; c += 256) {
-        const int r = c / CH, ch = c % CH;
-        const int sl = r >> 4, rr = r & 15;
-        const bool ok = sl < t.n_slabs && rr < t.slab_n[sl];
-        const __nv_bfloat16* src = ok ? a.q + static_cast<size_t>(t.slab_row0[sl] + rr) * d + head * HD + ch * 8 : a.q;
-        cp_async16(sQ + swz<HD>(r, ch), src, ok);
-    }
     auto load_tile = [&](int tile, int buf) {
         for (int c = threadIdx.x; c < kTileK * CH; c += 256) {
             const int key = c / CH, ch = c % CH;
@@ -349,9 +355,25 @@ __global__ void __launch_bounds__(256) step_attention_kernel(StepAttnArgs a) {
             if (ch == 0) sValid[buf * kTileK + key] = ok ? flag : 0;
         }
     };
-    if (t0 < t1) load_tile(t0, 0);
+    // four cp.async groups: cached tiles t0 and t0 + 1 (before the wait), then Q with the fresh split's
+    // first tile, then its second
+    if (!fresh_cta && t0 < t1) load_tile(t0, 0);
     asm volatile("cp.async.commit_group;" ::: "memory");
-    if (t0 + 1 < t1) load_tile(t0 + 1, 1);
+    if (!fresh_cta && t0 + 1 < t1) load_tile(t0 + 1, 1);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    pdl_wait();
+    l2_prefetch_slice(a.pf, (blockIdx.z * gridDim.y + blockIdx.y) * gridDim.x + blockIdx.x, gridDim.x * gridDim.y * gridDim.z);
+    // ---- Q: slab w holds the rows slab_row0[w] .. + slab_n[w] ----
+    for (int c = threadIdx.x; c < 128 * CH; c += 256) {
+        const int r = c / CH, ch = c % CH;
+        const int sl = r >> 4, rr = r & 15;
+        const bool ok = sl < t.n_slabs && rr < t.slab_n[sl];
+        const __nv_bfloat16* src = ok ? a.q + static_cast<size_t>(t.slab_row0[sl] + rr) * d + head * HD + ch * 8 : a.q;
+        cp_async16(sQ + swz<HD>(r, ch), src, ok);
+    }
+    if (fresh_cta && t0 < t1) load_tile(t0, 0);
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    if (fresh_cta && t0 + 1 < t1) load_tile(t0 + 1, 1);
     asm volatile("cp.async.commit_group;" ::: "memory");
 
     const bool warp_active = warp < t.n_slabs;

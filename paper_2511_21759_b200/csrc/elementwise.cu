@@ -219,8 +219,13 @@ __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial
 
 }  // namespace
 
+// First kernel of a forward.  Launched WITHOUT programmatic stream serialization: it starts only when
+// everything enqueued before it (the row and tile tables, the previous accept) has completed, and every
+// later kernel of the chain starts after this one has started.  That is what allows the attention
+// kernels to read the tile table and the K/V cache before their own griddepcontrol.wait.
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d, cudaStream_t st) {
-    return launch_kernel(embed_kernel, dim3(M), dim3(256), 0, st, embed, row_tok, h, d);
+    embed_kernel<<<dim3(M), dim3(256), 0, st>>>(embed, row_tok, h, d);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,

@@ -156,36 +156,13 @@ struct alignas(8) GemmShared {
 // 64 (tile t = gate rows [64t, 64t+64) then up rows [64t, 64t+64)); the epilogue pairs TMEM lane r
 // (gate) with lane r + 64 (up) through shared memory and stores bf16(silu(gate) * up) to
 // g[m][64 t + r]; N is then the FFN width F and there is no K split.
-// EPI_RESIDUAL: the K splits of one output tile form a thread-block CLUSTER (1, 1, splits).  Each CTA
-// parks its fp32 accumulator tile in its shared memory; after a cluster barrier CTA r sums rows
-// [128 r / S, 128 (r+1) / S) of the tile over all S CTAs in split order through distributed shared
-// memory and finishes the layer's bookkeeping in place: h += y (residual), operand of the next
-// projection bf16(h * gain), and this slice's contribution to sum(h^2) per activation row.  The CTA
-// that arrives last at the grid's counter turns the per-slice sums into 1/rms per row (fixed order).
-// No partial sums go through HBM and no RMSNorm kernel is needed after this GEMM.
-constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_RESIDUAL = 2, EPI_CONF = 3;
-
-__device__ __forceinline__ uint32_t dsmem_addr(const void* p, uint32_t cta_rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(cta_rank));
-    return r;
-}
-
-__device__ __forceinline__ float ld_dsmem_f32(uint32_t addr) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
-    return v;
-}
-
-__device__ __forceinline__ void cluster_barrier() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
+constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_CONF = 3;
 
 template <int BN, int EPI>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
             float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, const float* __restrict__ row_scale,
-            ResidualEpilogue re, ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
+            ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
             int l2_prefetch,
             int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -383,19 +360,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
-        } else if constexpr (EPI == EPI_RESIDUAL) {
-            // park the accumulator tile in shared memory as acc[m][n] (n contiguous): the ring is free
-            float* acc = reinterpret_cast<float*>(tiles);
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                if (ok) {
-                    tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
-                    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                }
-#pragma unroll
-                for (int j = 0; j < 32; ++j) acc[(c * 32 + j) * kBM + q * 32 + lane] = ok ? __uint_as_float(v[j]) : 0.f;
-            }
         } else {
             // all MMAs have completed, so the stage ring is free: use it to hand the up values over.
             // Every epilogue warp executes every barrier, whether or not its wait succeeded.
@@ -428,104 +392,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-            }
-        }
-    }
-    if constexpr (EPI == EPI_RESIDUAL) {
-        const int S = gridDim.z;                        // cluster size = number of K splits (4 or 8)
-        float* acc = reinterpret_cast<float*>(tiles);
-        float* css = acc + BN * kBM;                    // in the cluster's rank-0 CTA: [S][BN] slice sums of h^2
-        cluster_barrier();                              // every CTA's tile is parked
-        if (warp >= 2) {
-            const int t = threadIdx.x - 64;             // 0..127
-            const int slice = kBM / S;                  // rows of the tile this CTA finishes: 32 or 16
-            const int nl0 = split * slice;
-            // BN * slice elements, 128 threads: ITER elements per thread.  All remote tile values and
-            // all residual values are requested before anything is consumed (one round trip each).
-            constexpr int kMaxIter = BN / 4;            // slice <= 32
-            const int iters = BN * slice / 128;
-            float part[kMaxIter <= 8 ? kMaxIter : 8][8];
-            float hold[kMaxIter <= 8 ? kMaxIter : 8];
-            for (int i0 = 0; i0 < iters; i0 += 8) {
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (u < kMaxIter && i0 + u < iters) {
-                        const int idx = (i0 + u) * 128 + t;
-                        const int m_l = idx / slice, n_l = nl0 + idx % slice;
-#pragma unroll
-                        for (int z = 0; z < 8; ++z)
-                            if (z < S) part[u][z] = ld_dsmem_f32(dsmem_addr(acc + m_l * kBM + n_l, z));
-                        const int m = m0 + m_l, n = n0 + n_l;
-                        hold[u] = (m < M && n < N) ? re.h[static_cast<size_t>(m) * N + n] : 0.f;
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    if (u < kMaxIter && i0 + u < iters) {
-                        const int idx = (i0 + u) * 128 + t;
-                        const int m_l = idx / slice, n_l = nl0 + idx % slice;
-                        const int m = m0 + m_l, n = n0 + n_l;
-                        float hn = 0.f;
-                        if (m < M && n < N) {
-                            const size_t o = static_cast<size_t>(m) * N + n;
-                            float y = 0.f;
-#pragma unroll
-                            for (int z = 0; z < 8; ++z)
-                                if (z < S) y += part[u][z];
-                            hn = hold[u] + y;
-                            re.h[o] = hn;
-                            re.a_out[o] = __float2bfloat16_rn(hn * re.gain[n]);
-                        }
-                        // sum of squares over the `slice` consecutive lanes that share one activation row
-                        float ss = hn * hn;
-                        for (int off = slice >> 1; off > 0; off >>= 1) ss += __shfl_down_sync(0xffffffffu, ss, off, slice);
-                        if (idx % slice == 0) {
-                            const uint32_t dst = dsmem_addr(css + split * BN + m_l, 0);
-                            asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(dst), "f"(ss) : "memory");
-                        }
-                    }
-                }
-            }
-        }
-        cluster_barrier();                              // tiles no longer needed; slice sums are in rank 0
-        // rank 0 adds the slice sums in split order -> one value per (row, n-tile); the rank-0 CTA that
-        // arrives last at the grid counter (nobody waits) turns them into 1/rms per row
-        if (split == 0 && warp >= 2) {
-            const int t = threadIdx.x - 64;
-            const int slots = gridDim.x;
-            for (int m_l = t; m_l < BN; m_l += 128) {
-                if (m0 + m_l < M) {
-                    float ss = 0.f;
-                    for (int z = 0; z < S; ++z) ss += css[z * BN + m_l];
-                    re.sumsq[static_cast<size_t>(m0 + m_l) * slots + blockIdx.x] = ss;
-                }
-            }
-            int* flag = reinterpret_cast<int*>(&sh->empty[0]);
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (t == 0) {
-                __threadfence();
-                const int total = gridDim.x * gridDim.y;
-                const int old = atomicAdd(re.counter, 1);
-                *flag = old == total - 1;
-                if (old == total - 1) *re.counter = 0;
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (*flag) {
-                __threadfence();
-                // four threads per row, each a strided quarter of the slots, combined in a fixed order
-                // (the row loop is uniform across the warp: every lane takes part in the shuffles)
-                const int part = t & 3;
-                for (int mb = 0; mb < M; mb += 32) {
-                    const int m = mb + (t >> 2);
-                    float ssum = 0.f;
-                    if (m < M) {
-#pragma unroll 8
-                        for (int i = part; i < slots; i += 4) ssum += __ldcg(re.sumsq + static_cast<size_t>(m) * slots + i);
-                    }
-                    ssum += __shfl_down_sync(0xffffffffu, ssum, 2, 4);
-                    ssum += __shfl_down_sync(0xffffffffu, ssum, 1, 4);
-                    if (m < M && part == 0) re.inv_rms[m] = 1.0f / sqrtf(ssum / static_cast<float>(N) + re.eps);
-                }
             }
         }
     }
@@ -651,10 +517,6 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
     int stages = static_cast<int>(budget / stage_bytes);
     if (stages > 16) stages = 16;
     if (stages > nkb_per_split) stages = nkb_per_split < 2 ? 2 : nkb_per_split;
-    if (EPI == EPI_RESIDUAL) {   // the ring later holds the parked accumulator tile and the slice sums
-        const int need = static_cast<int>((static_cast<size_t>(BN) * (kBM + 8) * 4 + stage_bytes - 1) / stage_bytes);
-        if (stages < need) stages = need;
-    }
     const size_t smem = static_cast<size_t>(stages) * stage_bytes + sizeof(GemmShared) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
@@ -669,30 +531,9 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
         const char* e = getenv("ODB_GEMM_L2_PREFETCH");
         l2_prefetch = e ? atoi(e) : 0;   // measured: prefetching into L2 slows the step down
     }
-    if constexpr (EPI == EPI_RESIDUAL) {
-        // the parked accumulator tile (BN x 128 fp32) must fit the stage ring
-        if (static_cast<size_t>(stages) * stage_bytes < static_cast<size_t>(BN) * (kBM + 8) * 4) return cudaErrorInvalidValue;
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = grid;
-        cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = smem;
-        cfg.stream = st;
-        cudaLaunchAttribute attr[2];
-        attr[0].id = cudaLaunchAttributeClusterDimension;
-        attr[0].val.clusterDim.x = 1;
-        attr[0].val.clusterDim.y = 1;
-        attr[0].val.clusterDim.z = a.splits;
-        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[1].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = attr;
-        cfg.numAttrs = pdl_enabled() ? 2 : 1;
-        return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.residual, a.conf,
-                                  a.M, a.N, nkb_total, nkb_per_split, stages, 0, a.status);
-    } else {
-        return launch_kernel(gemm_kernel<BN, EPI>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
-                             a.row_scale, a.residual, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
-                             pdl_enabled() ? l2_prefetch : 0, a.status);
-    }
+    return launch_kernel(gemm_kernel<BN, EPI>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
+                         a.row_scale, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
+                         pdl_enabled() ? l2_prefetch : 0, a.status);
 }
 
 template <int EPI>
@@ -756,16 +597,6 @@ static int target_ctas() {
     return v;
 }
 
-// Cluster size for the residual epilogue: 8 or 4 K splits, none of them empty; 0 if the shape does
-// not allow it (then the caller uses plain split-K partials and the RMSNorm kernel).
-int gemm_cluster_splits(int M, int K) {
-    if (pick_bn(M) > 128) return 0;
-    const int nkb = (K + kBK - 1) / kBK;
-    for (int sp = 8; sp >= 4; sp >>= 1)
-        if (((nkb + sp - 1) / sp) * (sp - 1) < nkb) return sp;
-    return 0;
-}
-
 int gemm_pick_splits(int M, int N, int K) {
     const int bn = pick_bn(M);
     const int tiles = ((N + kBM - 1) / kBM) * ((M + bn - 1) / bn);
@@ -793,11 +624,6 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
     CUtensorMap tmx;
     cudaError_t e = make_tmap_2d(&tmx, a.x, a.M, a.K, bn);
     if (e != cudaSuccess) return e;
-    if (a.residual.h) {
-        // cluster split-K: the cluster size must divide the 128 tile rows and stay portable (<= 8)
-        if ((a.splits != 4 && a.splits != 8) || bn > 128) return cudaErrorInvalidValue;
-        return launch_epi<EPI_RESIDUAL>(a, tmx, bn, st);
-    }
     if (a.act_out) {
         if (a.splits != 1) return cudaErrorInvalidValue;
         return launch_epi<EPI_SWIGLU>(a, tmx, bn, st);

@@ -47,7 +47,7 @@ int32_t check_config(const odb_config* c) {
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
     size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, step_tile_buf;
-    size_t h, a, inv, sumsq, counter, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
+    size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
     size_t total;
 };
 
@@ -82,8 +82,6 @@ Layout make_layout(const odb_config& c) {
     L.h = take(4 * L.rows * d);
     L.a = take(2 * L.rows * d);
     L.inv = take(4 * L.rows);
-    L.sumsq = take(4 * 256 * ((d + 127) / 128) * 8);   // decode steps only: <= 256 rows x (n-tiles x 8 splits)
-    L.counter = take(256);
     L.q = take(2 * L.rows * d);
     L.k = take(2 * L.rows * d);
     L.v = take(2 * L.rows * d);
@@ -277,7 +275,6 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(s->ws + L.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s->st);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->ws + L.state, 0, L.x - L.state, s->st);   // state, results, status
-    if (e == cudaSuccess) e = cudaMemsetAsync(s->ws + L.counter, 0, 256, s->st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->st);
     if (e != cudaSuccess) {
         odb_session_destroy(s);
@@ -468,11 +465,6 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     if (ks < 1) ks = 1;
     // L2 prefetch hints (decode steps only): while a short kernel runs between two GEMMs, HBM is
     // idle; the kernel asks L2 for the head of the next GEMM's weights.  Sizes in bytes.
-    // Measured on the 8B shape: alone, a cluster GEMM costs what the plain GEMM plus the RMSNorm kernel
-    // cost (18 vs 12 + 6 us for O-proj), but its CTAs hold their shared memory through the reduction
-    // tail, so the next GEMM's early-launched CTAs cannot move in and prefetch: the step gets 6 % slower
-    // (3.60 vs 3.39 ms).  Off unless ODB_CLUSTER_EPILOGUE=1.
-    static const bool cluster_epilogue = getenv("ODB_CLUSTER_EPILOGUE") && getenv("ODB_CLUSTER_EPILOGUE")[0] == '1';
     static const long long pf_mb = getenv("ODB_L2_PREFETCH_MB") ? atoll(getenv("ODB_L2_PREFETCH_MB")) : 8;   // measured: 8 MB helps, 24 MB and more lengthen the hinting kernel
     const bool hint = !write_cache && pdl_enabled() && pf_mb > 0;
     const unsigned long long pf_bytes = static_cast<unsigned long long>(pf_mb) << 20;
@@ -486,34 +478,9 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     };
     const size_t qkv_bytes = packed_weight_bytes(3 * d, d), o_bytes = packed_weight_bytes(d, d),
                  gu_bytes = packed_gate_up_bytes(F, d);
-    // Decode steps close both residual branches inside the GEMM (cluster split-K with the residual
-    // epilogue): `a` and `inv` then already hold the next projection's operand and 1/rms, and no
-    // RMSNorm kernel sits between the GEMMs.  The refresh (many rows) keeps split partials + kernel.
-    const int cs_o = (!write_cache && M <= 128 && cluster_epilogue) ? gemm_cluster_splits(M, d) : 0;
-    const int cs_d = (!write_cache && M <= 128 && cluster_epilogue) ? gemm_cluster_splits(M, F) : 0;
-    auto residual_gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, int K, int splits, const float* gain) {
-        GemmArgs ga;
-        ga.tmap_w = tw;
-        ga.x = x;
-        ga.partial = nullptr;
-        ga.act_out = nullptr;
-        ga.residual.h = h;
-        ga.residual.gain = gain;
-        ga.residual.a_out = a;
-        ga.residual.sumsq = s->at<float>(L.sumsq);
-        ga.residual.inv_rms = inv;
-        ga.residual.counter = s->at<int>(L.counter);
-        ga.residual.eps = c.rms_eps;
-        ga.M = M; ga.N = d; ga.K = K;
-        ga.splits = splits;
-        ga.status = status;
-        return launch_gemm(ga, st);
-    };
-    bool prepped = false;   // `a` / `inv` already hold the operand and scalar of the next normed projection
     for (int l = 0; l < c.n_layers; ++l) {
-        if (!prepped)
-            ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
-                                                            c.rms_eps, hint_of(m->p_qkv[l], qkv_bytes, 0), st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
+                                                        c.rms_eps, hint_of(m->p_qkv[l], qkv_bytes, 0), st));
         int sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
         QkvRopeArgs qa;
@@ -550,18 +517,15 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
         aa.part_o = s->at<float>(L.part_o); aa.part_ml = s->at<float>(L.part_ml);
         aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = ks;
+        aa.early = write_cache ? 0 : 1;   // a refresh writes the cache it attends to: nothing may be read early
         aa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
         ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention(aa, st));
         if (ks > 1) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
         }
-        if (cs_o) {
-            ODB_LAUNCH(ODB_KIND_GEMM, residual_gemm(m->tm_o[l], o, d, cs_o, m->norm2[l]));
-        } else {
-            sp = 0;
-            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
-            ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
-                                                            d, c.rms_eps, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
-        }
+        sp = 0;
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
+                                                        d, c.rms_eps, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
         {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
             GemmArgs ga;
             ga.tmap_w = m->tm_gu[l];
@@ -574,23 +538,14 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             ga.status = status;
             ODB_LAUNCH(ODB_KIND_GEMM, launch_gemm(ga, st));
         }
-        if (cs_d) {
-            const float* next_gain = l + 1 < c.n_layers ? m->norm1[l + 1] : m->final_norm;
-            ODB_LAUNCH(ODB_KIND_GEMM, residual_gemm(m->tm_d[l], g, F, cs_d, next_gain));
-            prepped = true;
-            res = nullptr; res_splits = 0; res_stride = 0;
-        } else {
-            sp = 0;
-            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, &sp));
-            res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
-            prepped = false;
-        }
+        sp = 0;
+        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, &sp));
+        res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
     }
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
-        if (!prepped)
-            ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
-                                                            c.rms_eps, L2Prefetch{nullptr, 0}, st));
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
+                                                        c.rms_eps, L2Prefetch{nullptr, 0}, st));
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
@@ -598,13 +553,8 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
         const __nv_bfloat16* x = a;
         const float* scale = inv;
-        if (prepped) {          // decode step: every row needs logits, rows are in order
-            x = a + static_cast<size_t>(r0) * d;
-            scale = inv + r0;
-        } else {
-            ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
-                                                            rows, d, c.rms_eps, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
-        }
+        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
+                                                        rows, d, c.rms_eps, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
         if (s->dump_logits) {
             int sp = 1;
             ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, &sp, scale));

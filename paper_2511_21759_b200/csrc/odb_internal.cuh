@@ -132,18 +132,6 @@ constexpr int kRowDecoded = 1;   // row_flags bit: the row's position is decoded
 
 struct TmaEncoder;   // wraps the driver's tensor-map encode entry point
 
-// Epilogue of a projection that closes a residual branch (O-proj, down-proj) in a decode step; see
-// EPI_RESIDUAL in gemm_tcgen05.cu.  h non-null selects it.
-struct ResidualEpilogue {
-    float* h = nullptr;             // residual stream [M][N], updated in place: h += x W^T
-    const float* gain = nullptr;    // gains [N] of the RMSNorm that follows
-    __nv_bfloat16* a_out = nullptr; // [M][N] bf16(h * gain): operand of the next projection
-    float* sumsq = nullptr;         // [M][n_tiles] per-tile sums of h^2
-    float* inv_rms = nullptr;       // [M] 1 / sqrt(mean(h^2) + eps)
-    int* counter = nullptr;         // grid arrival counter, zero between launches
-    float eps = 0.f;
-};
-
 // Softmax statistics of a slice of one row of logits: running max, sum of exp(l - max), argmax
 // (lowest id on ties; [MASK] excluded by the producer).  Merged in a fixed order.
 struct ConfPartial {
@@ -180,7 +168,6 @@ struct GemmArgs {
     float* partial;        // fp32 [splits][M][N]
     __nv_bfloat16* act_out; // non-null: gate/up GEMM with the SwiGLU epilogue, writes bf16 [M][N = F]; splits == 1
     ConfEpilogue conf;                  // conf.part non-null: LM head fused with the confidence statistics, splits == 1
-    ResidualEpilogue residual;          // residual.h non-null: cluster split-K with the fused residual epilogue
     const float* row_scale = nullptr;   // per activation row m: the output is multiplied by row_scale[m]
                                         // (the 1/rms of an RMSNorm folded behind the projection); needs splits == 1
     int M, N, K;
@@ -188,7 +175,6 @@ struct GemmArgs {
     int* status;           // device status word
 };
 int gemm_pick_splits(int M, int N, int K);
-int gemm_cluster_splits(int M, int K);   // 8, 4 or 0 (residual epilogue not applicable)
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
 size_t packed_weight_bytes(int N, int K);
 size_t packed_gate_up_bytes(int F, int K);
@@ -234,6 +220,7 @@ struct AttnArgs {
     __nv_bfloat16* o;                     // [M][H*hd]
     float* part_o; float* part_ml;        // split workspaces [ks][M][H][hd], [ks][M][H][2]
     int layer, n_layers, H, hd, max_seq, M, ksplit;
+    int early = 0;                        // 1: tiles and cache were complete before the launch chain began (decode steps)
     L2Prefetch pf;
 };
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
