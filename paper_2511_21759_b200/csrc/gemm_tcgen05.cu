@@ -126,6 +126,60 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
                  : "memory");
 }
 
+// ---- CTA pair (cta_group::2): two CTAs of a cluster on neighbouring SMs issue ONE MMA of 256 weight rows.
+// Each CTA stages its own 128 weight rows and HALF of the activation rows; the leader (cluster rank 0)
+// issues the MMAs, which read both CTAs' shared memory and write both CTAs' TMEM.  TMA loads of both
+// CTAs report their bytes to the leader's barrier (the shared::cluster address with the pair bit cleared).
+constexpr uint32_t kPeerBitMask = 0xFEFFFFFFu;
+
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tmap, uint64_t* leader_bar, int c0, int c1,
+                                                 uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4}], [%2], %5;" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(leader_bar) & kPeerBitMask), "r"(c0), "r"(c1), "l"(hint)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_3d_pair(void* dst, const CUtensorMap* tmap, uint64_t* leader_bar, int c0, int c1,
+                                                 int c2, uint64_t hint) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%3, %4, %5}], [%2], %6;" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(leader_bar) & kPeerBitMask), "r"(c0), "r"(c1), "r"(c2), "l"(hint)
+        : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                               uint32_t accumulate) {
+    const uint32_t zero = 0;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, {%5, %5, %5, %5, %5, %5, %5, %5}, p;\n\t}" ::"r"(tmem_d),
+        "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(zero)
+        : "memory");
+}
+
+// arrives (once the MMAs issued so far have completed) at the barrier with this shared-memory offset in BOTH CTAs
+__device__ __forceinline__ void umma_commit_pair(uint64_t* bar) {
+    const uint16_t mask = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(
+                     smem_u32(bar)),
+                 "h"(mask)
+                 : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
@@ -158,7 +212,7 @@ struct alignas(8) GemmShared {
 // g[m][64 t + r]; N is then the FFN width F and there is no K split.
 constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_CONF = 3;
 
-template <int BN, int EPI>
+template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
             float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, const float* __restrict__ row_scale,
@@ -167,9 +221,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
-    constexpr uint32_t kBBytes = BN * kBK * 2;
+    constexpr int kBRows = PAIR ? BN / 2 : BN;        // activation rows this CTA stages
+    constexpr uint32_t kBBytes = kBRows * kBK * 2;
     constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    constexpr uint32_t kTxBytes = PAIR ? 2 * kStageBytes : kStageBytes;   // bytes reported to a full barrier
     constexpr uint32_t kTmemCols = BN < 32 ? 32 : BN;
+    const uint32_t pair_rank = PAIR ? cluster_ctarank() : 0u;
+    const bool leader = pair_rank == 0;
 
     uint8_t* tiles = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     GemmShared* sh = reinterpret_cast<GemmShared*>(tiles + static_cast<size_t>(stages) * kStageBytes);
@@ -203,14 +261,22 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     }
     if (warp == 1) {   // whole warp: allocate the accumulator's TMEM columns
         __syncwarp();
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                     "r"(kTmemCols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if constexpr (PAIR) {   // the same warp of both CTAs allocates the same columns in both SMs
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                         "r"(kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                         "r"(kTmemCols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    if constexpr (PAIR) cluster_barrier();   // the peer's barriers are initialised before anything signals them
     const uint32_t tmem_acc = sh->tmem_base;
 
     if (warp == 0) {
@@ -219,10 +285,15 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             // The weights do not depend on the preceding kernel: fill the ring with weight tiles
             // first, then wait for the predecessor and fetch the activation tiles.
             const int pre = nkb < stages ? nkb : stages;
+            const int mb = m0 + static_cast<int>(pair_rank) * kBRows;   // first activation row this CTA stages
             for (int i = 0; i < pre; ++i) {
-                mbar_expect_tx(&sh->full[i], kStageBytes);
-                tma_load_3d(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], 0, 0, wtile0 + i,
-                            kEvictFirst);
+                if (leader) mbar_expect_tx(&sh->full[i], kTxBytes);
+                if constexpr (PAIR)
+                    tma_load_3d_pair(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], 0, 0, wtile0 + i,
+                                     kEvictFirst);
+                else
+                    tma_load_3d(tiles + static_cast<size_t>(i) * kStageBytes, &tmap_w, &sh->full[i], 0, 0, wtile0 + i,
+                                kEvictFirst);
             }
             // and ask L2 for the weight tiles that follow, so that HBM keeps streaming while the
             // predecessor (a short elementwise kernel) is still running
@@ -234,9 +305,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                              "r"(0), "r"(0), "r"(wtile0 + i)
                              : "memory");
             pdl_wait();
-            for (int i = 0; i < pre; ++i)
-                tma_load_2d(tiles + static_cast<size_t>(i) * kStageBytes + kABytes, &tmap_x, &sh->full[i], (kb0 + i) * kBK,
-                            m0, kEvictLast);
+            for (int i = 0; i < pre; ++i) {
+                if constexpr (PAIR)
+                    tma_load_2d_pair(tiles + static_cast<size_t>(i) * kStageBytes + kABytes, &tmap_x, &sh->full[i],
+                                     (kb0 + i) * kBK, mb, kEvictLast);
+                else
+                    tma_load_2d(tiles + static_cast<size_t>(i) * kStageBytes + kABytes, &tmap_x, &sh->full[i], (kb0 + i) * kBK,
+                                mb, kEvictLast);
+            }
             int issued = pre;
             for (int i = pre; i < nkb; ++i) {
                 const int st = i % stages;
@@ -244,13 +320,19 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 if (!mbar_wait(&sh->empty[st], ph ^ 1u, cta_abort, status)) break;
                 uint8_t* a_dst = tiles + static_cast<size_t>(st) * kStageBytes;
                 uint8_t* b_dst = a_dst + kABytes;
-                mbar_expect_tx(&sh->full[st], kStageBytes);
-                tma_load_3d(a_dst, &tmap_w, &sh->full[st], 0, 0, wtile0 + i, kEvictFirst);
-                tma_load_2d(b_dst, &tmap_x, &sh->full[st], (kb0 + i) * kBK, m0, kEvictLast);
+                if (leader) mbar_expect_tx(&sh->full[st], kTxBytes);
+                if constexpr (PAIR) {
+                    tma_load_3d_pair(a_dst, &tmap_w, &sh->full[st], 0, 0, wtile0 + i, kEvictFirst);
+                    tma_load_2d_pair(b_dst, &tmap_x, &sh->full[st], (kb0 + i) * kBK, mb, kEvictLast);
+                } else {
+                    tma_load_3d(a_dst, &tmap_w, &sh->full[st], 0, 0, wtile0 + i, kEvictFirst);
+                    tma_load_2d(b_dst, &tmap_x, &sh->full[st], (kb0 + i) * kBK, mb, kEvictLast);
+                }
                 issued = i + 1;
             }
-            if (*cta_abort) {
-                // aborted: let the copies still in flight land before the CTA's shared memory goes away
+            if (*cta_abort && leader) {
+                // aborted: let the copies still in flight land before the CTA's shared memory goes away (the
+                // peer of a pair cannot observe its own copies; it is held by the cluster barrier at the end)
                 const int first = issued > stages ? issued - stages : 0;
                 for (int i = first; i < issued; ++i) {
                     const long long t0 = clock64();
@@ -261,9 +343,9 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
-            // ---- MMA issuer ----
-            constexpr uint32_t idesc = make_instr_desc(kBM, BN);
+        if (lane == 0 && leader) {
+            // ---- MMA issuer (the leader's, for both CTAs of a pair) ----
+            constexpr uint32_t idesc = make_instr_desc(PAIR ? 2 * kBM : kBM, BN);
             bool ok = true;
             for (int i = 0; i < nkb && ok; ++i) {
                 const int st = i % stages;
@@ -275,12 +357,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 const uint32_t b_addr = a_addr + kABytes;
 #pragma unroll
                 for (int k = 0; k < kBK / kUmmaK; ++k) {
-                    umma_bf16(tmem_acc, make_smem_desc(a_addr + k * kUmmaK * 2), make_smem_desc(b_addr + k * kUmmaK * 2),
-                              idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    if constexpr (PAIR)
+                        umma_bf16_pair(tmem_acc, make_smem_desc(a_addr + k * kUmmaK * 2), make_smem_desc(b_addr + k * kUmmaK * 2),
+                                       idesc, (i > 0 || k > 0) ? 1u : 0u);
+                    else
+                        umma_bf16(tmem_acc, make_smem_desc(a_addr + k * kUmmaK * 2), make_smem_desc(b_addr + k * kUmmaK * 2),
+                                  idesc, (i > 0 || k > 0) ? 1u : 0u);
                 }
-                umma_commit(&sh->empty[st]);   // frees the stage once these MMAs have read it
+                // frees the stage (in both CTAs of a pair) once these MMAs have read it
+                if constexpr (PAIR) umma_commit_pair(&sh->empty[st]);
+                else umma_commit(&sh->empty[st]);
             }
-            if (ok) umma_commit(&sh->acc_full);
+            if (ok) {
+                if constexpr (PAIR) umma_commit_pair(&sh->acc_full);
+                else umma_commit(&sh->acc_full);
+            }
         }
     } else {
         // ---- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 ----
@@ -398,10 +489,14 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     pdl_wait();   // every thread: keeps completion of the launch chain transitive
     tc_fence_before();
     __syncthreads();
+    if constexpr (PAIR) cluster_barrier();   // neither CTA's shared memory or TMEM goes away while its peer may touch it
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
+        if constexpr (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_acc), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -496,31 +591,48 @@ __global__ void pack_gate_up_kernel(const __nv_bfloat16* __restrict__ src, __nv_
     reinterpret_cast<uint4*>(dst)[chunk] = v;
 }
 
-int pick_bn(int M) {
-    static int max_bn = 0;
-    if (!max_bn) {
-        const char* e = getenv("ODB_GEMM_MAX_BN");
-        max_bn = e ? atoi(e) : 128;   // 128-row tiles run two CTAs per SM: one's epilogue overlaps the other's main loop
+// CTA pairs (cta_group::2) are used whenever the number of weight tiles is even (ODB_GEMM_PAIR=0 turns them off).
+bool pair_enabled() {
+    static int v = -1;
+    if (v < 0) {
+        const char* e = getenv("ODB_GEMM_PAIR");
+        v = e ? atoi(e) : 1;
     }
-    const int bn = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : 256;
-    return bn < max_bn ? bn : max_bn;
+    return v != 0;
 }
 
-template <int BN, int EPI>
-cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st) {
+int pick_bn(int M, bool pair) {
+    static int max_bn = -1;
+    if (max_bn < 0) {
+        const char* e = getenv("ODB_GEMM_MAX_BN");
+        max_bn = e ? atoi(e) : 0;
+    }
+    // Up to 128 rows per tile two CTAs share an SM (one's epilogue overlaps the other's main loop).  A CTA
+    // pair stages only half of the rows per CTA, so it affords 256-row tiles at the same occupancy.
+    int bn = M <= 32 ? 32 : M <= 64 ? 64 : M <= 128 ? 128 : pair ? 256 : 128;
+    if (max_bn > 0 && bn > max_bn) bn = max_bn;
+    return bn;
+}
+
+template <int BN, int EPI, bool PAIR>
+cudaError_t launch_bn(const GemmArgs& a, cudaStream_t st) {
     constexpr bool SWIGLU = EPI == EPI_SWIGLU;
+    constexpr int kBRows = PAIR ? BN / 2 : BN;
+    CUtensorMap tmx;
+    cudaError_t e = make_tmap_2d(&tmx, a.x, a.M, a.K, kBRows);
+    if (e != cudaSuccess) return e;
     const int nkb_total = (a.K + kBK - 1) / kBK;
     const int nkb_per_split = (nkb_total + a.splits - 1) / a.splits;
-    const uint32_t stage_bytes = kBM * kBK * 2 + BN * kBK * 2;
-    // two CTAs per SM up to 128 activation rows (hides each CTA's prologue and drain), one for 256
-    const uint32_t budget = BN <= 128 ? 100 * 1024 : 200 * 1024;
+    const uint32_t stage_bytes = kBM * kBK * 2 + kBRows * kBK * 2;
+    // two CTAs per SM as long as two accumulators fit TMEM and a CTA stages at most 128 rows
+    const uint32_t budget = kBRows <= 128 ? 100 * 1024 : 200 * 1024;
     int stages = static_cast<int>(budget / stage_bytes);
     if (stages > 16) stages = 16;
     if (stages > nkb_per_split) stages = nkb_per_split < 2 ? 2 : nkb_per_split;
     const size_t smem = static_cast<size_t>(stages) * stage_bytes + sizeof(GemmShared) + 1024;
     static bool attr_done = false;
     if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(gemm_kernel<BN, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        e = cudaFuncSetAttribute(gemm_kernel<BN, EPI, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
@@ -528,23 +640,57 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& tmx, cudaStream_t st
     dim3 grid(SWIGLU ? (a.N + 63) / 64 : (a.N + kBM - 1) / kBM, (a.M + BN - 1) / BN, a.splits);
     static int l2_prefetch = -1;
     if (l2_prefetch < 0) {
-        const char* e = getenv("ODB_GEMM_L2_PREFETCH");
-        l2_prefetch = e ? atoi(e) : 0;   // measured: prefetching into L2 slows the step down
+        const char* env = getenv("ODB_GEMM_L2_PREFETCH");
+        l2_prefetch = env ? atoi(env) : 0;   // measured: prefetching into L2 slows the step down
     }
-    return launch_kernel(gemm_kernel<BN, EPI>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
-                         a.row_scale, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
-                         pdl_enabled() ? l2_prefetch : 0, a.status);
+    if constexpr (PAIR) {
+        if (grid.x & 1) return cudaErrorInvalidValue;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = grid;
+        cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = st;
+        cudaLaunchAttribute attr[2];
+        attr[0].id = cudaLaunchAttributeClusterDimension;   // neighbouring weight tiles form the pair
+        attr[0].val.clusterDim.x = 2;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = pdl_enabled() ? 2 : 1;
+        return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI, PAIR>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.conf,
+                                  a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
+    } else {
+        return launch_kernel(gemm_kernel<BN, EPI, PAIR>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
+                             a.row_scale, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
+                             pdl_enabled() ? l2_prefetch : 0, a.status);
+    }
 }
 
 template <int EPI>
-cudaError_t launch_epi(const GemmArgs& a, const CUtensorMap& tmx, int bn, cudaStream_t st) {
+cudaError_t launch_epi(const GemmArgs& a, int bn, bool pair, cudaStream_t st) {
+    if (pair) {
+        switch (bn) {
+            case 32: return launch_bn<32, EPI, true>(a, st);
+            case 64: return launch_bn<64, EPI, true>(a, st);
+            case 128: return launch_bn<128, EPI, true>(a, st);
+            default: return launch_bn<256, EPI, true>(a, st);
+        }
+    }
     switch (bn) {
-        case 32: return launch_bn<32, EPI>(a, tmx, st);
-        case 64: return launch_bn<64, EPI>(a, tmx, st);
-        case 128: return launch_bn<128, EPI>(a, tmx, st);
-        default: return launch_bn<256, EPI>(a, tmx, st);
+        case 32: return launch_bn<32, EPI, false>(a, st);
+        case 64: return launch_bn<64, EPI, false>(a, st);
+        case 128: return launch_bn<128, EPI, false>(a, st);
+        default: return launch_bn<256, EPI, false>(a, st);
     }
 }
+
+// Whether a projection of M activation rows with n_tiles weight tiles runs as CTA pairs.  Measured on the
+// 8B shape: with many rows (refresh, 768..1024 rows: tensor/L2 bound) pairs with 256-row tiles are 11 %
+// faster than single CTAs with 128-row tiles; up to 128 rows (decode steps: HBM bound) the pair's extra
+// synchronisation costs more than the halved activation traffic saves (3.55 vs 3.41 ms at 32 rows).
+bool use_pair(int M, int n_tiles) { return pair_enabled() && M > 128 && (n_tiles & 1) == 0; }
 
 }  // namespace
 
@@ -598,15 +744,21 @@ static int target_ctas() {
 }
 
 int gemm_pick_splits(int M, int N, int K) {
-    const int bn = pick_bn(M);
-    const int tiles = ((N + kBM - 1) / kBM) * ((M + bn - 1) / bn);
+    const int n_tiles = (N + kBM - 1) / kBM;
+    const int bn = pick_bn(M, use_pair(M, n_tiles));
+    const int tiles = n_tiles * ((M + bn - 1) / bn);
     const int nkb = (K + kBK - 1) / kBK;
     // all work units must be resident at once (two CTA slots per SM) and equal in size: a
     // second, partly filled wave would double the kernel's time
     if (M > 128) {
         // many rows (refresh): compute bound, and every K split costs M x N fp32 partials written and
         // read back, so split only when the tiles alone cannot occupy the SMs
-        int sp = tiles >= 148 ? 1 : 148 / tiles;
+        static int big_target = 0;
+        if (!big_target) {
+            const char* e = getenv("ODB_GEMM_BIG_TARGET_CTAS");
+            big_target = e ? atoi(e) : 296;
+        }
+        int sp = tiles >= big_target ? 1 : big_target / tiles;
         if (sp > nkb / 8) sp = nkb / 8;
         return sp < 1 ? 1 : sp;
     }
@@ -620,19 +772,18 @@ int gemm_pick_splits(int M, int N, int K) {
 }
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
-    const int bn = pick_bn(a.M);
-    CUtensorMap tmx;
-    cudaError_t e = make_tmap_2d(&tmx, a.x, a.M, a.K, bn);
-    if (e != cudaSuccess) return e;
-    if (a.act_out) {
+    const bool swiglu = a.act_out != nullptr;
+    const bool pair = use_pair(a.M, swiglu ? (a.N + 63) / 64 : (a.N + kBM - 1) / kBM);
+    const int bn = pick_bn(a.M, pair);
+    if (swiglu) {
         if (a.splits != 1) return cudaErrorInvalidValue;
-        return launch_epi<EPI_SWIGLU>(a, tmx, bn, st);
+        return launch_epi<EPI_SWIGLU>(a, bn, pair, st);
     }
     if (a.conf.part) {
         if (a.splits != 1) return cudaErrorInvalidValue;
-        return launch_epi<EPI_CONF>(a, tmx, bn, st);
+        return launch_epi<EPI_CONF>(a, bn, pair, st);
     }
-    return launch_epi<EPI_PARTIAL>(a, tmx, bn, st);
+    return launch_epi<EPI_PARTIAL>(a, bn, pair, st);
 }
 
 cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,

@@ -22,7 +22,10 @@ def _case(M, N, K, seed):
     (64, 1376, 256, 0),       # N tail: 1376 = 10 * 128 + 96; 64-row tile
     (100, 2048, 256, 0),      # ragged rows inside a 128-row tile
     (128, 512, 1024, 4),
-    (300, 640, 512, 0),       # two 256-row tiles, second ragged
+    (300, 640, 512, 0),       # many rows, odd number of weight tiles (5): single-CTA tiles of 128 rows, last ragged
+    (300, 768, 512, 0),       # many rows, even number of weight tiles: CTA pairs, two 256-row tiles, second ragged
+    (700, 1024, 688, 2),      # CTA pairs with a K split and a K tail; three row tiles, last ragged (188 rows)
+    (129, 256, 64, 1),        # CTA pair, one k-block, one row beyond the first half of the second CTA's rows
     (1, 128, 64, 1),          # smallest
     (48, 2048, 2048, 0),
 ])
