@@ -38,53 +38,47 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
     }
 }
 
-// One block per output row: the part of RMSNorm that is not a row scalar.  x = residual stream row
-// (after adding the split-K partials of the preceding projection in split order); writes
-// bf16(x * gain) as the projection's operand and 1 / sqrt(mean(x^2) + eps) for the projection's
-// consumer (the scalar commutes with the matrix product).  float4 accesses.
-__global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
-                                                       int splits, size_t pstride, const float* __restrict__ gain,
-                                                       __nv_bfloat16* __restrict__ out, float* __restrict__ inv_rms,
-                                                       const int32_t* __restrict__ row_map, int d, float eps,
-                                                       L2Prefetch pf) {
+// grid (output rows, slices of kNormSliceCols columns), one float4 per thread: the part of RMSNorm that is
+// not a row scalar.  x = residual stream row (after adding the split-K partials of the preceding projection
+// in split order; all splits are requested at once, one memory round trip); writes bf16(x * gain) as the
+// projection's operand and this slice's sum(x^2) for the projection's consumer.
+__global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
+                                                                     int splits, size_t pstride, const float* __restrict__ gain,
+                                                                     __nv_bfloat16* __restrict__ out, float* __restrict__ ssq,
+                                                                     const int32_t* __restrict__ row_map, int d, L2Prefetch pf) {
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
-    l2_prefetch_slice(pf, blockIdx.x, gridDim.x);
+    l2_prefetch_slice(pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
     const int orow = blockIdx.x;
     const int row = row_map ? row_map[orow] : orow;
-    float* hr = h + static_cast<size_t>(row) * d;
-    const int nvec = d >> 2, stride = blockDim.x;
+    const int i = blockIdx.y * (kNormSliceCols / 4) + threadIdx.x;   // float4 index within the row
     float ss = 0.f;
-    __nv_bfloat16* o = out + static_cast<size_t>(orow) * d;
-    for (int i = threadIdx.x; i < nvec; i += stride) {
+    if (i < (d >> 2)) {
+        float* hr = h + static_cast<size_t>(row) * d;
         float4 v = reinterpret_cast<const float4*>(hr)[i];
         if (partial) {
-            // split order is fixed; groups of four loads are issued together (uniform guard) so the
-            // reduction costs one memory round trip per group instead of one per split
             const float* p = partial + static_cast<size_t>(row) * d + 4 * i;
-            for (int sb = 0; sb < splits; sb += 4) {
-                float4 t[4];
+            float4 t[16];
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (sb + u < splits) t[u] = *reinterpret_cast<const float4*>(p + static_cast<size_t>(sb + u) * pstride);
+            for (int u = 0; u < 16; ++u)
+                if (u < splits) t[u] = *reinterpret_cast<const float4*>(p + static_cast<size_t>(u) * pstride);
 #pragma unroll
-                for (int u = 0; u < 4; ++u)
-                    if (sb + u < splits) { v.x += t[u].x; v.y += t[u].y; v.z += t[u].z; v.w += t[u].w; }
-            }
+            for (int u = 0; u < 16; ++u)
+                if (u < splits) { v.x += t[u].x; v.y += t[u].y; v.z += t[u].z; v.w += t[u].w; }
             reinterpret_cast<float4*>(hr)[i] = v;
         }
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        ss = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
         const float4 g = reinterpret_cast<const float4*>(gain)[i];
         const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x * g.x, v.y * g.y);
         const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z * g.z, v.w * g.w);
         uint2 pk;
         pk.x = *reinterpret_cast<const uint32_t*>(&lo);
         pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-        reinterpret_cast<uint2*>(o)[i] = pk;
+        reinterpret_cast<uint2*>(out + static_cast<size_t>(orow) * d)[i] = pk;
     }
     const float total = block_sum(ss, red);
-    if (threadIdx.x == 0) inv_rms[orow] = 1.0f / sqrtf(total / static_cast<float>(d) + eps);
+    if (threadIdx.x == 0) ssq[static_cast<size_t>(orow) * gridDim.y + blockIdx.y] = total;
 }
 
 // grid (rows, pair chunks), one thread per rotation pair.  Sums the QKV partials, rotates q and k (rotate-half pairing: element i
@@ -129,7 +123,7 @@ __global__ void qkv_rope_kernel(QkvRopeArgs a) {
                 }
             }
         }
-        const float inv = a.inv_rms[row];               // scalar of the RMSNorm folded behind the projection
+        const float inv = row_scale_of(a.scale, row);   // scalar of the RMSNorm folded behind the projection
         q0 *= inv; q1 *= inv; k0 *= inv; k1 *= inv; v0 *= inv; v1 *= inv;
         const float2 cs = rope[i];
         const __nv_bfloat16 rq0 = __float2bfloat16_rn(q0 * cs.x - q1 * cs.y);
@@ -229,12 +223,12 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 }
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, float* inv_rms, const int32_t* row_map, int rows_out, int d, float eps,
-                           L2Prefetch pf, cudaStream_t st) {
-    int threads = ((d / 4 + 31) / 32) * 32;
-    if (threads > 1024) threads = 1024;
-    return launch_kernel(rmsnorm_kernel, dim3(rows_out), dim3(threads), 0, st, h, partial, splits, pstride, gain, out, inv_rms,
-                         row_map, d, eps, pf);
+                           __nv_bfloat16* out, float* ssq, const int32_t* row_map, int rows_out, int d, L2Prefetch pf,
+                           cudaStream_t st) {
+    if (splits > 16) return cudaErrorInvalidValue;
+    const int slices = (d + kNormSliceCols - 1) / kNormSliceCols;
+    return launch_kernel(rmsnorm_kernel, dim3(rows_out, slices), dim3(kNormSliceCols / 4), 0, st, h, partial, splits, pstride,
+                         gain, out, ssq, row_map, d, pf);
 }
 
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {

@@ -203,6 +203,7 @@ struct alignas(8) GemmShared {
     uint64_t acc_full;
     uint32_t tmem_base;
     int abort;
+    float scale[256];      // RowScale of the tile's activation rows
 };
 
 // BN: activation rows per tile (MMA N): 32, 64, 128 or 256.
@@ -215,7 +216,7 @@ constexpr int EPI_PARTIAL = 0, EPI_SWIGLU = 1, EPI_CONF = 3;
 template <int BN, int EPI, bool PAIR>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-            float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, const float* __restrict__ row_scale,
+            float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, RowScale rs,
             ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
             int l2_prefetch,
             int* status) {
@@ -376,7 +377,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     } else {
         // ---- epilogue: warps 2..5 own TMEM lanes 32*(warp%4) .. +31 ----
         const int q = warp & 3;
-        pdl_wait();   // the previous reader of the output buffer has finished
+        pdl_wait();   // the previous reader of the output buffer has finished; the predecessor's results are visible
+        if (rs.ssq) {   // uniform: row scalars of this tile's activation rows, computed while the main loop runs
+            for (int i = threadIdx.x - 64; i < BN; i += 128) sh->scale[i] = m0 + i < M ? row_scale_of(rs, m0 + i) : 1.0f;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+        }
         const bool ok = nkb > 0 && mbar_wait(&sh->acc_full, 0, cta_abort, status);   // nkb == 0: empty K split
         if (ok) tc_fence_after();
         if constexpr (EPI == EPI_PARTIAL) {
@@ -388,13 +393,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                     uint32_t v[32];
                     tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                    // lane j holds the scale of activation row m0 + 32 c + j; broadcast per column
-                    const int ms = m0 + c * 32 + lane;
-                    const float my_scale = (row_scale && ms < M) ? row_scale[ms] : 1.0f;
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + c * 32 + j;
-                        const float sc = __shfl_sync(0xffffffffu, my_scale, j);
+                        const float sc = rs.ssq ? sh->scale[c * 32 + j] : 1.0f;
                         if (n < N && m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]) * sc;
                     }
                 }
@@ -420,7 +422,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 asm volatile("bar.sync 1, 128;" ::: "memory");
                 const int m_l = t >> 2, part = t & 3;
                 const int m = m0 + c * 32 + m_l;
-                const float sc = (row_scale && m < M) ? row_scale[m] : 1.0f;
+                const float sc = rs.ssq ? sh->scale[c * 32 + m_l] : 1.0f;
                 float mx = -INFINITY, sum = 0.f;
                 int idx = 0x7fffffff;
 #pragma unroll 8
@@ -468,13 +470,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                     for (int j = 0; j < 32; ++j) xch[((q & 1) * 32 + lane) * 33 + j] = __uint_as_float(v[j]);
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int ms = m0 + c * 32 + lane;
-                const float my_scale = (row_scale && ms < M) ? row_scale[ms] : 1.0f;
                 if (ok && q < 2) {
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         const int m = m0 + c * 32 + j;
-                        const float sc = __shfl_sync(0xffffffffu, my_scale, j);
+                        const float sc = rs.ssq ? sh->scale[c * 32 + j] : 1.0f;
                         if (m < M && f < N) {
                             const float gate = __uint_as_float(v[j]) * sc;
                             const float up = xch[((q & 1) * 32 + lane) * 33 + j] * sc;

@@ -81,7 +81,7 @@ Layout make_layout(const odb_config& c) {
     L.step_tile_buf = take(sizeof(StepTile) * static_cast<size_t>(c.max_batch) * c.max_copies);
     L.h = take(4 * L.rows * d);
     L.a = take(2 * L.rows * d);
-    L.inv = take(4 * L.rows);
+    L.inv = take(4 * L.rows * ((d + kNormSliceCols - 1) / kNormSliceCols));   // sum-of-squares slices of the current RMSNorm
     L.q = take(2 * L.rows * d);
     L.k = take(2 * L.rows * d);
     L.v = take(2 * L.rows * d);
@@ -420,7 +420,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     const int d = c.d_model, F = c.d_ffn, H = c.n_heads, hd = c.head_dim;
     float* h = s->at<float>(L.h);
     __nv_bfloat16* a = s->at<__nv_bfloat16>(L.a);
-    float* inv = s->at<float>(L.inv);   // 1/rms of the RMSNorm whose operand is in `a`
+    float* inv = s->at<float>(L.inv);   // sum(x^2) slices of the RMSNorm whose operand is in `a`
+    RowScale inv_scale;
+    inv_scale.ssq = inv;
+    inv_scale.slots = (d + kNormSliceCols - 1) / kNormSliceCols;
+    inv_scale.inv_d = 1.0f / static_cast<float>(d);
+    inv_scale.eps = c.rms_eps;
     __nv_bfloat16* q = s->at<__nv_bfloat16>(L.q);
     __nv_bfloat16* k = s->at<__nv_bfloat16>(L.k);
     __nv_bfloat16* v = s->at<__nv_bfloat16>(L.v);
@@ -431,13 +436,13 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     const size_t nmax = 3 * static_cast<size_t>(d) > 2 * static_cast<size_t>(F) ? 3 * static_cast<size_t>(d)
                                                                                 : 2 * static_cast<size_t>(F);
     auto gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, float* out, int rows, int N, int K, int* splits,
-                    const float* row_scale = nullptr) {
+                    const RowScale* row_scale = nullptr) {
         GemmArgs ga;
         ga.tmap_w = tw;
         ga.x = x;
         ga.partial = out;
         ga.act_out = nullptr;
-        ga.row_scale = row_scale;
+        if (row_scale) ga.row_scale = *row_scale;
         ga.M = rows; ga.N = N; ga.K = K;
         int sp = *splits > 0 ? *splits : gemm_pick_splits(rows, N, K);
         const size_t cap = L.partial_rows * nmax / (static_cast<size_t>(rows) * N);
@@ -480,12 +485,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
                  gu_bytes = packed_gate_up_bytes(F, d);
     for (int l = 0; l < c.n_layers; ++l) {
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
-                                                        c.rms_eps, hint_of(m->p_qkv[l], qkv_bytes, 0), st));
+                                                        hint_of(m->p_qkv[l], qkv_bytes, 0), st));
         int sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
         QkvRopeArgs qa;
         qa.partial = partial; qa.splits = sp; qa.pstride = static_cast<size_t>(M) * 3 * d;
-        qa.inv_rms = inv;
+        qa.scale = inv_scale;
         qa.rope = s->at<float2>(L.rope);
         qa.row_pos = s->cb.row_pos; qa.row_seq = s->cb.row_seq;
         qa.q = q; qa.k = k; qa.v = v;
@@ -525,14 +530,14 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         sp = 0;
         ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
-                                                        d, c.rms_eps, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
+                                                        d, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
         {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
             GemmArgs ga;
             ga.tmap_w = m->tm_gu[l];
             ga.x = a;
             ga.partial = nullptr;
             ga.act_out = g;
-            ga.row_scale = inv;
+            ga.row_scale = inv_scale;
             ga.M = M; ga.N = F; ga.K = d;
             ga.splits = 1;
             ga.status = status;
@@ -545,16 +550,16 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
-                                                        c.rms_eps, L2Prefetch{nullptr, 0}, st));
+                                                        L2Prefetch{nullptr, 0}, st));
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
     for (int r0 = 0; r0 < n_lm; r0 += static_cast<int>(L.lm_chunk)) {
         const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
         const __nv_bfloat16* x = a;
-        const float* scale = inv;
+        const RowScale* scale = &inv_scale;
         ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
-                                                        rows, d, c.rms_eps, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
+                                                        rows, d, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
         if (s->dump_logits) {
             int sp = 1;
             ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, &sp, scale));
@@ -568,7 +573,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             ga.x = x;
             ga.partial = nullptr;
             ga.act_out = nullptr;
-            ga.row_scale = scale;
+            ga.row_scale = *scale;
             ga.conf.part = reinterpret_cast<ConfPartial*>(s->ws + L.conf_part);
             ga.conf.mask_id = c.mask_id;
             ga.M = rows; ga.N = c.vocab; ga.K = d;

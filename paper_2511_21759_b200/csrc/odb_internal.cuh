@@ -132,6 +132,26 @@ constexpr int kRowDecoded = 1;   // row_flags bit: the row's position is decoded
 
 struct TmaEncoder;   // wraps the driver's tensor-map encode entry point
 
+// The row scalar of an RMSNorm folded behind a projection, kept as the partial sums of x^2 its producer
+// wrote (one per 1024-column slice of the row): scale[m] = 1 / sqrt(sum_t ssq[m * slots + t] / d + eps),
+// summed in slot order.  ssq null: scale 1.
+struct RowScale {
+    const float* ssq = nullptr;
+    int slots = 0;
+    float inv_d = 0.f, eps = 0.f;
+};
+constexpr int kNormSliceCols = 1024;   // columns of a row one RMSNorm block handles
+
+#ifdef __CUDACC__
+__device__ __forceinline__ float row_scale_of(const RowScale& rs, int m) {
+    if (!rs.ssq) return 1.0f;
+    const float* p = rs.ssq + static_cast<size_t>(m) * rs.slots;
+    float t = 0.f;
+    for (int i = 0; i < rs.slots; ++i) t += p[i];
+    return 1.0f / sqrtf(t * rs.inv_d + rs.eps);
+}
+#endif
+
 // Softmax statistics of a slice of one row of logits: running max, sum of exp(l - max), argmax
 // (lowest id on ties; [MASK] excluded by the producer).  Merged in a fixed order.
 struct ConfPartial {
@@ -168,7 +188,7 @@ struct GemmArgs {
     float* partial;        // fp32 [splits][M][N]
     __nv_bfloat16* act_out; // non-null: gate/up GEMM with the SwiGLU epilogue, writes bf16 [M][N = F]; splits == 1
     ConfEpilogue conf;                  // conf.part non-null: LM head fused with the confidence statistics, splits == 1
-    const float* row_scale = nullptr;   // per activation row m: the output is multiplied by row_scale[m]
+    RowScale row_scale;                 // per activation row m: the output is multiplied by scale[m]
                                         // (the 1/rms of an RMSNorm folded behind the projection); needs splits == 1
     int M, N, K;
     int splits;
@@ -187,15 +207,17 @@ cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stri
 
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d,
                          cudaStream_t st);
-// RMSNorm feeding a projection, with the row scalar deferred: h[row] += sum_s partial[s][row] (if
-// partial); out[i] = bf16(h[r] * gain), inv_rms[i] = 1 / sqrt(mean(h[r]^2) + eps), r = map ? map[i] : i.
-// The projection's consumer multiplies its fp32 output by inv_rms (the scalar commutes with the GEMM).
+// The part of RMSNorm that is not a row scalar, for rows r = map ? map[i] : i of the residual stream:
+// h[r] += sum_s partial[s][r] (if partial; split order), out[i] = bf16(h[r] * gain) is the projection's
+// operand, ssq[i][t] = sum of h[r]^2 over the t-th slice of kNormSliceCols columns; the projection's consumer
+// multiplies its fp32 output by 1 / sqrt(sum_t ssq / d + eps) (RowScale; the scalar commutes with the matrix
+// product).  splits <= 16.
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
-                           __nv_bfloat16* out, float* inv_rms, const int32_t* row_map, int rows_out, int d, float eps,
-                           L2Prefetch pf, cudaStream_t st);
+                           __nv_bfloat16* out, float* ssq, const int32_t* row_map, int rows_out, int d, L2Prefetch pf,
+                           cudaStream_t st);
 struct QkvRopeArgs {
     const float* partial; int splits; size_t pstride;      // [splits][M][3d]
-    const float* inv_rms;                                  // [M] scalar of the preceding RMSNorm
+    RowScale scale;                                        // scalar of the preceding RMSNorm
     const float2* rope;                                    // [max_seq][hd/2] (cos, sin)
     const int32_t* row_pos; const int32_t* row_seq;
     __nv_bfloat16 *q, *k, *v;                              // [M][d]
