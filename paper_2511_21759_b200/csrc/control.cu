@@ -21,9 +21,9 @@ __global__ void build_refresh_rows_kernel(ControlBuffers c, int batch, BlockInde
         if (threadIdx.x == 0) st->in_fwd = 0;
         return;
     }
-    __shared__ int row0, lm0, tile0;
+    __shared__ int row0, lm0, tile0, big0;
     if (threadIdx.x == 0) {
-        int r = 0, l = 0, t = 0;
+        int r = 0, l = 0, t = 0, tb = 0;
         for (int j = 0; j < seq; ++j) {
             const SeqState* o = c.state + j;
             if (!o->active || bp.block_index[j] < 0) continue;
@@ -31,8 +31,9 @@ __global__ void build_refresh_rows_kernel(ControlBuffers c, int batch, BlockInde
             r += o->T;
             l += o->T - sj;
             t += (o->T + 63) / 64;
+            tb += (o->T + 127) / 128;
         }
-        row0 = r; lm0 = l; tile0 = t;
+        row0 = r; lm0 = l; tile0 = t; big0 = tb;
         const int s = st->P + bp.block_index[seq] * bp.block_len;
         st->in_fwd = 1;
         st->block_idx = bp.block_index[seq];
@@ -70,6 +71,16 @@ __global__ void build_refresh_rows_kernel(ControlBuffers c, int batch, BlockInde
         q.f0 = row0; q.n0 = T;
         q.f1 = 0; q.n1 = 0;
         c.tiles[tile0 + j] = q;
+    }
+    for (int j = threadIdx.x; j < (T + 127) / 128; j += blockDim.x) {
+        QTile q;
+        q.q_row0 = row0 + 128 * j;
+        q.nq = min(128, T - 128 * j);
+        q.seq = seq;
+        q.cA = 0; q.cB0 = 0; q.cB1 = 0;
+        q.f0 = row0; q.n0 = T;
+        q.f1 = 0; q.n1 = 0;
+        c.big_tiles[big0 + j] = q;
     }
 }
 

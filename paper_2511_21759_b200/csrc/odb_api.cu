@@ -46,7 +46,7 @@ int32_t check_config(const odb_config* c) {
 // odb_session_create so that both always agree.
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
-    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, step_tile_buf;
+    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
     size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
     size_t total;
 };
@@ -78,6 +78,7 @@ Layout make_layout(const odb_config& c) {
     L.row_flags = take(4 * L.rows);
     L.lm_rows = take(4 * L.rows);
     L.tile_buf = take(sizeof(QTile) * L.tiles);
+    L.big_tile_buf = take(sizeof(QTile) * static_cast<size_t>(c.max_batch) * ((c.max_seq + 127) / 128));
     L.step_tile_buf = take(sizeof(StepTile) * static_cast<size_t>(c.max_batch) * c.max_copies);
     L.h = take(4 * L.rows * d);
     L.a = take(2 * L.rows * d);
@@ -291,6 +292,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     cb.row_flags = s->at<int32_t>(L.row_flags);
     cb.lm_rows = s->at<int32_t>(L.lm_rows);
     cb.tiles = s->at<QTile>(L.tile_buf);
+    cb.big_tiles = s->at<QTile>(L.big_tile_buf);
     cb.step_tiles = s->at<StepTile>(L.step_tile_buf);
     cb.conf = s->at<float>(L.conf);
     cb.tok = s->at<int32_t>(L.tok);
@@ -412,7 +414,7 @@ struct LaunchScope {
 };
 
 // One forward over the M rows of the row table already built on the device.
-int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0) {
+int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0, int n_big_tiles = 0) {
     const odb_model* m = s->m;
     const odb_config& c = m->cfg;
     const Layout& L = s->L;
@@ -463,6 +465,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     int res_splits = 0;
     size_t res_stride = 0;
     static const int ks_env = getenv("ODB_ATTN_KS") ? atoi(getenv("ODB_ATTN_KS")) : 0;
+    static const bool tc_attention = !(getenv("ODB_ATTN_TC") && getenv("ODB_ATTN_TC")[0] == '0');
     int ks = (2 * 148 + n_tiles * H - 1) / (n_tiles * H);
     if (ks_env > 0 && !write_cache) ks = ks_env;
     if (ks > 8) ks = 8;
@@ -516,6 +519,15 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             sa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
             ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
             ++s->launches[ODB_KIND_ATTENTION];
+        } else if (write_cache && hd == 128 && n_big_tiles > 0 && tc_attention) {
+            // refresh with head dim 128: 128-row work items on the tcgen05 tensor cores, no key split
+            AttnArgs aa;
+            aa.tiles = s->cb.big_tiles; aa.n_tiles = n_big_tiles;
+            aa.q = q; aa.k = k; aa.v = v; aa.cache = s->kv; aa.row_flags = s->cb.row_flags; aa.o = o;
+            aa.part_o = nullptr; aa.part_ml = nullptr;
+            aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = 1;
+            aa.pf = L2Prefetch{nullptr, 0};
+            ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_tc(aa, status, st));
         } else {
         AttnArgs aa;
         aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
@@ -604,7 +616,7 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
     const odb_config& c = s->m->cfg;
     if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
     if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;   // an accept is pending
-    int M = 0, n_lm = 0, n_tiles = 0;
+    int M = 0, n_lm = 0, n_tiles = 0, n_big = 0;
     for (int i = 0; i < c.max_batch; ++i) {
         const SeqState& st = s->mirror[i];
         if (!st.active || block_index[i] < 0) continue;
@@ -613,10 +625,11 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
         M += st.T;
         n_lm += st.T - bs;
         n_tiles += (st.T + 63) / 64;
+        n_big += (st.T + 127) / 128;
     }
     if (M == 0) return ODB_ERR_STATE;
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
-    int32_t rc = forward(s, M, c.with_lm_head ? n_lm : 0, n_tiles, true);
+    int32_t rc = forward(s, M, c.with_lm_head ? n_lm : 0, n_tiles, true, 0, n_big);
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
     s->last_lm_rows = n_lm;

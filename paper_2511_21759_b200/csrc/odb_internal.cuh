@@ -246,6 +246,9 @@ struct AttnArgs {
     L2Prefetch pf;
 };
 cudaError_t launch_attention(const AttnArgs& a, cudaStream_t st);
+// refresh attention on the tcgen05 tensor cores (head dim 128): a.tiles = work items of up to 128 query rows
+// whose keys are the fresh rows [f0, f0 + n0); status = device status word (bounded waits)
+cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st);
 
 // Decode-step attention over StepTiles (copies of a block share the cached K/V loads).
 struct StepAttnArgs {
@@ -268,6 +271,7 @@ struct ControlBuffers {
     int32_t* row_tok; int32_t* row_pos; int32_t* row_seq; int32_t* row_copy; int32_t* row_flags;
     int32_t* lm_rows;         // rows whose logits are needed
     QTile* tiles;
+    QTile* big_tiles;         // refresh: the same rows cut into work items of up to 128 query rows
     StepTile* step_tiles;     // decode steps with more than one copy
     const float* conf; const int32_t* tok;   // outputs of the last forward, per logit row
     odb_result* results;      // [batch] device copy

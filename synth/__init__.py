@@ -75,6 +75,9 @@ TINY = ModelShape(n_layers=2, d_model=256, n_heads=4, head_dim=64, d_ffn=688, vo
 # confidences straddle the accept threshold, so the threshold branch, multi-token accepts and
 # jump-share misses all occur (they never do with N(0, 0.02) weights)
 TINY_PEAKY = dataclasses.replace(TINY, w_std=0.0625, lm_std=0.5)
+# the tiny model with the 8B shape's head dimension (2 heads of 128): exercises the kernels that exist
+# for head dim 128 only, at a size the oracle finishes in seconds
+TINY_HD128 = dataclasses.replace(TINY, n_heads=2, head_dim=128)
 LLADA_8B = ModelShape(n_layers=32, d_model=4096, n_heads=32, head_dim=128, d_ffn=12288,
                       vocab=126464, mask_id=126336, eos_id=126081)
 

@@ -20,6 +20,10 @@ CASES = [
     ("block_3_c4",      "TINY_PEAKY", 17, 10, 3,    4,      None),   # fewer masked positions than candidate ranks
     ("block64_c8",      "TINY_PEAKY", 64, 128, 64,  8,      None),   # 512 query rows per step: the largest step
     ("long_2048",       "TINY",      1984, 64, 32,  4,      12),     # the longest sequence: 16 key splits in the step
+    # head dim 128: the refresh attention runs on the tcgen05 tensor cores (128-row work items, 64-key tiles)
+    ("hd128_ragged",    "TINY_HD128", 150, 77, 16,  4,      None),   # T = 227: second row tile 99 rows, last key tile 35 keys
+    ("hd128_one_tile",  "TINY_HD128", 20,  30, 16,  1,      None),   # T = 50: a single ragged row tile and key tile
+    ("hd128_long",      "TINY_HD128", 1000, 64, 32, 8,      6),      # T = 1064: 9 row tiles x 17 key tiles
 ]
 
 
