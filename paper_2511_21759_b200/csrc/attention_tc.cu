@@ -8,12 +8,14 @@
 //   pass 2  P = exp2(S - max), row sums, P rounded to a two-term bf16 sum (value + remainder, as in the
 //           mma.sync kernel) and written to shared memory as the A operand of O += P V
 //           (128 x 128 x 64, V taken MN-major straight from its [key][dim] tile), O in TMEM.
-// Exact softmax, no rescaling of O.  Q, K, V tiles are staged with 16-byte cp.async in the canonical
-// 128-byte-swizzled layout the MMA descriptors expect (two 64-column atoms per 128-wide row).
-// S is double buffered in TMEM and K in shared memory: the MMAs of tile t + 1 are issued before the
-// softmax of tile t.  Two CTAs share an SM (112 KB of shared memory, 256 TMEM columns each).  Every
-// mbarrier wait is bounded; on expiry the CTA records ODB_ERR_TIMEOUT, stops issuing work, releases its
-// TMEM and exits.
+// Exact softmax, no rescaling of O.  Warp-specialised: warps 0..3 = softmax (one query row per thread),
+// warp 4 lane 0 = MMA issuer, warp 5 lane 0 = loader (TMA: boxes of 64 rows x 64 columns with the 128-byte
+// swizzle land in the canonical operand layout, two 64-column atoms per 128-wide row; rows past the
+// forward's last row read as zero, rows of a neighbouring sequence are masked in the softmax).  S is double buffered in TMEM and K in shared
+// memory, so S(t + 1) is computed while the softmax warps work on tile t and P V(t) while they work on
+// tile t + 1; the roles meet only through mbarriers.  Two CTAs share an SM (112 KB of shared memory, 256
+// TMEM columns each).  Every mbarrier wait is bounded; on expiry the CTA records ODB_ERR_TIMEOUT, every
+// role stops, the CTA releases its TMEM and exits.
 #include "odb_internal.cuh"
 
 namespace odb {
@@ -23,22 +25,29 @@ namespace {
 constexpr int kTQ = 128;   // query rows per work item (MMA M)
 constexpr int kTK = 64;    // keys per tile
 constexpr int kHD = 128;
-constexpr int kThreads = 128;
+constexpr int kThreads = 192;   // 4 softmax warps, MMA warp, loader warp
 constexpr long long kWaitLimitCycles = 4000000000ll;
 
 constexpr uint32_t kQBytes = kTQ * kHD * 2;          // 32 KB: two atoms of 128 rows x 128 B
 constexpr uint32_t kKBytes = kTK * kHD * 2;          // 16 KB: two atoms of 64 rows x 128 B
 constexpr uint32_t kPBytes = kTQ * kTK * 2;          // 16 KB: one atom of 128 rows x 128 B
-constexpr uint32_t kSmemBytes = kQBytes + 3 * kKBytes + 2 * kPBytes + 64;   // the dynamic region starts 1024-aligned
+constexpr uint32_t kSmemBytes = kQBytes + 3 * kKBytes + 2 * kPBytes + 128;   // the dynamic region starts 1024-aligned
 constexpr uint32_t kTmemCols = 256;                  // S0: columns 0..63, O: 64..191, S1: 192..255
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
 }
 
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src, bool valid) {
-    const int sz = valid ? 16 : 0;   // size 0: destination is zero filled
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(sz) : "memory");
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// one box of 64 rows x 64 columns (8 KB): rows row0.., columns col0..
+__device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tmap, uint64_t* bar, int col0, int row0) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(dst),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(smem_u32(bar)), "r"(col0), "r"(row0)
+        : "memory");
 }
 
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -135,11 +144,23 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
 }
 
 struct alignas(8) TcShared {
-    uint64_t bar_s[2];     // S = Q K^T into S buffer 0 / 1 has completed
-    uint64_t bar_o;        // O += P V of the current tile has completed
+    uint64_t q_full;       // Q tile landed                                   (loader -> MMA)
+    uint64_t k_full[2];    // key tile landed in K buffer 0 / 1                (loader -> MMA)
+    uint64_t k_empty[2];   // the MMAs have read K buffer 0 / 1                (MMA -> loader)
+    uint64_t v_full;       // V tile landed                                    (loader -> MMA)
+    uint64_t v_empty;      // the MMAs have read the V tile                    (MMA -> loader)
+    uint64_t s_full[2];    // S = Q K^T into S buffer 0 / 1 has completed      (MMA -> softmax)
+    uint64_t s_empty[2];   // the softmax warps have read S buffer 0 / 1       (softmax -> MMA, 4 arrivals)
+    uint64_t p_full;       // P is in shared memory                            (softmax -> MMA, 4 arrivals)
+    uint64_t p_empty;      // the MMAs have read P                             (MMA -> softmax)
+    uint64_t o_full;       // the last O += P V has completed                  (MMA -> softmax)
     uint32_t tmem_base;
     int abort;
 };
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 
 // swizzled position of the 16-byte chunk `chunk` (0..15 across the 128-wide row) of row `row` in a tile of
 // `rows` rows: two atoms (columns 0..63, 64..127), each rows x 128 bytes, chunk index XOR (row mod 8)
@@ -147,7 +168,8 @@ __device__ __forceinline__ uint32_t tile_off(int rows, int row, int chunk) {
     return static_cast<uint32_t>((chunk >> 3) * rows * 128 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
-__global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int* status) {
+__global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
+                                                                const __grid_constant__ CUtensorMap tm_v, AttnArgs a, int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* sQ = smem_raw;
     uint8_t* sK0 = sQ + kQBytes;         // key tiles with even index
@@ -157,7 +179,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int*
     uint8_t* sPl = sPh + kPBytes;        // P minus its rounded value, rounded to bf16
     TcShared* sh = reinterpret_cast<TcShared*>(sPl + kPBytes);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     volatile int* cta_abort = &sh->abort;
 
     pdl_launch_dependents();
@@ -167,13 +189,22 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int*
         return;
     }
     if (tid == 0) {
-        mbar_init(&sh->bar_s[0], 1);
-        mbar_init(&sh->bar_s[1], 1);
-        mbar_init(&sh->bar_o, 1);
+        mbar_init(&sh->q_full, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&sh->k_full[b], 1);
+            mbar_init(&sh->k_empty[b], 1);
+            mbar_init(&sh->s_full[b], 1);
+            mbar_init(&sh->s_empty[b], 4);
+        }
+        mbar_init(&sh->v_full, 1);
+        mbar_init(&sh->v_empty, 1);
+        mbar_init(&sh->p_full, 4);
+        mbar_init(&sh->p_empty, 1);
+        mbar_init(&sh->o_full, 1);
         sh->abort = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 0) {
+    if (warp == 4) {
         __syncwarp();
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
                      "r"(kTmemCols)
@@ -186,7 +217,6 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int*
     const uint32_t tmem_s0 = sh->tmem_base;                // 64 columns
     const uint32_t tmem_o = sh->tmem_base + 64;            // 128 columns
     const uint32_t tmem_s1 = sh->tmem_base + 192;          // 64 columns
-    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
 
     pdl_wait();   // q, k, v of this layer come from the preceding kernel
     const QTile t = a.tiles[blockIdx.x];
@@ -194,150 +224,179 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int*
     const int d = a.H * kHD;
     const int NK = t.n0;                                   // keys: rows f0 .. f0 + n0 of the forward
     const int ntiles = (NK + kTK - 1) / kTK;
-    const __nv_bfloat16* qsrc = a.q + static_cast<size_t>(t.q_row0) * d + head * kHD;
-    const __nv_bfloat16* ksrc = a.k + static_cast<size_t>(t.f0) * d + head * kHD;
-    const __nv_bfloat16* vsrc = a.v + static_cast<size_t>(t.f0) * d + head * kHD;
-
-    auto load_kv = [&](const __nv_bfloat16* src, uint8_t* dst, int tile) {
-        const uint32_t dbase = smem_u32(dst);
-        for (int c = tid; c < kTK * 16; c += kThreads) {
-            const int key = c >> 4, ch = c & 15;
-            const int kv = tile * kTK + key;
-            const bool ok = kv < NK;
-            cp_async16(dbase + tile_off(kTK, key, ch), ok ? src + static_cast<size_t>(kv) * d + ch * 8 : src, ok);
-        }
-    };
-    auto commit = [] { asm volatile("cp.async.commit_group;" ::: "memory"); };
-    // copies landed (this thread's), visible to the tensor core, and every thread is here
-    auto publish = [] {
-        proxy_fence();
-        tc_fence_before();
-        __syncthreads();
-    };
-
-    // ---- Q, first two key tiles ----
-    {
-        const uint32_t qb = smem_u32(sQ);
-        for (int c = tid; c < kTQ * 16; c += kThreads) {
-            const int r = c >> 4, ch = c & 15;
-            const bool ok = r < t.nq;
-            cp_async16(qb + tile_off(kTQ, r, ch), ok ? qsrc + static_cast<size_t>(r) * d + ch * 8 : qsrc, ok);
-        }
-    }
-    load_kv(ksrc, sK0, 0);
-    commit();
-    if (1 < ntiles) load_kv(ksrc, sK1, 1);
-    commit();
-
-    constexpr uint32_t idesc_s = instr_desc(kTQ, kTK, 0);
-    constexpr uint32_t idesc_o = instr_desc(kTQ, kHD, 1);
     const float scale_log2 = rsqrtf(static_cast<float>(kHD)) * 1.4426950408889634f;
-    uint32_t ph_s[2] = {0, 0}, ph_o = 0;                   // mbarrier phases
-    bool ok = true;
-
-    // S(tile) = Q K^T over the 128-wide head dim: 8 MMAs of K = 16 into S buffer tile & 1
-    auto issue_s = [&](int tile) {
-        const uint32_t qa = smem_u32(sQ), kb = smem_u32((tile & 1) ? sK1 : sK0);
-        const uint32_t ts = (tile & 1) ? tmem_s1 : tmem_s0;
-#pragma unroll
-        for (int kk = 0; kk < kHD / 16; ++kk) {
-            const uint32_t atom = kk >> 2, within = (kk & 3) * 32;
-            umma(ts, desc_k_major(qa + atom * (kTQ * 128) + within), desc_k_major(kb + atom * (kTK * 128) + within), idesc_s,
-                 kk > 0 ? 1u : 0u);
-        }
-        umma_commit(&sh->bar_s[tile & 1]);
+    auto wait = [&](uint64_t* bar, uint32_t& phase) {
+        const bool ok = mbar_wait(bar, phase, cta_abort, status);
+        phase ^= 1u;
+        return ok;
     };
 
-    // ---- pass 1: row maxima ----
-    float m_row = -INFINITY;
-    asm volatile("cp.async.wait_group 1;" ::: "memory");   // Q and key tile 0 landed
-    publish();
-    if (tid == 0) {
-        tc_fence_after();
-        issue_s(0);
-    }
-    for (int tile = 0; tile < ntiles && ok; ++tile) {
-        const int b = tile & 1;
-        if (tile + 1 < ntiles) {                            // S(tile + 1) runs while S(tile) is read back
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            publish();                                      // also: every thread has read S(tile - 1) out of that buffer
-            if (tid == 0) {
-                tc_fence_after();
-                issue_s(tile + 1);
+    if (warp == 5) {
+        // ================= loader =================
+        if (lane == 0) {
+            const int col0 = head * kHD;
+            // a 64-key tile (or 64 of the 128 query rows): one box per 64-column atom
+            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst, uint64_t* bar, int row0) {
+                tma_box(smem_u32(dst), tm, bar, col0, row0);
+                tma_box(smem_u32(dst) + kTK * 128, tm, bar, col0 + 64, row0);
+            };
+            auto load_k = [&](int tile) {
+                if (tile >= ntiles) return;
+                const int b = tile & 1;
+                mbar_expect_tx(&sh->k_full[b], kKBytes);
+                load_tile(&tm_k, b ? sK1 : sK0, &sh->k_full[b], t.f0 + tile * kTK);
+            };
+            auto load_v = [&](int tile) {
+                if (tile >= ntiles) return;
+                mbar_expect_tx(&sh->v_full, kKBytes);
+                load_tile(&tm_v, sV, &sh->v_full, t.f0 + tile * kTK);
+            };
+            uint32_t ph_ke[2] = {0, 0}, ph_ve = 0;
+            bool ok = true;
+            // Q: rows 0..63 and 64..127 of each atom
+            mbar_expect_tx(&sh->q_full, kQBytes);
+            tma_box(smem_u32(sQ), &tm_q, &sh->q_full, col0, t.q_row0);
+            tma_box(smem_u32(sQ) + 64 * 128, &tm_q, &sh->q_full, col0, t.q_row0 + 64);
+            tma_box(smem_u32(sQ) + kTQ * 128, &tm_q, &sh->q_full, col0 + 64, t.q_row0);
+            tma_box(smem_u32(sQ) + kTQ * 128 + 64 * 128, &tm_q, &sh->q_full, col0 + 64, t.q_row0 + 64);
+            // ---- pass 1 ----
+            load_k(0);
+            load_k(1);
+            for (int tile = 0; tile + 2 < ntiles && ok; ++tile) {
+                const int b = tile & 1;
+                ok = wait(&sh->k_empty[b], ph_ke[b]);            // S(tile) has read this buffer
+                if (ok) load_k(tile + 2);
+            }
+            // the last two S of pass 1 must have read their buffers before pass 2 refills them
+            for (int tile = ntiles > 2 ? ntiles - 2 : 0; tile < ntiles && ok; ++tile) ok = wait(&sh->k_empty[tile & 1], ph_ke[tile & 1]);
+            // ---- pass 2 ----
+            if (ok) {
+                load_k(0);
+                load_v(0);
+                load_k(1);
+            }
+            for (int tile = 0; tile < ntiles && ok; ++tile) {
+                const int b = tile & 1;
+                if (tile + 1 < ntiles) {
+                    ok = wait(&sh->v_empty, ph_ve);             // P V(tile) has read the V tile
+                    if (!ok) break;
+                    load_v(tile + 1);
+                }
+                if (tile + 2 < ntiles) {
+                    ok = wait(&sh->k_empty[b], ph_ke[b]);        // S(tile) has read this buffer
+                    if (!ok) break;
+                    load_k(tile + 2);
+                }
             }
         }
-        ok = mbar_wait(&sh->bar_s[b], ph_s[b], cta_abort, status);
-        ph_s[b] ^= 1u;
-        if (!ok) break;
-        tc_fence_after();
-        if (tile + 2 < ntiles) load_kv(ksrc, b ? sK1 : sK0, tile + 2);   // the MMAs have read this buffer
-        commit();
+    } else if (warp == 4) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idesc_s = instr_desc(kTQ, kTK, 0);
+            constexpr uint32_t idesc_o = instr_desc(kTQ, kHD, 1);
+            uint32_t ph_q = 0, ph_kf[2] = {0, 0}, ph_se[2] = {0, 0}, ph_vf = 0, ph_pf = 0;
+            bool ok = wait(&sh->q_full, ph_q);
+            // S(tile) = Q K^T over the 128-wide head dim: 8 MMAs of K = 16 into S buffer tile & 1
+            auto issue_s = [&](int tile) {
+                const int b = tile & 1;
+                const uint32_t qa = smem_u32(sQ), kb = smem_u32(b ? sK1 : sK0);
+                const uint32_t ts = b ? tmem_s1 : tmem_s0;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t v[32];
-            tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+                for (int kk = 0; kk < kHD / 16; ++kk) {
+                    const uint32_t atom = kk >> 2, within = (kk & 3) * 32;
+                    umma(ts, desc_k_major(qa + atom * (kTQ * 128) + within), desc_k_major(kb + atom * (kTK * 128) + within),
+                         idesc_s, kk > 0 ? 1u : 0u);
+                }
+                umma_commit(&sh->k_empty[b]);
+                umma_commit(&sh->s_full[b]);
+            };
+            // ---- pass 1 ----
+            for (int tile = 0; tile < ntiles && ok; ++tile) {
+                const int b = tile & 1;
+                ok = wait(&sh->k_full[b], ph_kf[b]);
+                if (ok && tile >= 2) ok = wait(&sh->s_empty[b], ph_se[b]);   // S(tile - 2) has been read
+                if (!ok) break;
+                tc_fence_after();
+                issue_s(tile);
+            }
+            // ---- pass 2 ----
+            auto issue_pv = [&](int tile, bool last) {
+                const uint32_t pa = smem_u32(sPh), pb = smem_u32(sPl), vb = smem_u32(sV);
 #pragma unroll
-            for (int j = 0; j < 32; ++j)
-                if (tile * kTK + half * 32 + j < NK) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+                for (int kk = 0; kk < kTK / 16; ++kk) {             // 16 keys per MMA
+                    const uint64_t bdesc = desc_mn_major(vb + kk * 2048, kTK * 128);
+                    umma(tmem_o, desc_k_major(pa + kk * 32), bdesc, idesc_o, (tile > 0 || kk > 0) ? 1u : 0u);
+                    umma(tmem_o, desc_k_major(pb + kk * 32), bdesc, idesc_o, 1u);
+                }
+                umma_commit(&sh->v_empty);
+                umma_commit(&sh->p_empty);
+                if (last) umma_commit(&sh->o_full);
+            };
+            for (int tile = 0; tile < ntiles && ok; ++tile) {
+                const int b = tile & 1;
+                ok = wait(&sh->k_full[b], ph_kf[b]);
+                if (ok) ok = wait(&sh->s_empty[b], ph_se[b]);        // the buffer's previous S has been read
+                if (!ok) break;
+                tc_fence_after();
+                issue_s(tile);
+                if (tile > 0) {                                      // P V of the previous tile, behind S(tile)
+                    ok = wait(&sh->p_full, ph_pf);
+                    if (ok) ok = wait(&sh->v_full, ph_vf);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_pv(tile - 1, false);
+                }
+            }
+            if (ok && ntiles > 0) {
+                ok = wait(&sh->p_full, ph_pf);
+                if (ok) ok = wait(&sh->v_full, ph_vf);
+                if (ok) {
+                    tc_fence_after();
+                    issue_pv(ntiles - 1, true);
+                }
+            }
         }
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    tc_fence_before();
-    __syncthreads();
-    ok = ok && !*cta_abort;
-
-    // ---- pass 2: P = exp2(S - max), O += P V ----
-    const float m_log2 = m_row * scale_log2;
-    float l_row = 0.f;
-    if (ok) {
-        load_kv(ksrc, sK0, 0);
-        commit();
-        load_kv(vsrc, sV, 0);
-        commit();
-        if (1 < ntiles) load_kv(ksrc, sK1, 1);
-        commit();
-        asm volatile("cp.async.wait_group 2;" ::: "memory");   // key tile 0 landed
-        publish();
-        if (tid == 0) {
-            tc_fence_after();
-            issue_s(0);
-        }
-    }
-    for (int tile = 0; tile < ntiles && ok; ++tile) {
-        const int b = tile & 1;
-        if (tile > 0) {
-            ok = mbar_wait(&sh->bar_o, ph_o, cta_abort, status);   // P and V of the previous tile have been read
-            ph_o ^= 1u;
+    } else {
+        // ================= softmax: thread r = query row r = TMEM lane r =================
+        const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
+        uint32_t ph_sf[2] = {0, 0}, ph_pe = 0, ph_of = 0;
+        bool ok = true;
+        // ---- pass 1: row maxima ----
+        float m_row = -INFINITY;
+        for (int tile = 0; tile < ntiles && ok; ++tile) {
+            const int b = tile & 1;
+            ok = wait(&sh->s_full[b], ph_sf[b]);
             if (!ok) break;
-            load_kv(vsrc, sV, tile);
-            commit();
-            asm volatile("cp.async.wait_group 1;" ::: "memory");   // key tile + 1 landed (V may be in flight)
-        } else {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-        }
-        publish();                                          // also: every thread has read S(tile - 1)
-        if (tid == 0 && tile + 1 < ntiles) {
             tc_fence_after();
-            issue_s(tile + 1);
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t v[32];
+                tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+#pragma unroll
+                for (int j = 0; j < 32; ++j)
+                    if (tile * kTK + half * 32 + j < NK) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->s_empty[b]);
         }
-        ok = mbar_wait(&sh->bar_s[b], ph_s[b], cta_abort, status);
-        ph_s[b] ^= 1u;
-        if (!ok) break;
-        tc_fence_after();
-        if (tile + 2 < ntiles) load_kv(ksrc, b ? sK1 : sK0, tile + 2);
-        commit();
-        // thread r: row r of S -> P (two bf16 terms) into the swizzled A-operand tiles
+        // ---- pass 2: P = exp2(S - max), row sums ----
+        const float m_log2 = m_row * scale_log2;
+        float l_row = 0.f;
         const uint32_t ph_base = smem_u32(sPh) + tid * 128, pl_base = smem_u32(sPl) + tid * 128;
+        for (int tile = 0; tile < ntiles && ok; ++tile) {
+            const int b = tile & 1;
+            ok = wait(&sh->s_full[b], ph_sf[b]);
+            if (!ok) break;
+            tc_fence_after();
+            uint32_t hi[32], lo[32];                                 // row `tid` of P: 64 keys as bf16 pairs
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            uint32_t v[32];
-            tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+            for (int half = 0; half < 2; ++half) {
+                uint32_t v[32];
+                tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
 #pragma unroll
-            for (int c4 = 0; c4 < 4; ++c4) {                         // 8 keys = one 16-byte chunk
-                uint32_t hi[4], lo[4];
-#pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int j = c4 * 8 + u * 2;
+                for (int u = 0; u < 16; ++u) {
+                    const int j = 2 * u;
                     const int key = tile * kTK + half * 32 + j;
                     const float p0 = key < NK ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_log2) : 0.f;
                     const float p1 = key + 1 < NK ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_log2) : 0.f;
@@ -345,62 +404,61 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(AttnArgs a, int*
                     const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                     const float2 hf = __bfloat1622float2(h);
                     const __nv_bfloat162 l = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
-                    hi[u] = *reinterpret_cast<const uint32_t*>(&h);
-                    lo[u] = *reinterpret_cast<const uint32_t*>(&l);
+                    hi[half * 16 + u] = *reinterpret_cast<const uint32_t*>(&h);
+                    lo[half * 16 + u] = *reinterpret_cast<const uint32_t*>(&l);
                 }
-                const uint32_t off = static_cast<uint32_t>(((half * 4 + c4) ^ (tid & 7)) << 4);
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ph_base + off), "r"(hi[0]), "r"(hi[1]), "r"(hi[2]),
-                             "r"(hi[3])
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->s_empty[b]);             // S(tile) is in registers
+            if (tile > 0) {
+                ok = wait(&sh->p_empty, ph_pe);                      // P V(tile - 1) has read P
+                if (!ok) break;
+            }
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {                            // 8 keys = one 16-byte chunk
+                const uint32_t off = static_cast<uint32_t>((c ^ (tid & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(ph_base + off), "r"(hi[4 * c]), "r"(hi[4 * c + 1]),
+                             "r"(hi[4 * c + 2]), "r"(hi[4 * c + 3])
                              : "memory");
-                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pl_base + off), "r"(lo[0]), "r"(lo[1]), "r"(lo[2]),
-                             "r"(lo[3])
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(pl_base + off), "r"(lo[4 * c]), "r"(lo[4 * c + 1]),
+                             "r"(lo[4 * c + 2]), "r"(lo[4 * c + 3])
                              : "memory");
             }
+            proxy_fence();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->p_full);
         }
-        asm volatile("cp.async.wait_group 1;" ::: "memory");        // V tile landed (key tile + 2 may be in flight)
-        publish();
-        if (tid == 0) {
+        if (ok && ntiles > 0) ok = wait(&sh->o_full, ph_of);
+        if (ok) {
             tc_fence_after();
-            const uint32_t pa = smem_u32(sPh), pb = smem_u32(sPl), vb = smem_u32(sV);
-#pragma unroll
-            for (int kk = 0; kk < kTK / 16; ++kk) {                  // 16 keys per MMA
-                const uint64_t bdesc = desc_mn_major(vb + kk * 2048, kTK * 128);
-                umma(tmem_o, desc_k_major(pa + kk * 32), bdesc, idesc_o, (tile > 0 || kk > 0) ? 1u : 0u);
-                umma(tmem_o, desc_k_major(pb + kk * 32), bdesc, idesc_o, 1u);
-            }
-            umma_commit(&sh->bar_o);
-        }
-    }
-    if (ok) ok = mbar_wait(&sh->bar_o, ph_o, cta_abort, status);
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    if (ok) {
-        tc_fence_after();
-        const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
-        __nv_bfloat16* orow = a.o + static_cast<size_t>(t.q_row0 + tid) * d + head * kHD;
+            const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
+            __nv_bfloat16* orow = a.o + static_cast<size_t>(t.q_row0 + tid) * d + head * kHD;
 #pragma unroll 1
-        for (int c = 0; c < kHD / 32; ++c) {
-            uint32_t v[32];
-            tmem_ld32(tmem_o + lane_base + c * 32, v);
-            if (tid < t.nq) {
+            for (int c = 0; c < kHD / 32; ++c) {
+                uint32_t v[32];
+                tmem_ld32(tmem_o + lane_base + c * 32, v);
+                if (tid < t.nq) {
 #pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                    uint4 pk;
-                    __nv_bfloat162 x0 = __floats2bfloat162_rn(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
-                    __nv_bfloat162 x1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
-                    __nv_bfloat162 x2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
-                    __nv_bfloat162 x3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
-                    pk.x = *reinterpret_cast<const uint32_t*>(&x0);
-                    pk.y = *reinterpret_cast<const uint32_t*>(&x1);
-                    pk.z = *reinterpret_cast<const uint32_t*>(&x2);
-                    pk.w = *reinterpret_cast<const uint32_t*>(&x3);
-                    *reinterpret_cast<uint4*>(orow + c * 32 + j) = pk;
+                    for (int j = 0; j < 32; j += 8) {
+                        uint4 pk;
+                        __nv_bfloat162 x0 = __floats2bfloat162_rn(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
+                        __nv_bfloat162 x1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                        __nv_bfloat162 x2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
+                        __nv_bfloat162 x3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
+                        pk.x = *reinterpret_cast<const uint32_t*>(&x0);
+                        pk.y = *reinterpret_cast<const uint32_t*>(&x1);
+                        pk.z = *reinterpret_cast<const uint32_t*>(&x2);
+                        pk.w = *reinterpret_cast<const uint32_t*>(&x3);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + j) = pk;
+                    }
                 }
             }
         }
     }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) {
+    if (warp == 4) {
         __syncwarp();
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(sh->tmem_base), "r"(kTmemCols) : "memory");
@@ -421,7 +479,14 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
         if (e != cudaSuccess) return e;
         attr_done = true;
     }
-    return launch_kernel(attention_tc_kernel, dim3(a.n_tiles, a.H), dim3(kThreads), kSmemBytes, st, a, status);
+    // the fresh q / k / v of this forward: [M][H * 128] bf16; rows beyond M read as zero
+    CUtensorMap tq, tk, tv;
+    const int d = a.H * kHD;
+    cudaError_t e = make_rows_tmap(&tq, a.q, a.M, d, 64);
+    if (e == cudaSuccess) e = make_rows_tmap(&tk, a.k, a.M, d, 64);
+    if (e == cudaSuccess) e = make_rows_tmap(&tv, a.v, a.M, d, 64);
+    if (e != cudaSuccess) return e;
+    return launch_kernel(attention_tc_kernel, dim3(a.n_tiles, a.H), dim3(kThreads), kSmemBytes, st, tq, tk, tv, a, status);
 }
 
 }  // namespace odb

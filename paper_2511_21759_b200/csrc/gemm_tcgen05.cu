@@ -696,6 +696,10 @@ bool use_pair(int M, int n_tiles) { return pair_enabled() && M > 128 && (n_tiles
 
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w, int N, int K) { return make_tmap_packed(out, w, N, K); }
 
+cudaError_t make_rows_tmap(CUtensorMap* out, const void* base, int rows, int cols, int box_rows) {
+    return make_tmap_2d(out, base, rows, cols, box_rows);
+}
+
 size_t packed_weight_bytes(int N, int K) {
     return static_cast<size_t>((N + kBM - 1) / kBM) * ((K + kBK - 1) / kBK) * kBM * kBK * 2;
 }

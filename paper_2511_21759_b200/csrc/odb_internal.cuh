@@ -196,6 +196,8 @@ struct GemmArgs {
 };
 int gemm_pick_splits(int M, int N, int K);
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
+// bf16 [rows][cols] row-major; box = 64 columns x box_rows rows, 128-byte swizzle, rows beyond `rows` read as zero
+cudaError_t make_rows_tmap(CUtensorMap* out, const void* base, int rows, int cols, int box_rows);
 size_t packed_weight_bytes(int N, int K);
 size_t packed_gate_up_bytes(int F, int K);
 cudaError_t make_gate_up_tmap(CUtensorMap* out, const void* w_packed, int F, int K);
