@@ -578,6 +578,12 @@ cudaError_t launch_step_hd(const StepAttnArgs& a, cudaStream_t st) {
                          static_cast<const float*>(a.part_ml), a.o, a.M, a.H, HD, a.ksplit);
 }
 
+// merges the key-split partials (part_o, part_ml) of M rows x H heads in split order into the bf16 output
+cudaError_t launch_attention_combine(const float* part_o, const float* part_ml, __nv_bfloat16* o, int M, int H, int hd,
+                                     int ksplit, cudaStream_t st) {
+    return launch_kernel(attention_combine_kernel, dim3(M, H), dim3(hd / 4), 0, st, part_o, part_ml, o, M, H, hd, ksplit);
+}
+
 cudaError_t launch_step_attention(const StepAttnArgs& a, cudaStream_t st) {
     if (a.n_tiles == 0) return cudaSuccess;
     if (a.ksplit < 2 || a.ksplit > 8) return cudaErrorInvalidValue;

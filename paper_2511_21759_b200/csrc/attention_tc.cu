@@ -1,19 +1,28 @@
-// Bidirectional attention of a refresh prefill on the tcgen05 tensor cores (head dim 128).
+// Bidirectional block-query attention on the tcgen05 tensor cores (head dim 128): the refresh prefill and
+// the decode step over several block copies.
 //
-// Work item: 128 query rows of one sequence x one head; keys = every row of that sequence (fresh q/k/v
-// of the same forward, nothing is read from the cache: the refresh is what writes it).  No causal mask.
-// Two passes over the key tiles of 64, both with S = Q K^T as one 128 x 64 x 128 tcgen05.mma group whose
-// fp32 result lives in TMEM:
+// Work item: up to 128 consecutive query rows x one head (x one key split in a decode step).
+//   refresh: keys = every row of the sequence (fresh q/k/v of the same forward; nothing is read from the
+//            cache, the refresh is what writes it); the output is final.
+//   step:    the rows of all copies of one block (a StepTile).  Key splits 0 .. ks-2 stream the cached
+//            K/V of the positions outside the block, visible to every row; the last split takes the fresh
+//            rows, one key tile per source copy: a row sees its own copy's tile and, in the decoded-share
+//            layout, the decoded rows of copy 0's tile.  Copies stay mutually invisible through this
+//            per-row key mask, no mask tensor exists.  Outputs are per-split (max, sum, unnormalised
+//            output) partials merged in split order by the merge kernel of attention.cu.
+// No causal mask.  Two passes over the key tiles of 64, both with S = Q K^T as one 128 x 64 x 128
+// tcgen05.mma group whose fp32 result lives in TMEM:
 //   pass 1  row maxima of S (thread r owns TMEM lane r = query row r: no cross-thread reduction);
 //   pass 2  P = exp2(S - max), row sums, P rounded to a two-term bf16 sum (value + remainder, as in the
 //           mma.sync kernel) and written to shared memory as the A operand of O += P V
 //           (128 x 128 x 64, V taken MN-major straight from its [key][dim] tile), O in TMEM.
 // Exact softmax, no rescaling of O.  Warp-specialised: warps 0..3 = softmax (one query row per thread),
 // warp 4 lane 0 = MMA issuer, warp 5 lane 0 = loader (TMA: boxes of 64 rows x 64 columns with the 128-byte
-// swizzle land in the canonical operand layout, two 64-column atoms per 128-wide row; rows past the
-// forward's last row read as zero, rows of a neighbouring sequence are masked in the softmax).  S is double buffered in TMEM and K in shared
-// memory, so S(t + 1) is computed while the softmax warps work on tile t and P V(t) while they work on
-// tile t + 1; the roles meet only through mbarriers.  Two CTAs share an SM (112 KB of shared memory, 256
+// swizzle land in the canonical operand layout, two 64-column atoms per 128-wide row; rows past a buffer's
+// end read as zero, rows that are not keys of this work item are masked in the softmax and hold finite
+// values, the K/V cache being zeroed when a session is created).  S is double buffered in TMEM and K in
+// shared memory, so S(t + 1) is computed while the softmax warps work on tile t and P V(t) while they work
+// on tile t + 1; the roles meet only through mbarriers.  Two CTAs share an SM (112 KB of shared memory, 256
 // TMEM columns each).  Every mbarrier wait is bounded; on expiry the CTA records ODB_ERR_TIMEOUT, every
 // role stops, the CTA releases its TMEM and exits.
 #include "odb_internal.cuh"
@@ -168,8 +177,26 @@ __device__ __forceinline__ uint32_t tile_off(int rows, int row, int chunk) {
     return static_cast<uint32_t>((chunk >> 3) * rows * 128 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
+// One key tile of a work item: 64 consecutive rows of a [rows][128]-column view starting at row0, of which
+// the first `valid` are keys.  src: 0 = fresh k / v rows of this forward, 1 = the K/V cache.
+struct KeyTile {
+    int src, row0, v_row0, valid;
+    int copy;          // fresh tile of a step: the source copy; -1 otherwise (visible to every row)
+};
+
+struct TcArgs {
+    const QTile* qtiles;          // refresh work items
+    const StepTile* stiles;       // step work items
+    const int32_t* row_flags;
+    __nv_bfloat16* o;             // refresh: final output [M][H * 128]
+    float* part_o; float* part_ml;   // step: split partials [ks][M][H][128], [ks][M][H][2]
+    int layer, n_layers, H, max_seq, M;
+};
+
+template <bool STEP>
 __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_constant__ CUtensorMap tm_q, const __grid_constant__ CUtensorMap tm_k,
-                                                                const __grid_constant__ CUtensorMap tm_v, AttnArgs a, int* status) {
+                                                                const __grid_constant__ CUtensorMap tm_v, const __grid_constant__ CUtensorMap tm_c,
+                                                                TcArgs a, int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     uint8_t* sQ = smem_raw;
     uint8_t* sK0 = sQ + kQBytes;         // key tiles with even index
@@ -219,11 +246,47 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
     const uint32_t tmem_s1 = sh->tmem_base + 192;          // 64 columns
 
     pdl_wait();   // q, k, v of this layer come from the preceding kernel
-    const QTile t = a.tiles[blockIdx.x];
     const int head = blockIdx.y;
-    const int d = a.H * kHD;
-    const int NK = t.n0;                                   // keys: rows f0 .. f0 + n0 of the forward
-    const int ntiles = (NK + kTK - 1) / kTK;
+    const int z = blockIdx.z, ks = gridDim.z;
+    // ---- the work item: query rows and key tiles ----
+    int q_row0, nq, ntiles;
+    int f0 = 0, NK = 0;                                     // refresh: keys = fresh rows [f0, f0 + NK)
+    int cA = 0, cB0 = 0, cB1 = 0, nA_t = 0, t_first = 0;    // step, cached split: positions [0, cA) and [cB0, cB1)
+    int c_row = 0;                                          // step: row of position 0 of this head's keys in the cache view
+    bool fresh_split = false;
+    const StepTile* stp = nullptr;
+    if constexpr (!STEP) {
+        const QTile t = a.qtiles[blockIdx.x];
+        q_row0 = t.q_row0; nq = t.nq; f0 = t.f0; NK = t.n0;
+        ntiles = (NK + kTK - 1) / kTK;
+    } else {
+        stp = a.stiles + blockIdx.x;
+        q_row0 = stp->slab_row0[0];
+        nq = stp->slab_row0[stp->n_slabs - 1] + stp->slab_n[stp->n_slabs - 1] - q_row0;   // the slabs are consecutive rows
+        fresh_split = z == ks - 1;
+        cA = stp->cA; cB0 = stp->cB0; cB1 = stp->cB1;
+        nA_t = (cA + kTK - 1) / kTK;
+        const int nct = nA_t + (cB1 - cB0 + kTK - 1) / kTK;
+        const int tp = (nct + ks - 2) / (ks - 1);
+        t_first = fresh_split ? 0 : z * tp;
+        ntiles = fresh_split ? stp->n_src : max(0, min(nct, t_first + tp) - t_first);
+        c_row = ((stp->seq * a.n_layers + a.layer) * 2 * a.H + head) * a.max_seq;   // K; V is H * max_seq rows further
+    }
+    auto key_tile = [&](int i) {
+        KeyTile kt;
+        kt.copy = -1;
+        if constexpr (!STEP) {
+            kt.src = 0; kt.row0 = f0 + i * kTK; kt.v_row0 = kt.row0; kt.valid = min(kTK, NK - i * kTK);
+        } else if (fresh_split) {
+            kt.src = 0; kt.row0 = stp->src_row0[i]; kt.v_row0 = kt.row0; kt.valid = stp->src_n[i]; kt.copy = stp->src_copy[i];
+        } else {
+            const int j = t_first + i;
+            const int pos0 = j < nA_t ? j * kTK : cB0 + (j - nA_t) * kTK;
+            const int end = j < nA_t ? cA : cB1;
+            kt.src = 1; kt.row0 = c_row + pos0; kt.v_row0 = kt.row0 + a.H * a.max_seq; kt.valid = min(kTK, end - pos0);
+        }
+        return kt;
+    };
     const float scale_log2 = rsqrtf(static_cast<float>(kHD)) * 1.4426950408889634f;
     auto wait = [&](uint64_t* bar, uint32_t& phase) {
         const bool ok = mbar_wait(bar, phase, cta_abort, status);
@@ -235,30 +298,32 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         // ================= loader =================
         if (lane == 0) {
             const int col0 = head * kHD;
-            // a 64-key tile (or 64 of the 128 query rows): one box per 64-column atom
-            auto load_tile = [&](const CUtensorMap* tm, uint8_t* dst, uint64_t* bar, int row0) {
-                tma_box(smem_u32(dst), tm, bar, col0, row0);
-                tma_box(smem_u32(dst) + kTK * 128, tm, bar, col0 + 64, row0);
-            };
+            // 64 rows x 128 columns: one box per 64-column atom (the cache view has 128 columns per row)
             auto load_k = [&](int tile) {
                 if (tile >= ntiles) return;
                 const int b = tile & 1;
+                const KeyTile kt = key_tile(tile);
+                const uint32_t dst = smem_u32(b ? sK1 : sK0);
                 mbar_expect_tx(&sh->k_full[b], kKBytes);
-                load_tile(&tm_k, b ? sK1 : sK0, &sh->k_full[b], t.f0 + tile * kTK);
+                tma_box(dst, kt.src ? &tm_c : &tm_k, &sh->k_full[b], kt.src ? 0 : col0, kt.row0);
+                tma_box(dst + kTK * 128, kt.src ? &tm_c : &tm_k, &sh->k_full[b], kt.src ? 64 : col0 + 64, kt.row0);
             };
             auto load_v = [&](int tile) {
                 if (tile >= ntiles) return;
+                const KeyTile kt = key_tile(tile);
+                const uint32_t dst = smem_u32(sV);
                 mbar_expect_tx(&sh->v_full, kKBytes);
-                load_tile(&tm_v, sV, &sh->v_full, t.f0 + tile * kTK);
+                tma_box(dst, kt.src ? &tm_c : &tm_v, &sh->v_full, kt.src ? 0 : col0, kt.v_row0);
+                tma_box(dst + kTK * 128, kt.src ? &tm_c : &tm_v, &sh->v_full, kt.src ? 64 : col0 + 64, kt.v_row0);
             };
             uint32_t ph_ke[2] = {0, 0}, ph_ve = 0;
             bool ok = true;
             // Q: rows 0..63 and 64..127 of each atom
             mbar_expect_tx(&sh->q_full, kQBytes);
-            tma_box(smem_u32(sQ), &tm_q, &sh->q_full, col0, t.q_row0);
-            tma_box(smem_u32(sQ) + 64 * 128, &tm_q, &sh->q_full, col0, t.q_row0 + 64);
-            tma_box(smem_u32(sQ) + kTQ * 128, &tm_q, &sh->q_full, col0 + 64, t.q_row0);
-            tma_box(smem_u32(sQ) + kTQ * 128 + 64 * 128, &tm_q, &sh->q_full, col0 + 64, t.q_row0 + 64);
+            tma_box(smem_u32(sQ), &tm_q, &sh->q_full, col0, q_row0);
+            tma_box(smem_u32(sQ) + 64 * 128, &tm_q, &sh->q_full, col0, q_row0 + 64);
+            tma_box(smem_u32(sQ) + kTQ * 128, &tm_q, &sh->q_full, col0 + 64, q_row0);
+            tma_box(smem_u32(sQ) + kTQ * 128 + 64 * 128, &tm_q, &sh->q_full, col0 + 64, q_row0 + 64);
             // ---- pass 1 ----
             load_k(0);
             load_k(1);
@@ -291,7 +356,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         }
     } else if (warp == 4) {
         // ================= MMA issuer =================
-        if (lane == 0) {
+        if (lane == 0 && ntiles > 0) {
             constexpr uint32_t idesc_s = instr_desc(kTQ, kTK, 0);
             constexpr uint32_t idesc_o = instr_desc(kTQ, kHD, 1);
             uint32_t ph_q = 0, ph_kf[2] = {0, 0}, ph_se[2] = {0, 0}, ph_vf = 0, ph_pf = 0;
@@ -347,7 +412,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                     issue_pv(tile - 1, false);
                 }
             }
-            if (ok && ntiles > 0) {
+            if (ok) {
                 ok = wait(&sh->p_full, ph_pf);
                 if (ok) ok = wait(&sh->v_full, ph_vf);
                 if (ok) {
@@ -361,10 +426,35 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;   // this warp's TMEM lanes
         uint32_t ph_sf[2] = {0, 0}, ph_pe = 0, ph_of = 0;
         bool ok = true;
+        int my_copy = -1, stage2 = 0;
+        if constexpr (STEP) {
+            stage2 = stp->stage2;
+            const int grow = q_row0 + tid;
+            for (int sl = 0; sl < stp->n_slabs; ++sl)
+                if (grow >= stp->slab_row0[sl] && grow < stp->slab_row0[sl] + stp->slab_n[sl]) my_copy = stp->slab_copy[sl];
+        }
+        // which of the tile's 64 keys this row sees (bit j = key j).  Every lane of a warp calls this for the
+        // same tile: the branch that uses the ballots is uniform.
+        auto tile_mask = [&](const KeyTile& kt) -> unsigned long long {
+            const unsigned long long all = kt.valid >= 64 ? ~0ull : ((1ull << kt.valid) - 1ull);
+            if (kt.copy < 0) return all;                            // cached keys, or a refresh
+            unsigned long long shared = 0ull;
+            if constexpr (STEP) {
+                if (stage2 && kt.copy == 0) {                        // decoded rows of copy 0, shared with every copy
+                    const bool d0 = lane < kt.valid && (a.row_flags[kt.row0 + lane] & kRowDecoded);
+                    const bool d1 = lane + 32 < kt.valid && (a.row_flags[kt.row0 + lane + 32] & kRowDecoded);
+                    const unsigned lo = __ballot_sync(0xffffffffu, d0), hi = __ballot_sync(0xffffffffu, d1);
+                    shared = (static_cast<unsigned long long>(hi) << 32 | lo) & all;
+                }
+            }
+            return kt.copy == my_copy ? all : shared;
+        };
         // ---- pass 1: row maxima ----
         float m_row = -INFINITY;
         for (int tile = 0; tile < ntiles && ok; ++tile) {
             const int b = tile & 1;
+            const KeyTile kt = key_tile(tile);
+            const unsigned long long mask = tile_mask(kt);
             ok = wait(&sh->s_full[b], ph_sf[b]);
             if (!ok) break;
             tc_fence_after();
@@ -372,20 +462,23 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+                const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
 #pragma unroll
                 for (int j = 0; j < 32; ++j)
-                    if (tile * kTK + half * 32 + j < NK) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+                    if ((m32 >> j) & 1u) m_row = fmaxf(m_row, __uint_as_float(v[j]));
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->s_empty[b]);
         }
         // ---- pass 2: P = exp2(S - max), row sums ----
-        const float m_log2 = m_row * scale_log2;
+        const float m_log2 = m_row == -INFINITY ? 0.f : m_row * scale_log2;   // a row that sees no key of this split: every P is 0
         float l_row = 0.f;
         const uint32_t ph_base = smem_u32(sPh) + tid * 128, pl_base = smem_u32(sPl) + tid * 128;
         for (int tile = 0; tile < ntiles && ok; ++tile) {
             const int b = tile & 1;
+            const KeyTile kt = key_tile(tile);
+            const unsigned long long mask = tile_mask(kt);
             ok = wait(&sh->s_full[b], ph_sf[b]);
             if (!ok) break;
             tc_fence_after();
@@ -394,12 +487,12 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+                const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
                     const int j = 2 * u;
-                    const int key = tile * kTK + half * 32 + j;
-                    const float p0 = key < NK ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_log2) : 0.f;
-                    const float p1 = key + 1 < NK ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_log2) : 0.f;
+                    const float p0 = ((m32 >> j) & 1u) ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_log2) : 0.f;
+                    const float p1 = ((m32 >> (j + 1)) & 1u) ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_log2) : 0.f;
                     l_row += p0 + p1;
                     const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
                     const float2 hf = __bfloat1622float2(h);
@@ -432,25 +525,47 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         if (ok && ntiles > 0) ok = wait(&sh->o_full, ph_of);
         if (ok) {
             tc_fence_after();
-            const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
-            __nv_bfloat16* orow = a.o + static_cast<size_t>(t.q_row0 + tid) * d + head * kHD;
+            const int d = a.H * kHD;
+            const int row = q_row0 + tid;
+            if constexpr (!STEP) {
+                const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
+                __nv_bfloat16* orow = a.o + static_cast<size_t>(row) * d + head * kHD;
 #pragma unroll 1
-            for (int c = 0; c < kHD / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld32(tmem_o + lane_base + c * 32, v);
-                if (tid < t.nq) {
+                for (int c = 0; c < kHD / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem_o + lane_base + c * 32, v);
+                    if (tid < nq) {
 #pragma unroll
-                    for (int j = 0; j < 32; j += 8) {
-                        uint4 pk;
-                        __nv_bfloat162 x0 = __floats2bfloat162_rn(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
-                        __nv_bfloat162 x1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
-                        __nv_bfloat162 x2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
-                        __nv_bfloat162 x3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
-                        pk.x = *reinterpret_cast<const uint32_t*>(&x0);
-                        pk.y = *reinterpret_cast<const uint32_t*>(&x1);
-                        pk.z = *reinterpret_cast<const uint32_t*>(&x2);
-                        pk.w = *reinterpret_cast<const uint32_t*>(&x3);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + j) = pk;
+                        for (int j = 0; j < 32; j += 8) {
+                            uint4 pk;
+                            __nv_bfloat162 x0 = __floats2bfloat162_rn(__uint_as_float(v[j]) * inv, __uint_as_float(v[j + 1]) * inv);
+                            __nv_bfloat162 x1 = __floats2bfloat162_rn(__uint_as_float(v[j + 2]) * inv, __uint_as_float(v[j + 3]) * inv);
+                            __nv_bfloat162 x2 = __floats2bfloat162_rn(__uint_as_float(v[j + 4]) * inv, __uint_as_float(v[j + 5]) * inv);
+                            __nv_bfloat162 x3 = __floats2bfloat162_rn(__uint_as_float(v[j + 6]) * inv, __uint_as_float(v[j + 7]) * inv);
+                            pk.x = *reinterpret_cast<const uint32_t*>(&x0);
+                            pk.y = *reinterpret_cast<const uint32_t*>(&x1);
+                            pk.z = *reinterpret_cast<const uint32_t*>(&x2);
+                            pk.w = *reinterpret_cast<const uint32_t*>(&x3);
+                            *reinterpret_cast<uint4*>(orow + c * 32 + j) = pk;
+                        }
+                    }
+                }
+            } else {
+                // split partial: unnormalised output, (max in the log2 domain, sum); a split that saw no key has sum 0
+                const size_t pr = (static_cast<size_t>(z) * a.M + row) * a.H + head;
+                if (tid < nq) *reinterpret_cast<float2*>(a.part_ml + pr * 2) = make_float2(m_log2, l_row);
+                if (ntiles > 0) {
+                    float* po = a.part_o + pr * kHD;
+#pragma unroll 1
+                    for (int c = 0; c < kHD / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_o + lane_base + c * 32, v);
+                        if (tid < nq) {
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4)
+                                *reinterpret_cast<float4*>(po + c * 32 + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]),
+                                                                                          __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+                        }
                     }
                 }
             }
@@ -465,6 +580,27 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
     }
 }
 
+template <bool STEP>
+cudaError_t launch_tc(dim3 grid, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* cache,
+                      size_t cache_rows, const TcArgs& ta, int* status, cudaStream_t st) {
+    static bool attr_done = false;
+    if (!attr_done) {
+        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<STEP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(kSmemBytes));
+        if (e != cudaSuccess) return e;
+        attr_done = true;
+    }
+    // the fresh q / k / v of this forward: [M][H * 128] bf16, rows beyond M read as zero; the cache as rows of 128
+    CUtensorMap tq, tk, tv, tc;
+    const int d = ta.H * kHD;
+    cudaError_t e = make_rows_tmap(&tq, q, ta.M, d, 64);
+    if (e == cudaSuccess) e = make_rows_tmap(&tk, k, ta.M, d, 64);
+    if (e == cudaSuccess) e = make_rows_tmap(&tv, v, ta.M, d, 64);
+    if (e == cudaSuccess) e = STEP ? make_rows_tmap(&tc, cache, cache_rows, kHD, 64) : make_rows_tmap(&tc, k, ta.M, d, 64);
+    if (e != cudaSuccess) return e;
+    return launch_kernel(attention_tc_kernel<STEP>, grid, dim3(kThreads), kSmemBytes, st, tq, tk, tv, tc, ta, status);
+}
+
 }  // namespace
 
 // Refresh attention on the tensor cores: a.tiles = work items of up to 128 query rows whose keys are the
@@ -472,21 +608,25 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
 cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st) {
     if (a.n_tiles == 0) return cudaSuccess;
     if (a.hd != kHD) return cudaErrorInvalidValue;
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(kSmemBytes));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
-    }
-    // the fresh q / k / v of this forward: [M][H * 128] bf16; rows beyond M read as zero
-    CUtensorMap tq, tk, tv;
-    const int d = a.H * kHD;
-    cudaError_t e = make_rows_tmap(&tq, a.q, a.M, d, 64);
-    if (e == cudaSuccess) e = make_rows_tmap(&tk, a.k, a.M, d, 64);
-    if (e == cudaSuccess) e = make_rows_tmap(&tv, a.v, a.M, d, 64);
-    if (e != cudaSuccess) return e;
-    return launch_kernel(attention_tc_kernel, dim3(a.n_tiles, a.H), dim3(kThreads), kSmemBytes, st, tq, tk, tv, a, status);
+    TcArgs ta{};
+    ta.qtiles = a.tiles;
+    ta.row_flags = a.row_flags;
+    ta.o = a.o;
+    ta.layer = a.layer; ta.n_layers = a.n_layers; ta.H = a.H; ta.max_seq = a.max_seq; ta.M = a.M;
+    return launch_tc<false>(dim3(a.n_tiles, a.H), a.q, a.k, a.v, nullptr, 0, ta, status, st);
+}
+
+// Decode-step attention over StepTiles on the tensor cores (head dim 128); cache_rows = rows of the K/V cache
+// viewed as [rows][128] (batch x layers x 2 x heads x max_seq).  Partials only: the caller merges them.
+cudaError_t launch_step_attention_tc(const StepAttnArgs& a, size_t cache_rows, int* status, cudaStream_t st) {
+    if (a.n_tiles == 0) return cudaSuccess;
+    if (a.hd != kHD || a.ksplit < 2 || a.ksplit > 8) return cudaErrorInvalidValue;
+    TcArgs ta{};
+    ta.stiles = a.tiles;
+    ta.row_flags = a.row_flags;
+    ta.part_o = a.part_o; ta.part_ml = a.part_ml;
+    ta.layer = a.layer; ta.n_layers = a.n_layers; ta.H = a.H; ta.max_seq = a.max_seq; ta.M = a.M;
+    return launch_tc<true>(dim3(a.n_tiles, a.H, a.ksplit), a.q, a.k, a.v, a.cache, cache_rows, ta, status, st);
 }
 
 }  // namespace odb

@@ -276,6 +276,10 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     if (e == cudaSuccess)
         e = cudaMemcpyAsync(s->ws + L.rope, rope.data(), rope.size() * sizeof(float2), cudaMemcpyHostToDevice, s->st);
     if (e == cudaSuccess) e = cudaMemsetAsync(s->ws + L.state, 0, L.x - L.state, s->st);   // state, results, status
+    // The tensor-core attention loads whole 64-row boxes: cache rows that are not keys of a work item are masked
+    // in its softmax but still enter the P V product with weight zero, so they must hold finite values; the
+    // q / k / v and output rows past a forward's last row are never read (the tensor maps end at that row).
+    if (e == cudaSuccess) e = cudaMemsetAsync(kv, 0, odb_kv_bytes(&c), s->st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->st);
     if (e != cudaSuccess) {
         odb_session_destroy(s);
@@ -517,8 +521,18 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             if (sks < 2) sks = 2;
             sa.ksplit = sks;
             sa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
-            ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
-            ++s->launches[ODB_KIND_ATTENTION];
+            // tensor-core work items when there are enough of them to fill the machine (batched steps: 33.5 -> 22.5 ms
+            // at 16 sequences x 256 rows); a single 128-row item per head is bound by its own dependency chain on
+            // either path (1.20 vs 1.12 ms at batch 1) and stays on the mma.sync kernel
+            static const int tc_step_min = getenv("ODB_ATTN_TC_STEP_MIN") ? atoi(getenv("ODB_ATTN_TC_STEP_MIN")) : 2 * 148;
+            if (hd == 128 && tc_attention && n_step_tiles * H >= tc_step_min) {
+                const size_t cache_rows = static_cast<size_t>(c.max_batch) * c.n_layers * 2 * H * c.max_seq;
+                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention_tc(sa, cache_rows, status, st));
+                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_combine(sa.part_o, sa.part_ml, o, M, H, hd, sks, st));
+            } else {
+                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
+                ++s->launches[ODB_KIND_ATTENTION];
+            }
         } else if (write_cache && hd == 128 && n_big_tiles > 0 && tc_attention) {
             // refresh with head dim 128: 128-row work items on the tcgen05 tensor cores, no key split
             AttnArgs aa;

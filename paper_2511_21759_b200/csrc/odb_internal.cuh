@@ -264,6 +264,11 @@ struct StepAttnArgs {
     L2Prefetch pf;
 };
 cudaError_t launch_step_attention(const StepAttnArgs& a, cudaStream_t st);
+// the same work items on the tcgen05 tensor cores (head dim 128): writes the split partials only;
+// cache_rows = rows of the K/V cache viewed as [rows][128]
+cudaError_t launch_step_attention_tc(const StepAttnArgs& a, size_t cache_rows, int* status, cudaStream_t st);
+cudaError_t launch_attention_combine(const float* part_o, const float* part_ml, __nv_bfloat16* o, int M, int H, int hd,
+                                     int ksplit, cudaStream_t st);
 
 // control kernels (control.cu)
 struct ControlBuffers {

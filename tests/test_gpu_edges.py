@@ -24,6 +24,10 @@ CASES = [
     ("hd128_ragged",    "TINY_HD128", 150, 77, 16,  4,      None),   # T = 227: second row tile 99 rows, last key tile 35 keys
     ("hd128_one_tile",  "TINY_HD128", 20,  30, 16,  1,      None),   # T = 50: a single ragged row tile and key tile
     ("hd128_long",      "TINY_HD128", 1000, 64, 32, 8,      6),      # T = 1064: 9 row tiles x 17 key tiles
+    # decode steps with several copies on the tensor cores: cached key tiles for all rows, one fresh tile per copy
+    ("hd128_c8_stage2", "TINY_HD128", 40,  48, 16,  8,      None),   # runs into the decoded-share layout in every block
+    ("hd128_b64_c8",    "TINY_HD128", 70,  128, 64, 8,      None),   # 512 rows per step: several 128-row work items
+    ("hd128_c4_noprompt", "TINY_HD128", 0, 64, 32,  4,      None),   # first block: no cached key at all (empty key splits)
 ]
 
 
@@ -52,6 +56,23 @@ def test_edge_case_in_lockstep(name, shape_name, P, L, Bk, copies, max_iters):
     print(f"\n{name}: {st['iters']} iterations ({st['refreshes']} refreshes), worst logit {st['worst_logit']:.2f} x bound, "
           f"oracle-side decision diffs {st['oracle_decision_diff']}")
     sess.close(); gm.close()
+
+
+@requires_gpu
+def test_tensor_core_step_attention_on_small_batches():
+    """The decode-step attention on the tensor cores is selected only when a step has enough work items
+    to fill the machine (batched steps); an environment variable read once per process lowers that bar,
+    so the multi-copy head-dim-128 cases are run through it in a child process."""
+    import os, subprocess, sys
+    engine()
+    names = ["hd128_ragged", "hd128_c8_stage2", "hd128_b64_c8", "hd128_c4_noprompt"]
+    code = ("import sys; sys.path.insert(0, 'tests'); import test_gpu_edges as t\n"
+            f"for c in t.CASES:\n    if c[0] in {names!r}: t.test_edge_case_in_lockstep(*c)\n")
+    env = dict(os.environ, ODB_ATTN_TC_STEP_MIN="0")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+    assert r.stdout.count("iterations") == len(names), r.stdout[-2000:]
 
 
 @requires_gpu
