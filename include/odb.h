@@ -158,7 +158,9 @@ size_t odb_workspace_bytes(const odb_config* cfg);
 
 /* kv and workspace are device buffers, 256-byte aligned, of at least odb_kv_bytes /
  * odb_workspace_bytes; stream is a cudaStream_t (NULL = default stream).  The call initialises
- * the workspace (RoPE table, state) on the stream and waits for it. */
+ * the workspace (RoPE table, state) and zeroes the K/V cache on the stream and waits for it (the
+ * tensor-core attention loads whole 64-position boxes of the cache: positions that are not keys
+ * are masked but must hold finite values). */
 int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* workspace, size_t ws_bytes,
                            void* stream, odb_session** out);
 int32_t odb_session_destroy(odb_session* s);
