@@ -111,39 +111,64 @@ __device__ int step_tiles_of(const SeqState* st) {
 __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id) {
     const int seq = blockIdx.x;
     SeqState* st = c.state + seq;
-    if (threadIdx.x != 0) return;
     if (!st->active || st->n_masked <= 0) {
-        st->in_fwd = 0;
+        if (threadIdx.x == 0) st->in_fwd = 0;
         return;
     }
-    st->in_fwd = 1;
-    int row = 0, tile = 0;
-    for (int j = 0; j < seq; ++j) {
-        const SeqState* o = c.state + j;
-        if (!o->active || o->n_masked <= 0) continue;
-        row += step_rows_of(o);
-        tile += o->n_copies;
-    }
+    __shared__ int xs[kMaxBlock];      // the block's committed tokens
+    __shared__ int mpre[kMaxBlock];    // masked positions before position i of the block
+    __shared__ int row_base, tile_base, n_masked_blk;
     const int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
-    const int s = st->s, e = st->e;
-    st->row0 = row;
-    for (int cp = 0; cp < st->n_copies; ++cp) {
-        st->copy_row0[cp] = row;
-        for (int p = s; p < e; ++p) {
-            const bool decoded = x[p] != mask_id;
-            if (st->stage2 && cp > 0 && decoded) continue;
-            int tok = x[p];
-            for (int r = 0; r < st->n_ranks; ++r)
-                if (((st->copy_mask[cp] >> r) & 1) && st->rank_off[r] == p - s) tok = st->rank_tok[r];
-            c.row_tok[row] = tok;
-            c.row_pos[row] = p;
-            c.row_seq[row] = seq;
-            c.row_copy[row] = cp;
-            c.row_flags[row] = decoded ? kRowDecoded : 0;
-            c.lm_rows[row] = row;
-            ++row;
+    const int s = st->s, e = st->e, B = e - s;
+    for (int i = threadIdx.x; i < B; i += blockDim.x) xs[i] = x[s + i];
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        st->in_fwd = 1;
+        int row = 0, tile = 0;
+        for (int j = 0; j < seq; ++j) {
+            const SeqState* o = c.state + j;
+            if (!o->active || o->n_masked <= 0) continue;
+            row += step_rows_of(o);
+            tile += o->n_copies;
         }
-        st->copy_nrows[cp] = row - st->copy_row0[cp];
+        int nm = 0;
+        for (int i = 0; i < B; ++i) {
+            mpre[i] = nm;
+            nm += xs[i] == mask_id;
+        }
+        row_base = row; tile_base = tile; n_masked_blk = nm;
+        st->row0 = row;
+        // copy 0 holds the whole block; a speculative copy the whole block or, in the decoded-share layout, the
+        // positions still masked
+        for (int cp = 0; cp < st->n_copies; ++cp) {
+            st->copy_row0[cp] = row;
+            st->copy_nrows[cp] = (st->stage2 && cp > 0) ? nm : B;
+            row += st->copy_nrows[cp];
+        }
+    }
+    __syncthreads();
+    // one thread per (copy, position): the rows of the copies, copy after copy
+    for (int it = threadIdx.x; it < st->n_copies * B; it += blockDim.x) {
+        const int cp = it / B, i = it % B;
+        const bool decoded = xs[i] != mask_id;
+        const bool shared = st->stage2 && cp > 0;
+        if (shared && decoded) continue;
+        const int row = st->copy_row0[cp] + (shared ? mpre[i] : i);
+        int tok = xs[i];
+        for (int r = 0; r < st->n_ranks; ++r)
+            if (((st->copy_mask[cp] >> r) & 1) && st->rank_off[r] == i) tok = st->rank_tok[r];
+        c.row_tok[row] = tok;
+        c.row_pos[row] = s + i;
+        c.row_seq[row] = seq;
+        c.row_copy[row] = cp;
+        c.row_flags[row] = decoded ? kRowDecoded : 0;
+        c.lm_rows[row] = row;
+    }
+    if (threadIdx.x != 0) return;
+    int row = row_base;
+    const int tile = tile_base;
+    for (int cp = 0; cp < st->n_copies; ++cp) {
+        row += st->copy_nrows[cp];
         QTile q;
         q.q_row0 = st->copy_row0[cp];
         q.nq = st->copy_nrows[cp];
@@ -230,11 +255,33 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
     }
     __shared__ float conf[ODB_MAX_COPIES][kMaxBlock];
     __shared__ int tok[ODB_MAX_COPIES][kMaxBlock];
-    if (threadIdx.x != 0) return;
-
+    __shared__ int xs[kMaxBlock];          // the block's committed tokens (step only)
     int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
     const int s = st->s;
     int n_copies = 1;
+    // After a step the whole block gathers the copies' confidences and tokens and the block's tokens (the
+    // decisions below are taken by thread 0 alone, in the order the method states them)
+    const bool gathered = !dry && !after_refresh;
+    if (gathered) {
+        n_copies = st->n_copies;
+        for (int i = threadIdx.x; i < n_copies * kMaxBlock; i += blockDim.x) {
+            conf[i / kMaxBlock][i % kMaxBlock] = -1.f;
+            tok[i / kMaxBlock][i % kMaxBlock] = -1;
+        }
+        for (int i = threadIdx.x; i < st->e - s; i += blockDim.x) xs[i] = x[s + i];
+        __syncthreads();
+        for (int cp = 0; cp < n_copies; ++cp) {
+            const int r0 = st->copy_row0[cp], r1 = r0 + st->copy_nrows[cp];
+            for (int r = r0 + threadIdx.x; r < r1; r += blockDim.x) {
+                const int i = c.row_pos[r] - s;
+                conf[cp][i] = c.conf[r];
+                tok[cp][i] = c.tok[r];
+            }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x != 0) return;
+
     if (dry) {
         // model without LM head (layer microbenchmark): there is nothing to decide on, so commit
         // nothing and lay out the next step as if no position had been accepted; the speculative
@@ -283,20 +330,10 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
             conf[0][i] = c.conf[r];
             tok[0][i] = c.tok[r];
         }
-    } else {
-        n_copies = st->n_copies;
-        for (int cp = 0; cp < n_copies; ++cp) {
-            for (int i = 0; i < kMaxBlock; ++i) { conf[cp][i] = -1.f; tok[cp][i] = -1; }
-            for (int r = st->copy_row0[cp]; r < st->copy_row0[cp] + st->copy_nrows[cp]; ++r) {
-                const int i = c.row_pos[r] - s;
-                conf[cp][i] = c.conf[r];
-                tok[cp][i] = c.tok[r];
-            }
-        }
     }
     const int B = st->e - s;
     bool masked0[kMaxBlock], masked[kMaxBlock], acc[kMaxBlock], taken[kMaxBlock];
-    for (int i = 0; i < B; ++i) { masked0[i] = x[s + i] == mask_id; taken[i] = false; }
+    for (int i = 0; i < B; ++i) { masked0[i] = (gathered ? xs[i] : x[s + i]) == mask_id; taken[i] = false; }
 
     // accept-jump walk (Section 4.2.1): start in the main block; a candidate is hit if its
     // position was accepted with the token it had been filled with; jump to the largest copy
@@ -388,13 +425,13 @@ int step_tiles_host(int n_copies, int rows_copy0, int rows_other) {
 }
 
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st) {
-    build_step_rows_kernel<<<batch, 32, 0, st>>>(c, batch, mask_id);
+    build_step_rows_kernel<<<batch, 64, 0, st>>>(c, batch, mask_id);
     return cudaGetLastError();
 }
 
 cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
                           int mask_id, int eos_id, int dry, cudaStream_t st) {
-    accept_kernel<<<batch, 32, 0, st>>>(c, p, after_refresh, mask_id, eos_id, dry);
+    accept_kernel<<<batch, 64, 0, st>>>(c, p, after_refresh, mask_id, eos_id, dry);
     return cudaGetLastError();
 }
 

@@ -269,18 +269,20 @@ __global__ void __launch_bounds__(256) confidence_partial_kernel(const float* __
     }
 }
 
-// One warp per row: lane l merges triples l, l + 32, ... in ascending order, then the lanes are
-// merged by a fixed shuffle tree (an earlier lane's triple is always the left operand).
+// One block of 128 threads per row: thread t merges triples t, t + 128, ... in ascending order, the lanes of
+// a warp are merged by a fixed shuffle tree (an earlier lane's triple is always the left operand) and the
+// four warps in warp order.
 __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial* __restrict__ part, int chunks, int rows,
                                                               float* __restrict__ conf, int32_t* __restrict__ tok) {
+    __shared__ float sm[4], ss[4];
+    __shared__ int si[4];
     pdl_launch_dependents();
     pdl_wait();
-    const int row = blockIdx.x * 4 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
-    if (row >= rows) return;                            // whole warps leave together
+    const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const ConfPartial* p = part + static_cast<size_t>(row) * chunks;
     float m = -INFINITY, s = 0.f;
     int idx = 0x7fffffff;
-    for (int c = lane; c < chunks; c += 32) conf_merge(m, s, idx, p[c].m, p[c].s, p[c].idx);
+    for (int c = threadIdx.x; c < chunks; c += 128) conf_merge(m, s, idx, p[c].m, p[c].s, p[c].idx);
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
         const float om = __shfl_down_sync(0xffffffffu, m, o);
@@ -288,7 +290,10 @@ __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial
         const int oi = __shfl_down_sync(0xffffffffu, idx, o);
         if (lane + o < 32) conf_merge(m, s, idx, om, os, oi);
     }
-    if (lane == 0) {
+    if (lane == 0) { sm[warp] = m; ss[warp] = s; si[warp] = idx; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 4; ++w) conf_merge(m, s, idx, sm[w], ss[w], si[w]);
         conf[row] = 1.0f / s;
         tok[row] = idx;
     }
@@ -326,7 +331,7 @@ cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
 
 cudaError_t launch_confidence_final(const ConfPartial* part, int chunks, int rows, float* conf, int32_t* tok,
                                     cudaStream_t st) {
-    return launch_kernel(confidence_final_kernel, dim3((rows + 3) / 4), dim3(128), 0, st, part, chunks, rows, conf, tok);
+    return launch_kernel(confidence_final_kernel, dim3(rows), dim3(128), 0, st, part, chunks, rows, conf, tok);
 }
 
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,
