@@ -237,8 +237,8 @@ __device__ int accept_set(const float* conf, const bool* masked, int B, float ta
     return n;
 }
 
-__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id,
-                              int dry) {
+__device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p, int after_refresh, int mask_id, int eos_id,
+                            int dry) {
     const int seq = blockIdx.x;
     SeqState* st = c.state + seq;
     odb_result* res = c.results + seq;
@@ -416,6 +416,22 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
     res->gen_len = st->T - st->P;
     res->block_start = s;
     res->block_end = st->e;
+}
+
+// One block per sequence.  After the decisions, the block writes the sequence's state and result (and block 0
+// the status word) straight into pinned host memory.
+__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id, int dry) {
+    accept_body(c, p, after_refresh, mask_id, eos_id, dry);
+    __syncthreads();
+    const int seq = blockIdx.x;
+    const int* src_state = reinterpret_cast<const int*>(c.state + seq);
+    int* dst_state = reinterpret_cast<int*>(c.host_state + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) dst_state[i] = src_state[i];
+    const int* src_res = reinterpret_cast<const int*>(c.results + seq);
+    int* dst_res = reinterpret_cast<int*>(c.host_results + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) dst_res[i] = src_res[i];
+    if (seq == 0 && threadIdx.x == 0) *c.host_status = *c.status;
+    __threadfence_system();
 }
 
 }  // namespace

@@ -297,6 +297,8 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     cb.lm_rows = s->at<int32_t>(L.lm_rows);
     cb.tiles = s->at<QTile>(L.tile_buf);
     cb.big_tiles = s->at<QTile>(L.big_tile_buf);
+    cb.host_state = s->pinned_state; cb.host_results = s->pinned_results; cb.host_status = s->pinned_status;
+    cb.status = s->at<int>(L.status);
     cb.step_tiles = s->at<StepTile>(L.step_tile_buf);
     cb.conf = s->at<float>(L.conf);
     cb.tok = s->at<int32_t>(L.tok);
@@ -687,11 +689,10 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
     if (s->phase != (after_refresh ? 1 : 3)) return ODB_ERR_STATE;
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id,
                                            c.with_lm_head ? 0 : 1, s->st));
-    ODB_CUDA(cudaMemcpyAsync(s->pinned_results, s->cb.results, sizeof(odb_result) * c.max_batch, cudaMemcpyDeviceToHost, s->st));
     int* dev_status = s->at<int>(s->L.status);
-    ODB_CUDA(cudaMemcpyAsync(s->pinned_status, dev_status, sizeof(int), cudaMemcpyDeviceToHost, s->st));
-    int32_t rc = pull_state(s);
-    if (rc != ODB_OK) return rc;
+    // the kernel has written state, results and status into pinned host memory: one synchronisation, no copy
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    for (int i = 0; i < c.max_batch; ++i) s->mirror[i] = s->pinned_state[i];
     memcpy(results, s->pinned_results, sizeof(odb_result) * c.max_batch);
     s->phase = 2;
     if (*s->pinned_status != 0) {

@@ -282,6 +282,10 @@ struct ControlBuffers {
     StepTile* step_tiles;     // decode steps with more than one copy
     const float* conf; const int32_t* tok;   // outputs of the last forward, per logit row
     odb_result* results;      // [batch] device copy
+    // pinned host memory the accept kernel writes its outcome to (state, results, the status word): the host
+    // reads them after synchronising the stream, no copy is enqueued
+    SeqState* host_state; odb_result* host_results; int* host_status;
+    const int* status;        // device status word
 };
 // block_index[seq] < 0: the sequence takes no part in this refresh
 cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index, int block_len,
