@@ -218,7 +218,7 @@ __global__ void __launch_bounds__(kThreads, 1)
 gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
             float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, RowScale rs,
             ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
-            int l2_prefetch,
+            int l2_prefetch, int pair_tiles_x, int pair_tiles_y,
             int* status) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
@@ -235,15 +235,26 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int n0 = blockIdx.x * kBM;
-    const int m0 = blockIdx.y * BN;
-    const int split = blockIdx.z;
+    // Work unit of this CTA.  Single CTAs: grid (weight tiles, row tiles, K splits).  Pairs: grid (2, row tiles of
+    // a group, weight-tile pairs x row-tile groups x K splits), scheduled in that order: the row tiles of a group
+    // run side by side on one weight-tile pair (its weights come from HBM once, from L2 for the other row
+    // tiles), and a group's activation rows (a few MB) stay in L2 while every weight-tile pair passes over them.
+    const int n_pairs = PAIR ? pair_tiles_x >> 1 : 0;
+    const int n_tile = PAIR ? 2 * static_cast<int>(blockIdx.z % n_pairs) + static_cast<int>(blockIdx.x) : static_cast<int>(blockIdx.x);
+    const int n_tiles = PAIR ? pair_tiles_x : static_cast<int>(gridDim.x);
+    const int m_groups = PAIR ? (pair_tiles_y + static_cast<int>(gridDim.y) - 1) / static_cast<int>(gridDim.y) : 1;
+    const int m_tile = PAIR ? static_cast<int>((blockIdx.z / n_pairs) % m_groups) * static_cast<int>(gridDim.y) + static_cast<int>(blockIdx.y)
+                            : static_cast<int>(blockIdx.y);
+    if (PAIR && m_tile >= pair_tiles_y) return;   // ragged last group: both CTAs of the pair leave together
+    const int n0 = n_tile * kBM;
+    const int m0 = m_tile * BN;
+    const int split = PAIR ? static_cast<int>(blockIdx.z / (n_pairs * m_groups)) : static_cast<int>(blockIdx.z);
     const int kb0 = split * nkb_per_split;
     int nkb = nkb_total - kb0;
     if (nkb > nkb_per_split) nkb = nkb_per_split;
     volatile int* cta_abort = &sh->abort;
     // packed weights: tile (n-tile, k-block) is the contiguous 16 KB chunk number n_tile * nkb_total + k_block
-    const int wtile0 = blockIdx.x * nkb_total + kb0;
+    const int wtile0 = n_tile * nkb_total + kb0;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -409,7 +420,6 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             // is stored.  The RMSNorm scalar of the row is applied first; [MASK] and padding are skipped.
             float* xch = reinterpret_cast<float*>(tiles);           // [32 rows][129]
             const int t = threadIdx.x - 64;                            // 0..127
-            const int n_tiles = gridDim.x;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -449,7 +459,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 if (ok && part == 0 && m < M) {
                     ConfPartial p;
                     p.m = mx; p.s = sum; p.idx = idx;
-                    ce.part[static_cast<size_t>(m) * n_tiles + blockIdx.x] = p;
+                    ce.part[static_cast<size_t>(m) * n_tiles + n_tile] = p;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
@@ -457,7 +467,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             // all MMAs have completed, so the stage ring is free: use it to hand the up values over.
             // Every epilogue warp executes every barrier, whether or not its wait succeeded.
             float* xch = reinterpret_cast<float*>(tiles);           // [64][33]
-            const int f = blockIdx.x * 64 + (q & 1) * 32 + lane;       // FFN feature of this lane's pair
+            const int f = n_tile * 64 + (q & 1) * 32 + lane;          // FFN feature of this lane's pair
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -645,8 +655,14 @@ cudaError_t launch_bn(const GemmArgs& a, cudaStream_t st) {
     }
     if constexpr (PAIR) {
         if (grid.x & 1) return cudaErrorInvalidValue;
+        const int tiles_x = static_cast<int>(grid.x), tiles_y = static_cast<int>(grid.y);
+        // row tiles per group: 8 x 256 rows x K x 2 B stay in L2 (measured at 128 row tiles: groups of 2 / 4 / 8 / 16
+        // give 430 / 414 / 404 / 407 ms of GEMM time per refresh, no grouping 475, one row tile per weight pass 462)
+        const int group = tiles_y < 8 ? tiles_y : 8;
+        const int m_groups = (tiles_y + group - 1) / group;
+        if (static_cast<size_t>(tiles_x / 2) * m_groups * a.splits > 65535) return cudaErrorInvalidValue;
         cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = grid;
+        cfg.gridDim = dim3(2, group, (tiles_x / 2) * m_groups * a.splits);
         cfg.blockDim = dim3(kThreads);
         cfg.dynamicSmemBytes = smem;
         cfg.stream = st;
@@ -660,11 +676,11 @@ cudaError_t launch_bn(const GemmArgs& a, cudaStream_t st) {
         cfg.attrs = attr;
         cfg.numAttrs = pdl_enabled() ? 2 : 1;
         return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI, PAIR>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.conf,
-                                  a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, a.status);
+                                  a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, tiles_x, tiles_y, a.status);
     } else {
         return launch_kernel(gemm_kernel<BN, EPI, PAIR>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
                              a.row_scale, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
-                             pdl_enabled() ? l2_prefetch : 0, a.status);
+                             pdl_enabled() ? l2_prefetch : 0, 0, 0, a.status);
     }
 }
 
