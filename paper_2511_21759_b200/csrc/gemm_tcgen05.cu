@@ -793,7 +793,11 @@ int gemm_pick_splits(int M, int N, int K) {
 
 cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st) {
     const bool swiglu = a.act_out != nullptr;
-    const bool pair = use_pair(a.M, swiglu ? (a.N + 63) / 64 : (a.N + kBM - 1) / kBM);
+    // The gate/up projection has no K split to balance its CTAs over the SMs (192 tiles on 148 SMs at the 8B
+    // shape: some SMs stage for two CTAs), so from 65 rows up it also runs as pairs, each CTA staging half of
+    // the activation rows (measured at 128 rows: step 4.84 -> 4.72 ms; at 32 rows pairs lose, 3.27 vs 3.26).
+    const bool pair = use_pair(a.M, swiglu ? (a.N + 63) / 64 : (a.N + kBM - 1) / kBM) ||
+                      (swiglu && a.M > 64 && pair_enabled() && (((a.N + 63) / 64) & 1) == 0);
     const int bn = pick_bn(a.M, pair);
     if (swiglu) {
         if (a.splits != 1) return cudaErrorInvalidValue;
