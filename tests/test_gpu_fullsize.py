@@ -102,3 +102,73 @@ def test_cfg3_refresh_and_first_step_match_oracle():
           f"element-wise {worst_r:.2f} x / {worst_s:.2f} x the small-model bound; "
           f"conf rel err {cerr:.2e} / {cerr_s:.2e}, greedy tokens differing: "
           f"{int((g_tok != o_tok).sum())} of {L} (refresh), {int((s_tok != o_t[0]).sum())} of {Bk} (step)")
+
+
+@requires_gpu
+def test_cfg4_refresh_and_four_copy_step_match_oracle():
+    """The jump-share configuration at full size (prompt 512, response 512, block 32, 4 copies): one refresh at
+    T = 1024 and the 128-row step that follows it (copies {}, {r1}, {r2}, {r1, r2}), every logit of both against
+    the float32 oracle; row table, accept rule and jump walk reproduced from the kernels' own confidences."""
+    E = engine()
+    wl = synth.WORKLOADS["cfg4_8b_c4"]
+    shape, P, L, Bk = wl.shape, wl.prompt_len, wl.gen_len, wl.block_len
+    T = P + L
+    x0 = synth.sequence(0, 0, P, L, shape)
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=T, max_block=Bk, max_copies=4)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    sess.set_logit_dump(True)
+    gp = E.DecodeParams(block_len=Bk, n_copies=4)
+    sess.refresh_prefill(gp, 0)
+    g_logits = sess.debug_read("logits")[:Bk].copy()          # the block's rows are enough to keep (512 x 126464 floats otherwise)
+    g_conf, g_tok = sess.debug_read("conf"), sess.debug_read("tok")
+    res = sess.unmask_accept(gp, True)[0]
+    g_acc = sorted((res.accepted_pos[j], res.accepted_tok[j]) for j in range(res.n_accepted))
+    sess.block_decode_step(gp)
+    s_logits = sess.debug_read("logits")
+    s_conf, s_tok = sess.debug_read("conf"), sess.debug_read("tok")
+    r_copy, r_pos = sess.debug_read("row_copy"), sess.debug_read("row_pos")
+    res2 = sess.unmask_accept(gp, False)[0]
+    s_acc = sorted((res2.accepted_pos[j], res2.accepted_tok[j]) for j in range(res2.n_accepted))
+    s_chain = [res2.chain[j] for j in range(res2.chain_len)]
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    del gm
+
+    tau = wl.accept_threshold
+    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
+    l2_r = rel_l2(g_logits, o_logits[:Bk])
+    assert l2_r <= 2e-2, f"refresh logits: per-row relative L2 error {l2_r:.3e}"
+    ok, worst_r = logits_close(g_logits, o_logits[:Bk], 6 * 2e-2)
+    assert ok, f"refresh logits off by {6 * worst_r:.2f} x the small-model bound"
+    cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
+    masked = np.ones(Bk, dtype=bool)
+    acc = O.accept_set(g_conf[:Bk], masked, tau)
+    assert g_acc == [(int(P + i), int(g_tok[i])) for i in np.flatnonzero(acc)]
+
+    # the step, from the state and the candidates the GPU is in (its own accepted token and ranking)
+    x = x0.astype(np.int64).copy()
+    for p_, t_ in g_acc:
+        x[p_] = t_
+    masked = x[P:P + Bk] == shape.mask_id
+    ranks = O.rank_candidates(g_conf[:Bk], masked, 2)
+    rank_tok = [int(g_tok[i]) for i in ranks]
+    subsets = O.copy_subsets(len(ranks), 4, False)
+    o_c, o_t, os_logits, oc, op = O.block_decode_step(om, cache, x, T, P, P + Bk, subsets, [P + i for i in ranks], rank_tok,
+                                                      False, dtype=np.float32, return_logits=True)
+    assert np.array_equal(r_copy, oc) and np.array_equal(r_pos, op), "row table"
+    assert s_logits.shape == os_logits.shape == (4 * Bk, shape.vocab)
+    l2_s = rel_l2(s_logits, os_logits)
+    assert l2_s <= 2e-2, f"step logits: per-row relative L2 error {l2_s:.3e}"
+    ok, worst_s = logits_close(s_logits, os_logits, 6 * 2e-2)
+    assert ok, f"step logits off by {6 * worst_s:.2f} x the small-model bound"
+    g_c = np.full((len(subsets), Bk), -1.0, np.float32)
+    g_t = np.full((len(subsets), Bk), -1, np.int32)
+    g_c[r_copy, r_pos - P] = s_conf
+    g_t[r_copy, r_pos - P] = s_tok
+    new, chain, _ = O.jump_walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
+    assert s_acc == sorted((int(P + i), int(t)) for i, t in new.items()) and s_chain == [int(c) for c in chain], "jump walk"
+    print(f"\ncfg4 full size: per-row rel. L2 error {l2_r:.2e} (refresh, block rows) {l2_s:.2e} (4-copy step); "
+          f"element-wise {6 * worst_r:.2f} x / {6 * worst_s:.2f} x the small-model bound; conf rel err {cerr:.2e}; "
+          f"chain {s_chain}, accepted {len(s_acc)}")
