@@ -172,3 +172,88 @@ def test_cfg4_refresh_and_four_copy_step_match_oracle():
     print(f"\ncfg4 full size: per-row rel. L2 error {l2_r:.2e} (refresh, block rows) {l2_s:.2e} (4-copy step); "
           f"element-wise {6 * worst_r:.2f} x / {6 * worst_s:.2f} x the small-model bound; conf rel err {cerr:.2e}; "
           f"chain {s_chain}, accepted {len(s_acc)}")
+
+
+@requires_gpu
+def test_cfg5_batch16_sampled_sequence_matches_oracle():
+    """The batched configuration at full size (16 sequences, prompt 1024, ragged responses of up to 1024, block 64,
+    4 copies: 4096 query rows per step).  The oracle cannot run the whole batch; sequences are independent, so
+    one seeded sequence of the ragged batch is checked: its last-layer K rows and confidences after the refresh
+    (T = 1024 + its response length), its accept decision, the row table, confidences and jump walk of the
+    4-copy step that follows.  The product path is used (no logits are materialised)."""
+    E = engine()
+    wl = synth.WORKLOADS["cfg5_8b_b16"]
+    shape, P, L, Bk, nb = wl.shape, wl.prompt_len, wl.gen_len, wl.block_len, wl.batch
+    targets = synth.shrink_schedule(0, nb, L)
+    lens = [L if i % 4 == 0 else int(targets[i]) for i in range(nb)]       # ragged: a quarter keep the full allocation
+    pick = 5
+    xs = [synth.sequence(0, i, P, lens[i], shape) for i in range(nb)]
+    gm = E.Model.from_synth(shape, seed=0, max_batch=nb, max_seq=P + L, max_block=Bk, max_copies=4)
+    sess = E.Session(gm)
+    for i in range(nb):
+        sess.set_sequence(i, xs[i], P)
+    gp = E.DecodeParams(block_len=Bk, n_copies=4)
+    sess.refresh_prefill(gp, [0] * nb)
+    conf, tok = sess.debug_read("conf"), sess.debug_read("tok")
+    k_last = sess.debug_read("k")
+    r = sess.unmask_accept(gp, True)[pick]                     # the result array is reused by the next call: copy out now
+    g_acc = sorted((r.accepted_pos[j], r.accepted_tok[j]) for j in range(r.n_accepted))
+    assert r.gen_len == lens[pick] and (r.block_start, r.block_end) == (P, P + Bk)
+    sess.block_decode_step(gp)
+    s_conf, s_tok = sess.debug_read("conf"), sess.debug_read("tok")
+    r_copy, r_pos = sess.debug_read("row_copy"), sess.debug_read("row_pos")
+    r2 = sess.unmask_accept(gp, False)[pick]
+    s_acc = sorted((r2.accepted_pos[j], r2.accepted_tok[j]) for j in range(r2.n_accepted))
+    s_chain = [r2.chain[j] for j in range(r2.chain_len)]
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    del gm
+
+    assert len(conf) == sum(lens) and k_last.shape[0] == sum(P + n for n in lens)
+    row0 = sum(P + n for n in lens[:pick])                     # first refresh row of the picked sequence
+    lm0 = sum(lens[:pick])                                     # its first confidence row (block 0 starts at the prompt's end)
+    Lp = lens[pick]
+    T = P + Lp
+    g_conf, g_tok = conf[lm0:lm0 + Lp], tok[lm0:lm0 + Lp]
+    g_k = synth.bf16_bits_to_f32(k_last[row0:row0 + T]).astype(np.float64)
+    tau = wl.accept_threshold
+
+    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    cache, o_conf, o_tok = O.refresh_prefill(om, xs[pick], T, P, dtype=np.float32)
+    o_k = np.asarray(cache.k[-1], dtype=np.float64).reshape(T, -1)
+    k_err = rel_l2(g_k, o_k)
+    assert k_err <= 2e-2, f"last-layer K of the picked sequence: per-row relative L2 error {k_err:.3e}"
+    cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
+    assert cerr <= 0.2, cerr
+    assert (g_tok != o_tok).mean() <= 0.1
+    masked = np.ones(Bk, dtype=bool)
+    acc = O.accept_set(g_conf[:Bk], masked, tau)
+    assert g_acc == [(int(P + i), int(g_tok[i])) for i in np.flatnonzero(acc)]
+
+    # the step: every sequence has 4 copies of 64 rows
+    x = xs[pick].astype(np.int64).copy()
+    for p_, t_ in g_acc:
+        x[p_] = t_
+    masked = x[P:P + Bk] == shape.mask_id
+    ranks = O.rank_candidates(g_conf[:Bk], masked, 2)
+    rank_tok = [int(g_tok[i]) for i in ranks]
+    subsets = O.copy_subsets(len(ranks), 4, False)
+    o_c, o_t = O.block_decode_step(om, cache, x, T, P, P + Bk, subsets, [P + i for i in ranks], rank_tok, False,
+                                   dtype=np.float32)[:2]
+    assert len(r_copy) == nb * 4 * Bk                          # every sequence still has two candidates: 4 copies of the block
+    rows = slice(4 * Bk * pick, 4 * Bk * (pick + 1))
+    rc, rp = r_copy[rows], r_pos[rows]
+    oc, op, _ = O.build_rows(x, P, P + Bk, shape.mask_id, subsets, [P + i for i in ranks], rank_tok, False)
+    assert np.array_equal(rc, oc) and np.array_equal(rp, op), "row table"
+    sc, stok = s_conf[rows], s_tok[rows]
+    serr = float((np.abs(sc - o_c[rc, rp - P]) / o_c[rc, rp - P]).max())
+    assert serr <= 0.2, serr
+    g_c = np.full((4, Bk), -1.0, np.float32)
+    g_t = np.full((4, Bk), -1, np.int32)
+    g_c[rc, rp - P] = sc
+    g_t[rc, rp - P] = stok
+    new, chain, _ = O.jump_walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
+    assert s_acc == sorted((int(P + i), int(t)) for i, t in new.items()), "jump walk: accepted set"
+    assert s_chain == [int(c) for c in chain], "jump walk: chain"
+    print(f"\ncfg5 full size, sequence {pick} of 16 (response {Lp}): last-layer K rel. L2 error {k_err:.2e}; conf rel err "
+          f"{cerr:.2e} (refresh) {serr:.2e} (step); greedy tokens differing {int((g_tok != o_tok).sum())} of {Lp}; chain {chain}")
