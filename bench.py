@@ -246,10 +246,14 @@ def run_cuda(args, wl):
         res = sess.unmask_accept(params, True)
         toks, iters = sum(res[i].n_accepted for i in range(wl.batch)), 1
         while any(res[i].masks_left > 0 for i in range(wl.batch)):
-            sess.block_decode_step(params)
-            res = sess.unmask_accept(params, False)
-            toks += sum(res[i].n_accepted for i in range(wl.batch))
-            iters += 1
+            if not args.host_loop:
+                log = sess.decode_block_resident(params)
+            else:
+                sess.block_decode_step(params)
+                log = [sess.unmask_accept(params, False)]
+            for res in log:
+                toks += sum(res[i].n_accepted for i in range(wl.batch))
+                iters += 1
         state["block"] += 1
         if e2e:
             for i in range(wl.batch):
@@ -315,6 +319,19 @@ def run_cuda(args, wl):
         b_.record(sess.stream)
         res = sess.unmask_accept(params, False)
         step_ms.append(a.elapsed_time(b_))
+    # the same iteration inside the device-resident loop (row table + step + accept, no host in between)
+    loop_ms = None
+    if not args.host_loop:
+        reset()
+        sess.refresh_prefill(params, [0] * wl.batch)
+        sess.unmask_accept(params, True)
+        sess.decode_block_resident(params, 2)                  # records the loop body on first use
+        a, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(sess.stream)
+        n_loop = len(sess.decode_block_resident(params, 8))
+        b_.record(sess.stream)
+        torch.cuda.synchronize()
+        loop_ms = a.elapsed_time(b_) / n_loop
     state["block"] = n_blocks
 
     keys = T - wl.block_len                                   # cached positions outside the block
@@ -341,11 +358,15 @@ def run_cuda(args, wl):
                                 "achieved_gbs": step_bytes / (step_med * 1e-3) / 1e9 if step_med else None,
                                 "frac_of_measured": step_bytes / (step_med * 1e-3) / 1e9 / peaks["hbm_gbs"] if step_med else None,
                                 "frac_of_nominal_8tbs": step_bytes / (step_med * 1e-3) / 1e9 / 8000.0 if step_med else None,
+                                "ms_in_resident_loop": loop_ms,
+                                "frac_of_measured_in_resident_loop": step_bytes / (loop_ms * 1e-3) / 1e9 / peaks["hbm_gbs"] if loop_ms else None,
                                 "ms_by_kind": {k: v / max(n_prof, 1) for k, v in ms_step.items()}},
                 "refresh": {"ms_by_kind": ms_refresh, "T": T}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic", "config": config_of(wl),
+            "dtype": "bf16", "data": "synthetic",
+            "config": dict(config_of(wl), block_loop="device-resident (odb_decode_block_resident)" if not args.host_loop
+                           else "host (odb_block_decode_step + odb_unmask_accept per iteration)"),
             "tokens_per_step": toks / args.steps, "iterations_per_step": iters / args.steps,
             "clocks": clk,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 4 * T * wl.batch,
@@ -362,7 +383,7 @@ def run_cuda(args, wl):
             torch.cuda.synchronize()
             m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             m0.record(sess.stream)
-            _, mtrace = E.generate(sess, mp, cache_blocks=cache_blocks)
+            _, mtrace = E.generate(sess, mp, cache_blocks=cache_blocks, resident=not args.host_loop)
             m1.record(sess.stream)
             torch.cuda.synchronize()
             sess.set_active(0, True)
@@ -459,6 +480,10 @@ def main():
     ap.add_argument("--workload", default="cfg3_8b_c1")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--host-loop", action="store_true",
+                    help="take every iteration of a block as odb_block_decode_step + odb_unmask_accept from the host instead "
+                         "of odb_decode_block_resident (one host round trip per iteration instead of one per change of the "
+                         "step's shape)")
     ap.add_argument("--modes", action="store_true",
                     help="also run the whole response as cache-less baseline / DualCache block decoding / full method")
     args = ap.parse_args()

@@ -12,7 +12,9 @@
  *                             block-wise mask, Section 4.2; decoded-share layout, Section 4.2.2);
  *   - odb_unmask_accept     : the confidence-threshold accept rule (Section 3, Observation 3),
  *                             the accept-jump walk over the copies (Section 4.2.1) and, after a
- *                             refresh, adaptive length prediction (Section 4.1).
+ *                             refresh, adaptive length prediction (Section 4.1);
+ *   - odb_decode_block_resident : step + accept repeated on the device until the block closes or
+ *                             the step's shape changes (no host round trip per iteration).
  * Adaptive length prediction needs no call of its own: the [EOS] scan runs inside
  * odb_unmask_accept(after_refresh = 1), and the host can also shorten a response with
  * odb_session_set_gen_len, the same lever.
@@ -203,6 +205,25 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p);
  * masked positions with token id 0), so masks_left never decreases. */
 int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t after_refresh,
                           odb_result* results);
+
+/* Device-resident block loop: the iterations of the open blocks, each an odb_block_decode_step
+ * followed by the odb_unmask_accept of its outputs (Sections 2.1 and 4.2: a block is decoded by
+ * repeated steps until none of its positions is masked), run on the device without returning to the
+ * host in between.  The loop body is recorded once per step shape as a CUDA graph whose WHILE node
+ * the accept kernel controls; it runs again while (a) fewer than max_iters iterations have run, (b) a
+ * masked position is left in some open block, (c) the next step's row table has the shape of this one
+ * (same number of rows, copies and attention work items: it changes when a sequence closes its block,
+ * when fewer candidates than copies are left, and at the switch to the decoded-share layout), and
+ * (d) no device-side wait has expired.  The results are the ones the two calls would have produced,
+ * bit for bit.
+ * Requires the state after an odb_unmask_accept (a refresh + accept for the block came before).
+ * max_iters: upper bound on iterations, <= 0 or > 64 means 64, never more than log_cap.
+ * log: host array [log_cap][max_batch]; entry [i][seq] is the odb_result of iteration i.
+ * *n_iters: iterations run (>= 1 on success).  Waits for the stream.  When the loop stops with masked
+ * positions left (a shape change or max_iters), call again or continue with the two single calls.
+ * Not available while odb_session_profile is on (ODB_ERR_STATE). */
+int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, int32_t max_iters,
+                                  odb_result* log, int32_t log_cap, int32_t* n_iters);
 
 /* ---- test / measurement entry points --------------------------------------------------- */
 

@@ -92,17 +92,6 @@ __device__ int step_rows_of(const SeqState* st) {
     return st->stage2 ? B + (st->n_copies - 1) * st->n_masked : st->n_copies * B;
 }
 
-// Number of StepTiles of a sequence's next step: copies packed in order into items of <= 8 slabs.
-__host__ __device__ int step_tiles_of_counts(int n_copies, int rows_copy0, int rows_other) {
-    int tiles = 0, slabs = 0;
-    for (int cp = 0; cp < n_copies; ++cp) {
-        const int need = ((cp == 0 ? rows_copy0 : rows_other) + 15) / 16;
-        if (slabs == 0 || slabs + need > 8) { ++tiles; slabs = 0; }
-        slabs += need;
-    }
-    return tiles;
-}
-
 __device__ int step_tiles_of(const SeqState* st) {
     const int B = st->e - st->s;
     return step_tiles_of_counts(st->n_copies, B, st->stage2 ? st->n_masked : B);
@@ -434,10 +423,57 @@ __global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_r
     __threadfence_system();
 }
 
+// The accept of the device-resident loop: the same decisions, then the hand-over to the next iteration.
+__global__ void accept_loop_kernel(ControlBuffers c, odb_decode_params p, int mask_id, int eos_id, int dry, LoopControl lc) {
+    accept_body(c, p, 0, mask_id, eos_id, dry);
+    __syncthreads();
+    const int seq = blockIdx.x, batch = gridDim.x;
+    const int it = *lc.iter;      // stable until every block has arrived below
+    const int* src_state = reinterpret_cast<const int*>(c.state + seq);
+    int* dst_state = reinterpret_cast<int*>(c.host_state + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) dst_state[i] = src_state[i];
+    const int* src_res = reinterpret_cast<const int*>(c.results + seq);
+    int* dst_res = reinterpret_cast<int*>(lc.host_log + static_cast<size_t>(it) * batch + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) dst_res[i] = src_res[i];
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    // fail-safe: the loop ends unless the last block below asks for another pass (block 0 writes this before it
+    // arrives, the last block writes after every arrival, so the last block's word stands)
+    if (seq == 0) {
+        cudaGraphSetConditional(lc.handle, 0u);
+        __threadfence();
+    }
+    if (atomicAdd(lc.arrivals, 1) != batch - 1) return;
+    // last block of the iteration: every sequence's state is final
+    __threadfence();
+    StepShape next{0, 0, 0, 0};
+    for (int i = 0; i < batch; ++i) {
+        const volatile SeqState* vs = c.state + i;
+        SeqState st{};
+        st.active = vs->active; st.n_masked = vs->n_masked; st.s = vs->s; st.e = vs->e;
+        st.n_copies = vs->n_copies; st.stage2 = vs->stage2;
+        step_shape_add(next, st);
+    }
+    const int err = *reinterpret_cast<const volatile int*>(c.status);
+    const bool same = next.rows == lc.shape.rows && next.tiles == lc.shape.tiles &&
+                      next.step_tiles == lc.shape.step_tiles && next.multi == lc.shape.multi;
+    const int limit = min(*lc.max_iters, kMaxLoopIters);
+    const bool again = it + 1 < limit && err == 0 && next.rows > 0 && same;
+    *lc.arrivals = 0;
+    *lc.iter = it + 1;
+    *lc.host_iters = it + 1;
+    *c.host_status = err;
+    __threadfence_system();
+    cudaGraphSetConditional(lc.handle, again ? 1u : 0u);
+}
+
 }  // namespace
 
-int step_tiles_host(int n_copies, int rows_copy0, int rows_other) {
-    return step_tiles_of_counts(n_copies, rows_copy0, rows_other);
+cudaError_t launch_accept_loop(const ControlBuffers& c, int batch, const odb_decode_params& p, int mask_id, int eos_id,
+                               int dry, const LoopControl& lc, cudaStream_t st) {
+    accept_loop_kernel<<<batch, 64, 0, st>>>(c, p, mask_id, eos_id, dry, lc);
+    return cudaGetLastError();
 }
 
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st) {

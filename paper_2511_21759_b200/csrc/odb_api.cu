@@ -46,7 +46,7 @@ int32_t check_config(const odb_config* c) {
 // odb_session_create so that both always agree.
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
-    size_t rope, state, results, status, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
+    size_t rope, state, results, status, loop, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
     size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
     size_t total;
 };
@@ -70,6 +70,7 @@ Layout make_layout(const odb_config& c) {
     L.state = take(sizeof(SeqState) * c.max_batch);
     L.results = take(sizeof(odb_result) * c.max_batch);
     L.status = take(sizeof(int));
+    L.loop = take(4 * sizeof(int32_t));   // device-resident loop: iterations done, accept blocks arrived, iteration limit
     L.x = take(sizeof(int32_t) * c.max_batch * c.max_seq);
     L.row_tok = take(4 * L.rows);
     L.row_pos = take(4 * L.rows);
@@ -136,6 +137,20 @@ struct odb_session {
     std::vector<cudaEvent_t> ev;        // pairs (start, stop)
     std::vector<int> ev_kind;
     size_t ev_used;
+    // device-resident block loop: one instantiated graph per step shape and parameter set, recorded on a
+    // stream of the session's own (the caller's stream may be the default stream, which cannot record)
+    struct ResidentGraph {
+        StepShape shape;
+        odb_decode_params p;
+        bool dump_logits;
+        cudaGraph_t graph;
+        cudaGraphExec_t exec;
+        long long launches[ODB_PROFILE_KINDS];   // kernels of one pass of the loop body
+    };
+    std::vector<ResidentGraph> resident;
+    cudaStream_t record_st;
+    odb_result* pinned_log;   // [kMaxLoopIters][max_batch]
+    int32_t* pinned_iters;    // [0] iterations run (written by the device); [1..3] the loop words of the next launch
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
 
@@ -260,7 +275,13 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->pinned_state = nullptr;
     s->pinned_results = nullptr;
     s->pinned_status = nullptr;
+    s->record_st = nullptr;
+    s->pinned_log = nullptr;
+    s->pinned_iters = nullptr;
     cudaError_t e = cudaMallocHost(&s->pinned_state, sizeof(SeqState) * c.max_batch);
+    if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_log, sizeof(odb_result) * kMaxLoopIters * c.max_batch);
+    if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_iters, 4 * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&s->record_st, cudaStreamNonBlocking);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_results, sizeof(odb_result) * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_status, sizeof(int));
     // RoPE table: angle(pos, i) = pos * theta^(-2i/hd), evaluated in double, stored as fp32 (cos, sin)
@@ -312,6 +333,13 @@ int32_t odb_session_destroy(odb_session* s) {
     if (s->pinned_state) cudaFreeHost(s->pinned_state);
     if (s->pinned_results) cudaFreeHost(s->pinned_results);
     if (s->pinned_status) cudaFreeHost(s->pinned_status);
+    if (s->pinned_log) cudaFreeHost(s->pinned_log);
+    if (s->pinned_iters) cudaFreeHost(s->pinned_iters);
+    for (auto& g : s->resident) {
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+        if (g.graph) cudaGraphDestroy(g.graph);
+    }
+    if (s->record_st) cudaStreamDestroy(s->record_st);
     for (cudaEvent_t e : s->ev) cudaEventDestroy(e);
     delete s;
     return ODB_OK;
@@ -420,11 +448,12 @@ struct LaunchScope {
 };
 
 // One forward over the M rows of the row table already built on the device.
-int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0, int n_big_tiles = 0) {
+int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0, int n_big_tiles = 0,
+                cudaStream_t st = nullptr) {
     const odb_model* m = s->m;
     const odb_config& c = m->cfg;
     const Layout& L = s->L;
-    cudaStream_t st = s->st;
+    if (!st) st = s->st;
     const int d = c.d_model, F = c.d_ffn, H = c.n_heads, hd = c.head_dim;
     float* h = s->at<float>(L.h);
     __nv_bfloat16* a = s->at<__nv_bfloat16>(L.a);
@@ -615,6 +644,11 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     return ODB_OK;
 }
 
+// Work items of the multi-copy step attention for a step of this shape (0: the per-copy kernel is used)
+int step_items(const odb_session* s, const StepShape& sh) {
+    return (!sh.multi || static_cast<size_t>(2) * sh.rows > s->L.attn_rows) ? 0 : sh.step_tiles;
+}
+
 int32_t pull_state(odb_session* s) {
     const int nb = s->m->cfg.max_batch;
     ODB_CUDA(cudaMemcpyAsync(s->pinned_state, s->cb.state, sizeof(SeqState) * nb, cudaMemcpyDeviceToHost, s->st));
@@ -657,22 +691,13 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
     if (!s || !p) return ODB_ERR_ARG;
     const odb_config& c = s->m->cfg;
     if (s->phase != 2) return ODB_ERR_STATE;
-    int M = 0, n_tiles = 0, n_step_tiles = 0;
-    bool multi = false;
-    for (int i = 0; i < c.max_batch; ++i) {
-        const SeqState& st = s->mirror[i];
-        if (!st.active || st.n_masked <= 0) continue;
-        const int B = st.e - st.s;
-        M += st.stage2 ? B + (st.n_copies - 1) * st.n_masked : st.n_copies * B;
-        n_tiles += st.n_copies;
-        if (st.n_copies > 1) multi = true;
-        n_step_tiles += step_tiles_host(st.n_copies, B, st.stage2 ? st.n_masked : B);
-    }
-    if (!multi || static_cast<size_t>(2) * M > s->L.attn_rows) n_step_tiles = 0;   // plain kernel for single copies
+    StepShape sh{0, 0, 0, 0};
+    for (int i = 0; i < c.max_batch; ++i) step_shape_add(sh, s->mirror[i]);
+    const int M = sh.rows;
     if (M == 0) return ODB_ERR_STATE;
     if (static_cast<size_t>(M) > s->L.rows) return ODB_ERR_SHAPE;
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
-    int32_t rc = forward(s, M, c.with_lm_head ? M : 0, n_tiles, false, n_step_tiles);
+    int32_t rc = forward(s, M, c.with_lm_head ? M : 0, sh.tiles, false, step_items(s, sh));
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
     s->last_lm_rows = M;
@@ -697,6 +722,97 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
     s->phase = 2;
     if (*s->pinned_status != 0) {
         cudaMemsetAsync(dev_status, 0, sizeof(int), s->st);
+        return *s->pinned_status;
+    }
+    return ODB_OK;
+}
+
+int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, int32_t max_iters, odb_result* log,
+                                  int32_t log_cap, int32_t* n_iters) {
+    if (!s || !p || !log || !n_iters || log_cap < 1) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
+    if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
+    if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
+    if (s->phase != 2 || s->profiling) return ODB_ERR_STATE;   // event pairs cannot be recorded into the loop body
+    *n_iters = 0;
+    if (max_iters <= 0 || max_iters > kMaxLoopIters) max_iters = kMaxLoopIters;
+    if (max_iters > log_cap) max_iters = log_cap;
+    StepShape sh{0, 0, 0, 0};
+    for (int i = 0; i < c.max_batch; ++i) step_shape_add(sh, s->mirror[i]);
+    if (sh.rows == 0) return ODB_ERR_STATE;
+    if (static_cast<size_t>(sh.rows) > s->L.rows) return ODB_ERR_SHAPE;
+
+    odb_session::ResidentGraph* g = nullptr;
+    for (auto& r : s->resident)
+        if (memcmp(&r.shape, &sh, sizeof(sh)) == 0 && memcmp(&r.p, p, sizeof(*p)) == 0 && r.dump_logits == s->dump_logits)
+            g = &r;
+    int32_t* loop_words = s->at<int32_t>(s->L.loop);   // [0] iterations done, [1] arrivals, [2] iteration limit
+    if (!g) {
+        odb_session::ResidentGraph r{};
+        r.shape = sh; r.p = *p; r.dump_logits = s->dump_logits;
+        ODB_CUDA(cudaGraphCreate(&r.graph, 0));
+        LoopControl lc;
+        cudaError_t e = cudaGraphConditionalHandleCreate(&lc.handle, r.graph, 1, cudaGraphCondAssignDefault);
+        cudaGraphNodeParams np = {cudaGraphNodeTypeConditional};
+        np.conditional.handle = lc.handle;
+        np.conditional.type = cudaGraphCondTypeWhile;
+        np.conditional.size = 1;
+        cudaGraphNode_t node;
+        if (e == cudaSuccess) e = cudaGraphAddNode(&node, r.graph, nullptr, 0, &np);
+        if (e == cudaSuccess)
+            e = cudaStreamBeginCaptureToGraph(s->record_st, np.conditional.phGraph_out[0], nullptr, nullptr, 0,
+                                              cudaStreamCaptureModeThreadLocal);
+        if (e != cudaSuccess) {
+            cudaGraphDestroy(r.graph);
+            return cuda_fail(e);
+        }
+        lc.iter = loop_words;
+        lc.arrivals = loop_words + 1;
+        lc.max_iters = loop_words + 2;
+        lc.shape = sh;
+        lc.host_log = s->pinned_log;
+        lc.host_iters = s->pinned_iters;
+        long long before[ODB_PROFILE_KINDS];
+        memcpy(before, s->launches, sizeof(before));
+        // the body: row table, forward, accept.  Whatever a launch returns, the recording is closed before leaving.
+        int32_t rc = [&]() -> int32_t {
+            ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->record_st));
+            int32_t frc = forward(s, sh.rows, c.with_lm_head ? sh.rows : 0, sh.tiles, false, step_items(s, sh), 0, s->record_st);
+            if (frc != ODB_OK) return frc;
+            ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept_loop(s->cb, c.max_batch, *p, c.mask_id, c.eos_id,
+                                                            c.with_lm_head ? 0 : 1, lc, s->record_st));
+            return ODB_OK;
+        }();
+        for (int k = 0; k < ODB_PROFILE_KINDS; ++k) r.launches[k] = s->launches[k] - before[k];
+        memcpy(s->launches, before, sizeof(before));
+        cudaGraph_t body = nullptr;
+        e = cudaStreamEndCapture(s->record_st, &body);
+        if (rc == ODB_OK && e == cudaSuccess) e = cudaGraphInstantiate(&r.exec, r.graph, 0);
+        if (rc != ODB_OK || e != cudaSuccess) {
+            if (r.exec) cudaGraphExecDestroy(r.exec);
+            cudaGraphDestroy(r.graph);
+            return rc != ODB_OK ? rc : cuda_fail(e);
+        }
+        s->resident.push_back(r);
+        g = &s->resident.back();
+    }
+    s->pinned_iters[0] = 0;
+    s->pinned_iters[1] = 0; s->pinned_iters[2] = 0; s->pinned_iters[3] = max_iters;
+    ODB_CUDA(cudaMemcpyAsync(loop_words, s->pinned_iters + 1, 3 * sizeof(int32_t), cudaMemcpyHostToDevice, s->st));
+    ODB_CUDA(cudaGraphLaunch(g->exec, s->st));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    const int done = *s->pinned_iters;
+    if (done < 1 || done > max_iters) return ODB_ERR_STATE;
+    for (int k = 0; k < ODB_PROFILE_KINDS; ++k) s->launches[k] += g->launches[k] * done;
+    for (int i = 0; i < c.max_batch; ++i) s->mirror[i] = s->pinned_state[i];
+    memcpy(log, s->pinned_log, sizeof(odb_result) * static_cast<size_t>(done) * c.max_batch);
+    *n_iters = done;
+    s->last_rows = sh.rows;
+    s->last_lm_rows = sh.rows;
+    s->phase = 2;
+    if (*s->pinned_status != 0) {
+        cudaMemsetAsync(s->at<int>(s->L.status), 0, sizeof(int), s->st);
         return *s->pinned_status;
     }
     return ODB_OK;

@@ -71,6 +71,7 @@ cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_
 // ---------------------------------------------------------------------------------------
 
 constexpr int kMaxBlock = 64;
+constexpr int kMaxLoopIters = 64;   // iterations of one device-resident loop (a block needs at most its length)
 
 // Per-sequence control state, resident on the device and mirrored on the host after every
 // odb_unmask_accept.  Positions are absolute (prompt position 0 first).
@@ -291,9 +292,50 @@ struct ControlBuffers {
 cudaError_t launch_build_refresh_rows(const ControlBuffers& c, int batch, const int32_t* block_index, int block_len,
                                       cudaStream_t st);
 cudaError_t launch_build_step_rows(const ControlBuffers& c, int batch, int mask_id, cudaStream_t st);
-int step_tiles_host(int n_copies, int rows_copy0, int rows_other);   // StepTiles of one sequence's step
+
+// Number of StepTiles of a sequence's step: copies packed in order into items of <= 8 slabs of 16 rows.
+__host__ __device__ inline int step_tiles_of_counts(int n_copies, int rows_copy0, int rows_other) {
+    int tiles = 0, slabs = 0;
+    for (int cp = 0; cp < n_copies; ++cp) {
+        const int need = ((cp == 0 ? rows_copy0 : rows_other) + 15) / 16;
+        if (slabs == 0 || slabs + need > 8) { ++tiles; slabs = 0; }
+        slabs += need;
+    }
+    return tiles;
+}
+
+// Shape of the row table of the next step, summed over the sequences that take part in it: everything a
+// step's launch configuration depends on.  Evaluated by the host before it enqueues a step and by the
+// device-resident loop, which goes on only while the shape it was recorded for still holds.
+struct StepShape {
+    int32_t rows, tiles, step_tiles, multi;
+};
+__host__ __device__ inline void step_shape_add(StepShape& sh, const SeqState& st) {
+    if (!st.active || st.n_masked <= 0) return;
+    const int B = st.e - st.s;
+    sh.rows += st.stage2 ? B + (st.n_copies - 1) * st.n_masked : st.n_copies * B;
+    sh.tiles += st.n_copies;
+    if (st.n_copies > 1) sh.multi = 1;
+    sh.step_tiles += step_tiles_of_counts(st.n_copies, B, st.stage2 ? st.n_masked : B);
+}
 // dry: model without LM head; commits nothing, only lays out the next step
 cudaError_t launch_accept(const ControlBuffers& c, int batch, const odb_decode_params& p, int after_refresh,
                           int mask_id, int eos_id, int dry, cudaStream_t st);
+
+// Control words of the device-resident block loop (a CUDA graph whose body, one step and its accept, sits in a
+// WHILE node).  The accept kernel of the body appends the per-sequence results of iteration i to
+// host_log[i][batch], and its last block decides whether the body runs again: iterations < max_iters, a masked
+// position left, no device error, and the next step's row table has the shape the body was recorded for.
+struct LoopControl {
+    cudaGraphConditionalHandle handle;
+    int32_t* iter;          // device: iterations completed since the loop was launched
+    int32_t* arrivals;      // device: accept blocks that have finished the current iteration
+    const int32_t* max_iters;   // device: iteration limit of this launch (hard limit kMaxLoopIters)
+    StepShape shape;
+    odb_result* host_log;   // pinned host memory [kMaxLoopIters][batch]
+    int32_t* host_iters;    // pinned host memory: copy of *iter
+};
+cudaError_t launch_accept_loop(const ControlBuffers& c, int batch, const odb_decode_params& p, int mask_id, int eos_id,
+                               int dry, const LoopControl& lc, cudaStream_t st);
 
 }  // namespace odb

@@ -173,6 +173,18 @@ class Session:
                 "odb_unmask_accept")
         return self._results
 
+    def decode_block_resident(self, params: DecodeParams, max_iters: int = 0):
+        """The device-resident loop: steps and accepts of the open blocks until they close, the step's shape
+        changes or max_iters iterations have run.  Returns a list with one entry per iteration, each the
+        per-sequence results of that iteration's accept (copies: they stay valid)."""
+        p = params.c()
+        cap = 64 if max_iters <= 0 else min(max_iters, 64)
+        log = (B.odb_result * (cap * self.nb))()
+        n = C.c_int32()
+        B.check(B.lib().odb_decode_block_resident(self.handle, C.byref(p), max_iters, log, cap, C.byref(n)),
+                "odb_decode_block_resident")
+        return [[log[i * self.nb + j] for j in range(self.nb)] for i in range(n.value)]
+
     def set_logit_dump(self, enable: bool):
         """Test mode: the LM head writes fp32 logits (debug_read("logits")) instead of fusing the reduction."""
         B.check(B.lib().odb_debug_set_logit_dump(self.handle, 1 if enable else 0), "odb_debug_set_logit_dump")
@@ -235,7 +247,7 @@ def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> 
 
 def generate(sess: Session, params: DecodeParams, *,
              length_schedule: Optional[Callable[[int, int, int], Optional[int]]] = None,
-             max_iters: Optional[int] = None, cache_blocks: bool = True):
+             max_iters: Optional[int] = None, cache_blocks: bool = True, resident: bool = False):
     """Runs every sequence set on the session to completion.
 
     Per iteration: the sequences standing at a block boundary are refreshed and accepted
@@ -245,7 +257,8 @@ def generate(sess: Session, params: DecodeParams, *,
     prediction also pulls).  Returns ({seq: tokens}, trace); trace is a list of per-call dicts
     {"kind", "seqs": {seq: {"accepted", "chain", "masks_left", "gen_len", "block"}}}.
     cache_blocks=False is the cache-less baseline (Section 1): every iteration of a block is a
-    refresh prefill and no block step is taken."""
+    refresh prefill and no block step is taken.  resident=True runs the steps of a block through the
+    device-resident loop (same trace, one host round trip per block instead of one per iteration)."""
     seqs = sorted(sess.gen_len)
     block = {i: 0 for i in seqs}
     need_refresh = {i: True for i in seqs}
@@ -280,6 +293,11 @@ def generate(sess: Session, params: DecodeParams, *,
             res = sess.unmask_accept(params, True)
             record(res, "refresh", refresh)
             touched = refresh
+        elif resident:
+            left = 0 if max_iters is None else max_iters - len(trace)
+            for res in sess.decode_block_resident(params, left):
+                record(res, "step", todo)
+            touched = todo
         else:
             sess.block_decode_step(params)
             res = sess.unmask_accept(params, False)

@@ -19,7 +19,8 @@ from gpu_common import engine, requires_gpu, compare_traces, lockstep_generate, 
 NEAR_TIE = 1e-3
 
 
-def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=None, om=None, lm_head_bits=None):
+def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=None, om=None, lm_head_bits=None,
+              resident=False):
     E = engine()
     wl = synth.WORKLOADS[wl_name]
     shape = shape or wl.shape
@@ -33,7 +34,7 @@ def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=
               truncate_threshold=wl.truncate_threshold)
     kw.update(params_kw or {})
     gsched = (lambda seq, b, L: schedule(b, L)) if schedule else None
-    gtok, gtrace = E.generate(sess, E.DecodeParams(**kw), length_schedule=gsched)
+    gtok, gtrace = E.generate(sess, E.DecodeParams(**kw), length_schedule=gsched, resident=resident)
     otok, otrace = O.generate(om, x0, wl.prompt_len, O.DecodeParams(**kw), length_schedule=schedule)
     assert sess.status() == 0
     sess.close(); gm.close()
@@ -56,6 +57,84 @@ def test_generate_matches_oracle(wl):
     # free run: the sharp-logit model turns a logit error into a confidence error of the same
     # size (5e-2 .. 9e-2 measured by the lock-step test), so its near-tie band is wider
     _assert_parity(*_run_both(wl), near_tie=NEAR_TIE if wl.startswith("cfg1") else 0.2)
+
+
+@requires_gpu
+@pytest.mark.parametrize("wl", ["cfg1_tiny", "cfg1_tiny_c4", "peaky_c1", "peaky_c4", "peaky_c8"])
+def test_resident_loop_matches_oracle(wl):
+    """The same free run with the steps of every block taken by the device-resident loop."""
+    _assert_parity(*_run_both(wl, resident=True), near_tie=NEAR_TIE if wl.startswith("cfg1") else 0.2)
+
+
+@requires_gpu
+@pytest.mark.parametrize("copies", [1, 4, 8])
+def test_resident_loop_equals_call_by_call(copies):
+    """A ragged batch of three sequences, decoded call by call and through the device-resident loop: the
+    traces (accepted sets, chains, masks left, block bounds, per iteration and sequence), the final tokens
+    and the number of kernels launched are identical; the loop returns to the host once per change of the
+    step's shape instead of once per iteration."""
+    E = engine()
+    shape = synth.TINY_PEAKY
+    P, lens, Bk = 24, [48, 37, 16], 16
+    gm = E.Model.from_synth(shape, seed=2, max_batch=3, max_seq=P + max(lens), max_block=Bk, max_copies=8)
+    params = E.DecodeParams(block_len=Bk, n_copies=copies)
+    runs = []
+    for resident in (False, True):
+        sess = E.Session(gm)
+        for i, n in enumerate(lens):
+            sess.set_sequence(i, synth.sequence(2, i, P, n, shape), P)
+        calls = {"n": 0}
+        inner = sess.decode_block_resident
+
+        def counted(*a, _inner=inner, **k):
+            calls["n"] += 1
+            return _inner(*a, **k)
+        sess.decode_block_resident = counted
+        toks, trace = E.generate(sess, params, resident=resident)
+        assert sess.status() == 0
+        runs.append((toks, trace, sess.profile_read()[1], calls["n"]))
+        sess.close()
+    gm.close()
+    (t0, tr0, l0, _), (t1, tr1, l1, n_loops) = runs
+    assert tr0 == tr1
+    for i in range(3):
+        assert np.array_equal(t0[i], t1[i]) and (t0[i][P:] != shape.mask_id).all()
+    steps = sum(t["kind"] == "step" for t in tr0)
+    assert l0 == l1, (l0, l1)
+    assert 0 < n_loops < steps or steps <= 1
+    print(f"\n{copies} copies: {steps} step iterations in {n_loops} loop launches")
+
+
+@requires_gpu
+def test_resident_loop_respects_max_iters_and_state():
+    E = engine()
+    from paper_2511_21759_b200 import binding as B
+    shape = synth.TINY
+    P, L, Bk = 20, 32, 16
+    gm = E.Model.from_synth(shape, seed=1, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
+    sess = E.Session(gm)
+    sess.set_sequence(0, synth.sequence(1, 0, P, L, shape), P)
+    gp = E.DecodeParams(block_len=Bk, n_copies=1, accept_threshold=1.0)     # one token per iteration: 15 steps per block
+    with pytest.raises(B.OdbError) as err:                                  # nothing refreshed yet
+        sess.decode_block_resident(gp)
+    assert err.value.status == B.ODB_ERR_STATE
+    sess.refresh_prefill(gp, 0)
+    assert sess.unmask_accept(gp, True)[0].masks_left == 15
+    log = sess.decode_block_resident(gp, 4)
+    assert len(log) == 4 and [it[0].masks_left for it in log] == [14, 13, 12, 11]
+    log = sess.decode_block_resident(gp)                                     # runs the block to its end
+    assert len(log) == 11 and log[-1][0].masks_left == 0
+    with pytest.raises(B.OdbError) as err:                                  # the block is closed: no rows
+        sess.decode_block_resident(gp)
+    assert err.value.status == B.ODB_ERR_STATE
+    sess.refresh_prefill(gp, 1)                                             # the session goes on normally
+    assert sess.unmask_accept(gp, True)[0].masks_left == 15
+    sess.block_decode_step(gp)                                              # mixing with the single calls
+    assert sess.unmask_accept(gp, False)[0].masks_left == 14
+    log = sess.decode_block_resident(gp)
+    assert len(log) == 14 and log[-1][0].masks_left == 0
+    assert sess.status() == 0
+    sess.close(); gm.close()
 
 
 @requires_gpu
