@@ -390,6 +390,43 @@ def jump_walk(conf: np.ndarray, tok: np.ndarray, masked0: np.ndarray, subsets: l
     return new, chain, cur
 
 
+def pick_best_walk(conf: np.ndarray, tok: np.ndarray, masked0: np.ndarray, subsets: list,
+                   rank_off: list, rank_tok: list, tau: float):
+    """The speculation the paper compares against ("traditional dLLM speculative", Fig. 7(a); the
+    "vanilla speculation" of Section 5.3): the same copies, but one of them is picked and its
+    decoding replaces the main block's.  The candidates are verified in the main block only (hit =
+    accepted there with the speculated token); the copy filling the largest set of hit candidates
+    is adopted (lowest ranks on a tie, the main block if nothing is hit): its fills and its own
+    accept set are committed, nothing else.  No candidate is verified inside a copy and no second
+    jump is made, so every step is one state change: the chain has the adopted copy as its only
+    link, which is why Section 5.3 can say that Eff_NFE equals NFE for this variant.
+    Reading: the paper describes this variant only by that property and by "pick"-ing among the
+    appended blocks; the main block's other accepted tokens are not carried over (they are the
+    output of a block that was not adopted).
+    Returns (new_tokens dict offset->token, chain [adopted copy], adopted copy index)."""
+    acc0 = accept_set(conf[0], masked0, tau)
+    hit = {r for r in range(1, len(rank_off) + 1)
+           if acc0[rank_off[r - 1]] and tok[0][rank_off[r - 1]] == rank_tok[r - 1]}
+    best = None
+    for ci, Y in enumerate(subsets):
+        if len(Y) > 0 and set(Y) <= hit:
+            key = (-len(Y), Y)
+            if best is None or key < best[0]:
+                best = (key, ci)
+    if best is None:
+        return {int(i): int(tok[0][i]) for i in np.flatnonzero(acc0)}, [0], 0
+    cur = best[1]
+    new = {int(rank_off[r - 1]): int(rank_tok[r - 1]) for r in subsets[cur]}
+    masked = masked0.copy()
+    for r in subsets[cur]:
+        masked[rank_off[r - 1]] = False
+    if masked.any():
+        acc = accept_set(conf[cur], masked, tau)
+        for i in np.flatnonzero(acc):
+            new[int(i)] = int(tok[cur][i])
+    return new, [cur], cur
+
+
 def alp_scan(conf: np.ndarray, tok: np.ndarray, s: int, P: int, eos_id: int, tau_trunc: float):
     """Adaptive length prediction (Section 4.1): scan the refresh's prediction of the whole
     response from the block start on; the first [EOS] whose confidence exceeds the truncate
@@ -409,6 +446,7 @@ class DecodeParams:
     truncate_threshold: float = 0.9
     stage2_min_decoded: int = -1      # -1: ceil(4 B / 7), the point where 8 copies fit 4 B rows
     alp: bool = True
+    pick_best: bool = False           # the compared "vanilla speculation": pick_best_walk instead of jump_walk
 
 
 def use_stage2(params: DecodeParams, B: int, n_decoded: int) -> bool:
@@ -477,7 +515,8 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             subsets = copy_subsets(len(ranks), 4 if (params.n_copies == 8 and not st2) else params.n_copies, st2)
             conf, tok = block_decode_step(model, cache, x, T, s, e, subsets, rank_pos, rank_tok,
                                           st2, faithful=faithful, dtype=dtype)
-            new, chain, last = jump_walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
+            walk = pick_best_walk if params.pick_best else jump_walk
+            new, chain, last = walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
             for i, t in new.items():
                 x[s + i] = t
             margin = min(decision_margin(conf[c], masked & (conf[c] >= 0), tau, k_ranks + 1) for c in chain)
@@ -494,7 +533,12 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
 # Fast-dLLM (DualCache block decoding with threshold acceptance, fixed length, no speculation),
 # and the paper's method (adaptive length prediction + jump-share speculation).
 def mode_settings(mode: str, block_len: int, n_copies: int = 4, accept_threshold: float = 0.9):
-    """Returns (DecodeParams, cache_blocks) for "vanilla", "fast_dllm" or "odb"."""
+    """Returns (DecodeParams, cache_blocks) for "vanilla", "fast_dllm" or "odb", and for the speculation
+    variants of Section 5.3 (Fig. 11), each on block decoding without length prediction: "spec_vanilla"
+    (pick one of four blocks), "accept_jump" (four copies, jump chain), "decoded_share" (eight copies)."""
+    if mode in ("spec_vanilla", "accept_jump", "decoded_share"):
+        return DecodeParams(block_len=block_len, n_copies=8 if mode == "decoded_share" else 4,
+                            accept_threshold=accept_threshold, alp=False, pick_best=mode == "spec_vanilla"), True
     if mode == "vanilla":
         return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=1.0, alp=False), False
     if mode == "fast_dllm":

@@ -706,7 +706,14 @@ cudaError_t launch_epi(const GemmArgs& a, int bn, bool pair, cudaStream_t st) {
 // 8B shape: with many rows (refresh, 768..1024 rows: tensor/L2 bound) pairs with 256-row tiles are 11 %
 // faster than single CTAs with 128-row tiles; up to 128 rows (decode steps: HBM bound) the pair's extra
 // synchronisation costs more than the halved activation traffic saves (3.55 vs 3.41 ms at 32 rows).
-bool use_pair(int M, int n_tiles) { return pair_enabled() && M > 128 && (n_tiles & 1) == 0; }
+bool use_pair(int M, int n_tiles) {
+    static int min_rows = -1;
+    if (min_rows < 0) {
+        const char* e = getenv("ODB_GEMM_PAIR_MIN_ROWS");
+        min_rows = e ? atoi(e) : 128;
+    }
+    return pair_enabled() && M > min_rows && (n_tiles & 1) == 0;
+}
 
 }  // namespace
 

@@ -140,6 +140,73 @@ def test_jump_walk_stage2_lattice():
     assert chain == [0, 4] and new == {2: 12, 5: 15}
 
 
+# ----------------------------------------------------------------------------- the compared "vanilla" speculation
+
+def _pick(conf_rows, tok_rows, masked, subsets, rank_off, rank_tok, tau=0.9):
+    return O.pick_best_walk(np.array(conf_rows, np.float32), np.array(tok_rows, np.int32), np.array(masked, bool),
+                            subsets, rank_off, rank_tok, tau)
+
+
+def test_pick_best_adopts_one_block_and_nothing_else():
+    """Fig. 7(a) / Section 5.3: candidates are checked in the main block, one appended block is picked and
+    its decoding replaces the main block's; one state change per step (chain of one link)."""
+    masked = [1] * 6
+    rank_off, rank_tok = [1, 5], [11, 15]
+    tok = [[20, 11, 22, 23, 24, 15]] * 4
+    # both candidates accepted in block 0, which also accepts position 0: the block filling both is adopted; its own
+    # accept set is position 3; position 0 (output of the block that was not adopted) is NOT committed
+    conf = [[.95, .95, .1, .1, .1, .95], [0] * 6, [0] * 6, [.5, 0, .1, .95, .1, 0]]
+    new, chain, last = _pick(conf, tok, masked, S1, rank_off, rank_tok)
+    assert (new, chain, last) == ({1: 11, 5: 15, 3: 23}, [3], 3)
+    # the jump chain on the same numbers keeps position 0 as well and has two links
+    new_j, chain_j, _ = _walk(conf, tok, masked, S1, rank_off, rank_tok)
+    assert new_j == {0: 20, 1: 11, 5: 15, 3: 23} and chain_j == [0, 3]
+    # only the first candidate is hit: its block is adopted; that block accepts the second candidate's position,
+    # which is committed as that block's output, but no second block is entered (the jump chain would go on to {1,2})
+    conf = [[.1, .95, .1, .1, .1, .3], [.1, 0, .1, .1, .1, .95], [0] * 6, [.1, 0, .95, .1, .1, 0]]
+    new, chain, last = _pick(conf, tok, masked, S1, rank_off, rank_tok)
+    assert (new, chain, last) == ({1: 11, 5: 15}, [1], 1)
+    new_j, chain_j, _ = _walk(conf, tok, masked, S1, rank_off, rank_tok)
+    assert chain_j == [0, 1, 3] and new_j == {1: 11, 5: 15, 2: 22}
+    # a candidate accepted with ANOTHER token is not a hit; nothing hit: the main block's own result
+    tok2 = [[20, 99, 22, 23, 24, 15]] + tok[1:]
+    conf = [[.1, .95, .1, .1, .1, .3]] + [[.95] * 6] * 3
+    new, chain, last = _pick(conf, tok2, masked, S1, rank_off, rank_tok)
+    assert (new, chain, last) == ({1: 99}, [0], 0)
+    # nothing above the threshold anywhere: top-1 fallback of the main block, which is a hit when it is the first
+    # candidate with its token -> that candidate's block, whose own fallback commits one more position
+    conf = [[.1, .6, .1, .1, .1, .3], [.1, 0, .1, .4, .1, .2], [0] * 6, [0] * 6]
+    new, chain, last = _pick(conf, tok, masked, S1, rank_off, rank_tok)
+    assert (new, chain, last) == ({1: 11, 3: 23}, [1], 1)
+    # the adopted block has nothing left to decode: only its fills are committed
+    new, chain, last = _pick([[.95, .95], [0, 0], [0, 0], [0, 0]], [[11, 15]] * 4, [1, 1], S1, [0, 1], [11, 15])
+    assert (new, chain, last) == ({0: 11, 1: 15}, [3], 3)
+
+
+def test_pick_best_generation_has_eff_nfe_equal_to_nfe(tiny_model):
+    """Section 5.3: for the compared speculation Eff_NFE equals NFE; the run still fills every position, never
+    needs more passes than plain block decoding needs in the worst case, and without a hit it IS plain block
+    decoding (one block's accept set per pass)."""
+    shape = synth.TINY
+    P, L, Bk = 12, 32, 16
+    x0 = synth.sequence(4, 0, P, L, shape)
+    pv, cb = O.mode_settings("spec_vanilla", Bk)
+    assert pv.pick_best and pv.n_copies == 4 and not pv.alp and cb
+    xv, tv = O.generate(tiny_model, x0, P, pv)
+    cv = O.trace_counters(tv)
+    assert (xv[P:] != shape.mask_id).all() and cv["tokens"] == L
+    assert cv["eff_nfe"] == cv["nfe"] <= L and all(len(t["chain"]) == 1 for t in tv)
+    pj, _ = O.mode_settings("accept_jump", Bk)
+    xj, tj = O.generate(tiny_model, x0, P, pj)
+    cj = O.trace_counters(tj)
+    assert not pj.pick_best and cj["tokens"] == L and cj["eff_nfe"] >= cj["nfe"]
+    pd, _ = O.mode_settings("decoded_share", Bk)
+    assert pd.n_copies == 8 and not pd.alp
+    # every committed token of a picked block is either a verified fill or in that block's own accept set: replay
+    for t in tv:
+        assert len(t["accepted"]) >= 1
+
+
 # ----------------------------------------------------------------------------- ALP
 
 def test_alp_scan_cases():
