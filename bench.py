@@ -203,7 +203,7 @@ def run_cuda(args, wl):
     shape = wl.shape
     T = wl.prompt_len + wl.gen_len
     gm = E.Model.from_synth(shape, seed=0, device=f"cuda:{local}", with_lm_head=wl.with_lm_head, max_batch=wl.batch,
-                            max_seq=T, max_block=wl.block_len, max_copies=4 if args.modes else max(wl.n_copies, 1))
+                            max_seq=T, max_block=wl.block_len, max_copies=8 if args.modes else max(wl.n_copies, 1))
     sess = E.Session(gm)
     params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies, accept_threshold=wl.accept_threshold,
                             truncate_threshold=wl.truncate_threshold)
@@ -375,10 +375,18 @@ def run_cuda(args, wl):
             "roofline": roofline}
     if args.modes and world == 1 and wl.batch == 1:
         # the three systems of the paper's tables on this workload's shapes, whole response each:
-        # cache-less baseline, DualCache block decoding, and the full method (speed relative to the first two)
+        # cache-less baseline, DualCache block decoding, and the full method (speed relative to the first two);
+        # then the speculation variants of the ablation (Section 5.3, Fig. 11), each on DualCache block decoding
+        # without length prediction: one picked block, the jump chain over four copies, eight copies with
+        # decoded-share (NFE and Eff_NFE relative to plain block decoding are the figure's other axis)
         modes = {}
-        for mode in ("vanilla", "fast_dllm", "odb"):
+        for mode in ("vanilla", "fast_dllm", "odb", "spec_vanilla", "accept_jump", "decoded_share"):
             mp, cache_blocks = E.mode_settings(mode, wl.block_len, n_copies=4, accept_threshold=wl.accept_threshold)
+            if cache_blocks and not args.host_loop:
+                # untimed first run: the device-resident loop records one graph per step shape on first use
+                reset()
+                E.generate(sess, mp, cache_blocks=cache_blocks, resident=True)
+                sess.set_active(0, True)
             reset()
             torch.cuda.synchronize()
             m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -393,6 +401,8 @@ def run_cuda(args, wl):
         for mode in modes:
             modes[mode]["speed_vs_vanilla"] = modes[mode]["tokens_per_s"] / modes["vanilla"]["tokens_per_s"]
             modes[mode]["speed_vs_fast_dllm"] = modes[mode]["tokens_per_s"] / modes["fast_dllm"]["tokens_per_s"]
+            modes[mode]["nfe_vs_fast_dllm"] = modes[mode]["nfe"] / modes["fast_dllm"]["nfe"]
+            modes[mode]["eff_nfe_vs_fast_dllm"] = modes[mode]["eff_nfe"] / modes["fast_dllm"]["eff_nfe"]
         line["modes"] = modes
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:

@@ -115,6 +115,10 @@ typedef struct odb_decode_params {
     int32_t stage2_min_decoded; /* decoded tokens in the block from which the 8-copy layout is used;
                                    -1 = ceil(4*block/7), where it fits the row budget of 4 full copies */
     int32_t alp;                /* 1: scan for [EOS] after a refresh and truncate */
+    int32_t pick_best;          /* 0: accept-jump walk (Section 4.2.1).  1: the speculation the paper compares
+                                   against (Fig. 7(a), Section 5.3): candidates are verified in the main block only,
+                                   the copy filling the largest set of verified candidates is adopted and its fills
+                                   and own accept set are the step's result (chain = that one copy) */
 } odb_decode_params;
 
 /* Per-sequence result of odb_unmask_accept (host memory, valid on return). */

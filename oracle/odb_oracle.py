@@ -36,7 +36,8 @@ single-accept regime of jump-share (tokens with 4 copies == tokens with 1 copy),
 cases and the truncated-refresh equivalence, batch == independent runs.
 PARITY UNPINNED (the paper prints no trace that could confirm them): the committed state
 after a multi-link jump (chain union), the stage-2 walk over eight copies, the stage switch
-point, and "truncate keeps the [EOS] slot, effective immediately".
+point, "truncate keeps the [EOS] slot, effective immediately", and the compared speculation
+variant of Section 5.3 (pick_best_walk: the paper gives its properties, not its rule).
 """
 from __future__ import annotations
 

@@ -43,7 +43,8 @@ class odb_weights(C.Structure):
 
 class odb_decode_params(C.Structure):
     _fields_ = [("block_len", C.c_int32), ("n_copies", C.c_int32), ("accept_threshold", C.c_float),
-                ("truncate_threshold", C.c_float), ("stage2_min_decoded", C.c_int32), ("alp", C.c_int32)]
+                ("truncate_threshold", C.c_float), ("stage2_min_decoded", C.c_int32), ("alp", C.c_int32),
+                ("pick_best", C.c_int32)]
 
 
 class odb_result(C.Structure):

@@ -329,7 +329,45 @@ __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p,
     // whose extra candidates are all hit; the accepted sets along the chain are committed,
     // an earlier link winning at a shared position
     int cur = 0, chain_len = 0, n_acc = 0;
-    while (true) {
+    const bool pick = p.pick_best && !after_refresh;
+    if (pick) {
+        // the compared speculation (Fig. 7(a), Section 5.3): candidates verified in the main block only; the copy
+        // filling the largest set of hits is adopted, and its fills and own accept set are the whole result
+        accept_set(conf[0], masked0, B, p.accept_threshold, acc);
+        int hit = 0;
+        for (int r = 0; r < st->n_ranks; ++r) {
+            const int o = st->rank_off[r];
+            if (acc[o] && tok[0][o] == st->rank_tok[r]) hit |= 1 << r;
+        }
+        for (int cp = 1; cp < n_copies; ++cp) {
+            const int Y = st->copy_mask[cp];
+            if (Y & ~hit) continue;
+            if (cur == 0 || __popc(Y) > __popc(st->copy_mask[cur]) ||
+                (__popc(Y) == __popc(st->copy_mask[cur]) && Y < st->copy_mask[cur]))
+                cur = cp;
+        }
+        auto commit = [&](int i, int t) {
+            taken[i] = true;
+            x[s + i] = t;
+            if (n_acc < 64) { res->accepted_pos[n_acc] = s + i; res->accepted_tok[n_acc] = t; }
+            ++n_acc;
+        };
+        if (cur != 0) {
+            const int Y = st->copy_mask[cur];
+            bool any = false;
+            for (int i = 0; i < B; ++i) masked[i] = masked0[i];
+            for (int r = 0; r < st->n_ranks; ++r)
+                if ((Y >> r) & 1) { masked[st->rank_off[r]] = false; commit(st->rank_off[r], st->rank_tok[r]); }
+            for (int i = 0; i < B; ++i) any |= masked[i];
+            if (any) accept_set(conf[cur], masked, B, p.accept_threshold, acc);
+            else for (int i = 0; i < B; ++i) acc[i] = false;
+        }
+        for (int i = 0; i < B; ++i)
+            if (acc[i] && !taken[i]) commit(i, tok[cur][i]);
+        res->chain[0] = cur;
+        chain_len = 1;
+    }
+    while (!pick) {
         res->chain[chain_len < ODB_MAX_CHAIN ? chain_len : ODB_MAX_CHAIN - 1] = cur;
         ++chain_len;
         const int X = after_refresh ? 0 : st->copy_mask[cur];

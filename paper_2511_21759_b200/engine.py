@@ -55,10 +55,11 @@ class DecodeParams:
     truncate_threshold: float = 0.9
     stage2_min_decoded: int = -1
     alp: bool = True
+    pick_best: bool = False
 
     def c(self) -> B.odb_decode_params:
         return B.odb_decode_params(self.block_len, self.n_copies, self.accept_threshold, self.truncate_threshold,
-                                   self.stage2_min_decoded, 1 if self.alp else 0)
+                                   self.stage2_min_decoded, 1 if self.alp else 0, 1 if self.pick_best else 0)
 
 
 class Model:
@@ -319,7 +320,12 @@ def generate(sess: Session, params: DecodeParams, *,
 def mode_settings(mode: str, block_len: int, n_copies: int = 4, accept_threshold: float = 0.9):
     """(DecodeParams, cache_blocks) of the three systems of Tables 2 and 3: "vanilla" (no cache, one
     token per full forward), "fast_dllm" (DualCache block decoding, threshold acceptance, fixed
-    length) and "odb" (adaptive length prediction + jump-share speculation)."""
+    length) and "odb" (adaptive length prediction + jump-share speculation); and of the speculation
+    variants of Section 5.3 (Fig. 11), each on block decoding without length prediction: "spec_vanilla"
+    (one of four blocks is picked), "accept_jump" (four copies, jump chain), "decoded_share" (eight copies)."""
+    if mode in ("spec_vanilla", "accept_jump", "decoded_share"):
+        return DecodeParams(block_len=block_len, n_copies=8 if mode == "decoded_share" else 4,
+                            accept_threshold=accept_threshold, alp=False, pick_best=mode == "spec_vanilla"), True
     if mode == "vanilla":
         return DecodeParams(block_len=block_len, n_copies=1, accept_threshold=1.0, alp=False), False
     if mode == "fast_dllm":

@@ -171,10 +171,11 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
             g_c[r_copy, r_pos - s] = g_cr
             g_t[r_copy, r_pos - s] = g_tr
             res = sess.unmask_accept(gp, False)[seq]
-            new, chain, last = O.jump_walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
+            walk = O.pick_best_walk if op.pick_best else O.jump_walk
+            new, chain, last = walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
             want = sorted((int(s + i), int(t)) for i, t in new.items())
             assert res_tuple(res) == (want, [int(c) for c in chain]), (res_tuple(res), want, chain)
-            new_o, chain_o, last_o = O.jump_walk(o_c, o_t, masked, subsets, ranks, rank_tok, tau)
+            new_o, chain_o, last_o = walk(o_c, o_t, masked, subsets, ranks, rank_tok, tau)
             if new_o != new or chain_o != chain:
                 margin = min(O.decision_margin(o_c[c], masked & (o_c[c] >= 0), tau, 0) for c in chain_o)
                 st["oracle_decision_diff"] += 1

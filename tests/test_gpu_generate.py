@@ -170,11 +170,12 @@ def test_lockstep_generate(wl_name, tol, fused):
 
 
 @requires_gpu
-@pytest.mark.parametrize("mode", ["vanilla", "fast_dllm", "odb"])
+@pytest.mark.parametrize("mode", ["vanilla", "fast_dllm", "odb", "spec_vanilla", "accept_jump", "decoded_share"])
 def test_baseline_modes_in_lockstep(mode):
     """The three systems the paper's tables compare, as settings of the same calls: the cache-less
     baseline (every iteration a refresh prefill, one token each), DualCache block decoding without
-    speculation or length prediction, and the full method."""
+    speculation or length prediction, and the full method; and the three speculation variants of the
+    ablation (Section 5.3): one picked block, the jump chain over four copies, eight copies."""
     E = engine()
     shape = synth.TINY_PEAKY
     P, L, Bk = 40, 24, 8
@@ -195,6 +196,31 @@ def test_baseline_modes_in_lockstep(mode):
     else:
         assert st["refreshes"] == L // Bk and st["iters"] <= L
     sess.close(); gm.close()
+
+
+@requires_gpu
+def test_pick_best_speculation_counters_and_resident_loop():
+    """The compared speculation: every step's chain is the one adopted copy, so Eff_NFE equals NFE
+    (Section 5.3); the device-resident loop gives the same trace as the call-by-call path."""
+    E = engine()
+    wl = synth.WORKLOADS["peaky_c4"]
+    gm = E.Model.from_synth(wl.shape, seed=0, max_batch=1, max_seq=wl.prompt_len + wl.gen_len, max_block=wl.block_len,
+                            max_copies=4)
+    gp, cache_blocks = E.mode_settings("spec_vanilla", wl.block_len)
+    traces = []
+    for resident in (False, True):
+        sess = E.Session(gm)
+        sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, wl.shape), wl.prompt_len)
+        toks, tr = E.generate(sess, gp, cache_blocks=cache_blocks, resident=resident)
+        assert sess.status() == 0 and (toks[0][wl.prompt_len:] != wl.shape.mask_id).all()
+        traces.append(tr)
+        sess.close()
+    gm.close()
+    assert traces[0] == traces[1]
+    c = E.trace_counters(traces[0])
+    assert c["tokens"] == wl.gen_len and c["eff_nfe"] == c["nfe"]
+    assert all(len(t["seqs"][0]["chain"]) == 1 for t in traces[0])
+    assert any(t["seqs"][0]["chain"] != [0] for t in traces[0]), "no speculative block was ever adopted"
 
 
 @requires_gpu
