@@ -177,6 +177,13 @@ __device__ __forceinline__ uint32_t tile_off(int rows, int row, int chunk) {
     return static_cast<uint32_t>((chunk >> 3) * rows * 128 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
 }
 
+// 2^x for x <= 0 on the special-function unit (flushes to zero far below zero, which is the wanted value)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 // One key tile of a work item: 64 consecutive rows of a [rows][128]-column view starting at row0, of which
 // the first `valid` are keys.  src: 0 = fresh k / v rows of this forward, 1 = the K/V cache.
 struct KeyTile {
@@ -458,14 +465,27 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             ok = wait(&sh->s_full[b], ph_sf[b]);
             if (!ok) break;
             tc_fence_after();
+            // a whole tile of cached keys (or of a refresh) is seen by every row: no per-key test (the softmax
+            // warps are bound by the instructions they issue per key)
+            const bool full = kt.copy < 0 && kt.valid >= 64;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
-                const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
+                if (full) {
+                    float m0 = m_row, m1 = -INFINITY;
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if ((m32 >> j) & 1u) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+                    for (int j = 0; j < 32; j += 4) {
+                        m0 = fmaxf(m0, fmaxf(__uint_as_float(v[j]), __uint_as_float(v[j + 1])));
+                        m1 = fmaxf(m1, fmaxf(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])));
+                    }
+                    m_row = fmaxf(m0, m1);
+                } else {
+                    const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if ((m32 >> j) & 1u) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+                }
             }
             tc_fence_before();
             __syncwarp();
@@ -483,23 +503,34 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             if (!ok) break;
             tc_fence_after();
             uint32_t hi[32], lo[32];                                 // row `tid` of P: 64 keys as bf16 pairs
+            const bool full = kt.copy < 0 && kt.valid >= 64;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
-                const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
+                const unsigned m32 = full ? 0xffffffffu : static_cast<unsigned>(mask >> (half * 32));
+                float l0 = 0.f, l1 = 0.f;
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
                     const int j = 2 * u;
-                    const float p0 = ((m32 >> j) & 1u) ? exp2f(__uint_as_float(v[j]) * scale_log2 - m_log2) : 0.f;
-                    const float p1 = ((m32 >> (j + 1)) & 1u) ? exp2f(__uint_as_float(v[j + 1]) * scale_log2 - m_log2) : 0.f;
-                    l_row += p0 + p1;
+                    // arguments are <= 0: the hardware exponential needs no range handling (far below zero it returns 0)
+                    float p0 = ex2_approx(fmaf(__uint_as_float(v[j]), scale_log2, -m_log2));
+                    float p1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), scale_log2, -m_log2));
+                    if (!full) {
+                        p0 = ((m32 >> j) & 1u) ? p0 : 0.f;
+                        p1 = ((m32 >> (j + 1)) & 1u) ? p1 : 0.f;
+                    }
+                    l0 += p0;
+                    l1 += p1;
                     const __nv_bfloat162 h = __floats2bfloat162_rn(p0, p1);
-                    const float2 hf = __bfloat1622float2(h);
-                    const __nv_bfloat162 l = __floats2bfloat162_rn(p0 - hf.x, p1 - hf.y);
-                    hi[half * 16 + u] = *reinterpret_cast<const uint32_t*>(&h);
+                    const uint32_t hb = *reinterpret_cast<const uint32_t*>(&h);
+                    // the bf16 halves widened back to fp32 are the bit patterns themselves, shifted into place
+                    const __nv_bfloat162 l = __floats2bfloat162_rn(p0 - __uint_as_float(hb << 16),
+                                                                   p1 - __uint_as_float(hb & 0xffff0000u));
+                    hi[half * 16 + u] = hb;
                     lo[half * 16 + u] = *reinterpret_cast<const uint32_t*>(&l);
                 }
+                l_row += l0 + l1;
             }
             tc_fence_before();
             __syncwarp();
