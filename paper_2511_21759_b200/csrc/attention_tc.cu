@@ -171,12 +171,6 @@ __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-// swizzled position of the 16-byte chunk `chunk` (0..15 across the 128-wide row) of row `row` in a tile of
-// `rows` rows: two atoms (columns 0..63, 64..127), each rows x 128 bytes, chunk index XOR (row mod 8)
-__device__ __forceinline__ uint32_t tile_off(int rows, int row, int chunk) {
-    return static_cast<uint32_t>((chunk >> 3) * rows * 128 + row * 128 + (((chunk & 7) ^ (row & 7)) << 4));
-}
-
 // 2^x for x <= 0 on the special-function unit (flushes to zero far below zero, which is the wanted value)
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;

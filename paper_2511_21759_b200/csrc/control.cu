@@ -106,7 +106,7 @@ __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id)
     }
     __shared__ int xs[kMaxBlock];      // the block's committed tokens
     __shared__ int mpre[kMaxBlock];    // masked positions before position i of the block
-    __shared__ int row_base, tile_base, n_masked_blk;
+    __shared__ int row_base, tile_base;
     const int32_t* x = c.x + static_cast<size_t>(seq) * c.max_seq;
     const int s = st->s, e = st->e, B = e - s;
     for (int i = threadIdx.x; i < B; i += blockDim.x) xs[i] = x[s + i];
@@ -125,7 +125,7 @@ __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id)
             mpre[i] = nm;
             nm += xs[i] == mask_id;
         }
-        row_base = row; tile_base = tile; n_masked_blk = nm;
+        row_base = row; tile_base = tile;
         st->row0 = row;
         // copy 0 holds the whole block; a speculative copy the whole block or, in the decoded-share layout, the
         // positions still masked
@@ -179,7 +179,7 @@ __global__ void build_step_rows_kernel(ControlBuffers c, int batch, int mask_id)
         if (!o->active || o->n_masked <= 0) continue;
         stile += step_tiles_of(o);
     }
-    StepTile cur;
+    StepTile cur{};
     int have = 0;
     auto add_src = [&](int cp) {
         for (int i = 0; i < cur.n_src; ++i)

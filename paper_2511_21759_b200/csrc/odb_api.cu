@@ -649,14 +649,6 @@ int step_items(const odb_session* s, const StepShape& sh) {
     return (!sh.multi || static_cast<size_t>(2) * sh.rows > s->L.attn_rows) ? 0 : sh.step_tiles;
 }
 
-int32_t pull_state(odb_session* s) {
-    const int nb = s->m->cfg.max_batch;
-    ODB_CUDA(cudaMemcpyAsync(s->pinned_state, s->cb.state, sizeof(SeqState) * nb, cudaMemcpyDeviceToHost, s->st));
-    ODB_CUDA(cudaStreamSynchronize(s->st));
-    for (int i = 0; i < nb; ++i) s->mirror[i] = s->pinned_state[i];
-    return ODB_OK;
-}
-
 }  // namespace
 
 extern "C" {
