@@ -13,6 +13,15 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
+__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
+    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b);
+    const __nv_bfloat162 hi = __floats2bfloat162_rn(c, d);
+    uint2 pk;
+    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
+    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
+    return pk;
+}
+
 // block-wide sum, same value returned to every thread; `red` has >= 32 floats
 __device__ __forceinline__ float block_sum(float v, float* red) {
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
@@ -81,6 +90,71 @@ __global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_kernel(float* __re
     if (threadIdx.x == 0) ssq[static_cast<size_t>(orow) * gridDim.y + blockIdx.y] = total;
 }
 
+// The same for many rows (a refresh): kNormRows rows per block, every load of the thread's rows and splits in
+// flight at once, so that the kernel runs nearer memory speed instead of at one short round trip per block
+// (768 rows x 4096, three splits: 21 -> 14.5 us per launch).  Same sums in the same order per row.
+constexpr int kNormRows = 4;
+constexpr int kNormRowsMaxSplits = 4;
+__global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_rows_kernel(float* __restrict__ h, const float* __restrict__ partial,
+                                                                          int splits, size_t pstride,
+                                                                          const float* __restrict__ gain,
+                                                                          __nv_bfloat16* __restrict__ out, float* __restrict__ ssq,
+                                                                          const int32_t* __restrict__ row_map, int rows_out, int d) {
+    __shared__ float red[kNormRows][32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.y * (kNormSliceCols / 4) + threadIdx.x;   // float4 index within the row
+    const int orow0 = blockIdx.x * kNormRows;
+    const bool in = i < (d >> 2);
+    float4 v[kNormRows], t[kNormRows][kNormRowsMaxSplits];
+    int row[kNormRows];
+#pragma unroll
+    for (int r = 0; r < kNormRows; ++r) {
+        const int orow = orow0 + r;
+        row[r] = orow < rows_out ? (row_map ? row_map[orow] : orow) : -1;
+    }
+#pragma unroll
+    for (int r = 0; r < kNormRows; ++r) {
+        if (!in || row[r] < 0) continue;
+        v[r] = reinterpret_cast<const float4*>(h + static_cast<size_t>(row[r]) * d)[i];
+        if (partial) {
+            const float* p = partial + static_cast<size_t>(row[r]) * d + 4 * i;
+#pragma unroll
+            for (int u = 0; u < kNormRowsMaxSplits; ++u)
+                if (u < splits) t[r][u] = *reinterpret_cast<const float4*>(p + static_cast<size_t>(u) * pstride);
+        }
+    }
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (in) g = reinterpret_cast<const float4*>(gain)[i];
+    float ss[kNormRows];
+#pragma unroll
+    for (int r = 0; r < kNormRows; ++r) {
+        ss[r] = 0.f;
+        if (!in || row[r] < 0) continue;
+        float4 x = v[r];
+        if (partial) {
+#pragma unroll
+            for (int u = 0; u < kNormRowsMaxSplits; ++u)
+                if (u < splits) { x.x += t[r][u].x; x.y += t[r][u].y; x.z += t[r][u].z; x.w += t[r][u].w; }
+            reinterpret_cast<float4*>(h + static_cast<size_t>(row[r]) * d)[i] = x;
+        }
+        ss[r] = x.x * x.x + x.y * x.y + x.z * x.z + x.w * x.w;
+        reinterpret_cast<uint2*>(out + static_cast<size_t>(orow0 + r) * d)[i] = pack4_bf16(x.x * g.x, x.y * g.y, x.z * g.z, x.w * g.w);
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nw = blockDim.x >> 5;
+#pragma unroll
+    for (int r = 0; r < kNormRows; ++r) {
+        const float w = warp_sum(ss[r]);
+        if (lane == 0) red[r][warp] = w;
+    }
+    __syncthreads();
+    if (threadIdx.x < kNormRows && orow0 + threadIdx.x < rows_out) {
+        float total = 0.f;
+        for (int w = 0; w < nw; ++w) total += red[threadIdx.x][w];
+        ssq[static_cast<size_t>(orow0 + threadIdx.x) * gridDim.y + blockIdx.y] = total;
+    }
+}
+
 // More than 64 rows: grid (rows, chunks), one thread per FOUR consecutive rotation pairs (float4 loads, 8-byte
 // stores; 1.5 x the throughput of the one-pair kernel below, which stays the faster one on the few rows of a
 // decode step, where the kernel is a single memory round trip on the dependency chain).  Sums the
@@ -88,14 +162,6 @@ __global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_kernel(float* __re
 // pairs with i + hd/2; angle = pos * theta^(-2i/hd), table precomputed), rounds to bf16 and writes the
 // row-major fresh q/k/v; in a refresh also the K/V cache [seq][layer][k|v][head][pos][hd].  hd/2 is a
 // multiple of 4, so the four pairs of a thread lie in one head.
-__device__ __forceinline__ uint2 pack4_bf16(float a, float b, float c, float d) {
-    const __nv_bfloat162 lo = __floats2bfloat162_rn(a, b);
-    const __nv_bfloat162 hi = __floats2bfloat162_rn(c, d);
-    uint2 pk;
-    pk.x = *reinterpret_cast<const uint32_t*>(&lo);
-    pk.y = *reinterpret_cast<const uint32_t*>(&hi);
-    return pk;
-}
 
 __device__ __forceinline__ void add4(float4& a, const float4& b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
 __device__ __forceinline__ void scale4(float4& a, float s) { a.x *= s; a.y *= s; a.z *= s; a.w *= s; }
@@ -315,6 +381,9 @@ cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t ps
                            cudaStream_t st) {
     if (splits > 16) return cudaErrorInvalidValue;
     const int slices = (d + kNormSliceCols - 1) / kNormSliceCols;
+    if (rows_out >= 256 && splits <= kNormRowsMaxSplits)
+        return launch_kernel(rmsnorm_rows_kernel, dim3((rows_out + kNormRows - 1) / kNormRows, slices), dim3(kNormSliceCols / 4), 0,
+                             st, h, partial, splits, pstride, gain, out, ssq, row_map, rows_out, d);
     return launch_kernel(rmsnorm_kernel, dim3(rows_out, slices), dim3(kNormSliceCols / 4), 0, st, h, partial, splits, pstride,
                          gain, out, ssq, row_map, d, pf);
 }
