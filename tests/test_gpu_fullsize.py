@@ -50,6 +50,12 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     s_conf, s_tok = sess.debug_read("conf"), sess.debug_read("tok")
     res2 = sess.unmask_accept(gp, False)[0]
     s_acc = sorted((res2.accepted_pos[j], res2.accepted_tok[j]) for j in range(res2.n_accepted))
+    # the launch configuration the benchmark times: the next two iterations inside the device-resident loop, LM head
+    # fused with the confidence reduction (no logits); the last iteration's confidences stay on the device
+    sess.set_logit_dump(False)
+    loop = [(sorted((it[0].accepted_pos[j], it[0].accepted_tok[j]) for j in range(it[0].n_accepted)), it[0].masks_left)
+            for it in sess.decode_block_resident(gp, 2)]
+    l_conf, l_tok = sess.debug_read("conf"), sess.debug_read("tok")
     assert sess.status() == 0
     sess.close(); gm.close()
     del gm
@@ -98,6 +104,20 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     if not np.array_equal(acc, acc_o):
         margin = O.decision_margin(o_c[0], masked, wl.accept_threshold, 0)
         assert margin <= max(1e-3, 4 * cerr_s), (margin, cerr_s)
+    # the loop's second iteration against the oracle, from the state the loop itself reached before it
+    assert len(loop) == 2 and len(l_conf) == Bk
+    for p_, t_ in s_acc + loop[0][0]:
+        x[p_] = t_
+    masked = x[P:P + Bk] == shape.mask_id
+    assert int(masked.sum()) == loop[0][1]
+    o_c2, o_t2 = O.block_decode_step(om, cache, x, T, P, P + Bk, [()], [], [], False, dtype=np.float32)
+    acc = O.accept_set(l_conf, masked, wl.accept_threshold)
+    assert loop[1][0] == [(int(P + i), int(l_tok[i])) for i in np.flatnonzero(acc)], "accept rule inside the resident loop"
+    assert loop[1][1] == int(masked.sum()) - int(acc.sum())
+    cerr_l = float((np.abs(l_conf - o_c2[0]) / o_c2[0]).max())
+    assert cerr_l <= 0.2, cerr_l
+    assert (l_tok != o_t2[0]).mean() <= 0.25
+    print(f"resident loop, iteration 2: conf rel err {cerr_l:.2e}, greedy tokens differing {int((l_tok != o_t2[0]).sum())} of {Bk}")
     print(f"\ncfg3 full size: per-row rel. L2 error {l2_r:.2e} (refresh) {l2_s:.2e} (step); "
           f"element-wise {worst_r:.2f} x / {worst_s:.2f} x the small-model bound; "
           f"conf rel err {cerr:.2e} / {cerr_s:.2e}, greedy tokens differing: "
