@@ -431,11 +431,14 @@ def run_layer_microbench(args, wl):
     peaks = load_peaks()
     shape, T = wl.shape, wl.prompt_len + wl.gen_len
     import synth
-    gm = E.Model.from_synth(shape, seed=0, with_lm_head=False, max_batch=1, max_seq=T, max_block=wl.block_len,
+    gm = E.Model.from_synth(shape, seed=0, with_lm_head=False, max_batch=wl.batch, max_seq=T, max_block=wl.block_len,
                             max_copies=max(wl.n_copies, 1))
     sess = E.Session(gm)
     params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies)
-    sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape), wl.prompt_len)
+    # a batch is ragged the way the full benchmark's is: seeded response lengths between a quarter and a half of the allocation
+    lens = [wl.gen_len] if wl.batch == 1 else [int(n) for n in synth.shrink_schedule(0, wl.batch, wl.gen_len)]
+    for i in range(wl.batch):
+        sess.set_sequence(i, synth.sequence(0, i, wl.prompt_len, lens[i], shape), wl.prompt_len)
     sess.refresh_prefill(params, 0)
     sess.unmask_accept(params, True)
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")

@@ -184,6 +184,9 @@ WORKLOADS = {
                               with_lm_head=False),
     "cfg2_layer_c4": Workload("cfg2_layer_c4", LLADA_8B.with_layers(1), 1, 256, 256, 32, 4,
                               with_lm_head=False),
+    # one 8B-shaped layer, 16 ragged sequences, block 64, 4 copies: the batched step's kernels on a small footprint
+    "cfg2_layer_b16_c4": Workload("cfg2_layer_b16_c4", LLADA_8B.with_layers(1), 16, 1024, 1024, 64, 4,
+                                  with_lm_head=False),
     # full 8B shape
     "cfg3_8b_c1": Workload("cfg3_8b_c1", LLADA_8B, 1, 512, 256, 32, 1),
     "cfg4_8b_c4": Workload("cfg4_8b_c4", LLADA_8B, 1, 512, 512, 32, 4),
