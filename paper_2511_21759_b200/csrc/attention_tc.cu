@@ -59,6 +59,13 @@ __device__ __forceinline__ void tma_box(uint32_t dst, const CUtensorMap* tmap, u
         : "memory");
 }
 
+// asks L2 for the same box (no shared-memory destination, nothing to wait for)
+__device__ __forceinline__ void tma_prefetch_box(const CUtensorMap* tmap, int col0, int row0) {
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(reinterpret_cast<uint64_t>(tmap)),
+                 "r"(col0), "r"(row0)
+                 : "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
@@ -317,6 +324,21 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                 tma_box(dst, kt.src ? &tm_c : &tm_v, &sh->v_full, kt.src ? 0 : col0, kt.v_row0);
                 tma_box(dst + kTK * 128, kt.src ? &tm_c : &tm_v, &sh->v_full, kt.src ? 64 : col0 + 64, kt.v_row0);
             };
+            // Two K buffers and one V buffer cover little of a load's latency from HBM: every load also asks L2 for
+            // the tile kAhead tiles further on, so that the load that later fills a buffer comes from L2.
+            constexpr int kAhead = 3;
+            auto hint_k = [&](int tile) {
+                if (tile >= ntiles) return;
+                const KeyTile kt = key_tile(tile);
+                tma_prefetch_box(kt.src ? &tm_c : &tm_k, kt.src ? 0 : col0, kt.row0);
+                tma_prefetch_box(kt.src ? &tm_c : &tm_k, kt.src ? 64 : col0 + 64, kt.row0);
+            };
+            auto hint_v = [&](int tile) {
+                if (tile >= ntiles) return;
+                const KeyTile kt = key_tile(tile);
+                tma_prefetch_box(kt.src ? &tm_c : &tm_v, kt.src ? 0 : col0, kt.v_row0);
+                tma_prefetch_box(kt.src ? &tm_c : &tm_v, kt.src ? 64 : col0 + 64, kt.v_row0);
+            };
             uint32_t ph_ke[2] = {0, 0}, ph_ve = 0;
             bool ok = true;
             // Q: rows 0..63 and 64..127 of each atom
@@ -328,10 +350,14 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             // ---- pass 1 ----
             load_k(0);
             load_k(1);
+            for (int t = 2; t < 2 + kAhead; ++t) hint_k(t);
             for (int tile = 0; tile + 2 < ntiles && ok; ++tile) {
                 const int b = tile & 1;
                 ok = wait(&sh->k_empty[b], ph_ke[b]);            // S(tile) has read this buffer
-                if (ok) load_k(tile + 2);
+                if (ok) {
+                    load_k(tile + 2);
+                    hint_k(tile + 2 + kAhead);
+                }
             }
             // the last two S of pass 1 must have read their buffers before pass 2 refills them
             for (int tile = ntiles > 2 ? ntiles - 2 : 0; tile < ntiles && ok; ++tile) ok = wait(&sh->k_empty[tile & 1], ph_ke[tile & 1]);
@@ -340,18 +366,24 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                 load_k(0);
                 load_v(0);
                 load_k(1);
+                for (int t = 1; t < 1 + kAhead; ++t) hint_v(t);
+                for (int t = 2; t < 2 + kAhead; ++t) hint_k(t);
             }
+            // S(tile) completes long before P V(tile) (the softmax of the tile lies between them), and S(tile + 2) is
+            // issued right behind P V(tile): the K buffer is refilled first, so that its load runs during that softmax
             for (int tile = 0; tile < ntiles && ok; ++tile) {
                 const int b = tile & 1;
-                if (tile + 1 < ntiles) {
-                    ok = wait(&sh->v_empty, ph_ve);             // P V(tile) has read the V tile
-                    if (!ok) break;
-                    load_v(tile + 1);
-                }
                 if (tile + 2 < ntiles) {
                     ok = wait(&sh->k_empty[b], ph_ke[b]);        // S(tile) has read this buffer
                     if (!ok) break;
                     load_k(tile + 2);
+                    hint_k(tile + 2 + kAhead);
+                }
+                if (tile + 1 < ntiles) {
+                    ok = wait(&sh->v_empty, ph_ve);             // P V(tile) has read the V tile
+                    if (!ok) break;
+                    load_v(tile + 1);
+                    hint_v(tile + 1 + kAhead);
                 }
             }
         }
