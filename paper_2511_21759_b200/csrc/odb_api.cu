@@ -786,6 +786,13 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
             cudaGraphDestroy(r.graph);
             return rc != ODB_OK ? rc : cuda_fail(e);
         }
+        // a ragged batch walks through many step shapes: keep the most recently recorded graphs only
+        constexpr size_t kMaxResidentGraphs = 64;
+        if (s->resident.size() >= kMaxResidentGraphs) {
+            cudaGraphExecDestroy(s->resident.front().exec);
+            cudaGraphDestroy(s->resident.front().graph);
+            s->resident.erase(s->resident.begin());
+        }
         s->resident.push_back(r);
         g = &s->resident.back();
     }
