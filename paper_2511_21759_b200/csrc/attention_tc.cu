@@ -262,6 +262,8 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
     int cA = 0, cB0 = 0, cB1 = 0, nA_t = 0, t_first = 0;    // step, cached split: positions [0, cA) and [cB0, cB1)
     int c_row = 0;                                          // step: row of position 0 of this head's keys in the cache view
     bool fresh_split = false;
+    const bool single = STEP && ks == 1;                    // step without key splits
+    int n_cached = 0;                                       // step: cached key tiles of this CTA (they come first)
     const StepTile* stp = nullptr;
     if constexpr (!STEP) {
         const QTile t = a.qtiles[blockIdx.x];
@@ -271,13 +273,20 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         stp = a.stiles + blockIdx.x;
         q_row0 = stp->slab_row0[0];
         nq = stp->slab_row0[stp->n_slabs - 1] + stp->slab_n[stp->n_slabs - 1] - q_row0;   // the slabs are consecutive rows
-        fresh_split = z == ks - 1;
         cA = stp->cA; cB0 = stp->cB0; cB1 = stp->cB1;
         nA_t = (cA + kTK - 1) / kTK;
         const int nct = nA_t + (cB1 - cB0 + kTK - 1) / kTK;
-        const int tp = (nct + ks - 2) / (ks - 1);
-        t_first = fresh_split ? 0 : z * tp;
-        ntiles = fresh_split ? stp->n_src : max(0, min(nct, t_first + tp) - t_first);
+        if (single) {
+            // one CTA takes every key of the item: the cached tiles, then the fresh ones; its output is final
+            n_cached = nct;
+            ntiles = nct + stp->n_src;
+        } else {
+            fresh_split = z == ks - 1;
+            const int tp = (nct + ks - 2) / (ks - 1);
+            t_first = fresh_split ? 0 : z * tp;
+            n_cached = fresh_split ? 0 : max(0, min(nct, t_first + tp) - t_first);
+            ntiles = fresh_split ? stp->n_src : n_cached;
+        }
         c_row = ((stp->seq * a.n_layers + a.layer) * 2 * a.H + head) * a.max_seq;   // K; V is H * max_seq rows further
     }
     auto key_tile = [&](int i) {
@@ -285,8 +294,9 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
         kt.copy = -1;
         if constexpr (!STEP) {
             kt.src = 0; kt.row0 = f0 + i * kTK; kt.v_row0 = kt.row0; kt.valid = min(kTK, NK - i * kTK);
-        } else if (fresh_split) {
-            kt.src = 0; kt.row0 = stp->src_row0[i]; kt.v_row0 = kt.row0; kt.valid = stp->src_n[i]; kt.copy = stp->src_copy[i];
+        } else if (i >= n_cached) {
+            const int f = i - n_cached;
+            kt.src = 0; kt.row0 = stp->src_row0[f]; kt.v_row0 = kt.row0; kt.valid = stp->src_n[f]; kt.copy = stp->src_copy[f];
         } else {
             const int j = t_first + i;
             const int pos0 = j < nA_t ? j * kTK : cB0 + (j - nA_t) * kTK;
@@ -584,7 +594,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             tc_fence_after();
             const int d = a.H * kHD;
             const int row = q_row0 + tid;
-            if constexpr (!STEP) {
+            if (!STEP || single) {
                 const float inv = l_row > 0.f ? 1.0f / l_row : 0.f;
                 __nv_bfloat16* orow = a.o + static_cast<size_t>(row) * d + head * kHD;
 #pragma unroll 1
@@ -674,13 +684,15 @@ cudaError_t launch_attention_tc(const AttnArgs& a, int* status, cudaStream_t st)
 }
 
 // Decode-step attention over StepTiles on the tensor cores (head dim 128); cache_rows = rows of the K/V cache
-// viewed as [rows][128] (batch x layers x 2 x heads x max_seq).  Partials only: the caller merges them.
+// viewed as [rows][128] (batch x layers x 2 x heads x max_seq).  ksplit = 1: every work item is one CTA over all of its
+// keys and writes the final output; ksplit >= 2: partials only, the caller merges them.
 cudaError_t launch_step_attention_tc(const StepAttnArgs& a, size_t cache_rows, int* status, cudaStream_t st) {
     if (a.n_tiles == 0) return cudaSuccess;
-    if (a.hd != kHD || a.ksplit < 2 || a.ksplit > 8) return cudaErrorInvalidValue;
+    if (a.hd != kHD || a.ksplit < 1 || a.ksplit > 8) return cudaErrorInvalidValue;
     TcArgs ta{};
     ta.stiles = a.tiles;
     ta.row_flags = a.row_flags;
+    ta.o = a.o;                                            // written when there is no key split
     ta.part_o = a.part_o; ta.part_ml = a.part_ml;
     ta.layer = a.layer; ta.n_layers = a.n_layers; ta.H = a.H; ta.max_seq = a.max_seq; ta.M = a.M;
     return launch_tc<true>(dim3(a.n_tiles, a.H, a.ksplit), a.q, a.k, a.v, a.cache, cache_rows, ta, status, st);

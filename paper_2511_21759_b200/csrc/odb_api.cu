@@ -558,8 +558,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             static const int tc_step_min = getenv("ODB_ATTN_TC_STEP_MIN") ? atoi(getenv("ODB_ATTN_TC_STEP_MIN")) : 2 * 148;
             if (hd == 128 && tc_attention && n_step_tiles * H >= tc_step_min) {
                 const size_t cache_rows = static_cast<size_t>(c.max_batch) * c.n_layers * 2 * H * c.max_seq;
+                // with a work item for every CTA slot there is nothing to gain from key splits: one CTA per item takes
+                // the cached and the fresh keys and writes the final output (no partials, no merge kernel)
+                if (ks_env == 1 || (ks_env <= 0 && n_step_tiles * H >= 2 * 148)) sa.ksplit = 1;
                 ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention_tc(sa, cache_rows, status, st));
-                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_combine(sa.part_o, sa.part_ml, o, M, H, hd, sks, st));
+                if (sa.ksplit > 1)
+                    ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_combine(sa.part_o, sa.part_ml, o, M, H, hd, sa.ksplit, st));
             } else {
                 ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
                 ++s->launches[ODB_KIND_ATTENTION];

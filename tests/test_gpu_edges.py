@@ -68,11 +68,14 @@ def test_tensor_core_step_attention_on_small_batches():
     names = ["hd128_ragged", "hd128_c8_stage2", "hd128_b64_c8", "hd128_c4_noprompt"]
     code = ("import sys; sys.path.insert(0, 'tests'); import test_gpu_edges as t\n"
             f"for c in t.CASES:\n    if c[0] in {names!r}: t.test_edge_case_in_lockstep(*c)\n")
-    env = dict(os.environ, ODB_ATTN_TC_STEP_MIN="0")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
-    assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
-    assert r.stdout.count("iterations") == len(names), r.stdout[-2000:]
+    # with key splits (the small-batch configuration) and without (one CTA per work item over cached and fresh
+    # keys, final output: what batched steps with a work item for every CTA slot use)
+    for extra in ({}, {"ODB_ATTN_KS": "1"}):
+        env = dict(os.environ, ODB_ATTN_TC_STEP_MIN="0", **extra)
+        r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
+        assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
+        assert r.stdout.count("iterations") == len(names), r.stdout[-2000:]
 
 
 @requires_gpu
