@@ -333,4 +333,18 @@ def test_argument_validation_and_state_errors():
     res = sess.unmask_accept(p, True)
     assert res[0].gen_len == 20 and res[0].block_end == 48
     assert len(sess.get_tokens(0)) == 52
+    # the device-resident loop validates the same way, and refuses to run while launches are being timed
+    import ctypes as C
+    lib, log, n = B.lib(), (B.odb_result * 4)(), C.c_int32()
+    pc = p.c()
+    assert lib.odb_decode_block_resident(sess.handle, C.byref(pc), 0, log, 0, C.byref(n)) == B.ODB_ERR_ARG      # no room in the log
+    assert lib.odb_decode_block_resident(sess.handle, C.byref(pc), 0, None, 4, C.byref(n)) == B.ODB_ERR_ARG
+    bad = E.DecodeParams(block_len=16, n_copies=8).c()
+    assert lib.odb_decode_block_resident(sess.handle, C.byref(bad), 0, log, 4, C.byref(n)) == B.ODB_ERR_SHAPE
+    sess.profile(True)
+    assert lib.odb_decode_block_resident(sess.handle, C.byref(pc), 0, log, 4, C.byref(n)) == B.ODB_ERR_STATE
+    sess.profile(False)
+    assert lib.odb_decode_block_resident(sess.handle, C.byref(pc), 0, log, 4, C.byref(n)) == B.ODB_OK
+    assert 1 <= n.value <= 4 and log[n.value - 1].masks_left < res[0].masks_left      # log_cap bounds the iterations
+    assert sess.status() == 0
     sess.close(); gm.close()
