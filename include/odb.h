@@ -238,6 +238,14 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
  * confidences agree to fp32 rounding of a differently ordered sum. */
 int32_t odb_debug_set_logit_dump(odb_session* s, int32_t enable);
 
+/* Test of the timeout path without a fault.  Every device-side wait of the library (TMA / MMA barriers) is the same
+ * bounded wait; this call enqueues one small kernel whose single wait cannot be satisfied (an mbarrier nothing
+ * arrives at) with a limit of limit_cycles SM clock cycles (1 .. the library's own limit).  The wait runs out, the
+ * kernel records ODB_ERR_TIMEOUT in the session's status word and returns normally; the next odb_session_status
+ * (or odb_unmask_accept / odb_decode_block_resident) reports it and clears it, and the session stays usable.
+ * Asynchronous. */
+int32_t odb_debug_expire_wait(odb_session* s, int64_t limit_cycles);
+
 /* Copies a device buffer of the last forward to the host.  which: 0 logits fp32 [rows][vocab]
  * (needs the logit dump);
  * 1 conf fp32 [rows]; 2 tok int32 [rows]; 3 residual stream fp32 [rows][d_model]; 4 q, 5 k,

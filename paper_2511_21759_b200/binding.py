@@ -79,6 +79,7 @@ SIGNATURES = {
     "odb_decode_block_resident": (C.c_int32, [C.c_void_p, C.POINTER(odb_decode_params), C.c_int32, C.POINTER(odb_result),
                                               C.c_int32, C.POINTER(C.c_int32)]),
     "odb_debug_set_logit_dump": (C.c_int32, [C.c_void_p, C.c_int32]),
+    "odb_debug_expire_wait": (C.c_int32, [C.c_void_p, C.c_int64]),
     "odb_debug_read": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_size_t, C.POINTER(C.c_int32)]),
     "odb_debug_gemm": (C.c_int32, [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_int32, C.c_void_p]),

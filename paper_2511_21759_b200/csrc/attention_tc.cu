@@ -35,7 +35,6 @@ constexpr int kTQ = 128;   // query rows per work item (MMA M)
 constexpr int kTK = 64;    // keys per tile
 constexpr int kHD = 128;
 constexpr int kThreads = 192;   // 4 softmax warps, MMA warp, loader warp
-constexpr long long kWaitLimitCycles = 4000000000ll;
 
 constexpr uint32_t kQBytes = kTQ * kHD * 2;          // 32 KB: two atoms of 128 rows x 128 B
 constexpr uint32_t kKBytes = kTK * kHD * 2;          // 16 KB: two atoms of 64 rows x 128 B
@@ -70,31 +69,9 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
 }
 
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false if the CTA has been aborted or the limit expired.
+// Bounded wait (shared implementation): false if the CTA has been aborted or the limit expired.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* cta_abort, int* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*cta_abort) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *cta_abort = 1;
-            atomicExch(status, ODB_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
+    return mbar_wait_bounded(bar, parity, cta_abort, status);
 }
 
 // K-major operand, rows of 128 bytes, 128-byte swizzle, 8-row groups 1024 bytes apart

@@ -506,7 +506,24 @@ __global__ void accept_loop_kernel(ControlBuffers c, odb_decode_params p, int ma
     cudaGraphSetConditional(lc.handle, again ? 1u : 0u);
 }
 
+// A wait that runs out by design: the barrier is initialised for one arrival that never comes.
+__global__ void expire_wait_kernel(long long limit_cycles, int* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_word;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(static_cast<uint32_t>(__cvta_generic_to_shared(&bar))));
+        abort_word = 0;
+    }
+    __syncthreads();
+    mbar_wait_bounded(&bar, 0, &abort_word, status, limit_cycles);
+}
+
 }  // namespace
+
+cudaError_t launch_expire_wait(long long limit_cycles, int* status, cudaStream_t st) {
+    expire_wait_kernel<<<1, 32, 0, st>>>(limit_cycles, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_accept_loop(const ControlBuffers& c, int batch, const odb_decode_params& p, int mask_id, int eos_id,
                                int dry, const LoopControl& lc, cudaStream_t st) {

@@ -30,7 +30,6 @@ constexpr int kBM = 128;          // weight rows per tile (MMA M)
 constexpr int kBK = 64;           // K elements per stage = one 128-byte swizzle span of bf16
 constexpr int kUmmaK = 16;        // K per tcgen05.mma for 16-bit inputs
 constexpr int kThreads = 192;
-constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s at the boost clock
 
 constexpr uint64_t kEvictFirst = 0x12F0000000000000ull;   // L2 policy: streamed once (weights)
 constexpr uint64_t kEvictLast = 0x14F0000000000000ull;    // L2 policy: re-read by every CTA (activations)
@@ -48,31 +47,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
                  : "memory");
 }
 
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(smem_u32(bar)), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false if the CTA has been aborted or the limit expired.
+// Bounded wait (shared implementation): false if the CTA has been aborted or the limit expired.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* cta_abort, int* status) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const long long t0 = clock64();
-    while (!mbar_try_wait(bar, parity)) {
-        if (*cta_abort) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
-            *cta_abort = 1;
-            atomicExch(status, ODB_ERR_TIMEOUT);
-            return false;
-        }
-    }
-    return true;
+    return mbar_wait_bounded(bar, parity, cta_abort, status);
 }
 
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tmap, uint64_t* bar, int c0, int c1,
@@ -348,7 +325,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 const int first = issued > stages ? issued - stages : 0;
                 for (int i = first; i < issued; ++i) {
                     const long long t0 = clock64();
-                    while (!mbar_try_wait(&sh->full[i % stages], static_cast<uint32_t>(i / stages) & 1u) &&
+                    while (!mbar_try_wait_parity(&sh->full[i % stages], static_cast<uint32_t>(i / stages) & 1u) &&
                            clock64() - t0 < kWaitLimitCycles / 8) {
                     }
                 }

@@ -849,6 +849,12 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap, in
     return ODB_OK;
 }
 
+int32_t odb_debug_expire_wait(odb_session* s, int64_t limit_cycles) {
+    if (!s || limit_cycles < 1 || limit_cycles > kWaitLimitCycles) return ODB_ERR_ARG;
+    ODB_CUDA(launch_expire_wait(limit_cycles, s->at<int>(s->L.status), s->st));
+    return ODB_OK;
+}
+
 int32_t odb_debug_set_logit_dump(odb_session* s, int32_t enable) {
     if (!s) return ODB_ERR_ARG;
     s->dump_logits = enable != 0;

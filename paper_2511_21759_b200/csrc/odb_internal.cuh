@@ -338,4 +338,41 @@ struct LoopControl {
 cudaError_t launch_accept_loop(const ControlBuffers& c, int batch, const odb_decode_params& p, int mask_id, int eos_id,
                                int dry, const LoopControl& lc, cudaStream_t st);
 
+// ---------------------------------------------------------------------------------------
+// Bounded mbarrier wait shared by every kernel that waits on one (GEMM, tensor-core attention): no wait on
+// the device spins forever.  Returns false if the CTA has been aborted by another of its waits or the limit
+// expired; on expiry the CTA's abort word is set and ODB_ERR_TIMEOUT recorded in the session's status word,
+// the kernel then finishes normally (its roles stop, TMEM is released) and the host reads the status.
+// ---------------------------------------------------------------------------------------
+constexpr long long kWaitLimitCycles = 4000000000ll;   // ~2 s at the boost clock
+
+__device__ __forceinline__ bool mbar_try_wait_parity(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(static_cast<uint32_t>(__cvta_generic_to_shared(bar))), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* cta_abort, int* status,
+                                                  long long limit_cycles = kWaitLimitCycles) {
+    if (mbar_try_wait_parity(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait_parity(bar, parity)) {
+        if (*cta_abort) return false;
+        if (clock64() - t0 > limit_cycles) {
+            *cta_abort = 1;
+            atomicExch(status, ODB_ERR_TIMEOUT);
+            return false;
+        }
+    }
+    return true;
+}
+// Test entry: one CTA waits, with the given limit, on an mbarrier that nothing ever arrives at.
+cudaError_t launch_expire_wait(long long limit_cycles, int* status, cudaStream_t st);
+
 }  // namespace odb

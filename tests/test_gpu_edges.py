@@ -99,3 +99,43 @@ def test_fully_decoded_block_is_a_state_error_not_a_launch():
     sess.refresh_prefill(gp, 1)                                # the session is still usable
     assert sess.unmask_accept(gp, True)[0].n_accepted == 1
     sess.close(); gm.close()
+
+
+@requires_gpu
+def test_an_expired_device_wait_is_reported_and_the_session_stays_usable():
+    """Every device-side wait of the library is the same bounded wait.  Here one runs out by design (a barrier
+    nothing arrives at, limit about a millisecond): the kernel returns normally, the status word carries the
+    timeout to the host (through odb_session_status, or through the next accept), is cleared by the read, and
+    the session goes on working.  Nothing faults or hangs."""
+    import ctypes as C
+    E = engine()
+    from paper_2511_21759_b200 import binding as B
+    shape = synth.TINY
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=48, max_block=16, max_copies=1)
+    sess = E.Session(gm)
+    sess.set_sequence(0, synth.sequence(0, 0, 16, 32, shape), 16)
+    gp = E.DecodeParams(block_len=16, n_copies=1)
+    lib = B.lib()
+    assert lib.odb_debug_expire_wait(sess.handle, C.c_int64(0)) == B.ODB_ERR_ARG
+    assert lib.odb_debug_expire_wait(sess.handle, C.c_int64(2_000_000)) == B.ODB_OK
+    assert sess.status() == B.ODB_ERR_TIMEOUT
+    assert sess.status() == 0                                   # reading clears it
+    # reported by the accept that follows, whose own work is done all the same
+    sess.refresh_prefill(gp, 0)
+    assert lib.odb_debug_expire_wait(sess.handle, C.c_int64(2_000_000)) == B.ODB_OK
+    with pytest.raises(B.OdbError) as err:
+        sess.unmask_accept(gp, True)
+    assert err.value.status == B.ODB_ERR_TIMEOUT
+    assert sess.status() == 0
+    sess.block_decode_step(gp)                                  # the accept had committed its token: the step has rows
+    res = sess.unmask_accept(gp, False)[0]
+    assert res.n_accepted >= 1 and res.masks_left <= 14
+    # and by the device-resident loop, which stops after the iteration that saw it
+    assert lib.odb_debug_expire_wait(sess.handle, C.c_int64(2_000_000)) == B.ODB_OK
+    with pytest.raises(B.OdbError) as err:
+        sess.decode_block_resident(gp)
+    assert err.value.status == B.ODB_ERR_TIMEOUT
+    assert sess.status() == 0
+    log = sess.decode_block_resident(gp)
+    assert log[-1][0].masks_left == 0
+    sess.close(); gm.close()
