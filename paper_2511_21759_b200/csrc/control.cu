@@ -226,11 +226,11 @@ __device__ int accept_set(const float* conf, const bool* masked, int B, float ta
     return n;
 }
 
+// st / res: the block's shared-memory copies of the sequence's state and result (the decisions are one thread's
+// serial walk: every field it touches would otherwise be a dependent global load)
 __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p, int after_refresh, int mask_id, int eos_id,
-                            int dry) {
+                            int dry, SeqState* st, odb_result* res) {
     const int seq = blockIdx.x;
-    SeqState* st = c.state + seq;
-    odb_result* res = c.results + seq;
     if (!st->active || !st->in_fwd) {
         if (threadIdx.x == 0) {
             res->masks_left = st->active ? st->n_masked : 0;
@@ -447,32 +447,50 @@ __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p,
 
 // One block per sequence.  After the decisions, the block writes the sequence's state and result (and block 0
 // the status word) straight into pinned host memory.
-__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id, int dry) {
-    accept_body(c, p, after_refresh, mask_id, eos_id, dry);
-    __syncthreads();
+struct AcceptShared {
+    SeqState st;
+    odb_result res;
+};
+__device__ __forceinline__ void accept_load(const ControlBuffers& c, AcceptShared* sh) {
     const int seq = blockIdx.x;
-    const int* src_state = reinterpret_cast<const int*>(c.state + seq);
-    int* dst_state = reinterpret_cast<int*>(c.host_state + seq);
-    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) dst_state[i] = src_state[i];
-    const int* src_res = reinterpret_cast<const int*>(c.results + seq);
-    int* dst_res = reinterpret_cast<int*>(c.host_results + seq);
-    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) dst_res[i] = src_res[i];
-    if (seq == 0 && threadIdx.x == 0) *c.host_status = *c.status;
+    const int* gs = reinterpret_cast<const int*>(c.state + seq);
+    const int* gr = reinterpret_cast<const int*>(c.results + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) reinterpret_cast<int*>(&sh->st)[i] = gs[i];
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) reinterpret_cast<int*>(&sh->res)[i] = gr[i];
+    __syncthreads();
+}
+// state and result back to the device copies and out to pinned host memory (host_res: where this call's results go)
+__device__ __forceinline__ void accept_store(const ControlBuffers& c, const AcceptShared* sh, odb_result* host_res) {
+    const int seq = blockIdx.x;
+    const int* ss = reinterpret_cast<const int*>(&sh->st);
+    const int* sr = reinterpret_cast<const int*>(&sh->res);
+    int* gs = reinterpret_cast<int*>(c.state + seq);
+    int* hs = reinterpret_cast<int*>(c.host_state + seq);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) { gs[i] = ss[i]; hs[i] = ss[i]; }
+    int* gr = reinterpret_cast<int*>(c.results + seq);
+    int* hr = reinterpret_cast<int*>(host_res);
+    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) { gr[i] = sr[i]; hr[i] = sr[i]; }
+}
+
+__global__ void accept_kernel(ControlBuffers c, odb_decode_params p, int after_refresh, int mask_id, int eos_id, int dry) {
+    __shared__ AcceptShared sh;
+    accept_load(c, &sh);
+    accept_body(c, p, after_refresh, mask_id, eos_id, dry, &sh.st, &sh.res);
+    __syncthreads();
+    accept_store(c, &sh, c.host_results + blockIdx.x);
+    if (blockIdx.x == 0 && threadIdx.x == 0) *c.host_status = *c.status;
     __threadfence_system();
 }
 
 // The accept of the device-resident loop: the same decisions, then the hand-over to the next iteration.
 __global__ void accept_loop_kernel(ControlBuffers c, odb_decode_params p, int mask_id, int eos_id, int dry, LoopControl lc) {
-    accept_body(c, p, 0, mask_id, eos_id, dry);
+    __shared__ AcceptShared sh;
+    accept_load(c, &sh);
+    accept_body(c, p, 0, mask_id, eos_id, dry, &sh.st, &sh.res);
     __syncthreads();
     const int seq = blockIdx.x, batch = gridDim.x;
     const int it = *lc.iter;      // stable until every block has arrived below
-    const int* src_state = reinterpret_cast<const int*>(c.state + seq);
-    int* dst_state = reinterpret_cast<int*>(c.host_state + seq);
-    for (int i = threadIdx.x; i < static_cast<int>(sizeof(SeqState) / 4); i += blockDim.x) dst_state[i] = src_state[i];
-    const int* src_res = reinterpret_cast<const int*>(c.results + seq);
-    int* dst_res = reinterpret_cast<int*>(lc.host_log + static_cast<size_t>(it) * batch + seq);
-    for (int i = threadIdx.x; i < static_cast<int>(sizeof(odb_result) / 4); i += blockDim.x) dst_res[i] = src_res[i];
+    accept_store(c, &sh, lc.host_log + static_cast<size_t>(it) * batch + seq);
     __threadfence_system();
     __syncthreads();
     if (threadIdx.x != 0) return;
