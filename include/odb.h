@@ -3,9 +3,8 @@
  *
  * What the library computes (paper: "Orchestrating Dual-Boundaries", arXiv 2511.21759):
  *   - odb_refresh_prefill   : the block-boundary cache refresh, a full bidirectional forward
- *                             that rewrites the K/V cache of every position (Sections 1, 2.1
- *                             and 4.1: "all tokens in the response sequence are computed and
- *                             the KV cache is updated");
+ *                             that recomputes every response position and rewrites the K/V
+ *                             cache of every position and layer (Sections 1, 2.1 and 4.1);
  *   - odb_block_decode_step : one decoding iteration of the current block over the main block
  *                             and its speculative copies, attending the cached K/V of every
  *                             token outside the block (DualCache, Section 2.1; copies and their
@@ -276,8 +275,9 @@ int32_t odb_debug_gemm(const void* x, const void* w, float* out, void* scratch, 
  * Limit: k_splits * M * N * 4 bytes must fit ODB_STATIC_SCRATCH_BYTES (k_splits after the library's
  * heuristic when 0 is passed), otherwise ODB_ERR_WORKSPACE is returned and nothing is launched.
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
- * The first call on a device looks up the array's device address (with that device current); make
- * that first call before any stream capture begins.
+ * The first call on a device looks up the array's device address (with that device current).  Every
+ * call ends by waiting for `stream` and reading the status word back to the host, so it cannot be
+ * issued on a stream that is being captured.
  * All calls on a device share the one array: two calls whose kernels overlap on the GPU (different
  * streams, or different host threads) race on it; serialise them.  The array keeps the previous
  * call's contents; the call itself clears the one word that has to start at zero.

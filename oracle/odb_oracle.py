@@ -322,20 +322,89 @@ def accept_set(conf: np.ndarray, masked: np.ndarray, tau: float) -> np.ndarray:
     return acc
 
 
-def decision_margin(conf: np.ndarray, masked: np.ndarray, tau: float, k_ranks: int = 0) -> float:
-    """How close the decisions taken on this row of confidences are to flipping: the smallest
-    relative gap among (a) any masked confidence and the threshold, (b) the top two masked
-    confidences when the top-1 fallback decides, (c) neighbours in the candidate ranking.
-    Diagnostic only (used to tell a near-tie from a real disagreement); decides nothing."""
-    c = np.sort(conf[masked].astype(np.float64))[::-1]
-    if len(c) == 0:
+def decision_margin(conf: np.ndarray, masked: np.ndarray, tau: float, k_ranks: int = 0,
+                    still_masked: Optional[np.ndarray] = None, relative: bool = True) -> float:
+    """How close the decisions taken on this row of confidences are to flipping.  Diagnostic only
+    (tells a near-tie from a real disagreement); decides nothing.
+
+    The decisions are those of `accept_set` followed by `rank_candidates` on what stays masked:
+      (a) threshold: every masked confidence against tau            -> |c - tau| / tau;
+      (b) fallback, only when nothing exceeds tau: best against runner-up -> (c0 - c1) / c0;
+      (c) ranking of the positions still masked AFTER the accept: the k_ranks most confident among
+          them, each against the next one down (the last of them against the first one left out)
+                                                                      -> (c_i - c_{i+1}) / c_i.
+    Returns the smallest of these gaps (relative as written, or plain differences with
+    relative=False); inf when no position is masked.  Positions that are accepted take no part in
+    (c): their order among themselves decides nothing.  `still_masked` names the positions ranked
+    in (c) when they are not simply `masked` minus this row's accept set (after a jump chain:
+    minus everything the chain committed)."""
+    idx = np.flatnonzero(masked)
+    if len(idx) == 0:
         return np.inf
-    m = float(np.min(np.abs(c - tau) / max(abs(tau), 1e-30)))
-    if not (c > tau).any() and len(c) > 1:
-        m = min(m, float((c[0] - c[1]) / max(c[0], 1e-30)))
-    for i in range(min(k_ranks + 1, len(c)) - 1):
-        m = min(m, float((c[i] - c[i + 1]) / max(c[i], 1e-30)))
+    c = conf[idx].astype(np.float32).astype(np.float64)
+    over = (lambda v: max(abs(v), 1e-30)) if relative else (lambda v: 1.0)
+    with np.errstate(invalid="ignore"):
+        m = float(np.min(np.abs(c - tau))) / over(tau)
+    acc = accept_set(conf, masked, tau)[idx]
+    if not (c > np.float32(tau)).any() and len(c) > 1:
+        top = np.sort(c)[::-1]
+        m = min(m, float(top[0] - top[1]) / over(top[0]))
+    if still_masked is None:
+        rest = np.sort(c[~acc])[::-1]
+    else:
+        rest = np.sort(conf[np.flatnonzero(still_masked)].astype(np.float32).astype(np.float64))[::-1]
+    for i in range(min(k_ranks, len(rest) - 1)):
+        m = min(m, float(rest[i] - rest[i + 1]) / over(rest[i]))
     return m
+
+
+def conf_logit(c):
+    """ln(c / (1 - c)) of a confidence, clipped to +-16.  A perturbation of every logit of the row by
+    at most eps moves this quantity by at most 2 eps (c is the softmax probability of the row's best
+    entry), so distances between decisions are measured in it.  Diagnostic only."""
+    c = np.clip(np.asarray(c, dtype=np.float64), 1e-7, 1.0 - 1e-7)
+    return np.log(c) - np.log1p(-c)
+
+
+def top2_gap(logits: np.ndarray, mask_id: int) -> np.ndarray:
+    """Per row: best logit minus second-best logit, on the fp32 values the greedy token is decided
+    on, [MASK] excluded.  Diagnostic only: the distance of each argmax from flipping."""
+    l = logits.astype(np.float32).astype(np.float64)
+    l[:, mask_id] = -np.inf
+    top = np.partition(l, -2, axis=1)[:, -2:]
+    return np.abs(top[:, 1] - top[:, 0])
+
+
+def walk_diagnostics(conf: np.ndarray, gaps: np.ndarray, masked0: np.ndarray, subsets: list, rank_off: list,
+                     visited: list, new: dict, tau: float, k_ranks: int) -> dict:
+    """Distance of one iteration's decisions from flipping.  Diagnostic only.
+
+    conf [copies][B] and gaps [copies][B] (top2_gap per row) are the iteration's outputs, `visited`
+    the copies whose outputs decided something (the jump chain; the main block too when one block is
+    picked), `new` what the iteration committed.  In every visited copy the accept decisions count
+    over the positions masked in that copy's input; the last visited copy also ranks what is left
+    for the next candidates.  Greedy tokens count where they are used: at accepted positions and at
+    the next candidates.
+    Returns margin (decision_margin, relative, in confidence), sep (the same gaps as plain
+    differences of conf_logit) and tok_gap (smallest top-2 logit gap among the tokens used)."""
+    left = masked0.copy()
+    left[np.array(list(new.keys()), dtype=np.int64)] = False
+    last = visited[-1]
+    tau_l = float(conf_logit(tau)) if 0.0 < tau < 1.0 else (np.inf if tau >= 1.0 else -np.inf)
+    out = {"margin": np.inf, "sep": np.inf, "tok_gap": np.inf}
+    for c in visited:
+        m_c = masked0.copy()
+        m_c[np.array([rank_off[r - 1] for r in subsets[c]], dtype=np.int64)] = False   # its fills are not masked in its input
+        if not m_c.any():
+            continue
+        kk, lm = (k_ranks, left) if c == last else (0, None)
+        out["margin"] = min(out["margin"], decision_margin(conf[c], m_c, tau, kk, lm))
+        out["sep"] = min(out["sep"], decision_margin(conf_logit(conf[c]), m_c, tau_l, kk, lm, relative=False))
+        used = [int(i) for i in np.flatnonzero(accept_set(conf[c], m_c, tau))]
+        if c == last:
+            used += rank_candidates(conf[c], left, k_ranks)
+        out["tok_gap"] = min(out["tok_gap"], float(gaps[c][used].min()))
+    return out
 
 
 def rank_candidates(conf: np.ndarray, masked: np.ndarray, k: int) -> list:
@@ -482,7 +551,8 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
         s = P + b * params.block_len
         if s >= T or (max_iters is not None and len(trace) >= max_iters):
             break
-        cache, conf_r, tok_r = refresh_prefill(model, x, T, s, faithful=faithful, dtype=dtype)
+        cache, conf_r, tok_r, logits_r = refresh_prefill(model, x, T, s, faithful=faithful, dtype=dtype,
+                                                         return_logits=True)
         newL = alp_scan(conf_r, tok_r, s, P, model.eos_id, params.truncate_threshold) if params.alp else None
         if length_schedule is not None:
             cand = length_schedule(b, T - P)
@@ -497,9 +567,10 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
         acc = accept_set(conf_r[:B], masked, tau)
         for i in np.flatnonzero(acc):
             x[s + i] = tok_r[i]
+        diag = walk_diagnostics(conf_r[None, :B], top2_gap(logits_r[:B], model.mask_id)[None, :], masked, [()], [], [0],
+                                {int(i): 0 for i in np.flatnonzero(acc)}, tau, k_ranks)
         trace.append({"kind": "refresh", "block": b, "T": T,
-                      "accepted": [(int(s + i), int(tok_r[i])) for i in np.flatnonzero(acc)],
-                      "chain": [0], "margin": decision_margin(conf_r[:B], masked, tau, k_ranks + 1)})
+                      "accepted": [(int(s + i), int(tok_r[i])) for i in np.flatnonzero(acc)], "chain": [0], **diag})
         last_conf, last_tok = conf_r[:B], tok_r[:B]
         if not cache_blocks:
             if not (x[s:e] == model.mask_id).any():
@@ -514,16 +585,19 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             rank_tok = [int(last_tok[i]) for i in ranks]
             st2 = use_stage2(params, B, int((~masked).sum()))
             subsets = copy_subsets(len(ranks), 4 if (params.n_copies == 8 and not st2) else params.n_copies, st2)
-            conf, tok = block_decode_step(model, cache, x, T, s, e, subsets, rank_pos, rank_tok,
-                                          st2, faithful=faithful, dtype=dtype)
+            conf, tok, logits, r_copy, r_pos = block_decode_step(model, cache, x, T, s, e, subsets, rank_pos, rank_tok,
+                                                                 st2, faithful=faithful, dtype=dtype, return_logits=True)
             walk = pick_best_walk if params.pick_best else jump_walk
             new, chain, last = walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
             for i, t in new.items():
                 x[s + i] = t
-            margin = min(decision_margin(conf[c], masked & (conf[c] >= 0), tau, k_ranks + 1) for c in chain)
+            gaps = np.full(conf.shape, np.inf)
+            gaps[r_copy, r_pos - s] = top2_gap(logits, model.mask_id)
+            visited = chain if not (params.pick_best and chain != [0]) else [0] + chain
+            diag = walk_diagnostics(conf, gaps, masked, subsets, ranks, visited, new, tau, k_ranks)
             trace.append({"kind": "step", "block": b, "T": T, "stage2": st2,
                           "accepted": sorted((int(s + i), int(t)) for i, t in new.items()),
-                          "chain": [int(c) for c in chain], "margin": margin})
+                          "chain": [int(c) for c in chain], **diag})
             last_conf, last_tok = conf[last], tok[last]
         b += 1
     return x.astype(np.int32), trace

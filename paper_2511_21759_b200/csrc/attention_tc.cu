@@ -42,10 +42,6 @@ constexpr uint32_t kPBytes = kTQ * kTK * 2;          // 16 KB: one atom of 128 r
 constexpr uint32_t kSmemBytes = kQBytes + 3 * kKBytes + 2 * kPBytes + 128;   // the dynamic region starts 1024-aligned
 constexpr uint32_t kTmemCols = 256;                  // S0: columns 0..63, O: 64..191, S1: 192..255
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
 __device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
 }
@@ -627,12 +623,10 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
 template <bool STEP>
 cudaError_t launch_tc(dim3 grid, const __nv_bfloat16* q, const __nv_bfloat16* k, const __nv_bfloat16* v, const __nv_bfloat16* cache,
                       size_t cache_rows, const TcArgs& ta, int* status, cudaStream_t st) {
-    static bool attr_done = false;
-    if (!attr_done) {
-        cudaError_t e = cudaFuncSetAttribute(attention_tc_kernel<STEP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(kSmemBytes));
-        if (e != cudaSuccess) return e;
-        attr_done = true;
+    static std::atomic<unsigned long long> attr_done{0};
+    {
+        cudaError_t e0 = set_smem_limit_once(attr_done, attention_tc_kernel<STEP>, static_cast<int>(kSmemBytes));
+        if (e0 != cudaSuccess) return e0;
     }
     // the fresh q / k / v of this forward: [M][H * 128] bf16, rows beyond M read as zero; the cache as rows of 128
     CUtensorMap tq, tk, tv, tc;

@@ -47,7 +47,7 @@ int32_t check_config(const odb_config* c) {
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
     size_t rope, state, results, status, loop, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
-    size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml;
+    size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml, ptable, pbars;
     size_t total;
 };
 
@@ -99,6 +99,9 @@ Layout make_layout(const odb_config& c) {
     }
     L.part_o = take(4 * L.attn_rows * d);
     L.part_ml = take(4 * L.attn_rows * c.n_heads * 2);
+    // persistent decode-step kernel: one table of projections per row-tile size (32, 64, 128), the grid barrier words
+    L.ptable = take(3 * align_up(step_persistent_table_bytes(c.n_layers)));
+    L.pbars = take(step_persistent_barrier_bytes(c.n_layers));
     L.total = off;
     return L;
 }
@@ -151,6 +154,7 @@ struct odb_session {
     cudaStream_t record_st;
     odb_result* pinned_log;   // [kMaxLoopIters][max_batch]
     int32_t* pinned_iters;    // [0] iterations run (written by the device); [1..3] the loop words of the next launch
+    bool ptable_built[3];     // persistent step kernel: projection table for 32 / 64 / 128 rows per tile is on the device
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
 
@@ -278,6 +282,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->record_st = nullptr;
     s->pinned_log = nullptr;
     s->pinned_iters = nullptr;
+    s->ptable_built[0] = s->ptable_built[1] = s->ptable_built[2] = false;
     cudaError_t e = cudaMallocHost(&s->pinned_state, sizeof(SeqState) * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_log, sizeof(odb_result) * kMaxLoopIters * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_iters, 4 * sizeof(int32_t));
@@ -447,6 +452,47 @@ struct LaunchScope {
     }
 };
 
+int bn_index(int M) { return M <= 32 ? 0 : M <= 64 ? 1 : 2; }
+
+// Whether a decode step of M rows runs as the persistent kernel (one cooperative launch for the whole forward).
+bool use_persistent(const odb_session* s, int M) {
+    const odb_config& c = s->m->cfg;
+    return step_persistent_supported(M, c.d_model, c.d_ffn, c.head_dim);
+}
+
+// The persistent kernel reads its projections (weight and operand tensor maps, split) from a table in the
+// workspace; built on first use per row-tile size, outside any stream capture (it is a synchronous copy).
+int32_t ensure_ptable(odb_session* s, int M) {
+    const int bi = bn_index(M);
+    if (s->ptable_built[bi]) return ODB_OK;
+    const odb_model* m = s->m;
+    const odb_config& c = m->cfg;
+    const Layout& L = s->L;
+    const int BN = 32 << bi, d = c.d_model, F = c.d_ffn, grid = step_persistent_grid();
+    const int rows_cap = static_cast<int>(L.rows);
+    CUtensorMap tx_a, tx_o, tx_g;
+    ODB_CUDA(make_rows_tmap(&tx_a, s->ws + L.a, rows_cap, d, BN));
+    ODB_CUDA(make_rows_tmap(&tx_o, s->ws + L.o, rows_cap, d, BN));
+    ODB_CUDA(make_rows_tmap(&tx_g, s->ws + L.g, rows_cap, F, BN));
+    std::vector<PGemmDesc> t(4 * c.n_layers + 1);
+    const int kb_d = (d + 63) / 64, kb_F = (F + 63) / 64;
+    for (int l = 0; l < c.n_layers; ++l) {
+        step_persistent_fill_desc(t[4 * l + 0], m->tm_qkv[l], tx_a, m->norm1[l], (3 * d + 127) / 128, kb_d, 0, grid);
+        step_persistent_fill_desc(t[4 * l + 1], m->tm_o[l], tx_o, nullptr, (d + 127) / 128, kb_d, 0, grid);
+        step_persistent_fill_desc(t[4 * l + 2], m->tm_gu[l], tx_a, m->norm2[l], (F + 63) / 64, kb_d, 0, grid);
+        step_persistent_fill_desc(t[4 * l + 3], m->tm_d[l], tx_g, nullptr, (d + 127) / 128, kb_F, 0, grid);
+    }
+    if (c.with_lm_head)
+        step_persistent_fill_desc(t[4 * c.n_layers], m->tm_lm, tx_a, m->final_norm, (c.vocab + 127) / 128, kb_d, 1, grid);
+    else
+        step_persistent_fill_desc(t[4 * c.n_layers], m->tm_o[0], tx_a, m->final_norm, 1, 1, 0, grid);   // unused slot
+    uint8_t* dst = s->ws + L.ptable + bi * align_up(step_persistent_table_bytes(c.n_layers));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
+    ODB_CUDA(cudaMemcpy(dst, t.data(), sizeof(PGemmDesc) * t.size(), cudaMemcpyHostToDevice));
+    s->ptable_built[bi] = true;
+    return ODB_OK;
+}
+
 // One forward over the M rows of the row table already built on the device.
 int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, int n_step_tiles = 0, int n_big_tiles = 0,
                 cudaStream_t st = nullptr) {
@@ -495,6 +541,45 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         LaunchScope scope__(s, kind);   \
         ODB_CUDA(call);                 \
     } while (0)
+    if (!write_cache && n_tiles > 0 && use_persistent(s, M) && s->ptable_built[bn_index(M)] && (!c.with_lm_head || n_lm == M)) {
+        // decode step as ONE persistent kernel: every projection, the short phases between them and the LM head
+        // with its confidence statistics; the per-row merge of the statistics follows as a second launch
+        StepPersistentArgs pa{};
+        pa.gemms = reinterpret_cast<const PGemmDesc*>(s->ws + L.ptable + bn_index(M) * align_up(step_persistent_table_bytes(c.n_layers)));
+        pa.n_layers = c.n_layers; pa.M = M;
+        pa.d = d; pa.F = F; pa.H = H; pa.hd = hd; pa.vocab = c.vocab; pa.mask_id = c.mask_id; pa.with_lm = (c.with_lm_head && !s->dump_logits) ? 1 : 0;
+        pa.rms_eps = c.rms_eps;
+        pa.embed = m->embed;
+        pa.row_tok = s->cb.row_tok; pa.row_pos = s->cb.row_pos; pa.row_flags = s->cb.row_flags;
+        pa.h = h; pa.a = a; pa.ssq = inv;
+        pa.q = q; pa.k = k; pa.v = v; pa.o = o; pa.g = g;
+        pa.partial = partial;
+        pa.rope = s->at<float2>(L.rope);
+        pa.cache = s->kv; pa.max_seq = c.max_seq;
+        pa.tiles = s->cb.tiles; pa.n_qtiles = n_tiles;
+        int pks = step_persistent_grid() / (n_tiles * H);
+        if (pks > 8) pks = 8;
+        if (static_cast<size_t>(pks) * M > L.attn_rows) pks = static_cast<int>(L.attn_rows / M);
+        if (pks < 1) pks = 1;
+        pa.ksplit = pks;
+        pa.part_o = s->at<float>(L.part_o); pa.part_ml = s->at<float>(L.part_ml);
+        pa.conf_part = reinterpret_cast<ConfPartial*>(s->ws + L.conf_part);
+        pa.bars = s->at<unsigned int>(L.pbars);
+        pa.status = status;
+        ODB_CUDA(step_persistent_configure(pa));
+        ODB_LAUNCH(ODB_KIND_GEMM, launch_step_persistent(pa, st));
+        if (pa.with_lm) {
+            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence_final(pa.conf_part, (c.vocab + 127) / 128, M, s->at<float>(L.conf),
+                                                                       s->at<int32_t>(L.tok), st));
+        } else if (c.with_lm_head) {
+            // test mode: the kernel ended with the LM head's operand; the logits are materialised by a plain launch
+            int sp = 1;
+            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, s->at<float>(L.logits), M, c.vocab, d, &sp, &inv_scale));
+            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(s->at<float>(L.logits), M, c.vocab, c.mask_id, s->at<float>(L.conf),
+                                                                 s->at<int32_t>(L.tok), s->ws + L.conf_part, st));
+        }
+        return ODB_OK;
+    }
     ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
     const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
     int res_splits = 0;
@@ -692,6 +777,10 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
     const int M = sh.rows;
     if (M == 0) return ODB_ERR_STATE;
     if (static_cast<size_t>(M) > s->L.rows) return ODB_ERR_SHAPE;
+    if (use_persistent(s, M)) {
+        const int32_t trc = ensure_ptable(s, M);
+        if (trc != ODB_OK) return trc;
+    }
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
     int32_t rc = forward(s, M, c.with_lm_head ? M : 0, sh.tiles, false, step_items(s, sh));
     if (rc != ODB_OK) return rc;
@@ -738,6 +827,10 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
     for (int i = 0; i < c.max_batch; ++i) step_shape_add(sh, s->mirror[i]);
     if (sh.rows == 0) return ODB_ERR_STATE;
     if (static_cast<size_t>(sh.rows) > s->L.rows) return ODB_ERR_SHAPE;
+    if (use_persistent(s, sh.rows)) {
+        const int32_t trc = ensure_ptable(s, sh.rows);
+        if (trc != ODB_OK) return trc;
+    }
 
     odb_session::ResidentGraph* g = nullptr;
     for (auto& r : s->resident)

@@ -8,9 +8,25 @@
 
 #include "../../include/odb.h"
 
+#include <atomic>
 #include <utility>
 
 namespace odb {
+
+// cudaFuncSetAttribute is a setting of one device: `done` (one word per kernel, kept by the caller) remembers
+// for which device indices the kernel already has its dynamic shared-memory limit.  The device is the current
+// one, which must be the device of the stream the launch goes to.
+template <class Kernel>
+cudaError_t set_smem_limit_once(std::atomic<unsigned long long>& done, Kernel kernel, int bytes) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const unsigned long long bit = dev >= 0 && dev < 64 ? 1ull << dev : 0ull;
+    if (bit && (done.load(std::memory_order_acquire) & bit)) return cudaSuccess;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e == cudaSuccess && bit) done.fetch_or(bit, std::memory_order_release);
+    return e;
+}
 
 // ---------------------------------------------------------------------------------------
 // programmatic dependent launch: every kernel of a forward lets its successor start early
@@ -21,6 +37,9 @@ namespace odb {
 // ---------------------------------------------------------------------------------------
 
 #ifdef __CUDACC__
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
@@ -270,6 +289,58 @@ cudaError_t launch_step_attention(const StepAttnArgs& a, cudaStream_t st);
 cudaError_t launch_step_attention_tc(const StepAttnArgs& a, size_t cache_rows, int* status, cudaStream_t st);
 cudaError_t launch_attention_combine(const float* part_o, const float* part_ml, __nv_bfloat16* o, int M, int H, int hd,
                                      int ksplit, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------
+// Persistent decode-step kernel (step_persistent.cu): ONE cooperative launch runs the whole forward of a
+// decode step of up to 128 query rows - every projection, RMSNorm, RoPE, attention and the LM head with its
+// confidence statistics - on one CTA per SM.  The k-blocks of every projection are divided evenly over the
+// CTAs (fixed assignment, partial tiles reduced in CTA order); a TMA producer warp per CTA keeps a ring of
+// shared-memory stages filled with weight tiles and runs ahead of the phase its consumers are in, so HBM keeps
+// streaming across the hand-overs between phases, which are grid-wide barriers with a bounded wait.
+// ---------------------------------------------------------------------------------------
+struct alignas(64) PGemmDesc {   // one projection of the step; an array of these lives in device memory
+    CUtensorMap tmap_w;          // packed weight tiles
+    CUtensorMap tmap_x;          // its bf16 activation rows [rows][K], box 64 x BN
+    const float* gain;           // gain of the RMSNorm that produces its operand (QKV, gate/up, LM head), else null
+    int32_t n_tiles, nkb;        // weight tiles of 128 rows, k-blocks of 64
+    int32_t conf;                // 1: LM head, tile aligned, epilogue = softmax statistics per vocabulary tile
+    int32_t g_use;               // CTAs its units are divided over (all of them unless the projection is tiny: a
+                                 // CTA's range is never shorter than a sixth of a tile's k-blocks, so that an
+                                 // output tile has at most 8 parts)
+    int32_t pad[10];
+};
+struct StepPersistentArgs {
+    const PGemmDesc* gemms;      // [4 * n_layers (qkv, o, gate/up, down per layer) + with_lm]
+    int n_layers, M, BN, stages, scratch_bytes;
+    int d, F, H, hd, vocab, mask_id, with_lm;
+    float rms_eps;
+    const __nv_bfloat16* embed;
+    const int32_t* row_tok; const int32_t* row_pos; const int32_t* row_flags;
+    float* h; __nv_bfloat16* a; float* ssq;
+    __nv_bfloat16 *q, *k, *v, *o, *g;
+    float* partial;
+    const float2* rope;
+    const __nv_bfloat16* cache; int max_seq;
+    const QTile* tiles; int n_qtiles, ksplit;
+    float* part_o; float* part_ml;
+    ConfPartial* conf_part;
+    unsigned int* bars;          // one word per grid barrier, zero when the kernel starts
+    int n_bars;
+    int* status;
+};
+// bytes of the PGemmDesc table and of the barrier words for a model of n_layers layers
+size_t step_persistent_table_bytes(int n_layers);
+size_t step_persistent_barrier_bytes(int n_layers);
+// whether this step can run as the persistent kernel (shape limits, cooperative launch available on the device)
+bool step_persistent_supported(int M, int d, int F, int hd);
+// rows per MMA tile and ring depth for M rows; fills a.BN, a.stages, a.scratch_bytes, a.n_bars
+cudaError_t step_persistent_configure(StepPersistentArgs& a);
+// CTAs of the launch (the SM count of the current device; 0: no cooperative launch there)
+int step_persistent_grid();
+void step_persistent_fill_desc(PGemmDesc& d, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x, const float* gain, int n_tiles,
+                               int nkb, int conf, int grid);
+// zeroes the barrier words and launches the kernel (cooperative, one CTA per SM) on st
+cudaError_t launch_step_persistent(const StepPersistentArgs& a, cudaStream_t st);
 
 // control kernels (control.cu)
 struct ControlBuffers {

@@ -248,7 +248,8 @@ def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> 
 
 def generate(sess: Session, params: DecodeParams, *,
              length_schedule: Optional[Callable[[int, int, int], Optional[int]]] = None,
-             max_iters: Optional[int] = None, cache_blocks: bool = True, resident: bool = False):
+             max_iters: Optional[int] = None, cache_blocks: bool = True, resident: bool = False,
+             start_block: int = 0):
     """Runs every sequence set on the session to completion.
 
     Per iteration: the sequences standing at a block boundary are refreshed and accepted
@@ -259,9 +260,11 @@ def generate(sess: Session, params: DecodeParams, *,
     {"kind", "seqs": {seq: {"accepted", "chain", "masks_left", "gen_len", "block"}}}.
     cache_blocks=False is the cache-less baseline (Section 1): every iteration of a block is a
     refresh prefill and no block step is taken.  resident=True runs the steps of a block through the
-    device-resident loop (same trace, one host round trip per block instead of one per iteration)."""
+    device-resident loop (same trace, one host round trip per block instead of one per iteration).
+    start_block: the block every sequence starts at (a resumed session: the blocks before it are already
+    decoded in the ids given to set_sequence; the refresh of start_block recomputes the whole cache)."""
     seqs = sorted(sess.gen_len)
-    block = {i: 0 for i in seqs}
+    block = {i: start_block for i in seqs}
     need_refresh = {i: True for i in seqs}
     done = {i: False for i in seqs}
     trace = []

@@ -76,7 +76,18 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
     x = np.array(x0, dtype=np.int64)
     T = len(x)
     st = {"iters": 0, "refreshes": 0, "steps": 0, "tokens": 0, "oracle_decision_diff": 0, "near_ties": [],
-          "worst_logit": 0.0, "worst_conf": 0.0, "tok_diff": 0}
+          "worst_logit": 0.0, "worst_conf": 0.0, "tok_diff": 0, "log": []}
+
+    def record(kind, diag, rows, g_conf, o_conf, g_logits, o_logits):
+        """Per iteration: the oracle's distance from flipping (walk_diagnostics) beside the errors measured on the
+        rows at masked positions: |d conf_logit| and the largest |d logit|."""
+        rows = np.flatnonzero(rows)
+        e = {"kind": kind, **diag, "cl_err": 0.0, "logit_err": None}
+        if len(rows):
+            e["cl_err"] = float(np.abs(O.conf_logit(g_conf[rows].astype(np.float64)) - O.conf_logit(o_conf[rows].astype(np.float64))).max())
+            if g_logits is not None:
+                e["logit_err"] = float(np.abs(g_logits[rows] - o_logits[rows]).max())
+        st["log"].append(e)
 
     def numerics(g_conf, g_tok, g_logits, o_conf, o_tok, o_logits):
         rel = np.abs(g_conf.astype(np.float64) - o_conf) / np.maximum(o_conf, 1e-30)
@@ -133,6 +144,9 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
         assert res_tuple(res) == (want, [0]), (res_tuple(res), want)
         acc_o = O.accept_set(o_conf[:B], masked, tau)
         want_o = [(int(s + i), int(o_tok[i])) for i in np.flatnonzero(acc_o)]
+        record("refresh", O.walk_diagnostics(o_conf[None, :B], O.top2_gap(o_logits[:B], shape_mask)[None, :], masked, [()], [], [0],
+                                             {int(i): 0 for i in np.flatnonzero(acc_o)}, tau, k_ranks),
+               masked, g_conf[:B], o_conf[:B], None if g_logits is None else g_logits[:B], o_logits[:B])
         if want_o != want or newL_o != newL:
             margin = O.decision_margin(o_conf[:B], masked, tau, 0)
             st["oracle_decision_diff"] += 1
@@ -176,6 +190,11 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
             want = sorted((int(s + i), int(t)) for i, t in new.items())
             assert res_tuple(res) == (want, [int(c) for c in chain]), (res_tuple(res), want, chain)
             new_o, chain_o, last_o = walk(o_c, o_t, masked, subsets, ranks, rank_tok, tau)
+            o_gaps = np.full(o_c.shape, np.inf)
+            o_gaps[r_copy, r_pos - s] = O.top2_gap(o_logits, shape_mask)
+            visited = chain_o if not (op.pick_best and chain_o != [0]) else [0] + chain_o
+            record("step", O.walk_diagnostics(o_c, o_gaps, masked, subsets, ranks, visited, new_o, tau, k_ranks),
+                   masked[r_pos - s], g_cr, o_c[r_copy, r_pos - s], g_logits, o_logits)
             if new_o != new or chain_o != chain:
                 margin = min(O.decision_margin(o_c[c], masked & (o_c[c] >= 0), tau, 0) for c in chain_o)
                 st["oracle_decision_diff"] += 1

@@ -139,3 +139,39 @@ def test_an_expired_device_wait_is_reported_and_the_session_stays_usable():
     log = sess.decode_block_resident(gp)
     assert log[-1][0].masks_left == 0
     sess.close(); gm.close()
+
+
+@requires_gpu
+@pytest.mark.parametrize("copies", [1, 4])
+def test_resumed_session_continues_identically(copies):
+    """Checkpoint / resume: the state of a sequence is its token ids (the K/V cache is recomputed by the next
+    refresh).  A generation stopped at a block boundary, read out with get_tokens, handed to a NEW session with
+    set_sequence and continued from the next block gives the same trace and the same final tokens as the
+    uninterrupted generation."""
+    E = engine()
+    shape = synth.TINY_PEAKY
+    P, L, Bk = 24, 48, 16
+    gm = E.Model.from_synth(shape, seed=3, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
+    gp = E.DecodeParams(block_len=Bk, n_copies=copies, alp=False)
+    x0 = synth.sequence(3, 0, P, L, shape)
+    s0 = E.Session(gm)
+    s0.set_sequence(0, x0, P)
+    full_tok, full_trace = E.generate(s0, gp)
+    s0.close()
+    # the iteration that closes block 0 of the uninterrupted run
+    n0 = next(i for i, t in enumerate(full_trace) if t["seqs"][0]["masks_left"] == 0) + 1
+    assert 0 < n0 < len(full_trace)
+    s1 = E.Session(gm)
+    s1.set_sequence(0, x0, P)
+    _, head = E.generate(s1, gp, max_iters=n0)
+    saved = s1.get_tokens(0)
+    s1.close()
+    assert head == full_trace[:n0]
+    assert (saved[P:P + Bk] != shape.mask_id).all() and (saved[P + Bk:] == shape.mask_id).all()
+    s2 = E.Session(gm)                               # nothing of the first session survives but the ids
+    s2.set_sequence(0, saved, P)
+    tok, tail = E.generate(s2, gp, start_block=1)
+    assert s2.status() == 0
+    s2.close(); gm.close()
+    assert tail == full_trace[n0:]
+    assert np.array_equal(tok[0], full_tok[0])

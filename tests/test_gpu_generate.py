@@ -1,12 +1,16 @@
 """End-to-end generation through the C ABI against the oracle's generate loop.
 
-Token ids and the per-iteration accepted sets / jump chains must be identical.  The one
-legitimate exception is a near-tie: where the oracle's own decision margin (distance of a
-confidence to the threshold, or between the two best candidates) is below 1e-3 relative, the
-two sides may take different branches; such a case is reported, never silently accepted as
-equal, and the comparison stops there.
+Two regimes, tested apart:
+  * separated workloads (tests/golden/separated_workloads.json): every decision of the oracle's own
+    run is far from flipping, measured against the error of the kernels; token ids and the
+    per-iteration accepted sets / jump chains must be IDENTICAL, free running, no exception;
+  * random-weight workloads, where some decision is always closer than bf16 rounding noise: the
+    first divergence, if any, must be a near-tie by the measured error at that very iteration
+    (oracle margin <= max(1e-3, 4 x confidence error)); it is printed, and the test fails otherwise.
 """
 import dataclasses
+import json
+import os
 
 import numpy as np
 import pytest
@@ -16,7 +20,8 @@ from oracle import odb_oracle as O
 from oracle.inputs import model_from_synth
 from gpu_common import engine, requires_gpu, compare_traces, lockstep_generate, assert_near_ties_only
 
-NEAR_TIE = 1e-3
+with open(os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "separated_workloads.json")) as _f:
+    SEPARATED = json.load(_f)
 
 
 def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=None, om=None, lm_head_bits=None,
@@ -37,33 +42,109 @@ def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=
     gtok, gtrace = E.generate(sess, E.DecodeParams(**kw), length_schedule=gsched, resident=resident)
     otok, otrace = O.generate(om, x0, wl.prompt_len, O.DecodeParams(**kw), length_schedule=schedule)
     assert sess.status() == 0
+    # where the two runs part (if they do), the error is measured on that very state: the lock-step harness
+    # replays the generation up to and including that iteration
+    n, div = compare_traces(gtrace, otrace)
+    measured = None
+    if div is not None and div["gpu"] is not None:
+        sess.set_sequence(0, x0, wl.prompt_len)
+        st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw),
+                               schedule=schedule, tol=1.0, max_iters=div["iter"] + 1)
+        measured = st
     sess.close(); gm.close()
-    return gtok[0], gtrace, otok, otrace
+    return gtok[0], gtrace, otok, otrace, measured
 
 
-def _assert_parity(gtok, gtrace, otok, otrace, near_tie=NEAR_TIE):
-    n, div = compare_traces(gtrace, otrace, near_tie=near_tie)
+def _assert_identical_or_near_tie(gtok, gtrace, otok, otrace, measured):
+    """Passes when the free runs are identical, or when they part at a measured near-tie; fails otherwise."""
+    n, div = compare_traces(gtrace, otrace)
     if div is None:
         assert np.array_equal(gtok, otok)
+        print(f"\nfree run identical over {n} iterations")
         return
-    assert div["near_tie"], f"real divergence at iteration {div['iter']}: {div}"
-    pytest.xfail(f"near-tie at iteration {div['iter']} (oracle margin {div['margin']:.2e}); "
-                 f"{n} iterations identical before it")
+    assert measured is not None, f"traces differ in length after {n} equal iterations: {div}"
+    g, o = div["gpu"], div["oracle"]
+    if [p_ for p_, _ in g["accepted"]] == [p_ for p_, _ in sorted(o["accepted"])] and g["chain"] == o["chain"]:
+        # same positions, another greedy token: the replay has already asserted that every differing token sits
+        # on a top-2 logit gap below twice the logit error measured there
+        print(f"\nfree runs part at iteration {div['iter']} after {n} identical ones on a greedy token whose top-2 "
+              f"logit gap is below twice the measured logit error ({measured['tok_diff']} such rows): a near-tie")
+        return
+    ties = [t for t in measured["near_ties"] if t[0] == div["iter"]]
+    assert ties, f"iteration {div['iter']}: the free runs part but the oracle decides like the kernels in lock step: {div}"
+    assert_near_ties_only({"near_ties": ties})
+    it, kind, margin, cerr = ties[0]
+    print(f"\nfree runs part at iteration {it} ({kind}) after {n} identical ones: oracle margin {margin:.2e}, "
+          f"measured confidence error {cerr:.2e}: a near-tie")
+
+
+def _separated(name):
+    w = SEPARATED["workloads"][name]
+    shape = dataclasses.replace(synth.TINY_PEAKY, w_std=w["w_std"], lm_std=w["lm_std"])
+    x0 = synth.sequence(w["seed"], 0, w["prompt_len"], w["gen_len"], shape)
+    kw = dict(block_len=w["block_len"], n_copies=w["n_copies"], accept_threshold=w["accept_threshold"], alp=False)
+    return w, shape, x0, kw
 
 
 @requires_gpu
-@pytest.mark.parametrize("wl", ["cfg1_tiny", "cfg1_tiny_c4", "peaky_c1", "peaky_c4", "peaky_c8"])
-def test_generate_matches_oracle(wl):
-    # free run: the sharp-logit model turns a logit error into a confidence error of the same
-    # size (5e-2 .. 9e-2 measured by the lock-step test), so its near-tie band is wider
-    _assert_parity(*_run_both(wl), near_tie=NEAR_TIE if wl.startswith("cfg1") else 0.2)
+@pytest.mark.parametrize("resident", [False, True])
+@pytest.mark.parametrize("name", sorted(SEPARATED["workloads"]))
+def test_free_run_identical_on_separated_workloads(name, resident):
+    """Free-running generation (call by call, and through the device-resident loop) of a workload whose every
+    decision is separated: final tokens and every iteration's accepted set and jump chain equal the stored
+    oracle trace exactly.  There is no excuse path."""
+    E = engine()
+    w, shape, x0, kw = _separated(name)
+    P = w["prompt_len"]
+    gm = E.Model.from_synth(shape, seed=w["seed"], max_batch=1, max_seq=len(x0), max_block=w["block_len"], max_copies=8)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    gtok, gtrace = E.generate(sess, E.DecodeParams(**kw), resident=resident)
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    assert len(gtrace) == len(w["trace"])
+    for i, (g, o) in enumerate(zip(gtrace, w["trace"])):
+        assert g["kind"] == o["kind"], i
+        assert g["seqs"][0]["accepted"] == sorted(tuple(a) for a in o["accepted"]), (i, g["seqs"][0], o)
+        assert g["seqs"][0]["chain"] == o["chain"], (i, g["seqs"][0], o)
+    assert gtok[0].tolist() == w["tokens"]
 
 
 @requires_gpu
+@pytest.mark.parametrize("name", sorted(SEPARATED["workloads"]))
+def test_separated_workloads_are_separated_by_the_measured_error(name):
+    """Lock step on the same workloads: at every iteration the oracle's distance from flipping a decision is at
+    least ten times the confidence error measured there (both in ln(c / (1 - c))), and every greedy token that
+    is used has a top-2 logit gap of at least four times the largest logit error; the oracle never decides
+    differently from the kernels."""
+    E = engine()
+    w, shape, x0, kw = _separated(name)
+    P = w["prompt_len"]
+    om = model_from_synth(shape, seed=w["seed"])
+    gm = E.Model.from_synth(shape, seed=w["seed"], max_batch=1, max_seq=len(x0), max_block=w["block_len"], max_copies=8)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    st = lockstep_generate(E, sess, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=4e-2)
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    assert st["oracle_decision_diff"] == 0 and st["tokens_final"].tolist() == w["tokens"]
+    worst_c = min(e["sep"] / max(e["cl_err"], 1e-12) for e in st["log"])
+    worst_t = min(e["tok_gap"] / max(e["logit_err"], 1e-12) for e in st["log"])
+    print(f"\n{name}: {len(st['log'])} iterations; decision distance / confidence error >= {worst_c:.1f}, "
+          f"top-2 gap / logit error >= {worst_t:.1f}")
+    for i, (e, o) in enumerate(zip(st["log"], w["trace"])):
+        assert e["sep"] == pytest.approx(o["sep"], rel=1e-6) and e["tok_gap"] == pytest.approx(o["tok_gap"], rel=1e-6), i
+        assert e["sep"] >= 10 * e["cl_err"], (i, e)
+        assert e["tok_gap"] >= 4 * e["logit_err"], (i, e)
+
+
+@requires_gpu
+@pytest.mark.parametrize("resident", [False, True])
 @pytest.mark.parametrize("wl", ["cfg1_tiny", "cfg1_tiny_c4", "peaky_c1", "peaky_c4", "peaky_c8"])
-def test_resident_loop_matches_oracle(wl):
-    """The same free run with the steps of every block taken by the device-resident loop."""
-    _assert_parity(*_run_both(wl, resident=True), near_tie=NEAR_TIE if wl.startswith("cfg1") else 0.2)
+def test_free_run_parts_only_at_a_measured_near_tie(wl, resident):
+    """Random weights: the free runs are compared until they part; the iteration where they do is replayed in
+    lock step, and the oracle's margin there must be within four times the confidence error measured there."""
+    _assert_identical_or_near_tie(*_run_both(wl, resident=resident))
 
 
 @requires_gpu
@@ -244,9 +325,9 @@ def test_trace_counters_match_the_oracle_definition():
 @requires_gpu
 def test_generate_with_length_schedule():
     sched = lambda b, L: {0: 40, 1: 24}.get(b)
-    gtok, gtrace, otok, otrace = _run_both("peaky_c4", schedule=sched)
+    gtok, gtrace, otok, otrace, measured = _run_both("peaky_c4", schedule=sched)
     assert [r["seqs"][0]["gen_len"] for r in gtrace if r["kind"] == "refresh"][:2] == [40, 24]
-    _assert_parity(gtok, gtrace, otok, otrace, near_tie=0.2)
+    _assert_identical_or_near_tie(gtok, gtrace, otok, otrace, measured)
 
 
 @requires_gpu
@@ -268,12 +349,12 @@ def test_generate_alp_truncates():
     wl = dataclasses.replace(synth.WORKLOADS["peaky_c1"], prompt_len=32, gen_len=64)
     synth.WORKLOADS["_alp"] = wl
     try:
-        gtok, gtrace, otok, otrace = _run_both("_alp", seed=5, shape=shape, x0=x0, om=om, lm_head_bits=bits,
-                                               params_kw=dict(truncate_threshold=0.0))
+        gtok, gtrace, otok, otrace, measured = _run_both("_alp", seed=5, shape=shape, x0=x0, om=om, lm_head_bits=bits,
+                                                         params_kw=dict(truncate_threshold=0.0))
     finally:
         del synth.WORKLOADS["_alp"]
     assert otrace[0]["T"] < 96 and gtrace[0]["seqs"][0]["gen_len"] == otrace[0]["T"] - 32
-    _assert_parity(gtok, gtrace, otok, otrace, near_tie=0.2)
+    _assert_identical_or_near_tie(gtok, gtrace, otok, otrace, measured)
 
 
 @requires_gpu
@@ -299,7 +380,7 @@ def test_ragged_batch_equals_independent_runs():
         assert np.array_equal(together[i], alone[0]), i
     om = model_from_synth(shape, seed=0)
     otok, otrace = O.generate(om, xs[2], 17, O.DecodeParams(block_len=16, n_copies=4))
-    if min(t["margin"] for t in otrace) > NEAR_TIE:
+    if min(t["margin"] for t in otrace) > 0.5:          # only when no decision of the oracle's run is close
         assert np.array_equal(together[2], otok)
     gm.close()
 

@@ -393,3 +393,100 @@ def test_counters_of_the_three_systems():
     assert o["eff_nfe"] >= o["nfe"]                                            # several state changes in one pass
     assert f["tokens"] == L and o["tokens"] == len(out["odb"][0]) - wl.prompt_len
 
+
+
+# ----------------------------------------------------------------------------- diagnostics (decide nothing)
+
+ALL4 = np.ones(4, bool)
+
+
+def test_decision_margin_threshold_term_binds():
+    # something passes tau: only the distances to the threshold count; .95 is the closest, (.95 - .9) / .9
+    m = O.decision_margin(f32(.95, .5, .1), np.ones(3, bool), 0.9)
+    assert m == pytest.approx(0.05 / 0.9, rel=1e-5)
+    # a position just BELOW the threshold binds the same way
+    assert O.decision_margin(f32(.99, .89, .1), np.ones(3, bool), 0.9) == pytest.approx(0.01 / 0.9, rel=1e-4)
+    # positions that are not masked take no part, however close to tau they are
+    assert O.decision_margin(f32(.9001, .5), np.array([0, 1], bool), 0.9) == pytest.approx(0.4 / 0.9, rel=1e-5)
+
+
+def test_decision_margin_fallback_term_binds():
+    # nothing passes: the best must beat the runner-up, (.5 - .45) / .5 = .1 < distance to tau .4 / .9
+    assert O.decision_margin(f32(.5, .45, .1), np.ones(3, bool), 0.9) == pytest.approx(0.1, rel=1e-5)
+    # as soon as one position passes, the top-2 gap decides nothing any more
+    assert O.decision_margin(f32(.95, .949, .1), np.ones(3, bool), 0.9) == pytest.approx(0.049 / 0.9, rel=1e-4)
+    # a single masked position has no runner-up
+    assert O.decision_margin(f32(.5, .49), np.array([1, 0], bool), 0.9) == pytest.approx(0.4 / 0.9, rel=1e-5)
+
+
+def test_decision_margin_ranking_term_binds():
+    conf = f32(.95, .6, .57, .2)
+    assert O.decision_margin(conf, ALL4, 0.9, 0) == pytest.approx(0.05 / 0.9, rel=1e-5)       # no ranking asked for
+    # one candidate: .6 against the first one left out, (.6 - .57) / .6 = .05 < .0556
+    assert O.decision_margin(conf, ALL4, 0.9, 1) == pytest.approx(0.05, rel=1e-5)
+    # two candidates add (.57 - .2) / .57, which does not bind
+    assert O.decision_margin(conf, ALL4, 0.9, 2) == pytest.approx(0.05, rel=1e-5)
+    # more candidates than positions left: only the gaps that exist
+    assert O.decision_margin(conf, ALL4, 0.9, 7) == pytest.approx(0.05, rel=1e-5)
+    # the last candidate against the first one left out binds too
+    assert O.decision_margin(f32(.95, .6, .3, .299), ALL4, 0.9, 2) == pytest.approx(0.001 / 0.3, rel=1e-3)
+    assert O.decision_margin(f32(.95, .6, .3, .299), ALL4, 0.9, 1) == pytest.approx(0.05 / 0.9, rel=1e-5)
+
+
+def test_decision_margin_ignores_order_among_accepted_positions():
+    # .99 and .9899 are both accepted: their near-tie decides nothing; the fallback's winner is accepted too
+    assert O.decision_margin(f32(.99, .9899, .3, .1), ALL4, 0.9, 2) == pytest.approx(0.0899 / 0.9, rel=1e-3)
+    assert O.decision_margin(f32(.5, .3, .299, .1), ALL4, 0.9, 1) == pytest.approx(0.001 / 0.3, rel=1e-3)   # .5 taken by fallback
+    assert O.decision_margin(f32(.5, .3, .299, .1), ALL4, 0.9, 0) == pytest.approx(0.4, rel=1e-5)          # (.5 - .3) / .5
+
+
+def test_decision_margin_empty_and_overrides():
+    assert O.decision_margin(f32(.5, .6), np.zeros(2, bool), 0.9, 2) == np.inf
+    # still_masked: rank only what a jump chain left ({2, 3}), not everything this row did not accept
+    conf = f32(.95, .6, .599, .2)
+    assert O.decision_margin(conf, ALL4, 0.9, 1) == pytest.approx(0.001 / 0.6, rel=1e-3)
+    assert O.decision_margin(conf, ALL4, 0.9, 1, np.array([0, 0, 1, 1], bool)) == pytest.approx(0.05 / 0.9, rel=1e-5)
+    # plain differences instead of relative gaps
+    assert O.decision_margin(f32(.5, .45, .1), np.ones(3, bool), 0.9, relative=False) == pytest.approx(0.05, rel=1e-5)
+    assert O.decision_margin(conf, ALL4, 0.9, 1, relative=False) == pytest.approx(0.001, rel=1e-3)
+
+
+def test_top2_gap_and_conf_logit():
+    logits = np.array([[1.0, 3.0, 2.5, 9.0], [0.0, -1.0, 7.0, 9.0]])
+    assert O.top2_gap(logits, 3).tolist() == [0.5, 7.0]                  # entry 3 is [MASK]: excluded
+    assert O.top2_gap(logits, 0).tolist() == [6.0, 2.0]
+    assert O.conf_logit(0.5) == pytest.approx(0.0, abs=1e-12)
+    assert O.conf_logit(0.9) == pytest.approx(np.log(9.0))
+    assert O.conf_logit(1.0) == pytest.approx(-O.conf_logit(0.0)) and np.isfinite(O.conf_logit(1.0))
+    # the property it is used for: moving every logit by at most eps moves conf_logit by at most 2 eps
+    rng = np.random.default_rng(0)
+    l = rng.normal(0, 3, (50, 40))
+    for eps in (1e-3, 0.1):
+        c0, _ = O.confidence(l, 39)
+        c1, _ = O.confidence(l + rng.uniform(-eps, eps, l.shape), 39)
+        ok = O.top2_gap(l, 39) > 2 * eps                                   # same greedy token on both sides
+        d = np.abs(O.conf_logit(c1.astype(np.float64)) - O.conf_logit(c0.astype(np.float64)))
+        assert (d[ok] <= 2 * eps * (1 + 1e-3) + 1e-6).all()
+
+
+def test_walk_diagnostics_on_the_worked_example():
+    """The six-position example above: chain 0 -> {r1} -> {r1, r2}; p1, p5, p3 committed, p4 left."""
+    n = -1.0
+    masked = np.array([0, 1, 0, 1, 1, 1], bool)
+    conf = np.array([[n, .92, n, .50, .20, .85],
+                     [n, n, n, .60, .25, .91],
+                     [n, .3, n, .1, .1, n],
+                     [n, n, n, .95, .30, n]], np.float32)
+    gaps = np.full((4, 6), 5.0)
+    gaps[0, 1], gaps[1, 5], gaps[3, 3], gaps[3, 4], gaps[0, 3] = 1.0, 0.7, 2.0, 0.9, 0.01
+    d = O.walk_diagnostics(conf, gaps, masked, S1, [1, 5], [0, 1, 3], {1: 11, 5: 15, 3: 13}, 0.9, 2)
+    # closest confidence decision: .91 against tau in copy {r1} (its own fill p1 is not masked there)
+    assert d["margin"] == pytest.approx(0.01 / 0.9, rel=1e-3)
+    assert d["sep"] == pytest.approx(float(O.conf_logit(.91) - O.conf_logit(.9)), rel=1e-3)
+    # tokens used: p1 in copy 0, p5 in copy {r1}, p3 in the last copy and the next candidate p4 there;
+    # the near-tie of p3's token in copy 0 (gap .01) is not used: p3 is not accepted there
+    assert d["tok_gap"] == 0.7
+    # with only the main block visited the closest decision is .92 against tau, and p1's token the one used,
+    # next candidates ranked from copy 0: p5 (.85), p3 (.50) -> p3's token there now counts
+    d0 = O.walk_diagnostics(conf, gaps, masked, S1, [1, 5], [0], {1: 11}, 0.9, 2)
+    assert d0["margin"] == pytest.approx(0.02 / 0.9, rel=1e-3) and d0["tok_gap"] == 0.01
