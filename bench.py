@@ -38,6 +38,18 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def recorded_layer_traffic():
+    """DRAM bytes (read + written) of the GEMM launches of one decode step of ONE 8B-shaped layer with 32 rows, as
+    the ncu capture summarised in profiles/ recorded them; None if the summary is not there."""
+    import re
+    path = os.path.join(ROOT, "profiles", "gemm_kernel_cfg2_layer_c1.md")
+    try:
+        m = re.search(r"dram_bytes_per_layer_step:\s*([0-9.eE+]+)", open(path).read())
+        return float(m.group(1)) if m else None
+    except OSError:
+        return None
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
 
@@ -127,6 +139,7 @@ def oracle_sample(wl, budget_layers=2):
     t_block = t_refresh + (Bk - 1) * t_step
     cores = len(os.sched_getaffinity(0)) if hasattr(os, "sched_getaffinity") else os.cpu_count()
     return {"tokens_per_s": Bk / t_block, "t_step_s": t_step, "t_refresh_s": t_refresh, "cores": cores,
+            "extrapolated": True, "measured_s": t_refresh_layers + t_step_layers + t_lm_step,
             "sample": f"{nl} of {shape.n_layers} layers of one refresh (T={T}) and one block step (M={len(subsets) * Bk}) "
                       f"in fp32 + LM head of the step rows, layer time scaled x{scale:g}; block cycle = 1 refresh + {Bk - 1} steps"}
 
@@ -146,7 +159,9 @@ def run_reference(args, wl):
             "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic", "config": config_of(wl),
             "cpu_baseline": {"value": v, "unit": UNIT, "cores": vals[-1]["cores"], "kind": "oracle",
-                             "sample": vals[-1]["sample"]},
+                             "sample": vals[-1]["sample"], "extrapolated": True,
+                             "measured_s_per_step": float(np.mean([r["measured_s"] for r in vals]))},
+            "extrapolated": True,   # ms_per_step is the block cycle estimated from the sample, not a block cycle run in full
             "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line))
 
@@ -340,27 +355,36 @@ def run_cuda(args, wl):
     gemm_bytes = nl * (3 * d * d + d * d + 2 * F * d + d * F) * 2 + (V * d * 2 if wl.with_lm_head else 0)
     gemm_launches = max(n_step["gemm"], 1)
     gemm_ms = ms_step["gemm"] / max(n_prof, 1)                # per decode step
-    achieved = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else None
+    gemm_gbs = gemm_bytes / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else None
     step_med = float(np.median(step_ms)) if step_ms else None
+    step_gbs = step_bytes / (step_med * 1e-3) / 1e9 if step_med else None
+    # the step is a READ stream; the measured peak is a read+write copy: a read-only probe in the same run
+    read_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}") if rank == 0 else None
+    layer_traffic = recorded_layer_traffic()
     rows = wl.batch * wl.block_len * wl.n_copies
-    bn = 32 if rows <= 32 else 64 if rows <= 64 else 128
-    roofline = {"bound": "hbm", "kernel": f"gemm_kernel<{bn}, *> (tcgen05 weight-streaming GEMM), all launches of one decode step",
-                "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": (achieved / peaks["hbm_gbs"]) if achieved else None, "peak_source": peaks["source"],
-                # DRAM bytes of the GEMM launches of one decode step: ncu capture of the four per-layer
-                # launches on the single-layer case (profiles/gemm_kernel_cfg2_layer_c1.md: 448.5 MB read +
-                # written per layer against 436.2 MB of weights), scaled by the layers; the LM-head launch
-                # is taken at its algorithmic bytes
-                "traffic": (nl * 448.5e6 + (V * d * 2 if wl.with_lm_head else 0)) if shape.d_model == 4096 and wl.n_copies == 1 else None,
-                "bytes_per_step": gemm_bytes, "launches_per_step": gemm_launches / max(n_prof, 1),
-                "ms_per_step": gemm_ms,
-                "decode_step": {"ms": step_med, "algorithmic_bytes": step_bytes,
-                                "achieved_gbs": step_bytes / (step_med * 1e-3) / 1e9 if step_med else None,
-                                "frac_of_measured": step_bytes / (step_med * 1e-3) / 1e9 / peaks["hbm_gbs"] if step_med else None,
-                                "frac_of_nominal_8tbs": step_bytes / (step_med * 1e-3) / 1e9 / 8000.0 if step_med else None,
-                                "ms_in_resident_loop": loop_ms,
-                                "frac_of_measured_in_resident_loop": step_bytes / (loop_ms * 1e-3) / 1e9 / peaks["hbm_gbs"] if loop_ms else None,
-                                "ms_by_kind": {k: v / max(n_prof, 1) for k, v in ms_step.items()}},
+    frac_of = lambda gbs, peak: (gbs / peak) if (gbs and peak) else None
+    roofline = {"bound": "hbm",
+                "kernel": "one decode step = every kernel of one odb_block_decode_step (weights once + visible K/V once)",
+                "achieved": step_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": frac_of(step_gbs, peaks["hbm_gbs"]),
+                "peak_source": peaks["source"],
+                "definition": "algorithmic bytes of a step / median device time of a whole step (enqueue to completion, CUDA "
+                              "events on the session's stream, nothing instrumented) / MEASURED_PEAKS.json hbm_gbs (a "
+                              "read+write copy)",
+                "algorithmic_bytes": step_bytes, "ms": step_med, "rows": rows,
+                "frac_of_nominal_8tbs": frac_of(step_gbs, 8000.0),
+                "hbm_read_gbs": read_gbs, "frac_of_read_probe": frac_of(step_gbs, read_gbs),
+                "ms_in_resident_loop": loop_ms,
+                "frac_in_resident_loop": frac_of(step_bytes / (loop_ms * 1e-3) / 1e9 if loop_ms else None, peaks["hbm_gbs"]),
+                # DRAM bytes of a step: the ncu capture of the single-layer case recorded under profiles/ (the full
+                # model holds 33 GB on the device: too large to capture), x layers + the LM head's weight bytes
+                "traffic": (nl * layer_traffic + (V * d * 2 if wl.with_lm_head else 0))
+                if (layer_traffic and shape.d_model == 4096 and rows == 32) else None,
+                "traffic_source": "recorded ncu capture (profiles/), scaled by the layer count; not a measurement of this run",
+                "gemm_only": {"definition": "weight bytes of the GEMM launches of one step / their summed device time with an "
+                                            "event pair around EVERY launch (serialises the launches: pessimistic)",
+                              "achieved": gemm_gbs, "frac": frac_of(gemm_gbs, peaks["hbm_gbs"]), "bytes_per_step": gemm_bytes,
+                              "launches_per_step": gemm_launches / max(n_prof, 1), "ms_per_step": gemm_ms},
+                "ms_by_kind": {k: v / max(n_prof, 1) for k, v in ms_step.items()},
                 "refresh": {"ms_by_kind": ms_refresh, "T": T}}
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -404,17 +428,151 @@ def run_cuda(args, wl):
             modes[mode]["nfe_vs_fast_dllm"] = modes[mode]["nfe"] / modes["fast_dllm"]["nfe"]
             modes[mode]["eff_nfe_vs_fast_dllm"] = modes[mode]["eff_nfe"] / modes["fast_dllm"]["eff_nfe"]
         line["modes"] = modes
+    if rank == 0 and world == 1 and args.workload == "cfg3_8b_c1" and not args.no_secondary:
+        line["secondary"] = secondary_measurements(E, synth, gm, peaks, args)
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             r = oracle_sample(wl)
             line["cpu_baseline"] = {"value": r["tokens_per_s"], "unit": UNIT, "cores": r["cores"], "kind": "oracle",
-                                    "sample": r["sample"], "t_step_s": r["t_step_s"], "t_refresh_s": r["t_refresh_s"]}
+                                    "sample": r["sample"], "t_step_s": r["t_step_s"], "t_refresh_s": r["t_refresh_s"],
+                                    "extrapolated": True, "measured_s": r["measured_s"]}
         print(json.dumps(line))
     sess.close()
     gm.close()
     if dist:
         dist.barrier()
         dist.destroy_process_group()
+
+
+def secondary_measurements(E, synth, gm, peaks, args):
+    """The other configurations the metric names, in the same process after the headline: the 4-copy workload on the
+    same weights (block cycle tokens/s and its 128-row decode step), and the single-layer decode step with 1 and 4
+    copies (L2 flushed before every step)."""
+    import torch
+    out = {}
+    # ---- 4 copies, prompt 512 + response 512, same weights, a session of its own ----
+    wl4 = synth.WORKLOADS["cfg4_8b_c4"]
+    T4 = wl4.prompt_len + wl4.gen_len
+    gm4 = E.Model(wl4.shape, gm.t, max_batch=1, max_seq=T4, max_block=wl4.block_len, max_copies=4)
+    s4 = E.Session(gm4)
+    p4 = E.DecodeParams(block_len=wl4.block_len, n_copies=4)
+    x4 = synth.sequence(0, 0, wl4.prompt_len, wl4.gen_len, wl4.shape)
+
+    def cycle(block):
+        s4.refresh_prefill(p4, block)
+        res = s4.unmask_accept(p4, True)
+        toks, its = res[0].n_accepted, 1
+        while res[0].masks_left > 0:
+            for res in (s4.decode_block_resident(p4) if not args.host_loop else [(s4.block_decode_step(p4), s4.unmask_accept(p4, False))[1]]):
+                toks += res[0].n_accepted
+                its += 1
+        return toks, its
+
+    s4.set_sequence(0, x4, wl4.prompt_len)
+    cycle(0)                                                   # warm-up (records the loop graphs of the shapes met)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(s4.stream)
+    toks = its = 0
+    for blk in range(1, 4):
+        t_, i_ = cycle(blk)
+        toks += t_; its += i_
+    b.record(s4.stream)
+    torch.cuda.synchronize()
+    ms4 = a.elapsed_time(b)
+    # the 128-row step on its own
+    s4.set_sequence(0, x4, wl4.prompt_len)
+    s4.refresh_prefill(p4, 0)
+    res = s4.unmask_accept(p4, True)
+    steps = []
+    for _ in range(8):
+        if res[0].masks_left <= 0:
+            break
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(s4.stream)
+        s4.block_decode_step(p4)
+        e1.record(s4.stream)
+        res = s4.unmask_accept(p4, False)
+        steps.append(e0.elapsed_time(e1))
+    bytes4 = gm4.step_algorithmic_bytes(T4 - wl4.block_len)
+    st4 = float(np.median(steps)) if steps else None
+    out["cfg4_8b_c4"] = {"tokens_per_s": toks / (ms4 * 1e-3), "block_cycles": 3, "iterations_per_block": its / 3,
+                         "step_rows": 4 * wl4.block_len, "step_ms": st4, "step_algorithmic_bytes": bytes4,
+                         "step_frac_of_measured": (bytes4 / (st4 * 1e-3) / 1e9 / peaks["hbm_gbs"]) if st4 else None}
+    s4.close(); gm4.close()
+    # ---- one 8B-shaped layer, context 512, block 32: the decode step with 1 and 4 copies ----
+    shape1 = synth.LLADA_8B.with_layers(1)
+    wl1 = synth.WORKLOADS["cfg2_layer_c1"]
+    T1 = wl1.prompt_len + wl1.gen_len
+    gm1 = E.Model.from_synth(shape1, seed=0, with_lm_head=False, max_batch=1, max_seq=T1, max_block=wl1.block_len, max_copies=4)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for name, copies in (("cfg2_layer_c1", 1), ("cfg2_layer_c4", 4)):
+        s1 = E.Session(gm1)
+        p1 = E.DecodeParams(block_len=wl1.block_len, n_copies=copies)
+        s1.set_sequence(0, synth.sequence(0, 0, wl1.prompt_len, wl1.gen_len, shape1), wl1.prompt_len)
+        s1.refresh_prefill(p1, 0)
+        s1.unmask_accept(p1, True)
+        times = []
+        for i in range(3 + 12):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(s1.stream)
+            s1.block_decode_step(p1)
+            e1.record(s1.stream)
+            s1.unmask_accept(p1, False)
+            if i >= 3:
+                times.append(e0.elapsed_time(e1))
+        ms1 = float(np.median(times))
+        b1 = gm1.step_algorithmic_bytes(T1 - wl1.block_len)
+        out[name] = {"step_us": ms1 * 1e3, "rows": copies * wl1.block_len, "algorithmic_bytes": b1,
+                     "frac_of_measured": b1 / (ms1 * 1e-3) / 1e9 / peaks["hbm_gbs"], "l2": "flushed before every step"}
+        s1.close()
+    gm1.close()
+    return out
+
+
+def run_persistent_phases(args, wl):
+    """Where the time of the persistent decode-step kernel goes: mean duration of every phase between two grid
+    barriers (from the release of the previous barrier to the last CTA's arrival at the next), and the barrier's
+    own latency (last arrival to release), over the layers of one step.  Prints one JSON line."""
+    os.environ["ODB_PERSISTENT"] = "1"
+    os.environ["ODB_PERSISTENT_TIMING"] = "1"
+    import torch
+    import synth
+    import __graft_entry__ as G
+    from paper_2511_21759_b200 import engine as E
+    G.build()
+    shape, T = wl.shape, wl.prompt_len + wl.gen_len
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=T, max_block=wl.block_len, max_copies=max(wl.n_copies, 1))
+    sess = E.Session(gm)
+    sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape), wl.prompt_len)
+    gp = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies)
+    sess.refresh_prefill(gp, 0)
+    sess.unmask_accept(gp, True)
+    step_ms = []
+    for _ in range(args.warmup + args.steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(sess.stream)
+        sess.block_decode_step(gp)
+        b.record(sess.stream)
+        sess.unmask_accept(gp, False)
+        step_ms.append(a.elapsed_time(b))
+    n_cta = torch.cuda.get_device_properties(0).multi_processor_count
+    ks = max(1, min(8, n_cta // (wl.n_copies * shape.n_heads)))
+    names = ["norm1", "qkv", "rope", "attention"] + (["merge"] if ks > 1 else []) + ["o", "norm2", "gate_up", "swiglu", "down"]
+    nb = len(names)
+    t = sess.persistent_barrier_times(n_cta, shape.n_layers * nb + 1)
+    arr, rel = t[:, :, 0], t[:, :, 1]
+    last_arr, last_rel = arr.max(0), rel.max(0)
+    phases = {}
+    for j, n in enumerate(names):
+        ids = [l * nb + j for l in range(1, shape.n_layers)]
+        phases[n] = {"us": float(np.mean([last_arr[i] - last_rel[i - 1] for i in ids])) / 1e3,
+                     "barrier_us": float(np.mean([last_rel[i] - last_arr[i] for i in ids])) / 1e3}
+    print(json.dumps({"kernel": "step_persistent_kernel", "workload": wl.name, "ctas": n_cta, "key_splits": ks,
+                      "step_ms": float(np.median(step_ms[args.warmup:])),
+                      "per_layer_us": float(sum(v["us"] + v["barrier_us"] for v in phases.values())), "phases": phases}))
+    sess.close(); gm.close()
 
 
 def run_layer_microbench(args, wl):
@@ -493,16 +651,31 @@ def main():
     ap.add_argument("--workload", default="cfg3_8b_c1")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the secondary object (4-copy workload and single-layer steps measured after the headline)")
     ap.add_argument("--host-loop", action="store_true",
                     help="take every iteration of a block as odb_block_decode_step + odb_unmask_accept from the host instead "
                          "of odb_decode_block_resident (one host round trip per iteration instead of one per change of the "
                          "step's shape)")
+    ap.add_argument("--persistent-phases", action="store_true",
+                    help="run decode steps through the persistent step kernel and print the mean time of each of its phases")
     ap.add_argument("--modes", action="store_true",
                     help="also run the whole response as cache-less baseline / DualCache block decoding / full method")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # not under a launcher: start the N local ranks (one process per GPU) and pass their output through
+        import socket
+        with socket.socket() as so:
+            so.bind(("127.0.0.1", 0))
+            port = so.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+               "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        raise SystemExit(subprocess.call(cmd))
     import synth
     wl = synth.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.persistent_phases:
+        run_persistent_phases(args, wl)
+    elif args.impl == "reference":
         run_reference(args, wl)
     elif not wl.with_lm_head:
         run_layer_microbench(args, wl)

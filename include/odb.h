@@ -249,8 +249,16 @@ int32_t odb_debug_expire_wait(odb_session* s, int64_t limit_cycles);
  * (needs the logit dump);
  * 1 conf fp32 [rows]; 2 tok int32 [rows]; 3 residual stream fp32 [rows][d_model]; 4 q, 5 k,
  * 6 v bf16 [rows][d_model] of the LAST layer; 7 attention output bf16 [rows][d_model];
- * 8 row tokens int32 [rows]; 9 row positions int32 [rows]; 10 row copy ids int32 [rows].
- * *rows gets the row count of that buffer.  Synchronous. */
+ * 8 row tokens int32 [rows]; 9 row positions int32 [rows]; 10 row copy ids int32 [rows];
+ * 11 the raw timing words of the persistent step kernel (see ODB_PERSISTENT_TIMING below; up to cap_bytes).
+ * *rows gets the row count of that buffer.  Synchronous.
+ *
+ * Environment switches of the decode step, read once per process: ODB_PERSISTENT=1 runs a step of up to 128 rows
+ * as ONE cooperative launch (all projections, the short phases between them and the LM head's statistics; same
+ * results to rounding order, measured slower than the separate kernels, off by default); with it,
+ * ODB_PERSISTENT_TIMING=1 records per CTA the global-timer value at which it arrived at and was released from
+ * every grid barrier of the step: uint64 [CTAs][barriers][2] in the logits buffer, 10 barriers per layer (9
+ * without key splits) and one before the LM head. */
 int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap_bytes, int32_t* rows);
 
 /* out[M][N] (fp32, device) = x[M][K] (bf16, device) * w[N][K]^T (PACKED bf16, device) with the
@@ -295,6 +303,13 @@ int32_t odb_gemm_static_scratch(const void* x, const void* w_packed, float* out,
  * Launches are counted whether profiling is on or off. */
 int32_t odb_session_profile(odb_session* s, int32_t enable);
 int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* launches_by_kind);
+
+/* Measurement: the rate at which this GPU streams `bytes` (a multiple of 16, 16-byte aligned, at least 1 MiB; use
+ * far more than the L2 holds) of device memory with a read-only kernel of 16-byte loads, `reps` passes after one
+ * warm-up pass, timed with CUDA events on `stream`.  The decode step is a read stream (weights and K/V are read
+ * once, almost nothing is written), so this is the ceiling it is measured against beside the copy bandwidth.
+ * Synchronous. */
+int32_t odb_measure_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s);
 
 /* Algorithmic bytes one odb_block_decode_step must move for `rows` query rows and `keys`
  * visible cached positions per sequence (weights once + K/V once); used by the benchmark. */

@@ -365,7 +365,29 @@ __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial
     }
 }
 
+// Read-only streaming probe: every thread reads 16-byte vectors grid-stride over the buffer and folds them into
+// one word, written out only if it has an (impossible) value, so that the loads cannot be removed.
+__global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restrict__ src, size_t n_vec, unsigned int* sink) {
+    const size_t stride = static_cast<size_t>(gridDim.x) * blockDim.x;
+    unsigned int acc = 0;
+    size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    for (; i + 3 * stride < n_vec; i += 4 * stride) {
+        const uint4 a = __ldcs(src + i), b = __ldcs(src + i + stride), c = __ldcs(src + i + 2 * stride), d = __ldcs(src + i + 3 * stride);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w ^ b.x ^ b.y ^ b.z ^ b.w ^ c.x ^ c.y ^ c.z ^ c.w ^ d.x ^ d.y ^ d.z ^ d.w;
+    }
+    for (; i < n_vec; i += stride) {
+        const uint4 a = __ldcs(src + i);
+        acc ^= a.x ^ a.y ^ a.z ^ a.w;
+    }
+    if (acc == 0x9E3779B9u && sink) atomicAdd(sink, 1u);
+}
+
 }  // namespace
+
+cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned int* sink, int grid, cudaStream_t st) {
+    read_stream_kernel<<<grid, 512, 0, st>>>(static_cast<const uint4*>(src), bytes / 16, sink);
+    return cudaGetLastError();
+}
 
 // First kernel of a forward.  Launched WITHOUT programmatic stream serialization: it starts only when
 // everything enqueued before it (the row and tile tables, the previous accept) has completed, and every

@@ -154,6 +154,8 @@ struct odb_session {
     cudaStream_t record_st;
     odb_result* pinned_log;   // [kMaxLoopIters][max_batch]
     int32_t* pinned_iters;    // [0] iterations run (written by the device); [1..3] the loop words of the next launch
+    int pmaxp[4];             // persistent step kernel: most parts per output tile of the four projections of a layer
+    bool persistent_off;      // the model is beyond the persistent step kernel's limits: steps run as separate kernels
     bool ptable_built[3];     // persistent step kernel: projection table for 32 / 64 / 128 rows per tile is on the device
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
@@ -283,6 +285,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->pinned_log = nullptr;
     s->pinned_iters = nullptr;
     s->ptable_built[0] = s->ptable_built[1] = s->ptable_built[2] = false;
+    s->persistent_off = false;
     cudaError_t e = cudaMallocHost(&s->pinned_state, sizeof(SeqState) * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_log, sizeof(odb_result) * kMaxLoopIters * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_iters, 4 * sizeof(int32_t));
@@ -457,7 +460,7 @@ int bn_index(int M) { return M <= 32 ? 0 : M <= 64 ? 1 : 2; }
 // Whether a decode step of M rows runs as the persistent kernel (one cooperative launch for the whole forward).
 bool use_persistent(const odb_session* s, int M) {
     const odb_config& c = s->m->cfg;
-    return step_persistent_supported(M, c.d_model, c.d_ffn, c.head_dim);
+    return !s->persistent_off && step_persistent_supported(M, c.d_model, c.d_ffn, c.head_dim);
 }
 
 // The persistent kernel reads its projections (weight and operand tensor maps, split) from a table in the
@@ -486,6 +489,15 @@ int32_t ensure_ptable(odb_session* s, int M) {
         step_persistent_fill_desc(t[4 * c.n_layers], m->tm_lm, tx_a, m->final_norm, (c.vocab + 127) / 128, kb_d, 1, grid);
     else
         step_persistent_fill_desc(t[4 * c.n_layers], m->tm_o[0], tx_a, m->final_norm, 1, 1, 0, grid);   // unused slot
+    for (int j = 0; j < 4; ++j) {
+        s->pmaxp[j] = step_persistent_max_parts(t[j]);
+        if (s->pmaxp[j] > 8 || t[j].n_tiles > 256) t[j].g_use = 0;   // beyond the kernel's fixed tables
+    }
+    for (const PGemmDesc& pd : t)
+        if (pd.g_use < 1) {   // a projection too large for the kernel's unit arithmetic: keep the separate kernels
+            s->persistent_off = true;
+            return ODB_OK;
+        }
     uint8_t* dst = s->ws + L.ptable + bi * align_up(step_persistent_table_bytes(c.n_layers));
     ODB_CUDA(cudaStreamSynchronize(s->st));
     ODB_CUDA(cudaMemcpy(dst, t.data(), sizeof(PGemmDesc) * t.size(), cudaMemcpyHostToDevice));
@@ -549,6 +561,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         pa.n_layers = c.n_layers; pa.M = M;
         pa.d = d; pa.F = F; pa.H = H; pa.hd = hd; pa.vocab = c.vocab; pa.mask_id = c.mask_id; pa.with_lm = (c.with_lm_head && !s->dump_logits) ? 1 : 0;
         pa.rms_eps = c.rms_eps;
+        for (int j = 0; j < 4; ++j) pa.maxp[j] = s->pmaxp[j];
         pa.embed = m->embed;
         pa.row_tok = s->cb.row_tok; pa.row_pos = s->cb.row_pos; pa.row_flags = s->cb.row_flags;
         pa.h = h; pa.a = a; pa.ssq = inv;
@@ -566,6 +579,9 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         pa.conf_part = reinterpret_cast<ConfPartial*>(s->ws + L.conf_part);
         pa.bars = s->at<unsigned int>(L.pbars);
         pa.status = status;
+        // measurement: per-CTA arrival / release times of every grid barrier, kept in the (unused) logits buffer
+        static const bool ptiming = getenv("ODB_PERSISTENT_TIMING") && getenv("ODB_PERSISTENT_TIMING")[0] == '1';
+        pa.timing = (ptiming && c.with_lm_head && !s->dump_logits) ? s->at<unsigned long long>(L.logits) : nullptr;
         ODB_CUDA(step_persistent_configure(pa));
         ODB_LAUNCH(ODB_KIND_GEMM, launch_step_persistent(pa, st));
         if (pa.with_lm) {
@@ -932,9 +948,11 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap, in
         case 8: off = L.row_tok; bytes = 4 * M; break;
         case 9: off = L.row_pos; bytes = 4 * M; break;
         case 10: off = L.row_copy; bytes = 4 * M; break;
+        case 11: off = L.logits; n = 1; bytes = cap < 4 * L.lm_chunk * c.vocab ? cap : 4 * L.lm_chunk * c.vocab; break;   // raw timing words
         default: return ODB_ERR_ARG;
     }
     if (which == 0 && (!c.with_lm_head || !s->dump_logits)) return ODB_ERR_STATE;
+    if (which == 11 && !c.with_lm_head) return ODB_ERR_STATE;
     if (cap < bytes) return ODB_ERR_WORKSPACE;
     ODB_CUDA(cudaStreamSynchronize(s->st));
     ODB_CUDA(cudaMemcpy(host, s->ws + off, bytes, cudaMemcpyDeviceToHost));
@@ -1005,6 +1023,30 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
         if (cudaEventElapsedTime(&ms, s->ev[i], s->ev[i + 1]) == cudaSuccess) ms_by_kind[s->ev_kind[i / 2]] += ms;
     }
     s->ev_used = 0;
+    return ODB_OK;
+}
+
+int32_t odb_measure_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s) {
+    if (!buf || !gb_per_s || reps < 1 || bytes < (1u << 20)) return ODB_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(buf) & 15) || (bytes & 15)) return ODB_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int dev = 0, sms = 0;
+    ODB_CUDA(cudaGetDevice(&dev));
+    ODB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    ODB_CUDA(cudaEventCreate(&e0));
+    cudaError_t e = cudaEventCreate(&e1);
+    if (e == cudaSuccess) e = launch_read_stream(buf, bytes, nullptr, 4 * sms, st);   // warm-up pass
+    if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+    for (int i = 0; i < reps && e == cudaSuccess; ++i) e = launch_read_stream(buf, bytes, nullptr, 4 * sms, st);
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *gb_per_s = static_cast<double>(bytes) * reps / (static_cast<double>(ms) * 1e-3) / 1e9;
     return ODB_OK;
 }
 

@@ -227,6 +227,8 @@ cudaError_t launch_gemm(const GemmArgs& a, cudaStream_t st);
 cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stride, float* out, size_t n,
                                    cudaStream_t st);
 
+// read-only streaming kernel over `bytes` of src (a multiple of 16), `grid` blocks of 512 threads
+cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned int* sink, int grid, cudaStream_t st);
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d,
                          cudaStream_t st);
 // The part of RMSNorm that is not a row scalar, for rows r = map ? map[i] : i of the residual stream:
@@ -312,6 +314,8 @@ struct alignas(64) PGemmDesc {   // one projection of the step; an array of thes
 struct StepPersistentArgs {
     const PGemmDesc* gemms;      // [4 * n_layers (qkv, o, gate/up, down per layer) + with_lm]
     int n_layers, M, BN, stages, scratch_bytes;
+    int maxp[4];                 // most parts any output tile of the layer's four projections has
+    int l2_ahead;                // weight tiles the producer asks L2 for ahead of the one it loads into shared memory
     int d, F, H, hd, vocab, mask_id, with_lm;
     float rms_eps;
     const __nv_bfloat16* embed;
@@ -327,6 +331,7 @@ struct StepPersistentArgs {
     unsigned int* bars;          // one word per grid barrier, zero when the kernel starts
     int n_bars;
     int* status;
+    unsigned long long* timing;  // measurement only (null: off): [cta][barrier][arrived, passed] global timer in ns
 };
 // bytes of the PGemmDesc table and of the barrier words for a model of n_layers layers
 size_t step_persistent_table_bytes(int n_layers);
@@ -339,6 +344,8 @@ cudaError_t step_persistent_configure(StepPersistentArgs& a);
 int step_persistent_grid();
 void step_persistent_fill_desc(PGemmDesc& d, const CUtensorMap& tmap_w, const CUtensorMap& tmap_x, const float* gain, int n_tiles,
                                int nkb, int conf, int grid);
+// most parts an output tile of this projection has under the kernel's split
+int step_persistent_max_parts(const PGemmDesc& d);
 // zeroes the barrier words and launches the kernel (cooperative, one CTA per SM) on st
 cudaError_t launch_step_persistent(const StepPersistentArgs& a, cudaStream_t st);
 

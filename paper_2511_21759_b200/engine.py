@@ -200,6 +200,14 @@ class Session:
         B.check(B.lib().odb_session_profile_read(self.handle, ms, n), "odb_session_profile_read")
         return dict(zip(B.KINDS, list(ms))), dict(zip(B.KINDS, list(n)))
 
+    def persistent_barrier_times(self, n_ctas: int, n_barriers: int) -> np.ndarray:
+        """[CTA][barrier][arrived, released] global-timer values (ns) of the last persistent step (needs
+        ODB_PERSISTENT=1 and ODB_PERSISTENT_TIMING=1 in the environment when the library was loaded)."""
+        buf = np.zeros(n_ctas * n_barriers * 2, dtype=np.uint64)
+        rows = C.c_int32()
+        B.check(B.lib().odb_debug_read(self.handle, 11, buf.ctypes.data, buf.nbytes, C.byref(rows)), "odb_debug_read")
+        return buf.reshape(n_ctas, n_barriers, 2).astype(np.int64)
+
     _READ = {"logits": (0, np.float32), "conf": (1, np.float32), "tok": (2, np.int32), "hidden": (3, np.float32),
              "q": (4, np.uint16), "k": (5, np.uint16), "v": (6, np.uint16), "o": (7, np.uint16),
              "row_tok": (8, np.int32), "row_pos": (9, np.int32), "row_copy": (10, np.int32)}
@@ -230,6 +238,17 @@ def debug_gemm(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Ten
     B.check(B.lib().odb_debug_gemm(x.data_ptr(), w.data_ptr(), out.data_ptr(), scratch.data_ptr(), scratch.numel(),
                                    M, N, K, k_splits, C.c_void_p(st.cuda_stream)), "odb_debug_gemm")
     return out
+
+
+def measure_read_bandwidth(n_bytes: int = 4 << 30, reps: int = 4, device="cuda") -> float:
+    """GB/s of a read-only streaming kernel over a buffer of n_bytes (odb_measure_read_bandwidth)."""
+    buf = torch.empty(n_bytes, dtype=torch.uint8, device=device)
+    buf.fill_(1)
+    st = torch.cuda.current_stream(buf.device)
+    out = C.c_double()
+    B.check(B.lib().odb_measure_read_bandwidth(buf.data_ptr(), buf.numel(), reps, C.c_void_p(st.cuda_stream), C.byref(out)),
+            "odb_measure_read_bandwidth")
+    return out.value
 
 
 def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Tensor:

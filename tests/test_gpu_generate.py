@@ -48,8 +48,16 @@ def _run_both(wl_name, *, seed=0, schedule=None, params_kw=None, shape=None, x0=
     measured = None
     if div is not None and div["gpu"] is not None:
         sess.set_sequence(0, x0, wl.prompt_len)
+        # the replay takes the same kernels as the free run (LM head fused with the confidence reduction)
         st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw),
-                               schedule=schedule, tol=1.0, max_iters=div["iter"] + 1)
+                               schedule=schedule, tol=1.0, max_iters=div["iter"] + 1, check_logits=False)
+        g, o = div["gpu"], div["oracle"]
+        if [p_ for p_, _ in g["accepted"]] == [p_ for p_, _ in sorted(o["accepted"])] and g["chain"] == o["chain"]:
+            # same positions, another greedy token: replayed once more with the logits materialised, which asserts
+            # that every differing token sits on a top-2 logit gap below twice the logit error
+            sess.set_sequence(0, x0, wl.prompt_len)
+            st = lockstep_generate(E, sess, om, x0, wl.prompt_len, E.DecodeParams(**kw), O.DecodeParams(**kw),
+                                   schedule=schedule, tol=1.0, max_iters=div["iter"] + 1)
         measured = st
     sess.close(); gm.close()
     return gtok[0], gtrace, otok, otrace, measured
