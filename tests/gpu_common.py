@@ -56,7 +56,7 @@ def compare_traces(gpu_trace, oracle_trace, seq=0, near_tie=1e-3):
 
 
 def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, check_logits=True, max_iters=None,
-                      seq=0, cache_blocks=True):
+                      seq=0, cache_blocks=True, dtype=np.float64, l2_tol=None, stop=None):
     """Lock-step parity harness for one sequence.
 
     Every iteration both sides start from the same state.  (1) Numerics: the GPU's logits /
@@ -68,7 +68,8 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
     oracle's decision margin must be below the confidence error measured in that iteration (a
     near-tie); these are counted and returned, never hidden.  The GPU's decision then advances
     both sides.  cache_blocks=False runs the cache-less baseline (every iteration a refresh).
-    Returns a stats dict."""
+    dtype: the oracle's arithmetic (float32 for the 8B shape); l2_tol: also bound the worst per-row relative L2
+    error of the logits; stop(stats) -> True ends the run after an iteration.  Returns a stats dict."""
     sess.set_logit_dump(check_logits)                   # logits are only materialised in the test mode
     shape_mask, eos = om.mask_id, om.eos_id
     Bk, tau = op.block_len, op.accept_threshold
@@ -76,7 +77,7 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
     x = np.array(x0, dtype=np.int64)
     T = len(x)
     st = {"iters": 0, "refreshes": 0, "steps": 0, "tokens": 0, "oracle_decision_diff": 0, "near_ties": [],
-          "worst_logit": 0.0, "worst_conf": 0.0, "tok_diff": 0, "log": []}
+          "worst_logit": 0.0, "worst_conf": 0.0, "tok_diff": 0, "log": [], "worst_l2": 0.0, "stage2_steps": 0}
 
     def record(kind, diag, rows, g_conf, o_conf, g_logits, o_logits):
         """Per iteration: the oracle's distance from flipping (walk_diagnostics) beside the errors measured on the
@@ -96,6 +97,10 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
             ok, worst = logits_close(g_logits, o_logits, tol)
             st["worst_logit"] = max(st["worst_logit"], worst)
             assert ok, f"logits off by {worst:.2f} x bound at iteration {st['iters']}"
+            if l2_tol is not None:
+                l2 = rel_l2(g_logits, o_logits)
+                st["worst_l2"] = max(st["worst_l2"], l2)
+                assert l2 <= l2_tol, f"per-row relative L2 error {l2:.3e} at iteration {st['iters']}"
             l32 = o_logits.astype(np.float32).astype(np.float64)
             l32[:, shape_mask] = -np.inf
             top2 = np.partition(l32, -2, axis=1)[:, -2:]
@@ -118,7 +123,7 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
         sess.refresh_prefill(gp, b)
         g_conf, g_tok = sess.debug_read("conf"), sess.debug_read("tok")
         g_logits = sess.debug_read("logits") if check_logits else None
-        out = O.refresh_prefill(om, x, T, s, return_logits=True)
+        out = O.refresh_prefill(om, x, T, s, return_logits=True, dtype=dtype)
         cache, o_conf, o_tok, o_logits = out
         assert len(g_conf) == T - s
         cerr = numerics(g_conf, g_tok, g_logits, o_conf, o_tok, o_logits)
@@ -170,7 +175,8 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
             st2 = O.use_stage2(op, B, int((~masked).sum()))
             subsets = O.copy_subsets(len(ranks), 4 if (op.n_copies == 8 and not st2) else op.n_copies, st2)
             o_c, o_t, o_logits, r_copy, r_pos = O.block_decode_step(om, cache, x, T, s, e, subsets, rank_pos,
-                                                                    rank_tok, st2, return_logits=True)
+                                                                    rank_tok, st2, return_logits=True, dtype=dtype)
+            st["stage2_steps"] += int(st2)
             _, _, r_tok = O.build_rows(x, s, e, shape_mask, subsets, rank_pos, rank_tok, st2)
             sess.block_decode_step(gp)
             assert np.array_equal(sess.debug_read("row_pos"), r_pos), "row positions"
@@ -204,6 +210,8 @@ def lockstep_generate(E, sess, om, x0, P, gp, op, *, schedule=None, tol=2e-2, ch
             st["iters"] += 1; st["steps"] += 1; st["tokens"] += len(want)
             assert res.masks_left == int((x[s:e] == shape_mask).sum())
             last_conf, last_tok = g_c[last], g_t[last]
+            if stop is not None and stop(st):
+                max_iters = st["iters"]
         b += 1
     st["tokens_final"] = x.astype(np.int32)
     return st
@@ -214,3 +222,15 @@ def assert_near_ties_only(st, floor=1e-3):
     decision margin no larger than four times the confidence error measured there (floor 1e-3)."""
     for it, kind, margin, cerr in st["near_ties"]:
         assert margin <= max(floor, 4 * cerr), f"iteration {it} ({kind}): margin {margin:.3e}, conf error {cerr:.3e}"
+
+
+def anchored_bounds(layers, n_elements):
+    """(per-row relative L2 bound, element-wise factor over the small-model bound) for a model of this depth, from
+    the oracle's measured distance between its own float32 and float64 runs (tests/golden/oracle_self_distance.py)."""
+    import importlib.util
+    import os
+    path = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "oracle_self_distance.py")
+    spec = importlib.util.spec_from_file_location("oracle_self_distance", path)
+    mod = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(mod)
+    return mod.l2_bound(layers), mod.elementwise_factor(layers, n_elements)

@@ -23,7 +23,7 @@ def _setup(shape, P, L, *, max_copies=8, seed=0, with_lm_head=True, block=16):
 
 
 @requires_gpu
-@pytest.mark.parametrize("shape_name", ["TINY", "TINY_PEAKY"])
+@pytest.mark.parametrize("shape_name", ["TINY", "TINY_PEAKY", "TINY_HD128"])
 def test_refresh_logits_conf_tok(shape_name):
     shape = getattr(synth, shape_name)
     P, L = 64, 64
@@ -34,8 +34,18 @@ def test_refresh_logits_conf_tok(shape_name):
     conf, tok = sess.debug_read("conf"), sess.debug_read("tok")
     cache, oconf, otok, ologits = O.refresh_prefill(om, x0, P + L, P, return_logits=True)
     assert logits.shape == ologits.shape == (L, shape.vocab)
-    ok, worst = logits_close(logits, ologits, 2e-2 if shape_name == "TINY" else 4e-2)
+    tol = 4e-2 if shape_name == "TINY_PEAKY" else 2e-2
+    ok, worst = logits_close(logits, ologits, tol)
     assert ok, worst
+    # and against the PLAIN definition (float64, nothing rounded to bf16 anywhere): parity does not rest on the
+    # oracle mode that rounds where the kernels round.  The benchmark spec's 2e-2 on the N(0, 0.02) models; the
+    # sharp-logit model's own bf16 mode is already 1.2 - 1.4 x 2e-2 away from its plain definition
+    # (tests/test_oracle_self_distance.py), hence 4e-2 there.
+    _, pconf, ptok, plogits = O.refresh_prefill(om, x0, P + L, P, return_logits=True, faithful=False)
+    ok_p, worst_p = logits_close(logits, plogits, tol)
+    print(f"\n{shape_name}: logits vs the bf16-faithful oracle {worst:.2f} x, vs the plain float64 definition {worst_p:.2f} x "
+          f"the bound of {tol:g}")
+    assert ok_p, worst_p
     # decisions: same greedy token unless the oracle's own top-2 logit gap is below the logit error
     l32 = ologits.astype(np.float32).astype(np.float64)
     l32[:, shape.mask_id] = -np.inf
@@ -44,7 +54,7 @@ def test_refresh_logits_conf_tok(shape_name):
     err = np.abs(logits - ologits).max(axis=1)
     bad = (tok != otok) & (gap > 2 * err)
     assert not bad.any()
-    assert np.allclose(conf, oconf, rtol=2e-2 if shape_name == "TINY" else 0.15)   # sharp logits: d(conf) ~ d(logit)
+    assert np.allclose(conf, oconf, rtol=0.15 if shape_name == "TINY_PEAKY" else 2e-2)   # sharp logits: d(conf) ~ d(logit)
     # the fresh K/V of the last layer and the K/V cache rows agree with the oracle to one bf16 step
     k = bf16_bits_to_f64(sess.debug_read("k")).reshape(P + L, shape.n_heads, shape.head_dim)
     v = bf16_bits_to_f64(sess.debug_read("v")).reshape(P + L, shape.n_heads, shape.head_dim)

@@ -11,10 +11,12 @@ of ~sqrt(delta * 2^-8): after three or four rounding points ANY two evaluation o
 fraction of a bf16 step in every activation, however close they started (the oracle's own float32
 and float64 runs do: 0.19 % rms in the residual stream after ONE 8B-shaped layer).  The logits of
 two correct implementations therefore differ by a few 1e-3 of their RMS per element, and the largest
-of 3.2e7 such differences sits 5-6 sigma out.  The 2e-2 figure is therefore applied to the per-row
-relative L2 error, and the element-wise check uses 6 x the small-model bound; on the 32-layer model
-the oracle's float32 and float64 runs differ from each other by about as much as the kernels differ
-from either (measured: 3.6 x vs 3.5 x the small-model bound at 16 layers).
+of 3.2e7 such differences sits 5-6 sigma out.  Both bounds used here are FUNCTIONS of the oracle's own
+distance between its float32 and float64 runs, measured by depth on the 8B shape
+(tests/golden/oracle_self_distance.py, checked on CPU by tests/test_oracle_self_distance.py): the
+per-row relative L2 bound is c * sqrt(layers) (1.99e-2 at 32 layers: the benchmark spec's 2e-2 is, at this
+depth, the distance between two correct evaluations) and the element-wise bound is sqrt(2 ln n) times
+that (5.9 x the small-model bound for the 3.2e7 logits of a refresh).
 Decisions are checked the lock-step way: the oracle's accept rule on the GPU's own confidences must
 give the GPU's accepted set; a differing oracle-side decision must be a measured near-tie.
 """
@@ -24,7 +26,7 @@ import pytest
 import synth
 from oracle import odb_oracle as O
 from oracle.inputs import model_from_synth
-from gpu_common import engine, requires_gpu, logits_close, rel_l2
+from gpu_common import engine, requires_gpu, logits_close, rel_l2, anchored_bounds
 
 
 @requires_gpu
@@ -64,9 +66,10 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
     assert g_logits.shape == o_logits.shape == (L, shape.vocab)
     l2_r = rel_l2(g_logits, o_logits)
-    assert l2_r <= 2e-2, f"refresh logits: per-row relative L2 error {l2_r:.3e}"
-    ok, worst_r = logits_close(g_logits, o_logits, 6 * 2e-2)
-    worst_r *= 6
+    l2_tol, factor = anchored_bounds(shape.n_layers, o_logits.size)
+    assert l2_r <= l2_tol, f"refresh logits: per-row relative L2 error {l2_r:.3e} (bound {l2_tol:.3e})"
+    ok, worst_r = logits_close(g_logits, o_logits, factor * 2e-2)
+    worst_r *= factor
     assert ok, f"refresh logits off by {worst_r:.2f} x the small-model bound"
     cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
     # control on the GPU's own numbers: bit exact
@@ -92,9 +95,9 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     o_c, o_t, os_logits, r_copy, r_pos = O.block_decode_step(om, cache, x, T, P, P + Bk, [()], [], [], False,
                                                              dtype=np.float32, return_logits=True)
     l2_s = rel_l2(s_logits, os_logits)
-    assert l2_s <= 2e-2, f"step logits: per-row relative L2 error {l2_s:.3e}"
-    ok, worst_s = logits_close(s_logits, os_logits, 6 * 2e-2)
-    worst_s *= 6
+    assert l2_s <= l2_tol, f"step logits: per-row relative L2 error {l2_s:.3e} (bound {l2_tol:.3e})"
+    ok, worst_s = logits_close(s_logits, os_logits, factor * 2e-2)
+    worst_s *= factor
     assert ok, f"step logits off by {worst_s:.2f} x the small-model bound"
     masked = x[P:P + Bk] == shape.mask_id
     acc = O.accept_set(s_conf, masked, wl.accept_threshold)
@@ -159,9 +162,10 @@ def test_cfg4_refresh_and_four_copy_step_match_oracle():
     om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
     cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
     l2_r = rel_l2(g_logits, o_logits[:Bk])
-    assert l2_r <= 2e-2, f"refresh logits: per-row relative L2 error {l2_r:.3e}"
-    ok, worst_r = logits_close(g_logits, o_logits[:Bk], 6 * 2e-2)
-    assert ok, f"refresh logits off by {6 * worst_r:.2f} x the small-model bound"
+    l2_tol, factor = anchored_bounds(shape.n_layers, L * shape.vocab)
+    assert l2_r <= l2_tol, f"refresh logits: per-row relative L2 error {l2_r:.3e} (bound {l2_tol:.3e})"
+    ok, worst_r = logits_close(g_logits, o_logits[:Bk], factor * 2e-2)
+    assert ok, f"refresh logits off by {factor * worst_r:.2f} x the small-model bound"
     cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
     masked = np.ones(Bk, dtype=bool)
     acc = O.accept_set(g_conf[:Bk], masked, tau)
@@ -180,9 +184,9 @@ def test_cfg4_refresh_and_four_copy_step_match_oracle():
     assert np.array_equal(r_copy, oc) and np.array_equal(r_pos, op), "row table"
     assert s_logits.shape == os_logits.shape == (4 * Bk, shape.vocab)
     l2_s = rel_l2(s_logits, os_logits)
-    assert l2_s <= 2e-2, f"step logits: per-row relative L2 error {l2_s:.3e}"
-    ok, worst_s = logits_close(s_logits, os_logits, 6 * 2e-2)
-    assert ok, f"step logits off by {6 * worst_s:.2f} x the small-model bound"
+    assert l2_s <= l2_tol, f"step logits: per-row relative L2 error {l2_s:.3e} (bound {l2_tol:.3e})"
+    ok, worst_s = logits_close(s_logits, os_logits, factor * 2e-2)
+    assert ok, f"step logits off by {factor * worst_s:.2f} x the small-model bound"
     g_c = np.full((len(subsets), Bk), -1.0, np.float32)
     g_t = np.full((len(subsets), Bk), -1, np.int32)
     g_c[r_copy, r_pos - P] = s_conf
@@ -190,7 +194,7 @@ def test_cfg4_refresh_and_four_copy_step_match_oracle():
     new, chain, _ = O.jump_walk(g_c, g_t, masked, subsets, ranks, rank_tok, tau)
     assert s_acc == sorted((int(P + i), int(t)) for i, t in new.items()) and s_chain == [int(c) for c in chain], "jump walk"
     print(f"\ncfg4 full size: per-row rel. L2 error {l2_r:.2e} (refresh, block rows) {l2_s:.2e} (4-copy step); "
-          f"element-wise {6 * worst_r:.2f} x / {6 * worst_s:.2f} x the small-model bound; conf rel err {cerr:.2e}; "
+          f"element-wise {factor * worst_r:.2f} x / {factor * worst_s:.2f} x the small-model bound; conf rel err {cerr:.2e}; "
           f"chain {s_chain}, accepted {len(s_acc)}")
 
 
@@ -242,7 +246,7 @@ def test_cfg5_batch16_sampled_sequence_matches_oracle():
     cache, o_conf, o_tok = O.refresh_prefill(om, xs[pick], T, P, dtype=np.float32)
     o_k = np.asarray(cache.k[-1], dtype=np.float64).reshape(T, -1)
     k_err = rel_l2(g_k, o_k)
-    assert k_err <= 2e-2, f"last-layer K of the picked sequence: per-row relative L2 error {k_err:.3e}"
+    assert k_err <= anchored_bounds(shape.n_layers, 1)[0], f"last-layer K of the picked sequence: per-row relative L2 error {k_err:.3e}"
     cerr = float((np.abs(g_conf - o_conf) / o_conf).max())
     assert cerr <= 0.2, cerr
     assert (g_tok != o_tok).mean() <= 0.1
@@ -277,3 +281,49 @@ def test_cfg5_batch16_sampled_sequence_matches_oracle():
     assert s_chain == [int(c) for c in chain], "jump walk: chain"
     print(f"\ncfg5 full size, sequence {pick} of 16 (response {Lp}): last-layer K rel. L2 error {k_err:.2e}; conf rel err "
           f"{cerr:.2e} (refresh) {serr:.2e} (step); greedy tokens differing {int((g_tok != o_tok).sum())} of {Lp}; chain {chain}")
+
+
+def _full_size_lockstep(wl_name, copies, max_iters=None, stop=None, prompt_len=None, gen_len=None):
+    from gpu_common import lockstep_generate, assert_near_ties_only, anchored_bounds
+    E = engine()
+    wl = synth.WORKLOADS[wl_name]
+    shape, Bk = wl.shape, wl.block_len
+    P, L = prompt_len or wl.prompt_len, gen_len or wl.gen_len
+    x0 = synth.sequence(0, 0, P, L, shape)
+    gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=copies)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    kw = dict(block_len=Bk, n_copies=copies, alp=False)
+    # bounds from the oracle's own float32-vs-float64 distance at this depth, not literals
+    l2_tol, factor = anchored_bounds(shape.n_layers, L * shape.vocab)
+    st = lockstep_generate(E, sess, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), tol=factor * 2e-2, l2_tol=l2_tol,
+                           dtype=np.float32, max_iters=max_iters, stop=stop)
+    assert sess.status() == 0
+    sess.close(); gm.close()
+    assert_near_ties_only(st)
+    print(f"\n{wl_name} x {copies} copies, full size in lock step: {st['iters']} iterations ({st['refreshes']} refreshes, "
+          f"{st['stage2_steps']} in the decoded-share layout), {st['tokens']} tokens; worst per-row rel. L2 {st['worst_l2']:.2e} "
+          f"(bound {l2_tol:.2e}), element-wise {st['worst_logit'] * factor:.2f} x the small-model bound (bound {factor:.2f} x); "
+          f"oracle-side decision differences {st['oracle_decision_diff']} (all measured near-ties), greedy tokens on a "
+          f"sub-error top-2 gap {st['tok_diff']}")
+    return st
+
+
+@requires_gpu
+def test_cfg3_whole_block_and_next_refresh_in_lockstep():
+    """Every iteration of block 0 of the benchmarked configuration (32 layers, prompt 512, response 256, block 32, one
+    copy) and the refresh of block 1, whose prefix then holds decoded tokens: per iteration all logits against the
+    float32 oracle, accept set and next row table reproduced bit for bit from the kernels' own confidences."""
+    wl = synth.WORKLOADS["cfg3_8b_c1"]
+    st = _full_size_lockstep("cfg3_8b_c1", 1, max_iters=wl.block_len + 1)
+    assert st["refreshes"] == 2 and st["steps"] == wl.block_len - 1 and st["tokens"] == wl.block_len + 1
+
+
+@requires_gpu
+def test_cfg4_eight_copies_until_the_decoded_share_switch_in_lockstep():
+    """The 8B shape with eight copies (block 32): steps of 128 rows (four copies) until enough of the block is decoded,
+    then the first step in the decoded-share layout (eight copies, speculative copies hold the masked positions
+    only) at full width and depth; prompt 512 and one block of response keep the oracle's part to a few minutes."""
+    st = _full_size_lockstep("cfg4_8b_c4", 8, gen_len=64, stop=lambda s: s["stage2_steps"] >= 1)
+    assert st["stage2_steps"] == 1 and st["refreshes"] == 1

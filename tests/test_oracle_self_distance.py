@@ -1,0 +1,77 @@
+"""Anchors of the GPU tests' tolerances: how far two correct evaluations of the same forward are from each other.
+
+Nothing here runs a kernel.  The oracle is compared with itself (float32 against float64 arithmetic between the
+bf16 rounding points, and the bf16-faithful mode against the unrounded definition); the tolerances the GPU parity
+tests apply are functions of, or multiples of, these distances."""
+import importlib.util
+import json
+import math
+import os
+
+import numpy as np
+
+import synth
+from oracle import odb_oracle as O
+from oracle.inputs import model_from_synth
+
+GOLDEN = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden")
+_spec = importlib.util.spec_from_file_location("oracle_self_distance", os.path.join(GOLDEN, "oracle_self_distance.py"))
+SD = importlib.util.module_from_spec(_spec)
+_spec.loader.exec_module(SD)
+
+
+def _in_bound_units(got, want, tol=2e-2):
+    """largest |got - want| in units of tol * max(|want|, rms(row)): the element bound of the small-model tests"""
+    want = np.asarray(want, np.float64)
+    rms = np.sqrt((want * want).mean(-1, keepdims=True))
+    return float((np.abs(np.asarray(got, np.float64) - want) / (tol * np.maximum(np.abs(want), rms))).max())
+
+
+def test_stored_self_distance_follows_the_square_root_law():
+    """The stored measurement (six 8B-shaped layers): layer 0's K is an exact function of the embeddings (distance
+    at float32 rounding level); from layer 1 on the per-row relative L2 distance is c * sqrt(layer) to within 10 %."""
+    d = json.load(open(os.path.join(GOLDEN, "oracle_self_distance.json")))
+    assert d["layers"] >= 6 and d["per_layer"][0]["rel_l2"] < 1e-3
+    assert d["c"] == SD.fit_c(d["per_layer"])
+    for p in d["per_layer"][1:]:
+        assert abs(p["rel_l2"] / (d["c"] * math.sqrt(p["layer"])) - 1.0) < 0.10, p
+
+
+def test_self_distance_measured_again_on_three_layers():
+    """The measurement itself, re-run small (three 8B-shaped layers, 8 rows): the same law with the stored constant."""
+    per_layer = SD.measure(3, 8)
+    assert per_layer[0]["rel_l2"] < 1e-3
+    c = SD.stored_c()
+    for p in per_layer[1:]:
+        assert 0.6 < p["rel_l2"] / (c * math.sqrt(p["layer"])) < 1.5, p
+
+
+def test_full_depth_bounds_come_out_of_the_measurement():
+    """What the full-size GPU test applies at 32 layers: a per-row relative L2 bound of c * sqrt(32) (it is the
+    the benchmark spec's 2e-2 to within a few per cent: at that depth the bound IS the oracle's own self-distance) and an
+    element-wise factor of sqrt(2 ln n) * that / 2e-2 over the small-model bound."""
+    assert 1.7e-2 < SD.l2_bound(32) < 2.3e-2
+    f = SD.elementwise_factor(32, 256 * 126464)
+    assert 5.0 < f < 7.0
+    assert SD.elementwise_factor(2, 64 * 2048) < f
+
+
+def test_small_model_tolerances_against_the_oracles_own_distances():
+    """Why the small-model GPU tests use 2e-2 on the N(0, 0.02) models and 4e-2 on the sharp-logit one.  On the
+    former the oracle's float32 and float64 runs differ by less than half of the 2e-2 element bound and its bf16
+    mode is within the bound of the unrounded definition.  On the sharp-logit model the bf16 mode is ALREADY more
+    than 2e-2 away from the unrounded definition (rounding noise is amplified by logits of rms 8) and the two
+    precisions differ by most of it; confidences, which move like the logits, by 2 to 3e-2 relative."""
+    out = {}
+    for name in ("TINY", "TINY_PEAKY"):
+        shape, P, L = getattr(synth, name), 64, 64
+        x0 = synth.sequence(0, 0, P, L, shape)
+        om64, om32 = model_from_synth(shape, seed=0), model_from_synth(shape, seed=0, dtype=np.float32)
+        _, c64, _, l64 = O.refresh_prefill(om64, x0, P + L, P, return_logits=True)
+        _, c32, _, l32 = O.refresh_prefill(om32, x0, P + L, P, return_logits=True, dtype=np.float32)
+        _, _, _, lp = O.refresh_prefill(om64, x0, P + L, P, return_logits=True, faithful=False)
+        out[name] = (_in_bound_units(l32, l64), _in_bound_units(l64, lp), float((np.abs(c32 - c64) / c64).max()))
+    prec, rnd, conf = out["TINY"]
+    assert prec < 0.6 and rnd < 1.0 and conf < 5e-3
+    prec, rnd, conf = out["TINY_PEAKY"]
+    assert 0.5 < prec < 1.2 and 1.0 < rnd < 2.0 and 1e-2 < conf < 0.15
