@@ -322,6 +322,24 @@ def accept_set(conf: np.ndarray, masked: np.ndarray, tau: float) -> np.ndarray:
     return acc
 
 
+def reverse_step_unmask(masked: np.ndarray, u: np.ndarray, k: int, n_steps: int) -> np.ndarray:
+    """The stochastic reverse step of the masked-diffusion process (Section 2.1, Eq. 1), as the unmask decision
+    of iteration k = 0 .. n_steps-1 of a block decoded in n_steps iterations.
+
+    Noise levels fall linearly over the block's iterations, t = 1 - k / n_steps to s = 1 - (k + 1) / n_steps.
+    A position that is not masked keeps its token (first case of Eq. 1).  A masked position stays masked with
+    probability s / t = (n_steps - k - 1) / (n_steps - k) (second case) and is otherwise given a token of the
+    model's clean-token distribution (third case); u holds one uniform [0, 1) deviate per position, and a
+    position is unmasked iff u >= s / t, compared in fp32.  The last iteration (s = 0) unmasks everything left.
+    Reading: the token itself is taken greedily (the distribution sampled at temperature 0, as everywhere in this
+    build); the paper's method replaces this stochastic schedule by the confidence threshold (Section 3).
+    masked bool [B], u fp32 [B] -> bool [B]."""
+    if k >= n_steps - 1:
+        return masked.copy()
+    stay = np.float32(n_steps - k - 1) / np.float32(n_steps - k)
+    return masked & (np.asarray(u, dtype=np.float32) >= stay)
+
+
 def decision_margin(conf: np.ndarray, masked: np.ndarray, tau: float, k_ranks: int = 0,
                     still_masked: Optional[np.ndarray] = None, relative: bool = True) -> float:
     """How close the decisions taken on this row of confidences are to flipping.  Diagnostic only
@@ -517,6 +535,8 @@ class DecodeParams:
     stage2_min_decoded: int = -1      # -1: ceil(4 B / 7), the point where 8 copies fit 4 B rows
     alp: bool = True
     pick_best: bool = False           # the compared "vanilla speculation": pick_best_walk instead of jump_walk
+    sampling: bool = False            # Eq. 1's stochastic unmasking (reverse_step_unmask) instead of the threshold rule
+    sample_steps: int = 0             # iterations a block is decoded in when sampling (<= 64)
 
 
 def use_stage2(params: DecodeParams, B: int, n_decoded: int) -> bool:
@@ -530,7 +550,8 @@ def use_stage2(params: DecodeParams, B: int, n_decoded: int) -> bool:
 
 def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, faithful=True,
              dtype=np.float64, length_schedule: Optional[Callable[[int, int], Optional[int]]] = None,
-             max_iters: Optional[int] = None, cache_blocks: bool = True):
+             max_iters: Optional[int] = None, cache_blocks: bool = True,
+             noise: Optional[Callable[[int, int], np.ndarray]] = None):
     """Whole-response generation: per block a refresh (itself a decoding iteration restricted
     to the block), adaptive length prediction, then block steps until the block is full.
 
@@ -539,8 +560,12 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
     workload).  cache_blocks=False is the cache-less baseline of Section 1 (bidirectional
     attention without a KV cache: every iteration re-executes the whole prefill), i.e. every
     iteration of a block is a refresh and no block step is ever taken.
+    With params.sampling the accept rule of every iteration is Eq. 1's stochastic unmasking
+    (reverse_step_unmask; one copy only): noise(block_index, k) gives the uniforms [block_len] of
+    iteration k of a block (k = 0 is the refresh); an iteration may unmask nothing.
     Returns (tokens [P + final length], trace list of per-iteration dicts).
     """
+    assert not params.sampling or (params.n_copies == 1 and 1 <= params.sample_steps <= 64 and noise is not None)
     x = np.array(x0, dtype=np.int64)
     T = len(x)
     tau = params.accept_threshold
@@ -564,11 +589,17 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
         e = min(s + params.block_len, T)
         B = e - s
         masked = x[s:e] == model.mask_id
-        acc = accept_set(conf_r[:B], masked, tau)
+        k_iter = 0                                                   # iteration of the block (sampling schedule)
+        acc = (reverse_step_unmask(masked, noise(b, 0)[:B], 0, params.sample_steps) if params.sampling
+               else accept_set(conf_r[:B], masked, tau))
         for i in np.flatnonzero(acc):
             x[s + i] = tok_r[i]
-        diag = walk_diagnostics(conf_r[None, :B], top2_gap(logits_r[:B], model.mask_id)[None, :], masked, [()], [], [0],
-                                {int(i): 0 for i in np.flatnonzero(acc)}, tau, k_ranks)
+        if params.sampling:   # no confidence decides anything; the greedy tokens of the unmasked positions do
+            g_ = top2_gap(logits_r[:B], model.mask_id)[acc]
+            diag = {"margin": np.inf, "sep": np.inf, "tok_gap": float(g_.min()) if len(g_) else np.inf}
+        else:
+            diag = walk_diagnostics(conf_r[None, :B], top2_gap(logits_r[:B], model.mask_id)[None, :], masked, [()], [], [0],
+                                    {int(i): 0 for i in np.flatnonzero(acc)}, tau, k_ranks)
         trace.append({"kind": "refresh", "block": b, "T": T,
                       "accepted": [(int(s + i), int(tok_r[i])) for i in np.flatnonzero(acc)], "chain": [0], **diag})
         last_conf, last_tok = conf_r[:B], tok_r[:B]
@@ -587,14 +618,23 @@ def generate(model: Model, x0: np.ndarray, P: int, params: DecodeParams, *, fait
             subsets = copy_subsets(len(ranks), 4 if (params.n_copies == 8 and not st2) else params.n_copies, st2)
             conf, tok, logits, r_copy, r_pos = block_decode_step(model, cache, x, T, s, e, subsets, rank_pos, rank_tok,
                                                                  st2, faithful=faithful, dtype=dtype, return_logits=True)
-            walk = pick_best_walk if params.pick_best else jump_walk
-            new, chain, last = walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
+            k_iter += 1
+            if params.sampling:
+                acc = reverse_step_unmask(masked, noise(b, k_iter)[:B], k_iter, params.sample_steps)
+                new, chain, last = {int(i): int(tok[0][i]) for i in np.flatnonzero(acc)}, [0], 0
+            else:
+                walk = pick_best_walk if params.pick_best else jump_walk
+                new, chain, last = walk(conf, tok, masked, subsets, ranks, rank_tok, tau)
             for i, t in new.items():
                 x[s + i] = t
             gaps = np.full(conf.shape, np.inf)
             gaps[r_copy, r_pos - s] = top2_gap(logits, model.mask_id)
             visited = chain if not (params.pick_best and chain != [0]) else [0] + chain
-            diag = walk_diagnostics(conf, gaps, masked, subsets, ranks, visited, new, tau, k_ranks)
+            if params.sampling:
+                g_ = gaps[0][np.array(list(new.keys()), dtype=np.int64)]
+                diag = {"margin": np.inf, "sep": np.inf, "tok_gap": float(g_.min()) if len(g_) else np.inf}
+            else:
+                diag = walk_diagnostics(conf, gaps, masked, subsets, ranks, visited, new, tau, k_ranks)
             trace.append({"kind": "step", "block": b, "T": T, "stage2": st2,
                           "accepted": sorted((int(s + i), int(t)) for i, t in new.items()),
                           "chain": [int(c) for c in chain], **diag})

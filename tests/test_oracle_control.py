@@ -490,3 +490,64 @@ def test_walk_diagnostics_on_the_worked_example():
     # next candidates ranked from copy 0: p5 (.85), p3 (.50) -> p3's token there now counts
     d0 = O.walk_diagnostics(conf, gaps, masked, S1, [1, 5], [0], {1: 11}, 0.9, 2)
     assert d0["margin"] == pytest.approx(0.02 / 0.9, rel=1e-3) and d0["tok_gap"] == 0.01
+
+
+# ----------------------------------------------------------------------------- stochastic reverse step (Eq. 1)
+
+def test_reverse_step_keeps_unmasked_and_ends_unmasking_everything():
+    masked = np.array([1, 0, 1, 1, 0, 1], bool)
+    u = f32(.99, .99, .0, .5, .0, .74)
+    acc = O.reverse_step_unmask(masked, u, 0, 4)            # stay with probability 3/4: unmask iff u >= .75
+    assert acc.tolist() == [True, False, False, False, False, False]      # unmasked positions never change (first case)
+    assert O.reverse_step_unmask(masked, u, 2, 4).tolist() == [True, False, False, True, False, True]   # stay 1/2
+    # the boundary is "stay masked iff u < s / t", in fp32
+    assert O.reverse_step_unmask(np.ones(2, bool), f32(0.75, np.nextafter(np.float32(0.75), np.float32(0))), 0, 4).tolist() == [True, False]
+    # last iteration: s = 0, nothing stays masked, whatever the deviates
+    assert O.reverse_step_unmask(masked, np.zeros(6, np.float32), 3, 4).tolist() == masked.tolist()
+    assert O.reverse_step_unmask(masked, np.zeros(6, np.float32), 0, 1).tolist() == masked.tolist()
+
+
+def test_reverse_step_stay_probability_and_linear_survival():
+    """Second case of Eq. 1: a masked position stays masked with probability s / t.  With t falling linearly over
+    the n iterations of a block, the probability of still being masked after iteration k is the product of the
+    stay probabilities = (n - k - 1) / n: every position is unmasked at a uniformly distributed iteration."""
+    n, N = 8, 200000
+    alive = np.ones(N, bool)
+    for k in range(n):
+        u = synth.uniform(7, 100 + k, N)
+        acc = O.reverse_step_unmask(alive, u, k, n)
+        frac_stay = 1.0 - acc.sum() / alive.sum()
+        want = (n - k - 1) / (n - k)
+        assert abs(frac_stay - want) < 4 * np.sqrt(max(want * (1 - want), 1e-9) / alive.sum()) + 1e-12, (k, frac_stay, want)
+        alive &= ~acc
+        assert abs(alive.mean() - (n - k - 1) / n) < 4 * np.sqrt(0.25 / N), (k, alive.mean())
+    assert not alive.any()
+
+
+def test_generate_with_sampling(tiny_model):
+    om, P = tiny_model, 64
+    x0 = synth.sequence(0, 0, P, 64, synth.TINY)
+    L, Bk, n = len(x0) - P, 16, 6
+    noise = lambda b, k: synth.uniform(3, 1000 * b + k, Bk)
+    p = O.DecodeParams(block_len=Bk, sampling=True, sample_steps=n, alp=False)
+    x, tr = O.generate(om, x0, P, p, noise=noise)
+    assert (x[P:] != om.mask_id).all() and sum(len(t["accepted"]) for t in tr) == L
+    per_block = [sum(t["block"] == b for t in tr) for b in range(L // Bk)]
+    assert all(1 <= c <= n for c in per_block) and max(per_block) > 1
+    # what is committed at an iteration is the greedy token of THAT iteration's forward at the unmasked positions,
+    # and which positions are unmasked depends on the deviates alone: replay the schedule without the model
+    b, k, masked = -1, 0, None
+    for t in tr:
+        if t["kind"] == "refresh":
+            b, k, masked = t["block"], 0, np.ones(Bk, bool)
+        else:
+            k += 1
+        acc = O.reverse_step_unmask(masked, noise(b, k), k, n)
+        assert [p_ - (P + b * Bk) for p_, _ in t["accepted"]] == np.flatnonzero(acc).tolist()
+        masked &= ~acc
+    # same deviates, same run; one iteration per block is the "accept everything at the refresh" regime
+    x2, tr2 = O.generate(om, x0, P, p, noise=noise)
+    assert np.array_equal(x, x2) and [t["accepted"] for t in tr] == [t["accepted"] for t in tr2]
+    x1, tr1 = O.generate(om, x0, P, O.DecodeParams(block_len=Bk, sampling=True, sample_steps=1, alp=False), noise=noise)
+    x0_, tr0 = O.generate(om, x0, P, O.DecodeParams(block_len=Bk, accept_threshold=-1.0, alp=False))
+    assert np.array_equal(x1, x0_) and len(tr1) == len(tr0) == L // Bk
