@@ -118,6 +118,12 @@ typedef struct odb_decode_params {
                                    against (Fig. 7(a), Section 5.3): candidates are verified in the main block only,
                                    the copy filling the largest set of verified candidates is adopted and its fills
                                    and own accept set are the step's result (chain = that one copy) */
+    int32_t sampling;           /* 1: instead of the threshold rule, the stochastic reverse step of the masked-diffusion
+                                   process (Section 2.1, Eq. 1): iteration k = 0 .. sample_steps-1 of a block (the
+                                   refresh is k = 0) leaves a masked position masked with probability
+                                   (sample_steps-k-1)/(sample_steps-k) and otherwise commits its greedy token; the
+                                   uniform deviates come from odb_session_set_sampling_noise.  One copy only. */
+    int32_t sample_steps;       /* iterations a block is decoded in when sampling, 1 .. 64 */
 } odb_decode_params;
 
 /* Per-sequence result of odb_unmask_accept (host memory, valid on return). */
@@ -181,6 +187,11 @@ int32_t odb_session_set_gen_len(odb_session* s, int32_t seq, int32_t new_gen_len
 /* Copies the sequence's ids (prompt + current response length) to ids_host[0..cap); *len gets
  * the count.  Synchronous. */
 int32_t odb_session_get_tokens(odb_session* s, int32_t seq, int32_t* ids_host, int32_t cap, int32_t* len);
+/* Uniform [0, 1) deviates for the stochastic reverse step (odb_decode_params.sampling) of the block of `seq` that
+ * the next refresh opens: u_host[k * block_len + i] decides position i of the block at iteration k (k = 0 is the
+ * refresh's accept), n_iters <= 64 rows.  The deviates are data of the caller's (a counter-based stream, so that a
+ * run can be reproduced); the library draws no random numbers.  Synchronous. */
+int32_t odb_session_set_sampling_noise(odb_session* s, int32_t seq, const float* u_host, int32_t n_iters, int32_t block_len);
 /* Marks a sequence inactive (finished) / active; inactive sequences take no part in later calls. */
 int32_t odb_session_set_active(odb_session* s, int32_t seq, int32_t active);
 /* Reads and clears the device status word (ODB_OK or ODB_ERR_TIMEOUT).  Synchronous. */

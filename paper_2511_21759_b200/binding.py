@@ -44,7 +44,7 @@ class odb_weights(C.Structure):
 class odb_decode_params(C.Structure):
     _fields_ = [("block_len", C.c_int32), ("n_copies", C.c_int32), ("accept_threshold", C.c_float),
                 ("truncate_threshold", C.c_float), ("stage2_min_decoded", C.c_int32), ("alp", C.c_int32),
-                ("pick_best", C.c_int32)]
+                ("pick_best", C.c_int32), ("sampling", C.c_int32), ("sample_steps", C.c_int32)]
 
 
 class odb_result(C.Structure):
@@ -71,6 +71,7 @@ SIGNATURES = {
     "odb_session_set_sequence": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32]),
     "odb_session_set_gen_len": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
     "odb_session_get_tokens": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.POINTER(C.c_int32)]),
+    "odb_session_set_sampling_noise": (C.c_int32, [C.c_void_p, C.c_int32, C.c_void_p, C.c_int32, C.c_int32]),
     "odb_session_set_active": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
     "odb_session_status": (C.c_int32, [C.c_void_p]),
     "odb_refresh_prefill": (C.c_int32, [C.c_void_p, C.POINTER(odb_decode_params), C.c_void_p]),

@@ -226,6 +226,20 @@ __device__ int accept_set(const float* conf, const bool* masked, int B, float ta
     return n;
 }
 
+// Stochastic reverse step (Section 2.1, Eq. 1) at iteration k of the n_steps a block is decoded in: a masked
+// position stays masked with probability s / t = (n_steps - k - 1) / (n_steps - k), decided by its uniform
+// deviate u (unmask iff u >= s / t, in fp32); the last iteration unmasks everything left.
+__device__ int sample_set(const float* u, const bool* masked, int B, int k, int n_steps, bool* acc) {
+    const bool all = k >= n_steps - 1;
+    const float stay = all ? 0.f : static_cast<float>(n_steps - k - 1) / static_cast<float>(n_steps - k);
+    int n = 0;
+    for (int i = 0; i < B; ++i) {
+        acc[i] = masked[i] && (all || u[i] >= stay);
+        n += acc[i];
+    }
+    return n;
+}
+
 // st / res: the block's shared-memory copies of the sequence's state and result (the decisions are one thread's
 // serial walk: every field it touches would otherwise be a dependent global load)
 __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p, int after_refresh, int mask_id, int eos_id,
@@ -321,6 +335,10 @@ __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p,
         }
     }
     const int B = st->e - s;
+    if (after_refresh) st->block_iter = 0;
+    const int k_iter = st->block_iter < kMaxLoopIters ? st->block_iter : kMaxLoopIters - 1;
+    const float* noise = c.noise + (static_cast<size_t>(seq) * kMaxLoopIters + k_iter) * kMaxBlock;
+    ++st->block_iter;
     bool masked0[kMaxBlock], masked[kMaxBlock], acc[kMaxBlock], taken[kMaxBlock];
     for (int i = 0; i < B; ++i) { masked0[i] = (gathered ? xs[i] : x[s + i]) == mask_id; taken[i] = false; }
 
@@ -377,7 +395,8 @@ __device__ void accept_body(const ControlBuffers& c, const odb_decode_params& p,
             if ((X >> r) & 1) masked[st->rank_off[r]] = false;
         for (int i = 0; i < B; ++i) any |= masked[i];
         if (!any) break;
-        accept_set(conf[cur], masked, B, p.accept_threshold, acc);
+        if (p.sampling) sample_set(noise, masked, B, k_iter, p.sample_steps, acc);
+        else accept_set(conf[cur], masked, B, p.accept_threshold, acc);
         for (int i = 0; i < B; ++i) {
             if (acc[i] && !taken[i]) {
                 taken[i] = true;

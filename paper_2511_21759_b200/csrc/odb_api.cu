@@ -47,7 +47,7 @@ int32_t check_config(const odb_config* c) {
 struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
     size_t rope, state, results, status, loop, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
-    size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml, ptable, pbars;
+    size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml, ptable, pbars, noise;
     size_t total;
 };
 
@@ -102,6 +102,7 @@ Layout make_layout(const odb_config& c) {
     // persistent decode-step kernel: one table of projections per row-tile size (32, 64, 128), the grid barrier words
     L.ptable = take(3 * align_up(step_persistent_table_bytes(c.n_layers)));
     L.pbars = take(step_persistent_barrier_bytes(c.n_layers));
+    L.noise = take(sizeof(float) * c.max_batch * kMaxLoopIters * kMaxBlock);   // deviates of the stochastic reverse step
     L.total = off;
     return L;
 }
@@ -332,6 +333,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     cb.conf = s->at<float>(L.conf);
     cb.tok = s->at<int32_t>(L.tok);
     cb.results = s->at<odb_result>(L.results);
+    cb.noise = s->at<float>(L.noise);
     *out = s;
     return ODB_OK;
 }
@@ -405,6 +407,18 @@ int32_t odb_session_get_tokens(odb_session* s, int32_t seq, int32_t* ids, int32_
     if (cap < T) return ODB_ERR_WORKSPACE;
     ODB_CUDA(cudaMemcpy(ids, s->cb.x + static_cast<size_t>(seq) * c.max_seq, sizeof(int32_t) * T, cudaMemcpyDeviceToHost));
     *len = T;
+    return ODB_OK;
+}
+
+int32_t odb_session_set_sampling_noise(odb_session* s, int32_t seq, const float* u, int32_t n_iters, int32_t block_len) {
+    if (!s || !u) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (seq < 0 || seq >= c.max_batch || n_iters < 1 || n_iters > kMaxLoopIters) return ODB_ERR_ARG;
+    if (block_len < 1 || block_len > c.max_block) return ODB_ERR_SHAPE;
+    float* dst = s->at<float>(s->L.noise) + static_cast<size_t>(seq) * kMaxLoopIters * kMaxBlock;
+    ODB_CUDA(cudaMemcpy2DAsync(dst, sizeof(float) * kMaxBlock, u, sizeof(float) * block_len, sizeof(float) * block_len, n_iters,
+                               cudaMemcpyHostToDevice, s->st));
+    ODB_CUDA(cudaStreamSynchronize(s->st));
     return ODB_OK;
 }
 
@@ -811,6 +825,7 @@ int32_t odb_unmask_accept(odb_session* s, const odb_decode_params* p, int32_t af
     const odb_config& c = s->m->cfg;
     if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
     if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
+    if (p->sampling && (p->n_copies != 1 || p->sample_steps < 1 || p->sample_steps > kMaxLoopIters)) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != (after_refresh ? 1 : 3)) return ODB_ERR_STATE;
     ODB_LAUNCH(ODB_KIND_CONTROL, launch_accept(s->cb, c.max_batch, *p, after_refresh, c.mask_id, c.eos_id,
@@ -834,6 +849,7 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
     const odb_config& c = s->m->cfg;
     if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
     if (p->n_copies != 1 && p->n_copies != 4 && p->n_copies != 8) return ODB_ERR_ARG;
+    if (p->sampling && (p->n_copies != 1 || p->sample_steps < 1 || p->sample_steps > kMaxLoopIters)) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != 2 || s->profiling) return ODB_ERR_STATE;   // event pairs cannot be recorded into the loop body
     *n_iters = 0;

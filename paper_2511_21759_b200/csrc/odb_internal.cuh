@@ -100,6 +100,7 @@ struct SeqState {
     int32_t P, T;                 // prompt length, current total length (prompt + response)
     int32_t block_idx, s, e;      // current block [s, e)
     int32_t n_masked;             // masked positions left in [s, e)
+    int32_t block_iter;           // iterations taken in the current block (0: the refresh's accept comes next)
     // speculative candidates for the next step (Section 4.2): offsets inside the block and the
     // tokens they would be filled with, most confident first
     int32_t n_ranks;
@@ -360,6 +361,7 @@ struct ControlBuffers {
     QTile* big_tiles;         // refresh: the same rows cut into work items of up to 128 query rows
     StepTile* step_tiles;     // decode steps with more than one copy
     const float* conf; const int32_t* tok;   // outputs of the last forward, per logit row
+    const float* noise;       // [batch][kMaxLoopIters][kMaxBlock] uniform deviates of the stochastic reverse step
     odb_result* results;      // [batch] device copy
     // pinned host memory the accept kernel writes its outcome to (state, results, the status word): the host
     // reads them after synchronising the stream, no copy is enqueued

@@ -56,10 +56,13 @@ class DecodeParams:
     stage2_min_decoded: int = -1
     alp: bool = True
     pick_best: bool = False
+    sampling: bool = False
+    sample_steps: int = 0
 
     def c(self) -> B.odb_decode_params:
         return B.odb_decode_params(self.block_len, self.n_copies, self.accept_threshold, self.truncate_threshold,
-                                   self.stage2_min_decoded, 1 if self.alp else 0, 1 if self.pick_best else 0)
+                                   self.stage2_min_decoded, 1 if self.alp else 0, 1 if self.pick_best else 0,
+                                   1 if self.sampling else 0, self.sample_steps)
 
 
 class Model:
@@ -145,6 +148,13 @@ class Session:
     def set_gen_len(self, seq: int, new_len: int):
         B.check(B.lib().odb_session_set_gen_len(self.handle, seq, new_len), "odb_session_set_gen_len")
         self.gen_len[seq] = new_len
+
+    def set_sampling_noise(self, seq: int, u: np.ndarray):
+        """u [iterations][block_len]: the uniform deviates of the stochastic reverse step for the block the next
+        refresh opens (data of the caller's; nothing is drawn here)."""
+        u = np.ascontiguousarray(u, dtype=np.float32)
+        B.check(B.lib().odb_session_set_sampling_noise(self.handle, seq, u.ctypes.data, u.shape[0], u.shape[1]),
+                "odb_session_set_sampling_noise")
 
     def set_active(self, seq: int, active: bool):
         B.check(B.lib().odb_session_set_active(self.handle, seq, 1 if active else 0), "odb_session_set_active")
@@ -268,7 +278,7 @@ def gemm_static_scratch(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> 
 def generate(sess: Session, params: DecodeParams, *,
              length_schedule: Optional[Callable[[int, int, int], Optional[int]]] = None,
              max_iters: Optional[int] = None, cache_blocks: bool = True, resident: bool = False,
-             start_block: int = 0):
+             start_block: int = 0, noise: Optional[Callable[[int, int], np.ndarray]] = None):
     """Runs every sequence set on the session to completion.
 
     Per iteration: the sequences standing at a block boundary are refreshed and accepted
@@ -281,7 +291,9 @@ def generate(sess: Session, params: DecodeParams, *,
     refresh prefill and no block step is taken.  resident=True runs the steps of a block through the
     device-resident loop (same trace, one host round trip per block instead of one per iteration).
     start_block: the block every sequence starts at (a resumed session: the blocks before it are already
-    decoded in the ids given to set_sequence; the refresh of start_block recomputes the whole cache)."""
+    decoded in the ids given to set_sequence; the refresh of start_block recomputes the whole cache).
+    noise(seq, block_index) -> [sample_steps][block_len] uniforms, handed to the session before the block's refresh
+    when params.sampling is set."""
     seqs = sorted(sess.gen_len)
     block = {i: start_block for i in seqs}
     need_refresh = {i: True for i in seqs}
@@ -307,6 +319,9 @@ def generate(sess: Session, params: DecodeParams, *,
             bi = [-1] * sess.nb
             for i in refresh:
                 bi[i] = block[i]
+            if params.sampling:
+                for i in refresh:
+                    sess.set_sampling_noise(i, noise(i, block[i]))
             sess.refresh_prefill(params, bi)
             if length_schedule is not None:
                 for i in refresh:

@@ -81,7 +81,7 @@ def _assert_identical_or_near_tie(gtok, gtrace, otok, otrace, measured):
     ties = [t for t in measured["near_ties"] if t[0] == div["iter"]]
     assert ties, f"iteration {div['iter']}: the free runs part but the oracle decides like the kernels in lock step: {div}"
     assert_near_ties_only({"near_ties": ties})
-    it, kind, margin, cerr = ties[0]
+    it, kind, margin, cerr = ties[0][:4]
     print(f"\nfree runs part at iteration {it} ({kind}) after {n} identical ones: oracle margin {margin:.2e}, "
           f"measured confidence error {cerr:.2e}: a near-tie")
 
@@ -436,4 +436,52 @@ def test_argument_validation_and_state_errors():
     assert lib.odb_decode_block_resident(sess.handle, C.byref(pc), 0, log, 4, C.byref(n)) == B.ODB_OK
     assert 1 <= n.value <= 4 and log[n.value - 1].masks_left < res[0].masks_left      # log_cap bounds the iterations
     assert sess.status() == 0
+    sess.close(); gm.close()
+
+
+@requires_gpu
+@pytest.mark.parametrize("shape_name", ["TINY", "TINY_PEAKY"])
+def test_stochastic_reverse_step_in_lockstep_and_free_running(shape_name):
+    """The stochastic unmasking of Section 2.1, Eq. 1 as the accept rule (odb_decode_params.sampling): which
+    positions an iteration unmasks depends on the caller's uniform deviates alone, so the accepted POSITIONS of every
+    iteration must equal the oracle's exactly; the tokens are the greedy tokens of that iteration's forward.  Lock
+    step first, then the same generation free running, call by call and through the device-resident loop."""
+    E = engine()
+    from paper_2511_21759_b200 import binding as B
+    shape = getattr(synth, shape_name)
+    P, L, Bk, n = 40, 48, 16, 6
+    om = model_from_synth(shape, seed=4)
+    gm = E.Model.from_synth(shape, seed=4, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
+    x0 = synth.sequence(4, 0, P, L, shape)
+    noise = lambda b, k: synth.uniform(9, 1000 * b + k, Bk)
+    kw = dict(block_len=Bk, n_copies=1, alp=False, sampling=True, sample_steps=n)
+    sess = E.Session(gm)
+    sess.set_sequence(0, x0, P)
+    st = lockstep_generate(E, sess, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), noise=noise,
+                           tol=4e-2 if shape_name == "TINY_PEAKY" else 2e-2)
+    assert sess.status() == 0 and st["tokens"] == L and st["refreshes"] == L // Bk and st["iters"] <= n * (L // Bk)
+    assert st["iters"] > L // Bk                      # some block needed more than its refresh
+    locked = st["tokens_final"]
+    # the oracle's own free run: identical positions per iteration; tokens identical unless a greedy token sits on
+    # a top-2 logit gap below the logit error (counted by the harness)
+    otok, otrace = O.generate(om, x0, P, O.DecodeParams(**kw), noise=noise)
+    runs = []
+    for resident in (False, True):
+        sess.set_sequence(0, x0, P)
+        gtok, gtrace = E.generate(sess, E.DecodeParams(**kw), noise=lambda seq, b: np.stack([noise(b, k) for k in range(n)]),
+                                  resident=resident)
+        assert sess.status() == 0
+        runs.append((gtok[0], gtrace))
+        assert [[p_ for p_, _ in t["seqs"][0]["accepted"]] for t in gtrace] == [[p_ for p_, _ in t["accepted"]] for t in otrace]
+    assert np.array_equal(runs[0][0], runs[1][0]) and runs[0][1] == runs[1][1]
+    assert np.array_equal(runs[0][0], locked)
+    if st["tok_diff"] == 0:
+        assert np.array_equal(runs[0][0], otok)
+    # only with one copy, and with a step count the schedule can hold
+    sess.set_sequence(0, x0, P)
+    sess.refresh_prefill(E.DecodeParams(**kw), 0)
+    for bad in (dict(kw, n_copies=4), dict(kw, sample_steps=0), dict(kw, sample_steps=65)):
+        with pytest.raises(B.OdbError) as err:
+            sess.unmask_accept(E.DecodeParams(**bad), True)
+        assert err.value.status == B.ODB_ERR_ARG
     sess.close(); gm.close()
