@@ -500,6 +500,60 @@ def secondary_measurements(E, synth, gm, peaks, args):
                          "step_rows": 4 * wl4.block_len, "step_ms": st4, "step_algorithmic_bytes": bytes4,
                          "step_frac_of_measured": (bytes4 / (st4 * 1e-3) / 1e9 / peaks["hbm_gbs"]) if st4 else None}
     s4.close(); gm4.close()
+    # ---- batch 16, prompt 1024, response 1024 shrunk per sequence, block 64, 4 copies: one block cycle ----
+    wl5 = synth.WORKLOADS["cfg5_8b_b16"]
+    T5 = wl5.prompt_len + wl5.gen_len
+    gm5 = E.Model(wl5.shape, gm.t, max_batch=wl5.batch, max_seq=T5, max_block=wl5.block_len, max_copies=4)
+    s5 = E.Session(gm5)
+    p5 = E.DecodeParams(block_len=wl5.block_len, n_copies=4)
+    targets = synth.shrink_schedule(0, wl5.batch, wl5.gen_len)
+    for i in range(wl5.batch):
+        s5.set_sequence(i, synth.sequence(0, i, wl5.prompt_len, wl5.gen_len, wl5.shape), wl5.prompt_len)
+
+    def cycle5(block, timed_steps=None):
+        bi = [block if block * wl5.block_len < s5.gen_len[i] else -1 for i in range(wl5.batch)]
+        s5.refresh_prefill(p5, bi)
+        for i in range(wl5.batch):       # every sequence gives up half of its excess over its seeded target length
+            cur = s5.gen_len[i]
+            new = max(int(targets[i]), cur - (cur - int(targets[i]) + 1) // 2, (block + 1) * wl5.block_len)
+            if bi[i] >= 0 and block * wl5.block_len < new < cur:
+                s5.set_gen_len(i, new)
+        res = s5.unmask_accept(p5, True)
+        toks = sum(res[i].n_accepted for i in range(wl5.batch))
+        while any(res[i].masks_left > 0 for i in range(wl5.batch)):
+            if timed_steps is not None and len(timed_steps) < 4:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(s5.stream)
+                s5.block_decode_step(p5)
+                e1.record(s5.stream)
+                log = [s5.unmask_accept(p5, False)]
+                timed_steps.append(e0.elapsed_time(e1))
+            else:
+                log = s5.decode_block_resident(p5) if not args.host_loop else [(s5.block_decode_step(p5), s5.unmask_accept(p5, False))[1]]
+            for res in log:
+                toks += sum(res[i].n_accepted for i in range(wl5.batch))
+        for i in range(wl5.batch):
+            s5.gen_len[i] = res[i].gen_len
+        return toks
+
+    cycle5(0)                                                  # warm-up block (graphs of the shapes met)
+    steps5 = []
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record(s5.stream)
+    toks5 = cycle5(1, steps5)
+    b.record(s5.stream)
+    torch.cuda.synchronize()
+    rows5 = wl5.batch * wl5.block_len * 4
+    d_, F_, V_, nl_ = wl5.shape.d_model, wl5.shape.d_ffn, wl5.shape.vocab, wl5.shape.n_layers
+    flops5 = 2.0 * rows5 * (nl_ * (4 * d_ * d_ + 3 * d_ * F_) + V_ * d_)      # projections of one full step (attention excluded)
+    st5 = float(np.median(steps5)) if steps5 else None
+    out["cfg5_8b_b16"] = {"tokens_per_s": toks5 / (a.elapsed_time(b) * 1e-3), "block_cycles": 1, "batch": wl5.batch,
+                          "response_lengths_after_two_refreshes": [int(s5.gen_len[i]) for i in range(wl5.batch)],
+                          "step_rows_at_block_start": rows5, "step_ms": st5, "bound": "tensor",
+                          "step_tflops": flops5 / (st5 * 1e-3) / 1e12 if st5 else None,
+                          "step_frac_of_sustained_bf16": (flops5 / (st5 * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]) if st5 else None}
+    s5.close(); gm5.close()
     # ---- one 8B-shaped layer, context 512, block 32: the decode step with 1 and 4 copies ----
     shape1 = synth.LLADA_8B.with_layers(1)
     wl1 = synth.WORKLOADS["cfg2_layer_c1"]
