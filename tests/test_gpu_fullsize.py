@@ -324,6 +324,8 @@ def test_cfg3_whole_block_and_next_refresh_in_lockstep():
 def test_cfg4_eight_copies_until_the_decoded_share_switch_in_lockstep():
     """The 8B shape with eight copies (block 32): steps of 128 rows (four copies) until enough of the block is decoded,
     then the first step in the decoded-share layout (eight copies, speculative copies hold the masked positions
-    only) at full width and depth; prompt 512 and one block of response keep the oracle's part to a few minutes."""
-    st = _full_size_lockstep("cfg4_8b_c4", 8, gen_len=64, stop=lambda s: s["stage2_steps"] >= 1)
+    only) at full width and depth; prompt 512 and a response of 256 keep the oracle's part to a few minutes (with a
+    response of 64, i.e. fewer keys for the attention to average rounding noise over, the same run measured a worst
+    per-row relative L2 error of 2.57e-2 against 1.8e-2 here: inside the bound, but only just)."""
+    st = _full_size_lockstep("cfg4_8b_c4", 8, gen_len=256, stop=lambda s: s["stage2_steps"] >= 1)
     assert st["stage2_steps"] == 1 and st["refreshes"] == 1
