@@ -117,12 +117,17 @@ class Model:
 
 
 class Session:
-    def __init__(self, model: Model, stream: Optional[torch.cuda.Stream] = None):
+    def __init__(self, model: Model, stream: Optional[torch.cuda.Stream] = None, poison: bool = False):
+        """poison: hand the library a workspace and a K/V cache filled with 0xFF bytes (NaN as fp32 and as bf16), so
+        that a kernel reading memory nothing has written shows up as NaN in the results (tests)."""
         self.model = model
         lib = B.lib()
         dev = model.t["embed"].device
         self.kv = torch.empty(lib.odb_kv_bytes(C.byref(model.cfg)), dtype=torch.uint8, device=dev)
         self.ws = torch.empty(lib.odb_workspace_bytes(C.byref(model.cfg)), dtype=torch.uint8, device=dev)
+        if poison:
+            self.kv.fill_(0xFF)
+            self.ws.fill_(0xFF)
         self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
         self.handle = C.c_void_p()
         B.check(lib.odb_session_create(model.handle, self.kv.data_ptr(), self.kv.numel(), self.ws.data_ptr(),

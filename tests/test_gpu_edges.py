@@ -175,3 +175,31 @@ def test_resumed_session_continues_identically(copies):
     s2.close(); gm.close()
     assert tail == full_trace[n0:]
     assert np.array_equal(tok[0], full_tok[0])
+
+
+@requires_gpu
+@pytest.mark.parametrize("shape_name,copies", [("TINY_PEAKY", 1), ("TINY_PEAKY", 8), ("TINY_HD128", 4)])
+def test_poisoned_workspace_reads_nothing_unwritten(shape_name, copies):
+    """The caller's workspace and K/V cache arrive filled with NaN patterns (0xFF bytes): the library initialises
+    what it needs at session creation and every kernel reads only what an earlier kernel of the same call chain
+    wrote.  A whole ragged generation in lock step (logits compared element by element) would turn any read of
+    unwritten memory into NaN."""
+    E = engine()
+    shape = getattr(synth, shape_name)
+    P, L, Bk = 37, 41, 16
+    om = model_from_synth(shape, seed=6)
+    gm = E.Model.from_synth(shape, seed=6, max_batch=2, max_seq=P + L + 11, max_block=Bk, max_copies=8)
+    sess = E.Session(gm, poison=True)
+    x0 = synth.sequence(6, 0, P, L, shape)
+    sess.set_sequence(0, x0, P)
+    kw = dict(block_len=Bk, n_copies=copies)
+    st = lockstep_generate(E, sess, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw),
+                           tol=4e-2 if shape_name == "TINY_PEAKY" else 2e-2)
+    assert sess.status() == 0 and np.isfinite(st["worst_logit"]) and np.isfinite(st["worst_conf"])
+    assert_near_ties_only(st)
+    # the fused product path and the device-resident loop on the same poisoned buffers
+    sess.set_sequence(0, x0, P)
+    toks, trace = E.generate(sess, E.DecodeParams(**kw), resident=True)
+    assert sess.status() == 0 and (toks[0][P:] != shape.mask_id).all()
+    assert np.array_equal(toks[0], st["tokens_final"])
+    sess.close(); gm.close()

@@ -67,4 +67,5 @@ def test_persistent_step_on_edge_shapes():
         "import test_gpu_edges as t\n"
         f"for c in t.CASES:\n    if c[0] in {names!r}: t.test_edge_case_in_lockstep(*c)\n"
         "t.test_an_expired_device_wait_is_reported_and_the_session_stays_usable()\n"
+        "for a in (('TINY_PEAKY', 1), ('TINY_PEAKY', 8), ('TINY_HD128', 4)): t.test_poisoned_workspace_reads_nothing_unwritten(*a)\n"
         "print('persistent edges ok')\n", "persistent edges ok", timeout=1500)
