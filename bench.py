@@ -359,7 +359,10 @@ def run_cuda(args, wl):
     step_med = float(np.median(step_ms)) if step_ms else None
     step_gbs = step_bytes / (step_med * 1e-3) / 1e9 if step_med else None
     # the step is a READ stream; the measured peak is a read+write copy: a read-only probe in the same run
-    read_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}") if rank == 0 else None
+    try:
+        read_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}") if rank == 0 else None
+    except Exception:
+        read_gbs = None
     layer_traffic = recorded_layer_traffic()
     rows = wl.batch * wl.block_len * wl.n_copies
     frac_of = lambda gbs, peak: (gbs / peak) if (gbs and peak) else None
@@ -429,7 +432,10 @@ def run_cuda(args, wl):
             modes[mode]["eff_nfe_vs_fast_dllm"] = modes[mode]["eff_nfe"] / modes["fast_dllm"]["eff_nfe"]
         line["modes"] = modes
     if rank == 0 and world == 1 and args.workload == "cfg3_8b_c1" and not args.no_secondary:
-        line["secondary"] = secondary_measurements(E, synth, gm, peaks, args)
+        try:
+            line["secondary"] = secondary_measurements(E, synth, gm, peaks, args)
+        except Exception as exc:      # the headline line must come out whatever happens to the extras
+            line["secondary"] = {"error": f"{type(exc).__name__}: {exc}"}
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             r = oracle_sample(wl)
