@@ -359,10 +359,14 @@ def run_cuda(args, wl):
     step_med = float(np.median(step_ms)) if step_ms else None
     step_gbs = step_bytes / (step_med * 1e-3) / 1e9 if step_med else None
     # the step is a READ stream; the measured peak is a read+write copy: a read-only probe in the same run
-    try:
-        read_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}") if rank == 0 else None
-    except Exception:
-        read_gbs = None
+    # (16-byte loads), and the same through rings of bulk copies, the way the projections fetch their weights
+    read_gbs = bulk_gbs = None
+    if rank == 0:
+        try:
+            read_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}")
+            bulk_gbs = E.measure_read_bandwidth(4 << 30, 4, f"cuda:{local}", bulk=True)
+        except Exception:
+            pass
     layer_traffic = recorded_layer_traffic()
     rows = wl.batch * wl.block_len * wl.n_copies
     frac_of = lambda gbs, peak: (gbs / peak) if (gbs and peak) else None
@@ -376,6 +380,7 @@ def run_cuda(args, wl):
                 "algorithmic_bytes": step_bytes, "ms": step_med, "rows": rows,
                 "frac_of_nominal_8tbs": frac_of(step_gbs, 8000.0),
                 "hbm_read_gbs": read_gbs, "frac_of_read_probe": frac_of(step_gbs, read_gbs),
+                "hbm_bulk_read_gbs": bulk_gbs, "frac_of_bulk_read_probe": frac_of(step_gbs, bulk_gbs),
                 "ms_in_resident_loop": loop_ms,
                 "frac_in_resident_loop": frac_of(step_bytes / (loop_ms * 1e-3) / 1e9 if loop_ms else None, peaks["hbm_gbs"]),
                 # DRAM bytes of a step: the ncu capture of the single-layer case recorded under profiles/ (the full

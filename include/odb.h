@@ -322,6 +322,13 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
  * Synchronous. */
 int32_t odb_measure_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s);
 
+/* The same measurement through the path the projections' weights take: one thread per SM keeps a ring of seven
+ * 16 KiB bulk copies (global to shared memory, completion on an mbarrier) in flight over its contiguous share of
+ * the buffer; the bytes are not consumed.  Same arguments (bytes at least 16 KiB per SM); the whole 16 KiB chunks
+ * of every SM's share are what is read and counted.  Waits are bounded: ODB_ERR_TIMEOUT if a copy never
+ * completed.  Allocates and frees one status word (synchronous, not for use inside a capture). */
+int32_t odb_measure_bulk_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s);
+
 /* Algorithmic bytes one odb_block_decode_step must move for `rows` query rows and `keys`
  * visible cached positions per sequence (weights once + K/V once); used by the benchmark. */
 double odb_step_algorithmic_bytes(const odb_config* cfg, int32_t keys);

@@ -89,6 +89,7 @@ SIGNATURES = {
     "odb_session_profile": (C.c_int32, [C.c_void_p, C.c_int32]),
     "odb_session_profile_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "odb_measure_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),
+    "odb_measure_bulk_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),
     "odb_step_algorithmic_bytes": (C.c_double, [C.POINTER(odb_config), C.c_int32]),
 }
 

@@ -382,7 +382,66 @@ __global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restric
     if (acc == 0x9E3779B9u && sink) atomicAdd(sink, 1u);
 }
 
+// The same probe through the copy engine the projections use: one thread per CTA keeps a ring of kBulkStages
+// bulk copies (global -> shared, completion on an mbarrier) of kBulkChunk bytes in flight over the CTA's
+// contiguous share of the buffer; nothing consumes the bytes.  Waits are bounded: on expiry the thread stops
+// issuing, waits (bounded again) for the copies it has in flight, and reports through `status`.
+constexpr int kBulkStages = 7;
+constexpr int kBulkChunk = 16384;
+
+__global__ void __launch_bounds__(32) bulk_read_stream_kernel(const uint8_t* __restrict__ src, long long chunks_per_cta, int* status) {
+    extern __shared__ __align__(1024) uint8_t ring[];
+    __shared__ __align__(8) uint64_t full[kBulkStages];
+    __shared__ int abort_flag;
+    if (threadIdx.x != 0) return;
+    abort_flag = 0;
+    for (int i = 0; i < kBulkStages; ++i)
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&full[i])));
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    const uint8_t* base = src + static_cast<size_t>(blockIdx.x) * chunks_per_cta * kBulkChunk;
+    auto issue = [&](long long i, int st) {
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&full[st])), "r"(kBulkChunk) : "memory");
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                         smem_u32(ring + static_cast<size_t>(st) * kBulkChunk)),
+                     "l"(base + static_cast<size_t>(i) * kBulkChunk), "r"(kBulkChunk), "r"(smem_u32(&full[st]))
+                     : "memory");
+    };
+    const long long pre = chunks_per_cta < kBulkStages ? chunks_per_cta : kBulkStages;
+    uint32_t in_flight = 0;   // bit s: stage s holds a copy that has not been waited for
+    for (long long i = 0; i < pre; ++i) { issue(i, static_cast<int>(i)); in_flight |= 1u << i; }
+    long long issued = pre;
+    int st = 0;
+    uint32_t ph = 0;
+    bool ok = true;
+    for (long long i = 0; i < chunks_per_cta; ++i) {
+        if (!mbar_wait_bounded(&full[st], ph, &abort_flag, status)) { ok = false; break; }
+        in_flight &= ~(1u << st);
+        if (issued < chunks_per_cta) { issue(issued, st); ++issued; in_flight |= 1u << st; }
+        if (++st == kBulkStages) { st = 0; ph ^= 1; }
+    }
+    if (!ok) {   // wait (bounded) for the copies still in flight before the shared memory is given back
+        int ignored = 0;
+        for (int s = 0; s < kBulkStages; ++s) {
+            if (!(in_flight & (1u << s))) continue;
+            abort_flag = 0;
+            mbar_wait_bounded(&full[s], s >= st ? ph : ph ^ 1, &abort_flag, &ignored);   // stages behind the ring position are one phase on
+        }
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_bulk_read_stream(const void* src, size_t bytes, int grid, int* status, size_t* streamed, cudaStream_t st) {
+    const long long chunks_per_cta = static_cast<long long>(bytes / (static_cast<size_t>(grid) * kBulkChunk));
+    if (chunks_per_cta < 1) return cudaErrorInvalidValue;
+    const int smem = kBulkStages * kBulkChunk;
+    static std::atomic<unsigned long long> limit_set{0};
+    cudaError_t e = set_smem_limit_once(limit_set, bulk_read_stream_kernel, smem);
+    if (e != cudaSuccess) return e;
+    *streamed = static_cast<size_t>(chunks_per_cta) * grid * kBulkChunk;
+    bulk_read_stream_kernel<<<grid, 32, smem, st>>>(static_cast<const uint8_t*>(src), chunks_per_cta, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned int* sink, int grid, cudaStream_t st) {
     read_stream_kernel<<<grid, 512, 0, st>>>(static_cast<const uint4*>(src), bytes / 16, sink);

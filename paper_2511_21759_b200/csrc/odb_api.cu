@@ -1042,28 +1042,57 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
     return ODB_OK;
 }
 
-int32_t odb_measure_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s) {
+namespace {
+
+// kind 0: 16-byte loads from every thread; kind 1: a ring of bulk copies per SM (the projections' weight path)
+int32_t measure_read(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s, int kind) {
     if (!buf || !gb_per_s || reps < 1 || bytes < (1u << 20)) return ODB_ERR_ARG;
     if ((reinterpret_cast<uintptr_t>(buf) & 15) || (bytes & 15)) return ODB_ERR_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int dev = 0, sms = 0;
     ODB_CUDA(cudaGetDevice(&dev));
     ODB_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    int* status = nullptr;
+    if (kind == 1) {
+        if (bytes < static_cast<size_t>(sms) * 16384) return ODB_ERR_ARG;
+        ODB_CUDA(cudaMalloc(&status, sizeof(int)));
+        cudaError_t z = cudaMemsetAsync(status, 0, sizeof(int), st);
+        if (z != cudaSuccess) { cudaFree(status); return cuda_fail(z); }
+    }
+    size_t per_pass = bytes;
+    auto pass = [&]() -> cudaError_t {
+        return kind == 1 ? launch_bulk_read_stream(buf, bytes, sms, status, &per_pass, st)
+                         : launch_read_stream(buf, bytes, nullptr, 4 * sms, st);
+    };
     cudaEvent_t e0 = nullptr, e1 = nullptr;
-    ODB_CUDA(cudaEventCreate(&e0));
-    cudaError_t e = cudaEventCreate(&e1);
-    if (e == cudaSuccess) e = launch_read_stream(buf, bytes, nullptr, 4 * sms, st);   // warm-up pass
+    cudaError_t e = cudaEventCreate(&e0);
+    if (e == cudaSuccess) e = cudaEventCreate(&e1);
+    if (e == cudaSuccess) e = pass();   // warm-up pass
     if (e == cudaSuccess) e = cudaEventRecord(e0, st);
-    for (int i = 0; i < reps && e == cudaSuccess; ++i) e = launch_read_stream(buf, bytes, nullptr, 4 * sms, st);
+    for (int i = 0; i < reps && e == cudaSuccess; ++i) e = pass();
     if (e == cudaSuccess) e = cudaEventRecord(e1, st);
     if (e == cudaSuccess) e = cudaEventSynchronize(e1);
     float ms = 0.f;
     if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
-    cudaEventDestroy(e0);
+    int waited_out = 0;
+    if (e == cudaSuccess && status) e = cudaMemcpy(&waited_out, status, sizeof(int), cudaMemcpyDeviceToHost);
+    if (e0) cudaEventDestroy(e0);
     if (e1) cudaEventDestroy(e1);
+    if (status) cudaFree(status);
     if (e != cudaSuccess) return cuda_fail(e);
-    *gb_per_s = static_cast<double>(bytes) * reps / (static_cast<double>(ms) * 1e-3) / 1e9;
+    if (waited_out != 0) return ODB_ERR_TIMEOUT;
+    *gb_per_s = static_cast<double>(per_pass) * reps / (static_cast<double>(ms) * 1e-3) / 1e9;
     return ODB_OK;
+}
+
+}  // namespace
+
+int32_t odb_measure_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s) {
+    return measure_read(buf, bytes, reps, stream, gb_per_s, 0);
+}
+
+int32_t odb_measure_bulk_read_bandwidth(const void* buf, size_t bytes, int32_t reps, void* stream, double* gb_per_s) {
+    return measure_read(buf, bytes, reps, stream, gb_per_s, 1);
 }
 
 double odb_step_algorithmic_bytes(const odb_config* c, int32_t keys) {

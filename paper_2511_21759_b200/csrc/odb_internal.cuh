@@ -230,6 +230,8 @@ cudaError_t launch_reduce_partials(const float* partial, int splits, size_t stri
 
 // read-only streaming kernel over `bytes` of src (a multiple of 16), `grid` blocks of 512 threads
 cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned int* sink, int grid, cudaStream_t st);
+// bulk-copy ring probe; *streamed = the bytes one launch reads (whole chunks per CTA); `status` is a device word
+cudaError_t launch_bulk_read_stream(const void* src, size_t bytes, int grid, int* status, size_t* streamed, cudaStream_t st);
 cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, float* h, int M, int d,
                          cudaStream_t st);
 // The part of RMSNorm that is not a row scalar, for rows r = map ? map[i] : i of the residual stream:

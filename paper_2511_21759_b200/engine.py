@@ -255,14 +255,15 @@ def debug_gemm(x: torch.Tensor, w: torch.Tensor, k_splits: int = 0) -> torch.Ten
     return out
 
 
-def measure_read_bandwidth(n_bytes: int = 4 << 30, reps: int = 4, device="cuda") -> float:
-    """GB/s of a read-only streaming kernel over a buffer of n_bytes (odb_measure_read_bandwidth)."""
+def measure_read_bandwidth(n_bytes: int = 4 << 30, reps: int = 4, device="cuda", bulk: bool = False) -> float:
+    """GB/s of a read-only stream over a buffer of n_bytes: 16-byte loads (odb_measure_read_bandwidth) or, with
+    bulk=True, rings of bulk copies as the projections' weights are fetched (odb_measure_bulk_read_bandwidth)."""
     buf = torch.empty(n_bytes, dtype=torch.uint8, device=device)
     buf.fill_(1)
     st = torch.cuda.current_stream(buf.device)
     out = C.c_double()
-    B.check(B.lib().odb_measure_read_bandwidth(buf.data_ptr(), buf.numel(), reps, C.c_void_p(st.cuda_stream), C.byref(out)),
-            "odb_measure_read_bandwidth")
+    name = "odb_measure_bulk_read_bandwidth" if bulk else "odb_measure_read_bandwidth"
+    B.check(getattr(B.lib(), name)(buf.data_ptr(), buf.numel(), reps, C.c_void_p(st.cuda_stream), C.byref(out)), name)
     return out.value
 
 

@@ -203,3 +203,26 @@ def test_poisoned_workspace_reads_nothing_unwritten(shape_name, copies):
     assert sess.status() == 0 and (toks[0][P:] != shape.mask_id).all()
     assert np.array_equal(toks[0], st["tokens_final"])
     sess.close(); gm.close()
+
+
+@requires_gpu
+def test_read_bandwidth_probes_are_sane_and_validate_their_arguments():
+    """The two read-stream probes the benchmark quotes beside the copy bandwidth: both land between 3 and 9 TB/s on
+    a buffer far larger than L2, the bulk-copy ring (the projections' weight path) is not slower than 90 % of the
+    plain loads, and bad arguments are refused before any launch."""
+    import ctypes as C
+    import torch
+    from paper_2511_21759_b200 import binding as B
+    E = engine()
+    ld = E.measure_read_bandwidth(1 << 30, 3)
+    bulk = E.measure_read_bandwidth(1 << 30, 3, bulk=True)
+    print(f"\nread probes: 16-byte loads {ld:.0f} GB/s, bulk-copy rings {bulk:.0f} GB/s")
+    assert 3000 < ld < 9000 and 3000 < bulk < 9000
+    assert bulk > 0.9 * ld
+    buf = torch.empty(1 << 21, dtype=torch.uint8, device="cuda")
+    out = C.c_double()
+    for fn in (B.lib().odb_measure_read_bandwidth, B.lib().odb_measure_bulk_read_bandwidth):
+        assert fn(buf.data_ptr() + 8, 1 << 20, 1, None, C.byref(out)) == B.ODB_ERR_ARG      # misaligned
+        assert fn(buf.data_ptr(), 1 << 10, 1, None, C.byref(out)) == B.ODB_ERR_ARG          # too small
+        assert fn(buf.data_ptr(), 1 << 20, 0, None, C.byref(out)) == B.ODB_ERR_ARG          # no passes
+        assert fn(None, 1 << 20, 1, None, C.byref(out)) == B.ODB_ERR_ARG
