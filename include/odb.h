@@ -84,7 +84,28 @@ typedef struct odb_config {
     int32_t max_block;  /* block length upper bound (<= 64) */
     int32_t max_copies; /* 1, 4 or 8 */
     int32_t with_lm_head; /* 0: single-layer microbench without LM head (no conf/tok outputs) */
+    int32_t tp_world;   /* tensor-parallel ranks sharing this model: 0 or 1 = none; else 2, 4 or 8 (see below) */
+    int32_t tp_rank;    /* this rank, 0 .. tp_world-1 */
 } odb_config;
+
+/* Tensor-parallel shards (tp_world = R > 1; beyond the paper, which runs on one GPU: the forward of Section 4.1
+ * with its weights divided over R GPUs).  The shape fields above keep their GLOBAL values; requirements:
+ * n_heads % R == 0, d_ffn % (64 R) == 0.  Rank r holds, and odb_weights describes, only its shard:
+ *   wqkv  [3*Hl*head_dim][d_model]  rows = [Wq; Wk; Wv] of heads [r*Hl, (r+1)*Hl), Hl = n_heads / R
+ *   wo    [d_model][Hl*head_dim]    the input columns of those heads
+ *   wgu   gate/up-packed, the FFN features [r*Fl, (r+1)*Fl), Fl = d_ffn / R
+ *   wd    [d_model][Fl]             the input columns of those features
+ *   lm_head [Vl][d_model]           the vocabulary rows of tiles [r*Tl, min(T, (r+1)*Tl)), T = ceil(vocab / 128),
+ *                                   Tl = ceil(T / R), a tile = 128 consecutive ids (odb_tp_vocab_range)
+ * embedding, gains and the residual stream are replicated; the K/V cache holds the rank's own heads
+ * (odb_kv_bytes shrinks accordingly).  The O and down projections produce partial sums of the full d_model
+ * width: their epilogue stores every fp32 partial tile straight into the receive buffer of EVERY rank (plain
+ * stores to peer memory, no bulk or multicast copy from a peer anywhere), a one-thread kernel then raises this
+ * rank's flag on every rank, and the consuming RMSNorm kernel, behind a bounded wait on the R flags, adds all
+ * partials in (rank, split) order - the same order on every rank, so the residual streams stay bit-identical.
+ * The LM head's per-tile confidence statistics are exchanged the same way and merged in tile order.
+ * Not available under TP: the device-resident loop, the logits test mode, the persistent step kernel. */
+#define ODB_TP_MAX_WORLD 8
 
 /* Device pointers to the weights; per-layer arrays are HOST arrays of n_layers device pointers.
  * wqkv = [Wq; Wk; Wv] stacked on the output dimension, wgu = [Wgate; Wup] likewise.
@@ -314,6 +335,34 @@ int32_t odb_gemm_static_scratch(const void* x, const void* w_packed, float* out,
  * Launches are counted whether profiling is on or off. */
 int32_t odb_session_profile(odb_session* s, int32_t enable);
 int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* launches_by_kind);
+
+/* ---- tensor parallelism (sessions of a model created with tp_world > 1) ----
+ * odb_session_tp_buffers: device pointers (inside this session's workspace) of the three regions its peers
+ * write into - receive slots for the partial sums, flag words, confidence statistics - and their sizes.  The
+ * caller carries them to the other ranks (same process: as they are; other processes: as offsets into an
+ * inter-process mapping of the workspace allocation) and hands every rank the R pointers of each kind with
+ * odb_session_tp_attach (entry tp_rank is this session's own).  Until attached, refresh / step calls return
+ * ODB_ERR_STATE.  Every rank must issue the same sequence of refresh / step / accept calls.
+ * The library never waits on the host for a peer: a rank that never arrives makes the bounded device-side wait
+ * expire, which the next odb_unmask_accept or odb_session_status reports as ODB_ERR_TIMEOUT. */
+int32_t odb_session_tp_buffers(odb_session* s, void** recv, size_t* recv_bytes, void** flags, size_t* flags_bytes,
+                               void** conf, size_t* conf_bytes);
+int32_t odb_session_tp_attach(odb_session* s, void* const* peer_recv, void* const* peer_flags, void* const* peer_conf);
+/* first and one-past-last vocabulary id of rank `rank`'s LM-head shard; ODB_ERR_ARG for a bad rank, the
+ * configuration's own error for a configuration odb_model_create would refuse */
+int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, int32_t* last);
+/* Test facility for running all ranks of a group on ONE GPU without kernels that wait on one another: a forward
+ * is cut into odb_tp_segment_count segments at its exchange points (after a flag is raised, before it is waited
+ * for).  With a range set, a refresh / step call launches only the kernels of segments [first, last) of the
+ * forward; the caller issues segment k on every rank before segment k+1 on any, on one stream, so that every
+ * flag is up before its wait kernel starts.  first = 0 begins a forward, later ranges continue it; the accept
+ * follows the last segment.  first < 0 restores whole forwards. */
+int32_t odb_tp_segment_count(const odb_config* cfg);
+int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last);
+/* Test facility: one launch of the flag wait for exchange `kind` (0, 1: partial-sum slots, 2: statistics) with the
+ * next sequence number and the given cycle limit; nothing raises the flags, so the wait expires and the status
+ * word reports ODB_ERR_TIMEOUT (read and cleared by odb_session_status). */
+int32_t odb_debug_tp_expire_wait(odb_session* s, int32_t kind, int64_t limit_cycles);
 
 /* Measurement: the rate at which this GPU streams `bytes` (a multiple of 16, 16-byte aligned, at least 1 MiB; use
  * far more than the L2 holds) of device memory with a read-only kernel of 16-byte loads, `reps` passes after one

@@ -32,7 +32,8 @@ class odb_config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_heads", "head_dim", "d_ffn", "vocab",
                                          "mask_id", "eos_id")] + \
                [("rope_theta", C.c_float), ("rms_eps", C.c_float)] + \
-               [(n, C.c_int32) for n in ("max_batch", "max_seq", "max_block", "max_copies", "with_lm_head")]
+               [(n, C.c_int32) for n in ("max_batch", "max_seq", "max_block", "max_copies", "with_lm_head",
+                                         "tp_world", "tp_rank")]
 
 
 class odb_weights(C.Structure):
@@ -88,6 +89,13 @@ SIGNATURES = {
                                             C.c_void_p]),
     "odb_session_profile": (C.c_int32, [C.c_void_p, C.c_int32]),
     "odb_session_profile_read": (C.c_int32, [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
+    "odb_session_tp_buffers": (C.c_int32, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t), C.POINTER(C.c_void_p),
+                                           C.POINTER(C.c_size_t), C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]),
+    "odb_session_tp_attach": (C.c_int32, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
+    "odb_tp_vocab_range": (C.c_int32, [C.POINTER(odb_config), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
+    "odb_tp_segment_count": (C.c_int32, [C.POINTER(odb_config)]),
+    "odb_debug_tp_segments": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
+    "odb_debug_tp_expire_wait": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
     "odb_measure_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),
     "odb_measure_bulk_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),
     "odb_step_algorithmic_bytes": (C.c_double, [C.POINTER(odb_config), C.c_int32]),

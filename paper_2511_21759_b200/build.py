@@ -7,7 +7,7 @@ import subprocess
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libodb.so")
-SOURCES = ["gemm_tcgen05.cu", "gemm_static.cu", "elementwise.cu", "attention.cu", "attention_tc.cu", "control.cu", "step_persistent.cu", "odb_api.cu"]
+SOURCES = ["gemm_tcgen05.cu", "gemm_static.cu", "elementwise.cu", "attention.cu", "attention_tc.cu", "control.cu", "tensor_parallel.cu", "step_persistent.cu", "odb_api.cu"]
 
 
 def _stale() -> bool:

@@ -392,7 +392,7 @@ constexpr int kBulkChunk = 16384;
 __global__ void __launch_bounds__(32) bulk_read_stream_kernel(const uint8_t* __restrict__ src, long long chunks_per_cta, int* status) {
     extern __shared__ __align__(1024) uint8_t ring[];
     __shared__ __align__(8) uint64_t full[kBulkStages];
-    __shared__ int abort_flag;
+    __shared__ int abort_flag, drain_status;
     if (threadIdx.x != 0) return;
     abort_flag = 0;
     for (int i = 0; i < kBulkStages; ++i)
@@ -420,11 +420,11 @@ __global__ void __launch_bounds__(32) bulk_read_stream_kernel(const uint8_t* __r
         if (++st == kBulkStages) { st = 0; ph ^= 1; }
     }
     if (!ok) {   // wait (bounded) for the copies still in flight before the shared memory is given back
-        int ignored = 0;
+        drain_status = 0;
         for (int s = 0; s < kBulkStages; ++s) {
             if (!(in_flight & (1u << s))) continue;
             abort_flag = 0;
-            mbar_wait_bounded(&full[s], s >= st ? ph : ph ^ 1, &abort_flag, &ignored);   // stages behind the ring position are one phase on
+            mbar_wait_bounded(&full[s], s >= st ? ph : ph ^ 1, &abort_flag, &drain_status);   // stages behind the ring position are one phase on
         }
     }
 }

@@ -49,7 +49,7 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
             float* __restrict__ partial, __nv_bfloat16* __restrict__ act_out, RowScale rs,
             ConfEpilogue ce, int M, int N, int nkb_total, int nkb_per_split, int stages,
             int l2_prefetch, int pair_tiles_x, int pair_tiles_y,
-            int* status) {
+            int* status, const __grid_constant__ PeerOut po) {
     extern __shared__ __align__(1024) uint8_t smem_raw[];
     constexpr uint32_t kABytes = kBM * kBK * 2;
     constexpr int kBRows = PAIR ? BN / 2 : BN;        // activation rows this CTA stages
@@ -228,19 +228,33 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
         if constexpr (EPI == EPI_PARTIAL) {
             const int n = n0 + q * 32 + lane;
             if (ok) {
-                float* out = partial + static_cast<size_t>(split) * M * N;
+                const size_t split_off = static_cast<size_t>(split) * M * N;
+                float* out = partial + split_off;
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
                     uint32_t v[32];
                     tmem_ld32(tmem_acc + (static_cast<uint32_t>(q * 32) << 16) + static_cast<uint32_t>(c * 32), v);
                     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                    if (po.n == 0) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int m = m0 + c * 32 + j;
-                        const float sc = rs.ssq ? sh->scale[c * 32 + j] : 1.0f;
-                        if (n < N && m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]) * sc;
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + c * 32 + j;
+                            const float sc = rs.ssq ? sh->scale[c * 32 + j] : 1.0f;
+                            if (n < N && m < M) out[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]) * sc;
+                        }
+                    } else {
+                        // tensor-parallel partial sums: the tile goes to the receive buffer of every rank
+                        for (int r = 0; r < po.n; ++r) {
+                            float* dst = po.partial[r] + split_off;
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int m = m0 + c * 32 + j;
+                                if (n < N && m < M) dst[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
+                            }
+                        }
                     }
                 }
+                if (po.n > 0) __threadfence_system();
             }
         } else if constexpr (EPI == EPI_CONF) {
             // LM head fused with the confidence reduction: the logits of this tile (128 vocabulary
@@ -268,12 +282,13 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
 #pragma unroll 8
                 for (int i = 0; i < 32; ++i) {
                     const int n = n0 + part * 32 + i;
+                    const int id = n + ce.tile0 * kBM;                  // vocabulary id (a shard starts at tile0)
                     const float l = xch[m_l * 129 + part * 32 + i] * sc;
-                    if (n < N && n != ce.mask_id) {
+                    if (n < N && id != ce.mask_id) {
                         if (l > mx) {
                             sum = sum * expf(mx - l) + 1.0f;            // first element: 0 * exp(-inf) + 1
                             mx = l;
-                            idx = n;
+                            idx = id;
                         } else {
                             sum += expf(l - mx);
                         }
@@ -289,7 +304,12 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                 if (ok && part == 0 && m < M) {
                     ConfPartial p;
                     p.m = mx; p.s = sum; p.idx = idx;
-                    ce.part[static_cast<size_t>(m) * n_tiles + n_tile] = p;
+                    if (po.n == 0) {
+                        ce.part[static_cast<size_t>(m) * n_tiles + n_tile] = p;
+                    } else {
+                        for (int r = 0; r < po.n; ++r) po.conf[r][static_cast<size_t>(m) * ce.tiles_total + ce.tile0 + n_tile] = p;
+                        __threadfence_system();
+                    }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
@@ -503,11 +523,11 @@ cudaError_t launch_bn(const GemmArgs& a, cudaStream_t st) {
         cfg.attrs = attr;
         cfg.numAttrs = pdl_enabled() ? 2 : 1;
         return cudaLaunchKernelEx(&cfg, gemm_kernel<BN, EPI, PAIR>, a.tmap_w, tmx, a.partial, a.act_out, a.row_scale, a.conf,
-                                  a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, tiles_x, tiles_y, a.status);
+                                  a.M, a.N, nkb_total, nkb_per_split, stages, pdl_enabled() ? l2_prefetch : 0, tiles_x, tiles_y, a.status, a.peers);
     } else {
         return launch_kernel(gemm_kernel<BN, EPI, PAIR>, grid, dim3(kThreads), smem, st, a.tmap_w, tmx, a.partial, a.act_out,
                              a.row_scale, a.conf, a.M, a.N, nkb_total, nkb_per_split, stages,
-                             pdl_enabled() ? l2_prefetch : 0, 0, 0, a.status);
+                             pdl_enabled() ? l2_prefetch : 0, 0, 0, a.status, a.peers);
     }
 }
 

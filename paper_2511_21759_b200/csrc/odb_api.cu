@@ -39,7 +39,32 @@ int32_t check_config(const odb_config* c) {
     if (c->max_block < 1 || c->max_block > kMaxBlock) return ODB_ERR_SHAPE;
     if (c->max_copies != 1 && c->max_copies != 4 && c->max_copies != 8) return ODB_ERR_SHAPE;
     if (c->mask_id < 0 || c->mask_id >= c->vocab || c->eos_id < 0 || c->eos_id >= c->vocab) return ODB_ERR_ARG;
+    if (c->tp_world > 1) {
+        const int R = c->tp_world;
+        if (R != 2 && R != 4 && R != 8) return ODB_ERR_SHAPE;
+        if (c->tp_rank < 0 || c->tp_rank >= R) return ODB_ERR_ARG;
+        if (c->n_heads % R || c->d_ffn % (64 * R)) return ODB_ERR_SHAPE;
+    } else if (c->tp_world < 0 || c->tp_rank != 0) {
+        return ODB_ERR_ARG;
+    }
     return ODB_OK;
+}
+
+// tensor-parallel shard sizes (the whole model when tp_world <= 1)
+int tp_ranks(const odb_config& c) { return c.tp_world > 1 ? c.tp_world : 1; }
+int heads_local(const odb_config& c) { return c.n_heads / tp_ranks(c); }
+int ffn_local(const odb_config& c) { return c.d_ffn / tp_ranks(c); }
+int vocab_tiles(const odb_config& c) { return (c.vocab + 127) / 128; }
+void vocab_shard(const odb_config& c, int rank, int* tile0, int* rows) {
+    const int T = vocab_tiles(c), R = tp_ranks(c), per = (T + R - 1) / R;
+    int t0 = rank * per, t1 = t0 + per;
+    if (t0 > T) t0 = T;
+    if (t1 > T) t1 = T;
+    const int first = t0 * 128;
+    int last = t1 * 128;
+    if (last > c.vocab) last = c.vocab;
+    *tile0 = t0;
+    *rows = last > first ? last - first : 0;
 }
 
 // Carve-up of the caller's workspace.  Offsets only; shared by odb_workspace_bytes and
@@ -48,6 +73,7 @@ struct Layout {
     size_t rows, lm_chunk, tiles, partial_rows, attn_rows;
     size_t rope, state, results, status, loop, x, row_tok, row_pos, row_seq, row_copy, row_flags, lm_rows, tile_buf, big_tile_buf, step_tile_buf;
     size_t h, a, inv, q, k, v, o, g, partial, logits, conf, tok, conf_part, part_o, part_ml, ptable, pbars, noise;
+    size_t tp_recv, tp_recv_slot, tp_flags, conf_part_bytes;   // tensor parallelism: two receive slots for partial sums, the flag words
     size_t total;
 };
 
@@ -62,7 +88,7 @@ Layout make_layout(const odb_config& c) {
     L.tiles = refresh_tiles > step_tiles ? refresh_tiles : step_tiles;
     L.partial_rows = L.rows > 4096 ? L.rows : 4096;
     L.attn_rows = L.rows > 2048 ? L.rows : 2048;
-    const size_t d = c.d_model, F = c.d_ffn;
+    const size_t d = c.d_model, F = ffn_local(c);
     const size_t nmax = 3 * d > 2 * F ? 3 * d : 2 * F;
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
@@ -95,7 +121,8 @@ Layout make_layout(const odb_config& c) {
     L.tok = take(4 * L.rows);
     {
         const size_t lm_tiles = (static_cast<size_t>(c.vocab) + 127) / 128;
-        L.conf_part = take(12 * L.lm_chunk * (lm_tiles > static_cast<size_t>(kConfMaxChunks) ? lm_tiles : kConfMaxChunks));
+        L.conf_part_bytes = 12 * L.lm_chunk * (lm_tiles > static_cast<size_t>(kConfMaxChunks) ? lm_tiles : kConfMaxChunks);
+        L.conf_part = take(L.conf_part_bytes);
     }
     L.part_o = take(4 * L.attn_rows * d);
     L.part_ml = take(4 * L.attn_rows * c.n_heads * 2);
@@ -103,6 +130,14 @@ Layout make_layout(const odb_config& c) {
     L.ptable = take(3 * align_up(step_persistent_table_bytes(c.n_layers)));
     L.pbars = take(step_persistent_barrier_bytes(c.n_layers));
     L.noise = take(sizeof(float) * c.max_batch * kMaxLoopIters * kMaxBlock);   // deviates of the stochastic reverse step
+    if (c.tp_world > 1) {
+        // a slot holds the [rank][split][rows][d_model] fp32 partials of one O or down projection: up to 16 partials
+        // of a decode step, fewer (whatever fits) of a refresh
+        const size_t all_ranks = 4 * static_cast<size_t>(c.tp_world) * L.rows * d;   // one partial per rank of the largest forward
+        L.tp_recv_slot = align_up(4 * L.partial_rows * nmax > all_ranks ? 4 * L.partial_rows * nmax : all_ranks);
+        L.tp_recv = take(2 * L.tp_recv_slot);
+        L.tp_flags = take(sizeof(unsigned int) * kTpKinds * kTpMaxWorld);
+    }
     L.total = off;
     return L;
 }
@@ -158,6 +193,17 @@ struct odb_session {
     int pmaxp[4];             // persistent step kernel: most parts per output tile of the four projections of a layer
     bool persistent_off;      // the model is beyond the persistent step kernel's limits: steps run as separate kernels
     bool ptable_built[3];     // persistent step kernel: projection table for 32 / 64 / 128 rows per tile is on the device
+    // tensor parallelism (model with tp_world > 1)
+    struct Tp {
+        bool attached = false;
+        float* recv[kTpMaxWorld] = {};          // every rank's receive region (two slots), own at index rank
+        ConfPartial* conf[kTpMaxWorld] = {};    // every rank's confidence-statistics buffer
+        TpPeers peers;                          // every rank's flag words
+        unsigned int seq[kTpKinds] = {0, 0, 0}; // sequence number of the latest completed exchange per kind
+        unsigned int fwd_base[kTpKinds] = {0, 0, 0};   // seq at the start of the forward in progress
+        int seg_first = -1, seg_last = -1;      // test facility: segments of a forward to launch (-1: all)
+        long long wait_limit = kWaitLimitCycles;
+    } tp;
     template <class T> T* at(size_t off) const { return reinterpret_cast<T*>(ws + off); }
 };
 
@@ -216,7 +262,7 @@ int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model*
     m->embed = static_cast<const __nv_bfloat16*>(w->embed);
     m->final_norm = w->final_norm;
     m->p_lm = w->lm_head;
-    const int d = cfg->d_model, F = cfg->d_ffn, nl = cfg->n_layers;
+    const int d = cfg->d_model, F = ffn_local(*cfg), da = heads_local(*cfg) * cfg->head_dim, nl = cfg->n_layers;
     m->tm_qkv.resize(nl); m->tm_o.resize(nl); m->tm_gu.resize(nl); m->tm_d.resize(nl);
     cudaError_t e = cudaSuccess;
     for (int l = 0; l < nl && e == cudaSuccess; ++l) {
@@ -229,12 +275,20 @@ int32_t odb_model_create(const odb_config* cfg, const odb_weights* w, odb_model*
         m->p_qkv.push_back(w->wqkv[l]);
         m->p_o.push_back(w->wo[l]);
         m->p_gu.push_back(w->wgu[l]);
-        e = make_weight_tmap(&m->tm_qkv[l], w->wqkv[l], 3 * d, d);
-        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_o[l], w->wo[l], d, d);
+        e = make_weight_tmap(&m->tm_qkv[l], w->wqkv[l], 3 * da, d);
+        if (e == cudaSuccess) e = make_weight_tmap(&m->tm_o[l], w->wo[l], d, da);
         if (e == cudaSuccess) e = make_gate_up_tmap(&m->tm_gu[l], w->wgu[l], F, d);
         if (e == cudaSuccess) e = make_weight_tmap(&m->tm_d[l], w->wd[l], d, F);
     }
-    if (e == cudaSuccess && cfg->with_lm_head) e = make_weight_tmap(&m->tm_lm, w->lm_head, cfg->vocab, d);
+    if (e == cudaSuccess && cfg->with_lm_head) {
+        int tile0 = 0, rows = cfg->vocab;
+        vocab_shard(*cfg, cfg->tp_rank, &tile0, &rows);
+        if (rows < 1) {   // more ranks than vocabulary tiles
+            delete m;
+            return ODB_ERR_SHAPE;
+        }
+        e = make_weight_tmap(&m->tm_lm, w->lm_head, rows, d);
+    }
     if (e != cudaSuccess) {
         delete m;
         return cuda_fail(e);
@@ -250,7 +304,7 @@ int32_t odb_model_destroy(odb_model* m) {
 
 size_t odb_kv_bytes(const odb_config* c) {
     if (check_config(c) != ODB_OK) return 0;
-    return static_cast<size_t>(c->max_batch) * c->n_layers * 2 * c->n_heads * c->max_seq * c->head_dim * 2;
+    return static_cast<size_t>(c->max_batch) * c->n_layers * 2 * heads_local(*c) * c->max_seq * c->head_dim * 2;
 }
 
 size_t odb_workspace_bytes(const odb_config* c) {
@@ -286,7 +340,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     s->pinned_log = nullptr;
     s->pinned_iters = nullptr;
     s->ptable_built[0] = s->ptable_built[1] = s->ptable_built[2] = false;
-    s->persistent_off = false;
+    s->persistent_off = c.tp_world > 1;
     cudaError_t e = cudaMallocHost(&s->pinned_state, sizeof(SeqState) * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_log, sizeof(odb_result) * kMaxLoopIters * c.max_batch);
     if (e == cudaSuccess) e = cudaMallocHost(&s->pinned_iters, 4 * sizeof(int32_t));
@@ -310,6 +364,8 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     // in its softmax but still enter the P V product with weight zero, so they must hold finite values; the
     // q / k / v and output rows past a forward's last row are never read (the tensor maps end at that row).
     if (e == cudaSuccess) e = cudaMemsetAsync(kv, 0, odb_kv_bytes(&c), s->st);
+    if (e == cudaSuccess && c.tp_world > 1)
+        e = cudaMemsetAsync(s->ws + L.tp_flags, 0, sizeof(unsigned int) * kTpKinds * kTpMaxWorld, s->st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->st);
     if (e != cudaSuccess) {
         odb_session_destroy(s);
@@ -526,7 +582,17 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     const odb_config& c = m->cfg;
     const Layout& L = s->L;
     if (!st) st = s->st;
-    const int d = c.d_model, F = c.d_ffn, H = c.n_heads, hd = c.head_dim;
+    // H, F, da: this rank's heads, FFN features and attention width (the whole model without tensor parallelism)
+    const int d = c.d_model, F = ffn_local(c), H = heads_local(c), hd = c.head_dim, da = H * hd;
+    const int R = tp_ranks(c);
+    odb_session::Tp& tp = s->tp;
+    // Tensor parallelism: a forward is a sequence of segments separated by its exchange points; `seg` counts them
+    // as the launches below are walked, and a launch is issued only if its segment is in the requested range.
+    int seg = 0;
+    if (tp.seg_first <= 0)   // a forward begins (always, unless a later segment range of one in progress is requested)
+        for (int k = 0; k < kTpKinds; ++k) tp.fwd_base[k] = tp.seq[k];
+    unsigned int xseq[kTpKinds] = {tp.fwd_base[0], tp.fwd_base[1], tp.fwd_base[2]};
+    auto seg_on = [&]() { return tp.seg_first < 0 || (seg >= tp.seg_first && seg < tp.seg_last); };
     float* h = s->at<float>(L.h);
     __nv_bfloat16* a = s->at<__nv_bfloat16>(L.a);
     float* inv = s->at<float>(L.inv);   // sum(x^2) slices of the RMSNorm whose operand is in `a`
@@ -544,8 +610,20 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     int* status = s->at<int>(L.status);
     const size_t nmax = 3 * static_cast<size_t>(d) > 2 * static_cast<size_t>(F) ? 3 * static_cast<size_t>(d)
                                                                                 : 2 * static_cast<size_t>(F);
-    auto gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, float* out, int rows, int N, int K, int* splits,
-                    const RowScale* row_scale = nullptr) {
+    // K splits of a projection with fp32 partial output; `exchanged`: the partials of all R ranks must fit a receive
+    // slot and the consumer's 16-partial limit
+    auto plan_splits = [&](int rows, int N, int K, bool exchanged) {
+        int sp = gemm_pick_splits(rows, N, K);
+        size_t cap = L.partial_rows * nmax / (static_cast<size_t>(rows) * N);
+        if (exchanged) {   // R blocks of `sp` partials in a receive slot (sized for at least one partial per rank)
+            cap = L.tp_recv_slot / sizeof(float) / (static_cast<size_t>(rows) * N * R);
+            if (cap > static_cast<size_t>(16 / R)) cap = 16 / R;
+        }
+        if (static_cast<size_t>(sp) > cap) sp = static_cast<int>(cap < 1 ? 1 : cap);
+        return sp;
+    };
+    auto gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, float* out, int rows, int N, int K, int sp,
+                    const RowScale* row_scale = nullptr, int slot = -1) {
         GemmArgs ga;
         ga.tmap_w = tw;
         ga.x = x;
@@ -553,19 +631,40 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         ga.act_out = nullptr;
         if (row_scale) ga.row_scale = *row_scale;
         ga.M = rows; ga.N = N; ga.K = K;
-        int sp = *splits > 0 ? *splits : gemm_pick_splits(rows, N, K);
-        const size_t cap = L.partial_rows * nmax / (static_cast<size_t>(rows) * N);
-        if (static_cast<size_t>(sp) > cap) sp = static_cast<int>(cap < 1 ? 1 : cap);
         ga.splits = sp;
         ga.status = status;
-        *splits = sp;
+        if (slot >= 0) {   // tensor-parallel partial sums: block `rank` of receive slot `slot` on every rank
+            ga.peers.n = R;
+            for (int r = 0; r < R; ++r)
+                ga.peers.partial[r] = tp.recv[r] + static_cast<size_t>(slot) * (L.tp_recv_slot / sizeof(float)) +
+                                      static_cast<size_t>(c.tp_rank) * sp * rows * N;
+        }
         return launch_gemm(ga, st);
+    };
+    // exchange point of kind `kind`: raise this rank's flag everywhere (end of a segment), wait for all flags
+    auto exchange = [&](int kind) -> int32_t {
+        const unsigned int sq = ++xseq[kind];
+        if (seg_on()) {
+            LaunchScope scope__(s, ODB_KIND_CONTROL);
+            ODB_CUDA(launch_tp_signal(tp.peers, kind, sq, st));
+        }
+        ++seg;
+        if (seg_on()) {
+            LaunchScope scope__(s, ODB_KIND_CONTROL);
+            ODB_CUDA(launch_tp_wait(tp.peers, kind, sq, tp.wait_limit, status, st));
+        }
+        return ODB_OK;
     };
 
 #define ODB_LAUNCH(kind, call)          \
     do {                                \
         LaunchScope scope__(s, kind);   \
         ODB_CUDA(call);                 \
+    } while (0)
+// a launch of the forward proper: only if its segment is requested (always, without tensor parallelism)
+#define ODB_FWD(kind, call)             \
+    do {                                \
+        if (seg_on()) ODB_LAUNCH(kind, call); \
     } while (0)
     if (!write_cache && n_tiles > 0 && use_persistent(s, M) && s->ptable_built[bn_index(M)] && (!c.with_lm_head || n_lm == M)) {
         // decode step as ONE persistent kernel: every projection, the short phases between them and the LM head
@@ -604,13 +703,13 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         } else if (c.with_lm_head) {
             // test mode: the kernel ended with the LM head's operand; the logits are materialised by a plain launch
             int sp = 1;
-            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, s->at<float>(L.logits), M, c.vocab, d, &sp, &inv_scale));
+            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, a, s->at<float>(L.logits), M, c.vocab, d, sp, &inv_scale));
             ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(s->at<float>(L.logits), M, c.vocab, c.mask_id, s->at<float>(L.conf),
                                                                  s->at<int32_t>(L.tok), s->ws + L.conf_part, st));
         }
         return ODB_OK;
     }
-    ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
+    ODB_FWD(ODB_KIND_ELEMENTWISE, launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
     const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
     int res_splits = 0;
     size_t res_stride = 0;
@@ -634,15 +733,15 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         }
         return pf;
     };
-    const size_t qkv_bytes = packed_weight_bytes(3 * d, d), o_bytes = packed_weight_bytes(d, d),
+    const size_t qkv_bytes = packed_weight_bytes(3 * da, d), o_bytes = packed_weight_bytes(d, da),
                  gu_bytes = packed_gate_up_bytes(F, d);
     for (int l = 0; l < c.n_layers; ++l) {
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
+        ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
                                                         hint_of(m->p_qkv[l], qkv_bytes, 0), st));
-        int sp = 0;
-        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * d, d, &sp));
+        int sp = plan_splits(M, 3 * da, d, false);
+        ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * da, d, sp));
         QkvRopeArgs qa;
-        qa.partial = partial; qa.splits = sp; qa.pstride = static_cast<size_t>(M) * 3 * d;
+        qa.partial = partial; qa.splits = sp; qa.pstride = static_cast<size_t>(M) * 3 * da;
         qa.scale = inv_scale;
         qa.rope = s->at<float2>(L.rope);
         qa.row_pos = s->cb.row_pos; qa.row_seq = s->cb.row_seq;
@@ -650,7 +749,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         qa.cache = write_cache ? s->kv : nullptr;
         qa.layer = l; qa.n_layers = c.n_layers; qa.H = H; qa.hd = hd; qa.max_seq = c.max_seq; qa.M = M;
         qa.pf = hint_of(m->p_o[l], o_bytes, 0);
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_qkv_rope(qa, st));
+        ODB_FWD(ODB_KIND_ELEMENTWISE, launch_qkv_rope(qa, st));
         if (n_step_tiles > 0) {
             // several copies: one work item serves all copies of a block, cached K/V loaded once
             StepAttnArgs sa;
@@ -676,12 +775,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
                 // with a work item for every CTA slot there is nothing to gain from key splits: one CTA per item takes
                 // the cached and the fresh keys and writes the final output (no partials, no merge kernel)
                 if (ks_env == 1 || (ks_env <= 0 && n_step_tiles * H >= 2 * 148)) sa.ksplit = 1;
-                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention_tc(sa, cache_rows, status, st));
+                ODB_FWD(ODB_KIND_ATTENTION, launch_step_attention_tc(sa, cache_rows, status, st));
                 if (sa.ksplit > 1)
-                    ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_combine(sa.part_o, sa.part_ml, o, M, H, hd, sa.ksplit, st));
+                    ODB_FWD(ODB_KIND_ATTENTION, launch_attention_combine(sa.part_o, sa.part_ml, o, M, H, hd, sa.ksplit, st));
             } else {
-                ODB_LAUNCH(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
-                ++s->launches[ODB_KIND_ATTENTION];
+                ODB_FWD(ODB_KIND_ATTENTION, launch_step_attention(sa, st));
+                if (seg_on()) ++s->launches[ODB_KIND_ATTENTION];
             }
         } else if (write_cache && hd == 128 && n_big_tiles > 0 && tc_attention) {
             // refresh with head dim 128: 128-row work items on the tcgen05 tensor cores, no key split
@@ -691,7 +790,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             aa.part_o = nullptr; aa.part_ml = nullptr;
             aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = 1;
             aa.pf = L2Prefetch{nullptr, 0};
-            ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention_tc(aa, status, st));
+            ODB_FWD(ODB_KIND_ATTENTION, launch_attention_tc(aa, status, st));
         } else {
         AttnArgs aa;
         aa.tiles = s->cb.tiles; aa.n_tiles = n_tiles;
@@ -700,12 +799,23 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         aa.layer = l; aa.n_layers = c.n_layers; aa.H = H; aa.hd = hd; aa.max_seq = c.max_seq; aa.M = M; aa.ksplit = ks;
         aa.early = write_cache ? 0 : 1;   // a refresh writes the cache it attends to: nothing may be read early
         aa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
-        ODB_LAUNCH(ODB_KIND_ATTENTION, launch_attention(aa, st));
-        if (ks > 1) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
+        ODB_FWD(ODB_KIND_ATTENTION, launch_attention(aa, st));
+        if (ks > 1 && seg_on()) ++s->launches[ODB_KIND_ATTENTION];   // the split merge is a second kernel
         }
-        sp = 0;
-        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, d, &sp));
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, partial, sp, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
+        sp = plan_splits(M, d, da, R > 1);
+        const float* o_sum = partial;   // the partial sums the next RMSNorm adds to the residual stream
+        int o_parts = sp;
+        if (R > 1) {
+            // every rank's partial tiles land in slot 0 of every rank; all R * sp partials are added in (rank, split) order
+            ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_o[l], o, nullptr, M, d, da, sp, nullptr, 0));
+            const int32_t xrc = exchange(0);
+            if (xrc != ODB_OK) return xrc;
+            o_sum = tp.recv[c.tp_rank];
+            o_parts = R * sp;
+        } else {
+            ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, da, sp));
+        }
+        ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, o_sum, o_parts, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
                                                         d, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
         {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
             GemmArgs ga;
@@ -717,29 +827,41 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             ga.M = M; ga.N = F; ga.K = d;
             ga.splits = 1;
             ga.status = status;
-            ODB_LAUNCH(ODB_KIND_GEMM, launch_gemm(ga, st));
+            ODB_FWD(ODB_KIND_GEMM, launch_gemm(ga, st));
         }
-        sp = 0;
-        ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, &sp));
-        res = partial; res_splits = sp; res_stride = static_cast<size_t>(M) * d;
+        sp = plan_splits(M, d, F, R > 1);
+        if (R > 1) {
+            ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_d[l], g, nullptr, M, d, F, sp, nullptr, 1));
+            const int32_t xrc = exchange(1);
+            if (xrc != ODB_OK) return xrc;
+            res = tp.recv[c.tp_rank] + L.tp_recv_slot / sizeof(float);
+            res_splits = R * sp;
+        } else {
+            ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_d[l], g, partial, M, d, F, sp));
+            res = partial; res_splits = sp;
+        }
+        res_stride = static_cast<size_t>(M) * d;
     }
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
+        ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
                                                         L2Prefetch{nullptr, 0}, st));
+        if (seg_on()) for (int k = 0; k < kTpKinds; ++k) tp.seq[k] = xseq[k];   // the forward's last segment was issued
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
+    int lm_tile0_local = 0, lm_rows_local = c.vocab;
+    vocab_shard(c, c.tp_rank, &lm_tile0_local, &lm_rows_local);
     for (int r0 = 0; r0 < n_lm; r0 += static_cast<int>(L.lm_chunk)) {
         const int rows = n_lm - r0 < static_cast<int>(L.lm_chunk) ? n_lm - r0 : static_cast<int>(L.lm_chunk);
         const __nv_bfloat16* x = a;
         const RowScale* scale = &inv_scale;
-        ODB_LAUNCH(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
-                                                        rows, d, hint_of(m->p_lm, packed_weight_bytes(c.vocab, d), 0), st));
+        ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
+                                                        rows, d, hint_of(m->p_lm, packed_weight_bytes(lm_rows_local, d), 0), st));
         if (s->dump_logits) {
             int sp = 1;
-            ODB_LAUNCH(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, &sp, scale));
-            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0,
+            ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, sp, scale));
+            ODB_FWD(ODB_KIND_CONFIDENCE, launch_confidence(logits, rows, c.vocab, c.mask_id, s->at<float>(L.conf) + r0,
                                                                  s->at<int32_t>(L.tok) + r0, s->ws + L.conf_part, st));
         } else {
             // LM head fused with the confidence reduction: per (row, vocabulary tile) statistics instead
@@ -752,14 +874,27 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             ga.row_scale = *scale;
             ga.conf.part = reinterpret_cast<ConfPartial*>(s->ws + L.conf_part);
             ga.conf.mask_id = c.mask_id;
-            ga.M = rows; ga.N = c.vocab; ga.K = d;
+            const int v_tile0 = lm_tile0_local, v_rows = lm_rows_local;
+            ga.M = rows; ga.N = v_rows; ga.K = d;
             ga.splits = 1;
             ga.status = status;
-            ODB_LAUNCH(ODB_KIND_GEMM, launch_gemm(ga, st));
-            ODB_LAUNCH(ODB_KIND_CONFIDENCE, launch_confidence_final(ga.conf.part, (c.vocab + 127) / 128, rows, s->at<float>(L.conf) + r0,
+            if (R > 1) {
+                // this rank's vocabulary tiles: their statistics go to every rank, which then merges all tiles in order
+                ga.conf.tile0 = v_tile0;
+                ga.conf.tiles_total = vocab_tiles(c);
+                ga.peers.n = R;
+                for (int r = 0; r < R; ++r) ga.peers.conf[r] = tp.conf[r];
+            }
+            ODB_FWD(ODB_KIND_GEMM, launch_gemm(ga, st));
+            if (R > 1) {
+                const int32_t xrc = exchange(2);
+                if (xrc != ODB_OK) return xrc;
+            }
+            ODB_FWD(ODB_KIND_CONFIDENCE, launch_confidence_final(ga.conf.part, vocab_tiles(c), rows, s->at<float>(L.conf) + r0,
                                                                        s->at<int32_t>(L.tok) + r0, st));
         }
     }
+    if (seg_on()) for (int k = 0; k < kTpKinds; ++k) tp.seq[k] = xseq[k];   // the forward's last segment was issued
     return ODB_OK;
 }
 
@@ -776,7 +911,10 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
     if (!s || !p || !block_index) return ODB_ERR_ARG;
     const odb_config& c = s->m->cfg;
     if (p->block_len < 1 || p->block_len > c.max_block) return ODB_ERR_SHAPE;
-    if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;   // an accept is pending
+    const bool tp_on = c.tp_world > 1;
+    const bool continuing = tp_on && s->tp.seg_first > 0;   // a later segment range of the refresh already begun
+    if (tp_on && (!s->tp.attached || s->dump_logits)) return ODB_ERR_STATE;
+    if (continuing ? s->phase != 1 : (s->phase == 1 || s->phase == 3)) return ODB_ERR_STATE;   // an accept is pending
     int M = 0, n_lm = 0, n_tiles = 0, n_big = 0;
     for (int i = 0; i < c.max_batch; ++i) {
         const SeqState& st = s->mirror[i];
@@ -789,7 +927,9 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
         n_big += (st.T + 127) / 128;
     }
     if (M == 0) return ODB_ERR_STATE;
-    ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
+    if (tp_on && static_cast<size_t>(n_lm) > s->L.lm_chunk) return ODB_ERR_SHAPE;   // one exchange of statistics per forward
+    if (!continuing)
+        ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_refresh_rows(s->cb, c.max_batch, block_index, p->block_len, s->st));
     int32_t rc = forward(s, M, c.with_lm_head ? n_lm : 0, n_tiles, true, 0, n_big);
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
@@ -801,7 +941,10 @@ int32_t odb_refresh_prefill(odb_session* s, const odb_decode_params* p, const in
 int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
     if (!s || !p) return ODB_ERR_ARG;
     const odb_config& c = s->m->cfg;
-    if (s->phase != 2) return ODB_ERR_STATE;
+    const bool tp_on = c.tp_world > 1;
+    const bool continuing = tp_on && s->tp.seg_first > 0;   // a later segment range of the step already begun
+    if (tp_on && (!s->tp.attached || s->dump_logits)) return ODB_ERR_STATE;
+    if (s->phase != (continuing ? 3 : 2)) return ODB_ERR_STATE;
     StepShape sh{0, 0, 0, 0};
     for (int i = 0; i < c.max_batch; ++i) step_shape_add(sh, s->mirror[i]);
     const int M = sh.rows;
@@ -811,7 +954,8 @@ int32_t odb_block_decode_step(odb_session* s, const odb_decode_params* p) {
         const int32_t trc = ensure_ptable(s, M);
         if (trc != ODB_OK) return trc;
     }
-    ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
+    if (tp_on && static_cast<size_t>(M) > s->L.lm_chunk) return ODB_ERR_SHAPE;
+    if (!continuing) ODB_LAUNCH(ODB_KIND_CONTROL, launch_build_step_rows(s->cb, c.max_batch, c.mask_id, s->st));
     int32_t rc = forward(s, M, c.with_lm_head ? M : 0, sh.tiles, false, step_items(s, sh));
     if (rc != ODB_OK) return rc;
     s->last_rows = M;
@@ -852,6 +996,7 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
     if (p->sampling && (p->n_copies != 1 || p->sample_steps < 1 || p->sample_steps > kMaxLoopIters)) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != 2 || s->profiling) return ODB_ERR_STATE;   // event pairs cannot be recorded into the loop body
+    if (c.tp_world > 1) return ODB_ERR_STATE;                  // the exchanges' sequence numbers are launch arguments
     *n_iters = 0;
     if (max_iters <= 0 || max_iters > kMaxLoopIters) max_iters = kMaxLoopIters;
     if (max_iters > log_cap) max_iters = log_cap;
@@ -951,16 +1096,17 @@ int32_t odb_debug_read(odb_session* s, int32_t which, void* host, size_t cap, in
     const odb_config& c = s->m->cfg;
     const Layout& L = s->L;
     const size_t M = s->last_rows, nlm = s->last_lm_rows, d = c.d_model;
+    const size_t da = static_cast<size_t>(heads_local(c)) * c.head_dim;   // row width of q / k / v / o (this rank's heads)
     size_t off = 0, bytes = 0, n = M;
     switch (which) {
         case 0: off = L.logits; n = nlm < L.lm_chunk ? nlm : L.lm_chunk; bytes = 4 * n * c.vocab; break;
         case 1: off = L.conf; n = nlm; bytes = 4 * n; break;
         case 2: off = L.tok; n = nlm; bytes = 4 * n; break;
         case 3: off = L.h; bytes = 4 * M * d; break;
-        case 4: off = L.q; bytes = 2 * M * d; break;
-        case 5: off = L.k; bytes = 2 * M * d; break;
-        case 6: off = L.v; bytes = 2 * M * d; break;
-        case 7: off = L.o; bytes = 2 * M * d; break;
+        case 4: off = L.q; bytes = 2 * M * da; break;
+        case 5: off = L.k; bytes = 2 * M * da; break;
+        case 6: off = L.v; bytes = 2 * M * da; break;
+        case 7: off = L.o; bytes = 2 * M * da; break;
         case 8: off = L.row_tok; bytes = 4 * M; break;
         case 9: off = L.row_pos; bytes = 4 * M; break;
         case 10: off = L.row_copy; bytes = 4 * M; break;
@@ -984,6 +1130,7 @@ int32_t odb_debug_expire_wait(odb_session* s, int64_t limit_cycles) {
 
 int32_t odb_debug_set_logit_dump(odb_session* s, int32_t enable) {
     if (!s) return ODB_ERR_ARG;
+    if (enable && s->m->cfg.tp_world > 1) return ODB_ERR_STATE;   // a rank holds a slice of the vocabulary only
     s->dump_logits = enable != 0;
     return ODB_OK;
 }
@@ -1039,6 +1186,85 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
         if (cudaEventElapsedTime(&ms, s->ev[i], s->ev[i + 1]) == cudaSuccess) ms_by_kind[s->ev_kind[i / 2]] += ms;
     }
     s->ev_used = 0;
+    return ODB_OK;
+}
+
+int32_t odb_session_tp_buffers(odb_session* s, void** recv, size_t* recv_bytes, void** flags, size_t* flags_bytes,
+                               void** conf, size_t* conf_bytes) {
+    if (!s || !recv || !recv_bytes || !flags || !flags_bytes || !conf || !conf_bytes) return ODB_ERR_ARG;
+    if (s->m->cfg.tp_world < 2) return ODB_ERR_STATE;
+    const Layout& L = s->L;
+    *recv = s->ws + L.tp_recv;
+    *recv_bytes = 2 * L.tp_recv_slot;
+    *flags = s->ws + L.tp_flags;
+    *flags_bytes = sizeof(unsigned int) * kTpKinds * kTpMaxWorld;
+    *conf = s->ws + L.conf_part;
+    *conf_bytes = L.conf_part_bytes;
+    return ODB_OK;
+}
+
+int32_t odb_session_tp_attach(odb_session* s, void* const* peer_recv, void* const* peer_flags, void* const* peer_conf) {
+    if (!s || !peer_recv || !peer_flags || !peer_conf) return ODB_ERR_ARG;
+    const odb_config& c = s->m->cfg;
+    if (c.tp_world < 2) return ODB_ERR_STATE;
+    if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;   // a forward is in flight
+    odb_session::Tp& tp = s->tp;
+    for (int r = 0; r < c.tp_world; ++r) {
+        const bool own = r == c.tp_rank;
+        void* pr = own ? static_cast<void*>(s->ws + s->L.tp_recv) : peer_recv[r];
+        void* pf = own ? static_cast<void*>(s->ws + s->L.tp_flags) : peer_flags[r];
+        void* pc = own ? static_cast<void*>(s->ws + s->L.conf_part) : peer_conf[r];
+        if (!pr || !pf || !pc) return ODB_ERR_ARG;
+        if ((reinterpret_cast<uintptr_t>(pr) | reinterpret_cast<uintptr_t>(pc)) & 15 || reinterpret_cast<uintptr_t>(pf) & 3)
+            return ODB_ERR_ARG;
+        tp.recv[r] = static_cast<float*>(pr);
+        tp.peers.flags[r] = static_cast<unsigned int*>(pf);
+        tp.conf[r] = static_cast<ConfPartial*>(pc);
+    }
+    tp.peers.world = c.tp_world;
+    tp.peers.rank = c.tp_rank;
+    tp.attached = true;
+    return ODB_OK;
+}
+
+int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, int32_t* last) {
+    if (!first || !last) return ODB_ERR_ARG;
+    const int32_t rc = check_config(cfg);
+    if (rc != ODB_OK) return rc;
+    if (rank < 0 || rank >= tp_ranks(*cfg)) return ODB_ERR_ARG;
+    int tile0 = 0, rows = 0;
+    vocab_shard(*cfg, rank, &tile0, &rows);
+    *first = tile0 * 128;
+    *last = tile0 * 128 + rows;
+    return ODB_OK;
+}
+
+int32_t odb_tp_segment_count(const odb_config* cfg) {
+    if (check_config(cfg) != ODB_OK) return 0;
+    if (cfg->tp_world < 2) return 1;
+    return 2 * cfg->n_layers + (cfg->with_lm_head ? 1 : 0) + 1;
+}
+
+int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last) {
+    if (!s) return ODB_ERR_ARG;
+    if (s->m->cfg.tp_world < 2) return ODB_ERR_STATE;
+    if (first < 0) {
+        if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;   // finish the forward in progress first
+        s->tp.seg_first = s->tp.seg_last = -1;
+        return ODB_OK;
+    }
+    if (last <= first || last > odb_tp_segment_count(&s->m->cfg)) return ODB_ERR_ARG;
+    s->tp.seg_first = first;
+    s->tp.seg_last = last;
+    return ODB_OK;
+}
+
+int32_t odb_debug_tp_expire_wait(odb_session* s, int32_t kind, int64_t limit_cycles) {
+    if (!s || kind < 0 || kind >= kTpKinds || limit_cycles < 1 || limit_cycles > kWaitLimitCycles) return ODB_ERR_ARG;
+    if (s->m->cfg.tp_world < 2 || !s->tp.attached) return ODB_ERR_STATE;
+    if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;
+    // a sequence number no rank has signalled: the flags stay below it, the wait runs into its limit
+    ODB_CUDA(launch_tp_wait(s->tp.peers, kind, s->tp.seq[kind] + 1, limit_cycles, s->at<int>(s->L.status), s->st));
     return ODB_OK;
 }
 

@@ -199,7 +199,19 @@ __device__ __forceinline__ void conf_merge(float& m, float& s, int& idx, float o
 // tile per activation row; see EPI_CONF in gemm_tcgen05.cu.  part non-null selects it.
 struct ConfEpilogue {
     ConfPartial* part = nullptr;   // [M][n_tiles]
-    int mask_id = -1;              // feature excluded from the statistics
+    int mask_id = -1;              // feature excluded from the statistics (a global vocabulary id)
+    // tensor-parallel shard of the vocabulary: this launch's tile t is global tile tile0 + t of tiles_total
+    // (row stride of `part`), its feature n is vocabulary id 128 * tile0 + n; tiles_total == 0: no shard
+    int tile0 = 0, tiles_total = 0;
+};
+
+// Tensor-parallel destinations of an epilogue: the same fp32 partial tiles (or confidence statistics) are stored to
+// n buffers, one per rank, this rank's own among them (plain stores; the others are peer memory).  n == 0: none.
+constexpr int kTpMaxWorld = 8;
+struct PeerOut {
+    float* partial[kTpMaxWorld] = {};       // each fp32 [splits][M][N], already offset to this rank's block
+    ConfPartial* conf[kTpMaxWorld] = {};    // each [M][tiles_total]
+    int n = 0;
 };
 
 // Weight-streaming GEMM: partial[s][M][N] (fp32) = x[M][K_s] * w[N][K_s]^T for each K split s.
@@ -211,11 +223,27 @@ struct GemmArgs {
     ConfEpilogue conf;                  // conf.part non-null: LM head fused with the confidence statistics, splits == 1
     RowScale row_scale;                 // per activation row m: the output is multiplied by scale[m]
                                         // (the 1/rms of an RMSNorm folded behind the projection); needs splits == 1
+    PeerOut peers;                      // peers.n > 0: the partial tiles (or statistics) go to these buffers instead
     int M, N, K;
     int splits;
     int* status;           // device status word
 };
 int gemm_pick_splits(int M, int N, int K);
+
+// ---- tensor parallelism: flags between ranks (tensor_parallel.cu) ----
+// Flag words of one rank: [kind][source rank], kind 0 / 1 = the two receive slots of partial sums, 2 = the
+// confidence statistics.  A flag holds the sequence number of the source's latest completed exchange of that kind.
+constexpr int kTpKinds = 3;
+struct TpPeers {
+    unsigned int* flags[kTpMaxWorld] = {};   // every rank's flag words (this rank's own at index rank)
+    int world = 0, rank = 0;
+};
+// One thread per rank: after everything this rank has stored to its peers is visible system-wide, writes `seq` into
+// flag [kind][rank] of every rank.
+cudaError_t launch_tp_signal(const TpPeers& p, int kind, unsigned int seq, cudaStream_t st);
+// One thread per source rank: waits (bounded by limit_cycles) until this rank's flag [kind][source] has reached
+// `seq`; on expiry writes ODB_ERR_TIMEOUT to *status and returns.
+cudaError_t launch_tp_wait(const TpPeers& p, int kind, unsigned int seq, long long limit_cycles, int* status, cudaStream_t st);
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
 // bf16 [rows][cols] row-major; box = 64 columns x box_rows rows, 128-byte swizzle, rows beyond `rows` read as zero
 cudaError_t make_rows_tmap(CUtensorMap* out, const void* base, int rows, int cols, int box_rows);

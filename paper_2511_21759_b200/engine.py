@@ -69,14 +69,15 @@ class Model:
     """Device-resident weights + the library's model handle."""
 
     def __init__(self, shape, tensors: dict, *, max_batch=1, max_seq=2048, max_block=64, max_copies=8,
-                 with_lm_head=True):
-        """tensors: embed, lm_head (or None), final_norm, and lists norm1, wqkv, wo, norm2, wgu, wd."""
+                 with_lm_head=True, tp=(0, 0)):
+        """tensors: embed, lm_head (or None), final_norm, and lists norm1, wqkv, wo, norm2, wgu, wd.
+        tp = (world, rank): the tensors are that tensor-parallel rank's shard (see odb.h); (0, 0): the whole model."""
         self.shape = shape
         self.t = tensors
         nl = shape.n_layers
         self.cfg = B.odb_config(nl, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
                                 shape.mask_id, shape.eos_id, shape.rope_theta, shape.rms_eps,
-                                max_batch, max_seq, max_block, max_copies, 1 if with_lm_head else 0)
+                                max_batch, max_seq, max_block, max_copies, 1 if with_lm_head else 0, tp[0], tp[1])
         arr = lambda name: (C.c_void_p * nl)(*[tensors[name][l].data_ptr() for l in range(nl)])
         self._arrays = {n: arr(n) for n in ("norm1", "wqkv", "wo", "norm2", "wgu", "wd")}
         w = B.odb_weights(_ptr(tensors["embed"]), _ptr(tensors.get("lm_head")) if with_lm_head else None,
@@ -230,8 +231,8 @@ class Session:
     def debug_read(self, what: str) -> np.ndarray:
         which, dt = self._READ[what]
         cfg = self.model.cfg
-        width = {"logits": cfg.vocab, "hidden": cfg.d_model, "q": cfg.d_model, "k": cfg.d_model, "v": cfg.d_model,
-                 "o": cfg.d_model}.get(what, 1)
+        da = cfg.d_model // max(cfg.tp_world, 1)      # q / k / v / o rows hold this rank's heads
+        width = {"logits": cfg.vocab, "hidden": cfg.d_model, "q": da, "k": da, "v": da, "o": da}.get(what, 1)
         cap_rows = self.ws.numel() // (width * np.dtype(dt).itemsize)
         cap_rows = min(cap_rows, cfg.max_batch * max(cfg.max_seq, cfg.max_copies * cfg.max_block))
         buf = np.empty(cap_rows * width, dtype=dt)

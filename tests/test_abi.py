@@ -48,7 +48,7 @@ def test_pure_host_calls_work_without_gpu():
 
 def test_struct_layouts_match_header():
     from paper_2511_21759_b200 import binding as B
-    assert ctypes.sizeof(B.odb_config) == 15 * 4
+    assert ctypes.sizeof(B.odb_config) == 17 * 4
     assert ctypes.sizeof(B.odb_decode_params) == 9 * 4
     assert ctypes.sizeof(B.odb_result) == (3 + 5 + 3 + 128) * 4
     assert ctypes.sizeof(B.odb_weights) == 9 * ctypes.sizeof(ctypes.c_void_p)

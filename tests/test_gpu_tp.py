@@ -1,0 +1,148 @@
+"""Tensor-parallel forward (weights divided over R ranks, partial sums and confidence statistics exchanged through
+the projections' epilogues) against the oracle of the WHOLE model.  One GPU: all ranks of a group run in this
+process on one stream, every forward issued segment by segment, so no kernel ever waits for a later launch; the
+kernels, the stores into the other ranks' buffers, the flags and their sequence numbers are the ones a group of
+R GPUs runs."""
+import dataclasses
+
+import numpy as np
+import pytest
+
+import synth
+from oracle import odb_oracle as O
+from oracle.inputs import model_from_synth
+from gpu_common import engine, requires_gpu, lockstep_generate, assert_near_ties_only, logits_close, bf16_bits_to_f64
+
+# shapes whose heads and FFN width divide over the ranks (d_ffn a multiple of 64 R)
+TP_TINY = dataclasses.replace(synth.TINY, d_ffn=768)                       # 4 heads of 64: R = 2, 4
+TP_PEAKY = dataclasses.replace(synth.TINY_PEAKY, d_ffn=768)
+TP_HD128 = dataclasses.replace(synth.TINY_HD128, d_ffn=768)               # 2 heads of 128: R = 2
+TP_WIDE = dataclasses.replace(synth.TINY, d_model=512, n_heads=8, d_ffn=1024)   # 8 heads: R = 8, two vocabulary tiles each
+SHAPES = {"tiny": TP_TINY, "peaky": TP_PEAKY, "hd128": TP_HD128, "wide": TP_WIDE}
+
+CASES = [
+    # name          shape    R  P   L   block copies poison  conf bound
+    ("r2_c1",       "tiny",  2, 64, 64, 16,   1,     False,  1e-2),
+    ("r4_c4",       "tiny",  4, 37, 41, 16,   4,     True,   1e-2),    # ragged tail, odd prompt, NaN-filled buffers
+    ("r2_peaky_c8", "peaky", 2, 51, 45, 16,   8,     False,  0.15),    # threshold accepts, jumps, decoded-share layout
+    ("r2_hd128_c4", "hd128", 2, 150, 77, 16,  4,     False,  1e-2),    # tcgen05 refresh attention, one head per rank
+    ("r8_c1",       "wide",  8, 40, 48, 16,   1,     False,  1e-2),
+    ("r4_b64_c8",   "peaky", 4, 64, 128, 64,  8,     False,  0.15),    # 512 query rows per step: CTA-pair projections
+]
+
+
+def _group(E, shape, R, P, L, Bk, *, seed=3, poison=False):
+    from paper_2511_21759_b200 import tp
+    g = tp.TPGroupOneGPU(shape, seed, R, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=8, poison=poison)
+    x0 = synth.sequence(seed, 0, P, L, shape)
+    g.set_sequence(0, x0, P)
+    return g, x0
+
+
+@requires_gpu
+@pytest.mark.parametrize("name,shape_name,R,P,L,Bk,copies,poison,conf_bound", CASES, ids=[c[0] for c in CASES])
+def test_tp_group_in_lockstep(name, shape_name, R, P, L, Bk, copies, poison, conf_bound):
+    """Whole generation of the group in lock step with the oracle of the unsharded model: confidences within the
+    bound every iteration, accept sets / chains / row tables bit-exact from the group's own confidences, the
+    oracle's own decisions equal except at measured near-ties; every rank ends with the same tokens (the group
+    object asserts rank-by-rank equality of confidences, tokens, row tables, results after every call)."""
+    E = engine()
+    shape = SHAPES[shape_name]
+    om = model_from_synth(shape, seed=3)
+    g, x0 = _group(E, shape, R, P, L, Bk, poison=poison)
+    kw = dict(block_len=Bk, n_copies=copies)
+    st = lockstep_generate(E, g, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), check_logits=False)
+    assert g.status() == [0] * R
+    assert_near_ties_only(st)
+    assert np.array_equal(g.get_tokens(0), st["tokens_final"])
+    assert (st["tokens_final"][P:] != shape.mask_id).all() and st["tokens"] == L
+    assert st["worst_conf"] < conf_bound, st["worst_conf"]
+    print(f"\n{name}: {R} ranks, {st['iters']} iterations ({st['refreshes']} refreshes), worst conf rel err {st['worst_conf']:.2e}, "
+          f"oracle-side decision diffs {st['oracle_decision_diff']}")
+    g.close()
+
+
+@requires_gpu
+@pytest.mark.parametrize("shape_name,R", [("tiny", 2), ("tiny", 4), ("hd128", 2), ("wide", 8)])
+def test_tp_refresh_shards_against_the_whole_model(shape_name, R):
+    """After a refresh: every rank's K / V rows of the last layer are the oracle's columns of that rank's heads (to
+    one bf16 step, most elements identical), the residual streams are bit-identical on all ranks, and the
+    confidences / greedy tokens agree with the oracle as the single-GPU path's do."""
+    E = engine()
+    shape = SHAPES[shape_name]
+    P, L = 64, 64
+    om = model_from_synth(shape, seed=0)
+    g, x0 = _group(E, shape, R, P, L, 16, seed=0)
+    p = E.DecodeParams(block_len=16)
+    g.refresh_prefill(p, 0)
+    conf, tok = g.debug_read("conf"), g.debug_read("tok")          # asserts the ranks agree
+    g.debug_read("hidden")
+    cache, oconf, otok, ologits = O.refresh_prefill(om, x0, P + L, P, return_logits=True)
+    hl = shape.n_heads // R
+    for r, sess in enumerate(g.ranks):
+        k = bf16_bits_to_f64(sess.debug_read("k")).reshape(P + L, hl, shape.head_dim)
+        v = bf16_bits_to_f64(sess.debug_read("v")).reshape(P + L, hl, shape.head_dim)
+        for got, want in ((k, cache.k[-1][:, r * hl:(r + 1) * hl]), (v, cache.v[-1][:, r * hl:(r + 1) * hl])):
+            ok, worst = logits_close(got.reshape(P + L, -1), want.reshape(P + L, -1), 4e-2)
+            assert ok, (r, worst)
+            assert (got == want).mean() > 0.7
+    assert np.allclose(conf, oconf, rtol=2e-2)
+    l32 = ologits.astype(np.float32).astype(np.float64)
+    l32[:, shape.mask_id] = -np.inf
+    top2 = np.sort(l32, axis=1)[:, -2:]
+    assert not ((tok != otok) & (top2[:, 1] - top2[:, 0] > 4e-2 * np.abs(l32[np.isfinite(l32)]).max())).any()
+    g.close()
+
+
+@requires_gpu
+def test_tp_expired_flag_wait_is_reported_and_the_group_stays_usable():
+    """A wait for a sequence number no rank has signalled runs into its (short) limit: the status word reports the
+    timeout to the host, nothing faults, and the group decodes on afterwards."""
+    from paper_2511_21759_b200 import binding as B
+    E = engine()
+    P, L = 32, 32
+    g, x0 = _group(E, TP_TINY, 2, P, L, 16)
+    p = E.DecodeParams(block_len=16)
+    g.refresh_prefill(p, 0)
+    g.unmask_accept(p, True)
+    for kind in range(3):
+        B.check(B.lib().odb_debug_tp_expire_wait(g.ranks[0].handle, kind, 2_000_000), "odb_debug_tp_expire_wait")
+        assert g.ranks[0].status() == B.ODB_ERR_TIMEOUT
+        assert g.ranks[0].status() == 0                            # read and cleared
+    assert g.ranks[1].status() == 0
+    g.block_decode_step(p)
+    res = g.unmask_accept(p, False)
+    assert res[0].n_accepted >= 1 and g.status() == [0, 0]
+    g.close()
+
+
+@requires_gpu
+def test_tp_state_errors():
+    """Unattached sessions, the logits test mode and the device-resident loop are refused; shard configurations the
+    library cannot divide are refused at model creation."""
+    import ctypes as C
+    from paper_2511_21759_b200 import binding as B, tp
+    E = engine()
+    m = tp.model_shard_from_synth(TP_TINY, 0, 0, 2, max_batch=1, max_seq=64, max_block=16, max_copies=4)
+    s = E.Session(m)
+    s.set_sequence(0, synth.sequence(0, 0, 32, 32, TP_TINY), 32)
+    p = E.DecodeParams(block_len=16)
+    with pytest.raises(B.OdbError) as e:
+        s.refresh_prefill(p, 0)
+    assert e.value.status == B.ODB_ERR_STATE                      # not attached
+    with pytest.raises(B.OdbError) as e:
+        s.set_logit_dump(True)
+    assert e.value.status == B.ODB_ERR_STATE
+    assert B.lib().odb_debug_tp_segments(s.handle, 0, 99) == B.ODB_ERR_ARG
+    assert B.lib().odb_debug_tp_expire_wait(s.handle, 0, 1000) == B.ODB_ERR_STATE
+    s.close(); m.close()
+    g, _ = _group(E, TP_TINY, 2, 32, 32, 16)
+    g.refresh_prefill(p, 0)
+    g.unmask_accept(p, True)
+    with pytest.raises(B.OdbError) as e:
+        g.ranks[0].decode_block_resident(p)
+    assert e.value.status == B.ODB_ERR_STATE
+    g.close()
+    with pytest.raises(B.OdbError) as e:                          # 688 FFN features do not divide into 2 x 64
+        tp.model_shard_from_synth(synth.TINY, 0, 0, 2, max_batch=1, max_seq=64, max_block=16, max_copies=4)
+    assert e.value.status == B.ODB_ERR_SHAPE
