@@ -42,31 +42,41 @@ def shard_layer(w: dict, shape, rank: int, world: int) -> dict:
             "wg": w["wg"][f0:f1], "wu": w["wu"][f0:f1], "wd": w["wd"][:, f0:f1]}
 
 
-def model_shard_from_synth(shape, seed, rank: int, world: int, device="cuda", *, with_lm_head=True, lm_head_bits=None,
-                           **kw) -> E.Model:
-    """The seeded synthetic model's shard of rank `rank` (data marshalling: slicing, upload, packing)."""
+def model_shards_from_synth(shape, seed, ranks: List[int], world: int, device="cuda", *, with_lm_head=True,
+                            lm_head_bits=None, **kw) -> List[E.Model]:
+    """The seeded synthetic model's shards of the given ranks (data marshalling: slicing, upload, packing); every
+    layer is generated once and sliced for each rank."""
     import synth
     d = shape.d_model
     ones = lambda: torch.ones(d, dtype=torch.float32, device=device)
-    probe = B.odb_config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
-                         shape.mask_id, shape.eos_id, shape.rope_theta, shape.rms_eps, 1, 2, 1, 1,
-                         1 if with_lm_head else 0, world, rank)
-    v0, v1 = vocab_range(probe, rank)
-    lm = None
-    if with_lm_head:
-        bits = lm_head_bits if lm_head_bits is not None else synth.lm_head_bits(shape, seed)
-        lm = E.pack_weight(E.bits_to_device(bits[v0:v1], device))
-    t = {"embed": E.bits_to_device(synth.embed_bits(shape, seed), device), "lm_head": lm,
-         "final_norm": ones(), "norm1": [], "wqkv": [], "wo": [], "norm2": [], "wgu": [], "wd": []}
+    embed = E.bits_to_device(synth.embed_bits(shape, seed), device)      # replicated: one device copy serves every rank here
+    lm_bits = (lm_head_bits if lm_head_bits is not None else synth.lm_head_bits(shape, seed)) if with_lm_head else None
+    ts = []
+    for r in ranks:
+        lm = None
+        if with_lm_head:
+            probe = B.odb_config(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab,
+                                 shape.mask_id, shape.eos_id, shape.rope_theta, shape.rms_eps, 1, 2, 1, 1, 1, world, r)
+            v0, v1 = vocab_range(probe, r)
+            lm = E.pack_weight(E.bits_to_device(lm_bits[v0:v1], device))
+        ts.append({"embed": embed, "lm_head": lm, "final_norm": ones(), "norm1": [], "wqkv": [], "wo": [], "norm2": [],
+                   "wgu": [], "wd": []})
     for l in range(shape.n_layers):
-        w = shard_layer(synth.layer_bits(shape, l, seed), shape, rank, world)
-        t["norm1"].append(ones())
-        t["norm2"].append(ones())
-        t["wqkv"].append(E.pack_weight(E.bits_to_device(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0), device)))
-        t["wo"].append(E.pack_weight(E.bits_to_device(w["wo"], device)))
-        t["wgu"].append(E.pack_gate_up(E.bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device)))
-        t["wd"].append(E.pack_weight(E.bits_to_device(w["wd"], device)))
-    return E.Model(shape, t, with_lm_head=with_lm_head, tp=(world, rank), **kw)
+        full = synth.layer_bits(shape, l, seed)
+        for t, r in zip(ts, ranks):
+            w = shard_layer(full, shape, r, world)
+            t["norm1"].append(ones())
+            t["norm2"].append(ones())
+            t["wqkv"].append(E.pack_weight(E.bits_to_device(np.concatenate([w["wq"], w["wk"], w["wv"]], axis=0), device)))
+            t["wo"].append(E.pack_weight(E.bits_to_device(w["wo"], device)))
+            t["wgu"].append(E.pack_gate_up(E.bits_to_device(np.concatenate([w["wg"], w["wu"]], axis=0), device)))
+            t["wd"].append(E.pack_weight(E.bits_to_device(w["wd"], device)))
+    return [E.Model(shape, t, with_lm_head=with_lm_head, tp=(world, r), **kw) for t, r in zip(ts, ranks)]
+
+
+def model_shard_from_synth(shape, seed, rank: int, world: int, device="cuda", **kw) -> E.Model:
+    """One rank's shard (what a process of a multi-process group uploads)."""
+    return model_shards_from_synth(shape, seed, [rank], world, device, **kw)[0]
 
 
 def tp_buffers(sess: E.Session):
@@ -93,8 +103,8 @@ class TPGroupOneGPU:
 
     def __init__(self, shape, seed=0, world=2, device="cuda", *, with_lm_head=True, lm_head_bits=None, poison=False, **kw):
         self.world = world
-        self.models = [model_shard_from_synth(shape, seed, r, world, device, with_lm_head=with_lm_head,
-                                              lm_head_bits=lm_head_bits, **kw) for r in range(world)]
+        self.models = model_shards_from_synth(shape, seed, list(range(world)), world, device, with_lm_head=with_lm_head,
+                                              lm_head_bits=lm_head_bits, **kw)
         self.ranks = [E.Session(m, poison=poison) for m in self.models]
         bufs = [tp_buffers(s) for s in self.ranks]
         for s in self.ranks:

@@ -329,3 +329,32 @@ def test_cfg4_eight_copies_until_the_decoded_share_switch_in_lockstep():
     per-row relative L2 error of 2.57e-2 against 1.8e-2 here: inside the bound, but only just)."""
     st = _full_size_lockstep("cfg4_8b_c4", 8, gen_len=256, stop=lambda s: s["stage2_steps"] >= 1)
     assert st["stage2_steps"] == 1 and st["refreshes"] == 1
+
+
+@requires_gpu
+def test_cfg4_tensor_parallel_group_of_four_in_lockstep():
+    """The 8B shape divided over four tensor-parallel ranks (8 heads, 3072 FFN features, 247 vocabulary tiles each; all
+    ranks on this one GPU, forwards issued segment by segment): the refresh at T = 768 (CTA-pair projections storing
+    their partial tiles into every rank's buffers) and two 128-row steps with four copies in lock step with the
+    float32 oracle of the WHOLE model.  No logits exist under tensor parallelism: confidences within the band the
+    single-GPU path is held to at this size, decisions reproduced from the group's own confidences, oracle-side
+    differences only at measured near-ties, every rank bit-identical to every other after each call."""
+    from gpu_common import lockstep_generate, assert_near_ties_only
+    from paper_2511_21759_b200 import tp
+    E = engine()
+    wl = synth.WORKLOADS["cfg4_8b_c4"]
+    shape, Bk, P, L = wl.shape, wl.block_len, 512, 256
+    x0 = synth.sequence(0, 0, P, L, shape)
+    g = tp.TPGroupOneGPU(shape, 0, 4, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
+    g.set_sequence(0, x0, P)
+    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    kw = dict(block_len=Bk, n_copies=4, alp=False)
+    st = lockstep_generate(E, g, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), check_logits=False,
+                           dtype=np.float32, max_iters=3)
+    assert g.status() == [0, 0, 0, 0]
+    g.close()
+    assert_near_ties_only(st)
+    assert st["refreshes"] == 1 and st["steps"] == 2
+    assert st["worst_conf"] < 0.2, st["worst_conf"]
+    print(f"\n8B shape over 4 tensor-parallel ranks, full size in lock step: {st['iters']} iterations, {st['tokens']} tokens; worst "
+          f"confidence rel. error {st['worst_conf']:.2e}; oracle-side decision differences {st['oracle_decision_diff']}")
