@@ -100,11 +100,13 @@ typedef struct odb_config {
  * embedding, gains and the residual stream are replicated; the K/V cache holds the rank's own heads
  * (odb_kv_bytes shrinks accordingly).  The O and down projections produce partial sums of the full d_model
  * width: their epilogue stores every fp32 partial tile straight into the receive buffer of EVERY rank (plain
- * stores to peer memory, no bulk or multicast copy from a peer anywhere), a one-thread kernel then raises this
- * rank's flag on every rank, and the consuming RMSNorm kernel, behind a bounded wait on the R flags, adds all
- * partials in (rank, split) order - the same order on every rank, so the residual streams stay bit-identical.
+ * stores to peer memory, no bulk or multicast copy from a peer anywhere), the last CTA of the projection to have
+ * stored its tiles raises this rank's flag on every rank, and the consuming RMSNorm kernel, which begins with a
+ * bounded wait on the R flags, adds all partials in (rank, split) order - the same order on every rank, so the residual streams stay bit-identical.
  * The LM head's per-tile confidence statistics are exchanged the same way and merged in tile order.
- * Not available under TP: the device-resident loop, the logits test mode, the persistent step kernel. */
+ * The exchanges' sequence numbers are counted on the device, so a tensor-parallel step can be captured like any
+ * other: odb_decode_block_resident works (every rank runs the same iterations: the accept decides from identical
+ * confidences).  Not available under TP: the logits test mode, the persistent step kernel. */
 #define ODB_TP_MAX_WORLD 8
 
 /* Device pointers to the weights; per-layer arrays are HOST arrays of n_layers device pointers.
@@ -359,6 +361,11 @@ int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, 
  * follows the last segment.  first < 0 restores whole forwards. */
 int32_t odb_tp_segment_count(const odb_config* cfg);
 int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last);
+/* Measurement facility: a rank timed WITHOUT its peers.  With enable != 0 the session raises, on itself, the flags
+ * of all sources at every exchange, so its waits pass although no peer runs; the partial sums and statistics of the
+ * absent ranks are whatever their blocks of the receive buffers hold (results are meaningless, device time is that
+ * of one rank's kernels).  Attach the session to its own three regions for every rank first. */
+int32_t odb_debug_tp_alone(odb_session* s, int32_t enable);
 /* Test facility: one launch of the flag wait for exchange `kind` (0, 1: partial-sum slots, 2: statistics) with the
  * next sequence number and the given cycle limit; nothing raises the flags, so the wait expires and the status
  * word reports ODB_ERR_TIMEOUT (read and cleared by odb_session_status). */

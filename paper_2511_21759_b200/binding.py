@@ -95,6 +95,7 @@ SIGNATURES = {
     "odb_tp_vocab_range": (C.c_int32, [C.POINTER(odb_config), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "odb_tp_segment_count": (C.c_int32, [C.POINTER(odb_config)]),
     "odb_debug_tp_segments": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),
+    "odb_debug_tp_alone": (C.c_int32, [C.c_void_p, C.c_int32]),
     "odb_debug_tp_expire_wait": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int64]),
     "odb_measure_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),
     "odb_measure_bulk_read_bandwidth": (C.c_int32, [C.c_void_p, C.c_size_t, C.c_int32, C.c_void_p, C.POINTER(C.c_double)]),

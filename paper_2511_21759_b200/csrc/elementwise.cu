@@ -54,10 +54,12 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
 __global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_kernel(float* __restrict__ h, const float* __restrict__ partial,
                                                                      int splits, size_t pstride, const float* __restrict__ gain,
                                                                      __nv_bfloat16* __restrict__ out, float* __restrict__ ssq,
-                                                                     const int32_t* __restrict__ row_map, int d, L2Prefetch pf) {
+                                                                     const int32_t* __restrict__ row_map, int d, L2Prefetch pf,
+                                                                     TpWait tw) {
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
+    tp_wait_flags(tw);   // tensor parallelism: the partials of every rank have arrived
     l2_prefetch_slice(pf, blockIdx.y * gridDim.x + blockIdx.x, gridDim.x * gridDim.y);
     const int orow = blockIdx.x;
     const int row = row_map ? row_map[orow] : orow;
@@ -99,10 +101,12 @@ __global__ void __launch_bounds__(kNormSliceCols / 4) rmsnorm_rows_kernel(float*
                                                                           int splits, size_t pstride,
                                                                           const float* __restrict__ gain,
                                                                           __nv_bfloat16* __restrict__ out, float* __restrict__ ssq,
-                                                                          const int32_t* __restrict__ row_map, int rows_out, int d) {
+                                                                          const int32_t* __restrict__ row_map, int rows_out, int d,
+                                                                          TpWait tw) {
     __shared__ float red[kNormRows][32];
     pdl_launch_dependents();
     pdl_wait();
+    tp_wait_flags(tw);
     const int i = blockIdx.y * (kNormSliceCols / 4) + threadIdx.x;   // float4 index within the row
     const int orow0 = blockIdx.x * kNormRows;
     const bool in = i < (d >> 2);
@@ -339,11 +343,12 @@ __global__ void __launch_bounds__(256) confidence_partial_kernel(const float* __
 // a warp are merged by a fixed shuffle tree (an earlier lane's triple is always the left operand) and the
 // four warps in warp order.
 __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial* __restrict__ part, int chunks, int rows,
-                                                              float* __restrict__ conf, int32_t* __restrict__ tok) {
+                                                              float* __restrict__ conf, int32_t* __restrict__ tok, TpWait tw) {
     __shared__ float sm[4], ss[4];
     __shared__ int si[4];
     pdl_launch_dependents();
     pdl_wait();
+    tp_wait_flags(tw);   // tensor parallelism: every rank's vocabulary tiles have arrived
     const int row = blockIdx.x, lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const ConfPartial* p = part + static_cast<size_t>(row) * chunks;
     float m = -INFINITY, s = 0.f;
@@ -459,14 +464,14 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
                            __nv_bfloat16* out, float* ssq, const int32_t* row_map, int rows_out, int d, L2Prefetch pf,
-                           cudaStream_t st) {
+                           cudaStream_t st, const TpWait& tw) {
     if (splits > 16) return cudaErrorInvalidValue;
     const int slices = (d + kNormSliceCols - 1) / kNormSliceCols;
     if (rows_out >= 256 && splits <= kNormRowsMaxSplits)
         return launch_kernel(rmsnorm_rows_kernel, dim3((rows_out + kNormRows - 1) / kNormRows, slices), dim3(kNormSliceCols / 4), 0,
-                             st, h, partial, splits, pstride, gain, out, ssq, row_map, rows_out, d);
+                             st, h, partial, splits, pstride, gain, out, ssq, row_map, rows_out, d, tw);
     return launch_kernel(rmsnorm_kernel, dim3(rows_out, slices), dim3(kNormSliceCols / 4), 0, st, h, partial, splits, pstride,
-                         gain, out, ssq, row_map, d, pf);
+                         gain, out, ssq, row_map, d, pf, tw);
 }
 
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
@@ -480,8 +485,8 @@ cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st) {
 }
 
 cudaError_t launch_confidence_final(const ConfPartial* part, int chunks, int rows, float* conf, int32_t* tok,
-                                    cudaStream_t st) {
-    return launch_kernel(confidence_final_kernel, dim3(rows), dim3(128), 0, st, part, chunks, rows, conf, tok);
+                                    cudaStream_t st, const TpWait& tw) {
+    return launch_kernel(confidence_final_kernel, dim3(rows), dim3(128), 0, st, part, chunks, rows, conf, tok, tw);
 }
 
 cudaError_t launch_confidence(const float* logits, int rows, int V, int mask_id, float* conf, int32_t* tok,

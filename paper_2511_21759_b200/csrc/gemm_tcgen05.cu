@@ -75,7 +75,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     const int m_groups = PAIR ? (pair_tiles_y + static_cast<int>(gridDim.y) - 1) / static_cast<int>(gridDim.y) : 1;
     const int m_tile = PAIR ? static_cast<int>((blockIdx.z / n_pairs) % m_groups) * static_cast<int>(gridDim.y) + static_cast<int>(blockIdx.y)
                             : static_cast<int>(blockIdx.y);
-    if (PAIR && m_tile >= pair_tiles_y) return;   // ragged last group: both CTAs of the pair leave together
+    if (PAIR && m_tile >= pair_tiles_y) {   // ragged last group: both CTAs of the pair leave together
+        if (po.n > 0 && threadIdx.x == 0) tp_arrive_and_signal(po, gridDim.x * gridDim.y * gridDim.z);
+        return;
+    }
     const int n0 = n_tile * kBM;
     const int m0 = m_tile * BN;
     const int split = PAIR ? static_cast<int>(blockIdx.z / (n_pairs * m_groups)) : static_cast<int>(blockIdx.z);
@@ -244,17 +247,21 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                         }
                     } else {
                         // tensor-parallel partial sums: the tile goes to the receive buffer of every rank
-                        for (int r = 0; r < po.n; ++r) {
-                            float* dst = po.partial[r] + split_off;
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int m = m0 + c * 32 + j;
-                                if (n < N && m < M) dst[static_cast<size_t>(m) * N + n] = __uint_as_float(v[j]);
+                        for (int j = 0; j < 32; ++j) {
+                            const int m = m0 + c * 32 + j;
+                            if (n < N && m < M) {
+                                const size_t off = split_off + static_cast<size_t>(m) * N + n;
+#pragma unroll 1
+                                for (int r = 0; r < po.n; ++r) po.partial[r][off] = __uint_as_float(v[j]);
                             }
                         }
                     }
                 }
-                if (po.n > 0) __threadfence_system();
+            }
+            if (po.n > 0) {   // uniform: the tile's stores of all four warps, then one arrival for the CTA
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (threadIdx.x == 64) tp_arrive_and_signal(po, gridDim.x * gridDim.y * gridDim.z);
             }
         } else if constexpr (EPI == EPI_CONF) {
             // LM head fused with the confidence reduction: the logits of this tile (128 vocabulary
@@ -308,11 +315,11 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
                         ce.part[static_cast<size_t>(m) * n_tiles + n_tile] = p;
                     } else {
                         for (int r = 0; r < po.n; ++r) po.conf[r][static_cast<size_t>(m) * ce.tiles_total + ce.tile0 + n_tile] = p;
-                        __threadfence_system();
                     }
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
             }
+            if (po.n > 0 && t == 0) tp_arrive_and_signal(po, gridDim.x * gridDim.y * gridDim.z);   // behind the loop's last barrier
         } else {
             // all MMAs have completed, so the stage ring is free: use it to hand the up values over.
             // Every epilogue warp executes every barrier, whether or not its wait succeeded.

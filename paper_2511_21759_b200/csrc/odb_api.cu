@@ -136,7 +136,7 @@ Layout make_layout(const odb_config& c) {
         const size_t all_ranks = 4 * static_cast<size_t>(c.tp_world) * L.rows * d;   // one partial per rank of the largest forward
         L.tp_recv_slot = align_up(4 * L.partial_rows * nmax > all_ranks ? 4 * L.partial_rows * nmax : all_ranks);
         L.tp_recv = take(2 * L.tp_recv_slot);
-        L.tp_flags = take(sizeof(unsigned int) * kTpKinds * kTpMaxWorld);
+        L.tp_flags = take(sizeof(unsigned int) * kTpFlagWords);   // flags, this rank's arrival and sequence counters
     }
     L.total = off;
     return L;
@@ -198,9 +198,8 @@ struct odb_session {
         bool attached = false;
         float* recv[kTpMaxWorld] = {};          // every rank's receive region (two slots), own at index rank
         ConfPartial* conf[kTpMaxWorld] = {};    // every rank's confidence-statistics buffer
-        TpPeers peers;                          // every rank's flag words
-        unsigned int seq[kTpKinds] = {0, 0, 0}; // sequence number of the latest completed exchange per kind
-        unsigned int fwd_base[kTpKinds] = {0, 0, 0};   // seq at the start of the forward in progress
+        unsigned int* flags[kTpMaxWorld] = {};  // every rank's flag words
+        bool alone = false;                     // measurement: all sources' flags are raised on this rank itself
         int seg_first = -1, seg_last = -1;      // test facility: segments of a forward to launch (-1: all)
         long long wait_limit = kWaitLimitCycles;
     } tp;
@@ -365,7 +364,7 @@ int32_t odb_session_create(odb_model* m, void* kv, size_t kv_bytes, void* worksp
     // q / k / v and output rows past a forward's last row are never read (the tensor maps end at that row).
     if (e == cudaSuccess) e = cudaMemsetAsync(kv, 0, odb_kv_bytes(&c), s->st);
     if (e == cudaSuccess && c.tp_world > 1)
-        e = cudaMemsetAsync(s->ws + L.tp_flags, 0, sizeof(unsigned int) * kTpKinds * kTpMaxWorld, s->st);
+        e = cudaMemsetAsync(s->ws + L.tp_flags, 0, sizeof(unsigned int) * kTpFlagWords, s->st);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s->st);
     if (e != cudaSuccess) {
         odb_session_destroy(s);
@@ -589,9 +588,6 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     // Tensor parallelism: a forward is a sequence of segments separated by its exchange points; `seg` counts them
     // as the launches below are walked, and a launch is issued only if its segment is in the requested range.
     int seg = 0;
-    if (tp.seg_first <= 0)   // a forward begins (always, unless a later segment range of one in progress is requested)
-        for (int k = 0; k < kTpKinds; ++k) tp.fwd_base[k] = tp.seq[k];
-    unsigned int xseq[kTpKinds] = {tp.fwd_base[0], tp.fwd_base[1], tp.fwd_base[2]};
     auto seg_on = [&]() { return tp.seg_first < 0 || (seg >= tp.seg_first && seg < tp.seg_last); };
     float* h = s->at<float>(L.h);
     __nv_bfloat16* a = s->at<__nv_bfloat16>(L.a);
@@ -622,6 +618,26 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         if (static_cast<size_t>(sp) > cap) sp = static_cast<int>(cap < 1 ? 1 : cap);
         return sp;
     };
+    // An exchange of kind `kind`: the projection that produces the data raises this rank's flags when its last CTA
+    // has stored (fill_peers); the segment ends behind that launch; the consumer waits on the flags of all ranks
+    // (end_exchange returns its argument).  Sequence numbers are counted on the device.
+    auto fill_peers = [&](PeerOut& po, int kind) {
+        po.n = R;
+        po.rank = c.tp_rank;
+        po.kind = kind;
+        po.alone = tp.alone ? 1 : 0;
+        for (int r = 0; r < R; ++r) po.flags[r] = tp.flags[r];
+    };
+    auto end_exchange = [&](int kind) {
+        ++seg;
+        TpWait tw;
+        tw.region = tp.flags[c.tp_rank];
+        tw.kind = kind;
+        tw.world = R;
+        tw.limit_cycles = tp.wait_limit;
+        tw.status = status;
+        return tw;
+    };
     auto gemm = [&](const CUtensorMap& tw, const __nv_bfloat16* x, float* out, int rows, int N, int K, int sp,
                     const RowScale* row_scale = nullptr, int slot = -1) {
         GemmArgs ga;
@@ -634,28 +650,13 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         ga.splits = sp;
         ga.status = status;
         if (slot >= 0) {   // tensor-parallel partial sums: block `rank` of receive slot `slot` on every rank
-            ga.peers.n = R;
+            fill_peers(ga.peers, slot);
             for (int r = 0; r < R; ++r)
                 ga.peers.partial[r] = tp.recv[r] + static_cast<size_t>(slot) * (L.tp_recv_slot / sizeof(float)) +
                                       static_cast<size_t>(c.tp_rank) * sp * rows * N;
         }
         return launch_gemm(ga, st);
     };
-    // exchange point of kind `kind`: raise this rank's flag everywhere (end of a segment), wait for all flags
-    auto exchange = [&](int kind) -> int32_t {
-        const unsigned int sq = ++xseq[kind];
-        if (seg_on()) {
-            LaunchScope scope__(s, ODB_KIND_CONTROL);
-            ODB_CUDA(launch_tp_signal(tp.peers, kind, sq, st));
-        }
-        ++seg;
-        if (seg_on()) {
-            LaunchScope scope__(s, ODB_KIND_CONTROL);
-            ODB_CUDA(launch_tp_wait(tp.peers, kind, sq, tp.wait_limit, status, st));
-        }
-        return ODB_OK;
-    };
-
 #define ODB_LAUNCH(kind, call)          \
     do {                                \
         LaunchScope scope__(s, kind);   \
@@ -711,6 +712,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     }
     ODB_FWD(ODB_KIND_ELEMENTWISE, launch_embed(m->embed, s->cb.row_tok, h, M, d, st));
     const float* res = nullptr;   // split-K partials of the projection not yet added to the residual stream
+    TpWait res_wait;              // tensor parallelism: the flags those partials are complete behind
     int res_splits = 0;
     size_t res_stride = 0;
     static const int ks_env = getenv("ODB_ATTN_KS") ? atoi(getenv("ODB_ATTN_KS")) : 0;
@@ -737,7 +739,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
                  gu_bytes = packed_gate_up_bytes(F, d);
     for (int l = 0; l < c.n_layers; ++l) {
         ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->norm1[l], a, inv, nullptr, M, d,
-                                                        hint_of(m->p_qkv[l], qkv_bytes, 0), st));
+                                                        hint_of(m->p_qkv[l], qkv_bytes, 0), st, res_wait));
         int sp = plan_splits(M, 3 * da, d, false);
         ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_qkv[l], a, partial, M, 3 * da, d, sp));
         QkvRopeArgs qa;
@@ -805,18 +807,18 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         sp = plan_splits(M, d, da, R > 1);
         const float* o_sum = partial;   // the partial sums the next RMSNorm adds to the residual stream
         int o_parts = sp;
+        TpWait o_wait;
         if (R > 1) {
             // every rank's partial tiles land in slot 0 of every rank; all R * sp partials are added in (rank, split) order
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_o[l], o, nullptr, M, d, da, sp, nullptr, 0));
-            const int32_t xrc = exchange(0);
-            if (xrc != ODB_OK) return xrc;
+            o_wait = end_exchange(0);
             o_sum = tp.recv[c.tp_rank];
             o_parts = R * sp;
         } else {
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_o[l], o, partial, M, d, da, sp));
         }
         ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, o_sum, o_parts, static_cast<size_t>(M) * d, m->norm2[l], a, inv, nullptr, M,
-                                                        d, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st));
+                                                        d, hint_of(m->p_gu[l], gu_bytes, pf_bytes), st, o_wait));
         {   // gate/up projection with the SwiGLU epilogue: writes bf16 g directly
             GemmArgs ga;
             ga.tmap_w = m->tm_gu[l];
@@ -832,8 +834,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         sp = plan_splits(M, d, F, R > 1);
         if (R > 1) {
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_d[l], g, nullptr, M, d, F, sp, nullptr, 1));
-            const int32_t xrc = exchange(1);
-            if (xrc != ODB_OK) return xrc;
+            res_wait = end_exchange(1);
             res = tp.recv[c.tp_rank] + L.tp_recv_slot / sizeof(float);
             res_splits = R * sp;
         } else {
@@ -845,8 +846,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
     if (!c.with_lm_head) {
         // fold the last projection into the residual stream (the normalised copy is not used)
         ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, nullptr, M, d,
-                                                        L2Prefetch{nullptr, 0}, st));
-        if (seg_on()) for (int k = 0; k < kTpKinds; ++k) tp.seq[k] = xseq[k];   // the forward's last segment was issued
+                                                        L2Prefetch{nullptr, 0}, st, res_wait));
         return ODB_OK;
     }
     float* logits = s->at<float>(L.logits);
@@ -857,7 +857,7 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         const __nv_bfloat16* x = a;
         const RowScale* scale = &inv_scale;
         ODB_FWD(ODB_KIND_ELEMENTWISE, launch_rmsnorm(h, res, res_splits, res_stride, m->final_norm, a, inv, s->cb.lm_rows + r0,
-                                                        rows, d, hint_of(m->p_lm, packed_weight_bytes(lm_rows_local, d), 0), st));
+                                                        rows, d, hint_of(m->p_lm, packed_weight_bytes(lm_rows_local, d), 0), st, res_wait));
         if (s->dump_logits) {
             int sp = 1;
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_lm, x, logits, rows, c.vocab, d, sp, scale));
@@ -882,19 +882,16 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
                 // this rank's vocabulary tiles: their statistics go to every rank, which then merges all tiles in order
                 ga.conf.tile0 = v_tile0;
                 ga.conf.tiles_total = vocab_tiles(c);
-                ga.peers.n = R;
+                fill_peers(ga.peers, 2);
                 for (int r = 0; r < R; ++r) ga.peers.conf[r] = tp.conf[r];
             }
             ODB_FWD(ODB_KIND_GEMM, launch_gemm(ga, st));
-            if (R > 1) {
-                const int32_t xrc = exchange(2);
-                if (xrc != ODB_OK) return xrc;
-            }
+            TpWait conf_wait;
+            if (R > 1) conf_wait = end_exchange(2);
             ODB_FWD(ODB_KIND_CONFIDENCE, launch_confidence_final(ga.conf.part, vocab_tiles(c), rows, s->at<float>(L.conf) + r0,
-                                                                       s->at<int32_t>(L.tok) + r0, st));
+                                                                       s->at<int32_t>(L.tok) + r0, st, conf_wait));
         }
     }
-    if (seg_on()) for (int k = 0; k < kTpKinds; ++k) tp.seq[k] = xseq[k];   // the forward's last segment was issued
     return ODB_OK;
 }
 
@@ -996,7 +993,7 @@ int32_t odb_decode_block_resident(odb_session* s, const odb_decode_params* p, in
     if (p->sampling && (p->n_copies != 1 || p->sample_steps < 1 || p->sample_steps > kMaxLoopIters)) return ODB_ERR_ARG;
     if (p->n_copies > c.max_copies) return ODB_ERR_SHAPE;
     if (s->phase != 2 || s->profiling) return ODB_ERR_STATE;   // event pairs cannot be recorded into the loop body
-    if (c.tp_world > 1) return ODB_ERR_STATE;                  // the exchanges' sequence numbers are launch arguments
+    if (c.tp_world > 1 && (!s->tp.attached || s->dump_logits || s->tp.seg_first >= 0)) return ODB_ERR_STATE;
     *n_iters = 0;
     if (max_iters <= 0 || max_iters > kMaxLoopIters) max_iters = kMaxLoopIters;
     if (max_iters > log_cap) max_iters = log_cap;
@@ -1197,7 +1194,7 @@ int32_t odb_session_tp_buffers(odb_session* s, void** recv, size_t* recv_bytes, 
     *recv = s->ws + L.tp_recv;
     *recv_bytes = 2 * L.tp_recv_slot;
     *flags = s->ws + L.tp_flags;
-    *flags_bytes = sizeof(unsigned int) * kTpKinds * kTpMaxWorld;
+    *flags_bytes = sizeof(unsigned int) * kTpFlagWords;   // peers write the flags; the counters behind them are this rank's own
     *conf = s->ws + L.conf_part;
     *conf_bytes = L.conf_part_bytes;
     return ODB_OK;
@@ -1218,11 +1215,9 @@ int32_t odb_session_tp_attach(odb_session* s, void* const* peer_recv, void* cons
         if ((reinterpret_cast<uintptr_t>(pr) | reinterpret_cast<uintptr_t>(pc)) & 15 || reinterpret_cast<uintptr_t>(pf) & 3)
             return ODB_ERR_ARG;
         tp.recv[r] = static_cast<float*>(pr);
-        tp.peers.flags[r] = static_cast<unsigned int*>(pf);
+        tp.flags[r] = static_cast<unsigned int*>(pf);
         tp.conf[r] = static_cast<ConfPartial*>(pc);
     }
-    tp.peers.world = c.tp_world;
-    tp.peers.rank = c.tp_rank;
     tp.attached = true;
     return ODB_OK;
 }
@@ -1259,12 +1254,27 @@ int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last) {
     return ODB_OK;
 }
 
+int32_t odb_debug_tp_alone(odb_session* s, int32_t enable) {
+    if (!s) return ODB_ERR_ARG;
+    if (s->m->cfg.tp_world < 2 || !s->tp.attached) return ODB_ERR_STATE;
+    if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;
+    s->tp.alone = enable != 0;
+    return ODB_OK;
+}
+
 int32_t odb_debug_tp_expire_wait(odb_session* s, int32_t kind, int64_t limit_cycles) {
     if (!s || kind < 0 || kind >= kTpKinds || limit_cycles < 1 || limit_cycles > kWaitLimitCycles) return ODB_ERR_ARG;
     if (s->m->cfg.tp_world < 2 || !s->tp.attached) return ODB_ERR_STATE;
     if (s->phase == 1 || s->phase == 3) return ODB_ERR_STATE;
     // a sequence number no rank has signalled: the flags stay below it, the wait runs into its limit
-    ODB_CUDA(launch_tp_wait(s->tp.peers, kind, s->tp.seq[kind] + 1, limit_cycles, s->at<int>(s->L.status), s->st));
+    TpWait tw;
+    tw.region = s->tp.flags[s->m->cfg.tp_rank];
+    tw.kind = kind;
+    tw.bias = 1;   // one more exchange than this rank has completed: nobody has signalled it
+    tw.world = s->m->cfg.tp_world;
+    tw.limit_cycles = limit_cycles;
+    tw.status = s->at<int>(s->L.status);
+    ODB_CUDA(launch_tp_wait(tw, s->st));
     return ODB_OK;
 }
 

@@ -207,12 +207,81 @@ struct ConfEpilogue {
 
 // Tensor-parallel destinations of an epilogue: the same fp32 partial tiles (or confidence statistics) are stored to
 // n buffers, one per rank, this rank's own among them (plain stores; the others are peer memory).  n == 0: none.
+// When every CTA of the launch has stored its tiles, the last one to arrive advances this rank's sequence counter of
+// exchange `kind` and raises this rank's flag of that kind to the new number on every rank (flag words of a rank:
+// [kind][source rank]; kind 0 / 1 = the two receive slots of partial sums, 2 = the confidence statistics; a flag
+// holds the number of exchanges of that kind its source has completed).  All numbers live on the device, so the
+// launches carry no per-call values and can be replayed from a CUDA graph.
 constexpr int kTpMaxWorld = 8;
+constexpr int kTpKinds = 3;
+// words of a rank's flag region: [kTpKinds][kTpMaxWorld] flags, then the arrival counter, then [kTpKinds] sequence counters
+constexpr int kTpArriveWord = kTpKinds * kTpMaxWorld;
+constexpr int kTpSeqWord = kTpArriveWord + 1;
+constexpr int kTpFlagWords = kTpSeqWord + kTpKinds;
 struct PeerOut {
-    float* partial[kTpMaxWorld] = {};       // each fp32 [splits][M][N], already offset to this rank's block
-    ConfPartial* conf[kTpMaxWorld] = {};    // each [M][tiles_total]
-    int n = 0;
+    float* partial[kTpMaxWorld] = {};        // each fp32 [splits][M][N], already offset to this rank's block
+    ConfPartial* conf[kTpMaxWorld] = {};     // each [M][tiles_total]
+    unsigned int* flags[kTpMaxWorld] = {};   // every rank's flag region
+    int n = 0, rank = 0, kind = 0;
+    int alone = 0;   // measurement: the flags of ALL sources are raised on this rank itself (a rank timed without peers)
 };
+
+// The consumer's side: wait until this rank's flags [kind][0 .. world) have reached the number of exchanges of that
+// kind this rank has itself completed (every rank performs the same exchanges; the consumer starts after this
+// rank's own producer has finished), plus `bias` (test: 1 = a number nobody has signalled).  world == 0: nothing.
+struct TpWait {
+    const unsigned int* region = nullptr;    // this rank's flag region
+    int kind = 0;
+    unsigned int bias = 0;
+    int world = 0;
+    long long limit_cycles = 0;
+    int* status = nullptr;
+};
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void st_release_sys(unsigned int* p, unsigned int v) {
+    asm volatile("st.release.sys.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned int ld_acquire_sys(const unsigned int* p) {
+    unsigned int v;
+    asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Called by ONE thread of a CTA after the CTA's storing threads have met at a barrier: makes the CTA's stores
+// visible system-wide, counts the CTA in, and - in the last CTA of the launch - raises the flags.
+__device__ __forceinline__ void tp_arrive_and_signal(const PeerOut& po, unsigned int total_ctas) {
+    unsigned int* own = po.flags[po.rank];
+    __threadfence_system();
+    const unsigned int before = atomicAdd(own + kTpArriveWord, 1u);
+    if (before + 1 != total_ctas) return;
+    own[kTpArriveWord] = 0;              // the next launch that uses the counter comes after this one in the stream
+    const unsigned int seq = atomicAdd(own + kTpSeqWord + po.kind, 1u) + 1u;
+    __threadfence_system();              // every CTA's fence happened before its arrival, which this thread has observed
+    for (int r = 0; r < po.n; ++r) {
+        if (po.alone) st_release_sys(own + po.kind * kTpMaxWorld + r, seq);
+        else st_release_sys(po.flags[r] + po.kind * kTpMaxWorld + po.rank, seq);
+    }
+}
+// Called by every thread of a block before it reads what the peers stored: threads 0 .. world-1 each poll one
+// source's flag (bounded; on expiry the status word gets ODB_ERR_TIMEOUT and the block carries on with whatever the
+// buffers hold), then the block meets.  Sequence numbers only grow; the signed difference survives a wrap.
+__device__ __forceinline__ void tp_wait_flags(const TpWait& tw) {
+    if (tw.world == 0) return;
+    if (static_cast<int>(threadIdx.x) < tw.world) {
+        const unsigned int want = *reinterpret_cast<const volatile unsigned int*>(tw.region + kTpSeqWord + tw.kind) + tw.bias;
+        const unsigned int* f = tw.region + tw.kind * kTpMaxWorld + threadIdx.x;
+        const long long t0 = clock64();
+        while (static_cast<int>(ld_acquire_sys(f) - want) < 0) {
+            if (clock64() - t0 > tw.limit_cycles) {
+                atomicExch(tw.status, ODB_ERR_TIMEOUT);
+                break;
+            }
+            __nanosleep(32);
+        }
+    }
+    __syncthreads();
+}
+#endif
 
 // Weight-streaming GEMM: partial[s][M][N] (fp32) = x[M][K_s] * w[N][K_s]^T for each K split s.
 struct GemmArgs {
@@ -230,20 +299,8 @@ struct GemmArgs {
 };
 int gemm_pick_splits(int M, int N, int K);
 
-// ---- tensor parallelism: flags between ranks (tensor_parallel.cu) ----
-// Flag words of one rank: [kind][source rank], kind 0 / 1 = the two receive slots of partial sums, 2 = the
-// confidence statistics.  A flag holds the sequence number of the source's latest completed exchange of that kind.
-constexpr int kTpKinds = 3;
-struct TpPeers {
-    unsigned int* flags[kTpMaxWorld] = {};   // every rank's flag words (this rank's own at index rank)
-    int world = 0, rank = 0;
-};
-// One thread per rank: after everything this rank has stored to its peers is visible system-wide, writes `seq` into
-// flag [kind][rank] of every rank.
-cudaError_t launch_tp_signal(const TpPeers& p, int kind, unsigned int seq, cudaStream_t st);
-// One thread per source rank: waits (bounded by limit_cycles) until this rank's flag [kind][source] has reached
-// `seq`; on expiry writes ODB_ERR_TIMEOUT to *status and returns.
-cudaError_t launch_tp_wait(const TpPeers& p, int kind, unsigned int seq, long long limit_cycles, int* status, cudaStream_t st);
+// Test entry: one block performs the consumers' flag wait (tensor_parallel.cu).
+cudaError_t launch_tp_wait(const TpWait& tw, cudaStream_t st);
 cudaError_t make_weight_tmap(CUtensorMap* out, const void* w_packed, int N, int K);
 // bf16 [rows][cols] row-major; box = 64 columns x box_rows rows, 128-byte swizzle, rows beyond `rows` read as zero
 cudaError_t make_rows_tmap(CUtensorMap* out, const void* base, int rows, int cols, int box_rows);
@@ -269,7 +326,7 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 // product).  splits <= 16.
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
                            __nv_bfloat16* out, float* ssq, const int32_t* row_map, int rows_out, int d, L2Prefetch pf,
-                           cudaStream_t st);
+                           cudaStream_t st, const TpWait& tw = TpWait());
 struct QkvRopeArgs {
     const float* partial; int splits; size_t pstride;      // [splits][M][3d]
     RowScale scale;                                        // scalar of the preceding RMSNorm
@@ -282,7 +339,7 @@ struct QkvRopeArgs {
 };
 cudaError_t launch_qkv_rope(const QkvRopeArgs& a, cudaStream_t st);
 cudaError_t launch_confidence_final(const ConfPartial* part, int chunks, int rows, float* conf, int32_t* tok,
-                                    cudaStream_t st);
+                                    cudaStream_t st, const TpWait& tw = TpWait());
 
 // scratch: rows * kConfMaxChunks * 12 bytes of per-chunk (max, sum, argmax) triples
 constexpr int kConfMaxChunks = 64;

@@ -94,6 +94,15 @@ def tp_attach(sess: E.Session, recv: List[Optional[int]], flags: List[Optional[i
     B.check(B.lib().odb_session_tp_attach(sess.handle, arr(recv), arr(flags), arr(conf)), "odb_session_tp_attach")
 
 
+def attach_alone(sess: E.Session):
+    """Measurement: the rank as its own peers (every rank's regions = its own) with all flags raised locally, so that
+    its steps can be timed on one GPU without the other ranks (odb_debug_tp_alone); results are meaningless."""
+    b = tp_buffers(sess)
+    n = sess.model.cfg.tp_world
+    tp_attach(sess, [b[0]] * n, [b[2]] * n, [b[4]] * n)
+    B.check(B.lib().odb_debug_tp_alone(sess.handle, 1), "odb_debug_tp_alone")
+
+
 def segment_count(cfg: B.odb_config) -> int:
     return B.lib().odb_tp_segment_count(C.byref(cfg))
 
