@@ -370,6 +370,33 @@ __global__ void __launch_bounds__(128) confidence_final_kernel(const ConfPartial
     }
 }
 
+// grid (rows, feature chunks of 256): one FFN feature per thread
+__global__ void __launch_bounds__(256) swiglu_combine_kernel(const float* __restrict__ partial, int splits, size_t pstride,
+                                                             RowScale scale, __nv_bfloat16* __restrict__ g, int F) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int m = blockIdx.x;
+    const int f = blockIdx.y * 256 + threadIdx.x;
+    if (f >= F) return;
+    const int tiles = (F + 63) / 64;
+    const size_t col = static_cast<size_t>(f >> 6) * 128 + (f & 63);   // the gate entry; its up entry sits 64 further
+    const float* p = partial + static_cast<size_t>(m) * tiles * 128 + col;
+    float gate = 0.f, up = 0.f;
+    for (int sb = 0; sb < splits; sb += 8) {
+        float t[8][2];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (sb + u < splits) { t[u][0] = p[(sb + u) * pstride]; t[u][1] = p[(sb + u) * pstride + 64]; }
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (sb + u < splits) { gate += t[u][0]; up += t[u][1]; }
+    }
+    const float sc = row_scale_of(scale, m);
+    gate *= sc;
+    up *= sc;
+    g[static_cast<size_t>(m) * F + f] = __float2bfloat16_rn(gate / (1.0f + expf(-gate)) * up);
+}
+
 // Read-only streaming probe: every thread reads 16-byte vectors grid-stride over the buffer and folds them into
 // one word, written out only if it has an (impossible) value, so that the loads cannot be removed.
 __global__ void __launch_bounds__(512) read_stream_kernel(const uint4* __restrict__ src, size_t n_vec, unsigned int* sink) {
@@ -446,6 +473,11 @@ cudaError_t launch_bulk_read_stream(const void* src, size_t bytes, int grid, int
     *streamed = static_cast<size_t>(chunks_per_cta) * grid * kBulkChunk;
     bulk_read_stream_kernel<<<grid, 32, smem, st>>>(static_cast<const uint8_t*>(src), chunks_per_cta, status);
     return cudaGetLastError();
+}
+
+cudaError_t launch_swiglu_combine(const float* partial, int splits, size_t pstride, const RowScale& scale, __nv_bfloat16* g,
+                                  int M, int F, cudaStream_t st) {
+    return launch_kernel(swiglu_combine_kernel, dim3(M, (F + 255) / 256), dim3(256), 0, st, partial, splits, pstride, scale, g, F);
 }
 
 cudaError_t launch_read_stream(const void* src, size_t bytes, unsigned int* sink, int grid, cudaStream_t st) {

@@ -247,11 +247,15 @@ __device__ __forceinline__ unsigned int ld_acquire_sys(const unsigned int* p) {
     asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-// Called by ONE thread of a CTA after the CTA's storing threads have met at a barrier: makes the CTA's stores
-// visible system-wide, counts the CTA in, and - in the last CTA of the launch - raises the flags.
+// Called by ONE thread of a CTA after the CTA's storing threads have met at a barrier: counts the CTA in and - in
+// the last CTA of the launch - raises the flags.  Ordering: the CTA's stores -> CTA barrier -> this thread's
+// GPU-scope fence -> arrival (atomic) -> observed by the last arriver -> its system-scope fence -> release store of
+// the flag at system scope -> the consumer's acquire load at system scope.  Causality order is transitive across
+// the scopes, so a consumer that sees the flag sees every CTA's stores; only the last arriver pays for a
+// system-scope fence (one per CTA, 296 of them per launch, measured 6 us per projection).
 __device__ __forceinline__ void tp_arrive_and_signal(const PeerOut& po, unsigned int total_ctas) {
     unsigned int* own = po.flags[po.rank];
-    __threadfence_system();
+    __threadfence();
     const unsigned int before = atomicAdd(own + kTpArriveWord, 1u);
     if (before + 1 != total_ctas) return;
     own[kTpArriveWord] = 0;              // the next launch that uses the counter comes after this one in the stream
@@ -327,6 +331,11 @@ cudaError_t launch_embed(const __nv_bfloat16* embed, const int32_t* row_tok, flo
 cudaError_t launch_rmsnorm(float* h, const float* partial, int splits, size_t pstride, const float* gain,
                            __nv_bfloat16* out, float* ssq, const int32_t* row_map, int rows_out, int d, L2Prefetch pf,
                            cudaStream_t st, const TpWait& tw = TpWait());
+// SwiGLU of a gate/up projection that ran with K splits (few weight tiles: a tensor-parallel shard): partial is fp32
+// [splits][M][tiles * 128] in the packed gate/up order (tile t = gate features [64t, 64t+64), then the same up
+// features); g[m][f] = bf16(silu(gate) * up) with gate, up = the split sums (split order) times the row scalar.
+cudaError_t launch_swiglu_combine(const float* partial, int splits, size_t pstride, const RowScale& scale, __nv_bfloat16* g,
+                                  int M, int F, cudaStream_t st);
 struct QkvRopeArgs {
     const float* partial; int splits; size_t pstride;      // [splits][M][3d]
     RowScale scale;                                        // scalar of the preceding RMSNorm
