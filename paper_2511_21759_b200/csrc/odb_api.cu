@@ -824,9 +824,9 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         // the others and a small kernel forms SwiGLU from the split sums (one rank of 4 / 8, timed alone: 3.43 -> 2.74
         // and 4.07 -> 3.38 ms per step).
         const int gu_tiles = (F + 63) / 64;
-        static const int gu_split_env = getenv("ODB_GU_SPLIT") ? atoi(getenv("ODB_GU_SPLIT")) : 0;   // experiment
-        int gu_sp = (R > 1 && gu_tiles * ((M + 127) / 128) <= 128) ? plan_splits(M, gu_tiles * 128, d, false) : 1;
-        if (gu_split_env > 1 && !write_cache) gu_sp = gu_split_env;
+        // (the whole model's 192 tiles on 148 SMs are unbalanced too, but there 2 or 3 K splits + the combine kernel
+        // measured slower than the fused epilogue: 3.52 / 3.43 against 3.28 ms per step, 5.02 / 4.97 against 4.74 at 128 rows)
+        const int gu_sp = (R > 1 && gu_tiles * ((M + 127) / 128) <= 128) ? plan_splits(M, gu_tiles * 128, d, false) : 1;
         if (gu_sp > 1) {
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_gu[l], a, partial, M, gu_tiles * 128, d, gu_sp));
             ODB_FWD(ODB_KIND_ELEMENTWISE, launch_swiglu_combine(partial, gu_sp, static_cast<size_t>(M) * gu_tiles * 128, inv_scale, g, M,
