@@ -28,6 +28,18 @@ from oracle import odb_oracle as O
 from oracle.inputs import model_from_synth
 from gpu_common import engine, requires_gpu, logits_close, rel_l2, anchored_bounds
 
+_ORACLE_MODELS = {}
+
+
+def _oracle_model(shape):
+    """The float32 oracle model of `shape` (seed 0), built once for the whole module: every test here uses the same
+    8B-shaped weights, and converting them is a minute of host time per test otherwise (30 GB of host memory, the
+    same a single test holds)."""
+    key = (shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn, shape.vocab)
+    if key not in _ORACLE_MODELS:
+        _ORACLE_MODELS[key] = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    return _ORACLE_MODELS[key]
+
 
 @requires_gpu
 def test_cfg3_refresh_and_first_step_match_oracle():
@@ -62,7 +74,7 @@ def test_cfg3_refresh_and_first_step_match_oracle():
     sess.close(); gm.close()
     del gm
 
-    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    om = _oracle_model(shape)
     cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
     assert g_logits.shape == o_logits.shape == (L, shape.vocab)
     l2_r = rel_l2(g_logits, o_logits)
@@ -159,7 +171,7 @@ def test_cfg4_refresh_and_four_copy_step_match_oracle():
     del gm
 
     tau = wl.accept_threshold
-    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    om = _oracle_model(shape)
     cache, o_conf, o_tok, o_logits = O.refresh_prefill(om, x0, T, P, dtype=np.float32, return_logits=True)
     l2_r = rel_l2(g_logits, o_logits[:Bk])
     l2_tol, factor = anchored_bounds(shape.n_layers, L * shape.vocab)
@@ -242,7 +254,7 @@ def test_cfg5_batch16_sampled_sequence_matches_oracle():
     g_k = synth.bf16_bits_to_f32(k_last[row0:row0 + T]).astype(np.float64)
     tau = wl.accept_threshold
 
-    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    om = _oracle_model(shape)
     cache, o_conf, o_tok = O.refresh_prefill(om, xs[pick], T, P, dtype=np.float32)
     o_k = np.asarray(cache.k[-1], dtype=np.float64).reshape(T, -1)
     k_err = rel_l2(g_k, o_k)
@@ -293,7 +305,7 @@ def _full_size_lockstep(wl_name, copies, max_iters=None, stop=None, prompt_len=N
     gm = E.Model.from_synth(shape, seed=0, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=copies)
     sess = E.Session(gm)
     sess.set_sequence(0, x0, P)
-    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    om = _oracle_model(shape)
     kw = dict(block_len=Bk, n_copies=copies, alp=False)
     # bounds from the oracle's own float32-vs-float64 distance at this depth, not literals
     l2_tol, factor = anchored_bounds(shape.n_layers, L * shape.vocab)
@@ -347,7 +359,7 @@ def test_cfg4_tensor_parallel_group_of_four_in_lockstep():
     x0 = synth.sequence(0, 0, P, L, shape)
     g = tp.TPGroupOneGPU(shape, 0, 4, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
     g.set_sequence(0, x0, P)
-    om = model_from_synth(shape, seed=0, dtype=np.float32, cache_layers=True)
+    om = _oracle_model(shape)
     kw = dict(block_len=Bk, n_copies=4, alp=False)
     st = lockstep_generate(E, g, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), check_logits=False,
                            dtype=np.float32, max_iters=3)
