@@ -118,9 +118,10 @@ class Model:
 
 
 class Session:
-    def __init__(self, model: Model, stream: Optional[torch.cuda.Stream] = None, poison: bool = False):
+    def __init__(self, model: Model, stream: Optional[torch.cuda.Stream] = None, poison: bool = False, zero: bool = False):
         """poison: hand the library a workspace and a K/V cache filled with 0xFF bytes (NaN as fp32 and as bf16), so
-        that a kernel reading memory nothing has written shows up as NaN in the results (tests)."""
+        that a kernel reading memory nothing has written shows up as NaN in the results (tests).  zero: zero-filled
+        buffers instead (a tensor-parallel rank run without its peers then adds zeros for their partial sums)."""
         self.model = model
         lib = B.lib()
         dev = model.t["embed"].device
@@ -129,6 +130,9 @@ class Session:
         if poison:
             self.kv.fill_(0xFF)
             self.ws.fill_(0xFF)
+        elif zero:
+            self.kv.zero_()
+            self.ws.zero_()
         self.stream = stream if stream is not None else torch.cuda.current_stream(dev)
         self.handle = C.c_void_p()
         B.check(lib.odb_session_create(model.handle, self.kv.data_ptr(), self.kv.numel(), self.ws.data_ptr(),

@@ -146,3 +146,32 @@ def test_tp_state_errors():
     with pytest.raises(B.OdbError) as e:                          # 688 FFN features do not divide into 2 x 64
         tp.model_shard_from_synth(synth.TINY, 0, 0, 2, max_batch=1, max_seq=64, max_block=16, max_copies=4)
     assert e.value.status == B.ODB_ERR_SHAPE
+
+
+@requires_gpu
+@pytest.mark.parametrize("shape_name,R,copies", [("tiny", 2, 1), ("peaky", 4, 4), ("hd128", 2, 8)])
+def test_tp_rank_alone_resident_loop_equals_call_by_call(shape_name, R, copies):
+    """A tensor-parallel step inside the device-resident loop (its exchanges count their sequence numbers on the
+    device, so the launches replay from a graph).  Ranks that wait for one another cannot share a GPU inside graphs,
+    so ONE rank runs alone: attached to its own buffers, the absent ranks' flags raised locally, their partial sums
+    zeros (zero-filled workspace).  The loop must reproduce the call-by-call run of the same rank bit for bit:
+    tokens, every iteration's accept set and chain, and no wait may have expired."""
+    from paper_2511_21759_b200 import tp
+    E = engine()
+    shape = SHAPES[shape_name]
+    P, L, Bk = 48, 64, 16
+    x0 = synth.sequence(5, 0, P, L, shape)
+    p = E.DecodeParams(block_len=Bk, n_copies=copies)
+    runs = []
+    for resident in (False, True):
+        gm = tp.model_shard_from_synth(shape, 5, R - 1, R, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=8)
+        sess = E.Session(gm, zero=True)
+        tp.attach_alone(sess)
+        sess.set_sequence(0, x0, P)
+        toks, trace = E.generate(sess, p, resident=resident)
+        assert sess.status() == 0
+        runs.append((toks[0], trace))
+        sess.close(); gm.close()
+    assert np.array_equal(runs[0][0], runs[1][0])
+    assert runs[0][1] == runs[1][1]
+    assert (runs[0][0][P:] != shape.mask_id).all()
