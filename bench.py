@@ -441,6 +441,10 @@ def run_cuda(args, wl):
             line["secondary"] = secondary_measurements(E, synth, gm, peaks, args)
         except Exception as exc:      # the headline line must come out whatever happens to the extras
             line["secondary"] = {"error": f"{type(exc).__name__}: {exc}"}
+        try:                          # the tensor-parallel path: one rank's step alone (a lower bound, no NVLink in it)
+            line["secondary"]["tp_rank_alone"] = tp_rank_alone(wl, peaks, 10, 3)
+        except Exception as exc:
+            line["secondary"]["tp_rank_alone"] = {"error": f"{type(exc).__name__}: {exc}"}
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
             r = oracle_sample(wl)
@@ -708,71 +712,77 @@ def run_layer_microbench(args, wl):
     gm.close()
 
 
-def run_tp_rank_step(args, wl):
+def tp_rank_alone(wl, peaks, steps, warmup):
     """Device time of ONE tensor-parallel rank's decode step, timed alone on this GPU, for groups of 2, 4 and 8: rank 0's
     shard of the workload's model, attached to its own buffers as if they were its peers', with the flags of the
     absent ranks raised locally (odb_debug_tp_alone).  Every kernel of the rank runs (its projections store their
-    partial tiles R times, the flag kernels run, the RMSNorm adds R blocks of partials); what is missing is the
-    NVLink latency of the stores and flags, so this is a lower bound of a rank's step time, not a scaling
-    measurement.  Results of the forward are meaningless (the peers' partial sums are absent).  One JSON line."""
+    partial tiles R times, the flags are raised and waited for, the RMSNorm adds R blocks of partials); what is missing
+    is the NVLink latency and bandwidth of the stores and flags, so this is a lower bound of a rank's step time, not a
+    scaling measurement.  Results of the forward are meaningless (the peers' partial sums are absent)."""
     import torch
-    import __graft_entry__ as G
     from paper_2511_21759_b200 import engine as E, tp
     import synth
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    G.build()
-    peaks = load_peaks()
     shape, T = wl.shape, wl.prompt_len + wl.gen_len
     worlds = [r for r in (2, 4, 8) if shape.n_heads % r == 0 and shape.d_ffn % (64 * r) == 0]
-    d, F, V, nl = shape.d_model, shape.d_ffn, shape.vocab, shape.n_layers
+    d, F, nl = shape.d_model, shape.d_ffn, shape.n_layers
     keys = T - wl.block_len
-    out = {}
+    out = {"definition": "one rank of R timed alone on one GPU (own buffers as peers, absent ranks' flags raised locally): "
+                         "lower bound of a rank's step time, no NVLink in it; not a scaling measurement"}
     params = E.DecodeParams(block_len=wl.block_len, n_copies=wl.n_copies, alp=False)
     for R in worlds:
         gm = tp.model_shard_from_synth(shape, 0, 0, R, max_batch=1, max_seq=T, max_block=wl.block_len,
                                        max_copies=max(wl.n_copies, 1))
         sess = E.Session(gm)
         tp.attach_alone(sess)
-        sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape), wl.prompt_len)
-        sess.refresh_prefill(params, 0)
-        sess.unmask_accept(params, True)
+
         def reopen():
             sess.set_sequence(0, synth.sequence(0, 0, wl.prompt_len, wl.gen_len, shape), wl.prompt_len)
             sess.refresh_prefill(params, 0)
             sess.unmask_accept(params, True)
+        reopen()
         times, loop_times = [], []
-        for i in range(args.warmup + args.steps):       # call by call: one launch sequence from the host per step
+        for i in range(warmup + steps):       # call by call: one launch sequence from the host per step
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(sess.stream)
             sess.block_decode_step(params)
             b.record(sess.stream)
             res = sess.unmask_accept(params, False)
-            if i >= args.warmup:
+            if i >= warmup:
                 times.append(a.elapsed_time(b))
             if res[0].masks_left == 0:      # block full (garbage confidences may accept anything): open it again
                 reopen()
         reopen()
-        for i in range(args.warmup + args.steps):       # the device-resident loop: the same kernels replayed from a graph
+        for i in range(warmup + steps):       # the device-resident loop: the same kernels replayed from a graph
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record(sess.stream)
             its = sess.decode_block_resident(params, 4)
             b.record(sess.stream)
             b.synchronize()
-            if i >= args.warmup:
+            if i >= warmup:
                 loop_times.append(a.elapsed_time(b) / len(its))
             if its[-1][0].masks_left == 0:
                 reopen()
-        ms = float(np.median(times))
+        ms, loop_ms = float(np.median(times)), float(np.median(loop_times))
         v0, v1 = tp.vocab_range(gm.cfg, 0)
         rank_bytes = nl * ((3 * d * d + d * d + 3 * F * d) * 2 / R + 2 * keys * d * 2 / R) + (v1 - v0) * d * 2
-        loop_ms = float(np.median(loop_times))
         out[f"ranks_{R}"] = {"ms_per_step_host_launched": ms, "ms_per_iteration_in_resident_loop": loop_ms,
                              "rank_algorithmic_bytes": rank_bytes, "achieved_gbs": rank_bytes / (loop_ms * 1e-3) / 1e9,
                              "frac_of_hbm_peak": rank_bytes / (loop_ms * 1e-3) / 1e9 / peaks["hbm_gbs"], "status": sess.status()}
         sess.close(); gm.close()
         del sess, gm
         torch.cuda.empty_cache()
+    return out
+
+
+def run_tp_rank_step(args, wl):
+    """bench.py --tp-rank-step: tp_rank_alone as one JSON line."""
+    import torch
+    import __graft_entry__ as G
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    G.build()
+    peaks = load_peaks()
+    out = tp_rank_alone(wl, peaks, args.steps, args.warmup)
     print(json.dumps({"metric": "device time of one tensor-parallel rank's decode step, timed alone (no peers, no NVLink)",
                       "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": False,
                       "dtype": "bf16", "data": "synthetic", "config": config_of(wl), "peak": peaks["hbm_gbs"],
