@@ -712,7 +712,7 @@ def run_layer_microbench(args, wl):
     gm.close()
 
 
-def tp_rank_alone(wl, peaks, steps, warmup):
+def tp_rank_alone(wl, peaks, steps, warmup, only=0):
     """Device time of ONE tensor-parallel rank's decode step, timed alone on this GPU, for groups of 2, 4 and 8: rank 0's
     shard of the workload's model, attached to its own buffers as if they were its peers', with the flags of the
     absent ranks raised locally (odb_debug_tp_alone).  Every kernel of the rank runs (its projections store their
@@ -723,7 +723,7 @@ def tp_rank_alone(wl, peaks, steps, warmup):
     from paper_2511_21759_b200 import engine as E, tp
     import synth
     shape, T = wl.shape, wl.prompt_len + wl.gen_len
-    worlds = [r for r in (2, 4, 8) if shape.n_heads % r == 0 and shape.d_ffn % (64 * r) == 0]
+    worlds = [r for r in (2, 4, 8) if shape.n_heads % r == 0 and shape.d_ffn % (64 * r) == 0 and only in (0, r)]
     d, F, nl = shape.d_model, shape.d_ffn, shape.n_layers
     keys = T - wl.block_len
     out = {"definition": "one rank of R timed alone on one GPU (own buffers as peers, absent ranks' flags raised locally): "
@@ -782,7 +782,7 @@ def run_tp_rank_step(args, wl):
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     G.build()
     peaks = load_peaks()
-    out = tp_rank_alone(wl, peaks, args.steps, args.warmup)
+    out = tp_rank_alone(wl, peaks, args.steps, args.warmup, args.tp_ranks)
     print(json.dumps({"metric": "device time of one tensor-parallel rank's decode step, timed alone (no peers, no NVLink)",
                       "unit": "ms", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "higher_is_better": False,
                       "dtype": "bf16", "data": "synthetic", "config": config_of(wl), "peak": peaks["hbm_gbs"],
@@ -808,6 +808,7 @@ def main():
     ap.add_argument("--tp-rank-step", action="store_true",
                     help="time one tensor-parallel rank's decode step alone on this GPU for groups of 2, 4 and 8 (lower bound "
                          "of a rank's step time: no peers, no NVLink latency)")
+    ap.add_argument("--tp-ranks", type=int, default=0, help="with --tp-rank-step: only this group size (2, 4 or 8)")
     ap.add_argument("--modes", action="store_true",
                     help="also run the whole response as cache-less baseline / DualCache block decoding / full method")
     args = ap.parse_args()
