@@ -76,7 +76,10 @@ gemm_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ 
     const int m_tile = PAIR ? static_cast<int>((blockIdx.z / n_pairs) % m_groups) * static_cast<int>(gridDim.y) + static_cast<int>(blockIdx.y)
                             : static_cast<int>(blockIdx.y);
     if (PAIR && m_tile >= pair_tiles_y) {   // ragged last group: both CTAs of the pair leave together
-        if (po.n > 0 && threadIdx.x == 0) tp_arrive_and_signal(po, gridDim.x * gridDim.y * gridDim.z);
+        if (po.n > 0 && threadIdx.x == 0) {
+            pdl_wait();   // the arrival counter is shared with the previous exchanging launch: count only once that one is complete
+            tp_arrive_and_signal(po, gridDim.x * gridDim.y * gridDim.z);
+        }
         return;
     }
     const int n0 = n_tile * kBM;

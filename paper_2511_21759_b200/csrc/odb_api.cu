@@ -809,7 +809,12 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
         int o_parts = sp;
         TpWait o_wait;
         if (R > 1) {
-            // every rank's partial tiles land in slot 0 of every rank; all R * sp partials are added in (rank, split) order
+            // every rank's partial tiles land in slot 0 of every rank; all R * sp partials are added in (rank, split) order.
+            // Reusing the slot every layer is safe: a peer stores its next O partials only after its wait on the down
+            // exchange of this layer, i.e. after this rank's down projection has raised its flag, and that projection's
+            // epilogue runs behind this rank's RMSNorm (the reader of slot 0) in the launch chain.  Slot 1 likewise,
+            // with the roles of the two exchanges swapped; the statistics buffer: a peer reaches its next LM head only
+            // through exchanges this rank signals after its merge of the current statistics.
             ODB_FWD(ODB_KIND_GEMM, gemm(m->tm_o[l], o, nullptr, M, d, da, sp, nullptr, 0));
             o_wait = end_exchange(0);
             o_sum = tp.recv[c.tp_rank];
