@@ -202,6 +202,7 @@ def share_workspace(sess: E.Session):
 
 def open_workspace(shared) -> torch.Tensor:
     """The peer's workspace as a uint8 tensor of this process (kept alive by the caller for the session's life)."""
+    torch.cuda.init()                       # the handle is opened by the CUDA runtime: it must be up in this process
     st = torch.UntypedStorage._new_shared_cuda(*shared["handle"])
     return torch.empty(0, dtype=torch.uint8, device=st.device).set_(st)[shared["tensor_offset"]:]
 

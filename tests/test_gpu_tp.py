@@ -175,3 +175,46 @@ def test_tp_rank_alone_resident_loop_equals_call_by_call(shape_name, R, copies):
     assert np.array_equal(runs[0][0], runs[1][0])
     assert runs[0][1] == runs[1][1]
     assert (runs[0][0][P:] != shape.mask_id).all()
+
+
+def _ipc_child(shared, offset, n, done):
+    """Second process of the mapping test: opens the first process's buffer through the inter-process handle and
+    writes a pattern through the mapping (no kernel of either process waits for the other)."""
+    try:
+        import torch
+        from paper_2511_21759_b200 import tp
+        view = tp.open_workspace(shared)
+        view[offset:offset + n] = torch.arange(n, device=view.device, dtype=torch.int64).to(torch.uint8)
+        torch.cuda.synchronize()
+        done.put(("ok", int(view.data_ptr())))
+    except Exception:                      # the parent reports it
+        import traceback
+        done.put(("error", traceback.format_exc()))
+
+
+@requires_gpu
+def test_tp_workspace_mapping_between_processes():
+    """The multi-process attach maps a peer's workspace through torch's CUDA inter-process storage handles and
+    addresses the peer's regions by offset.  Two processes on this one GPU: the second opens the first's buffer and
+    stores a pattern at an offset; the first sees it at that offset of its own tensor.  (Only the mapping is exercised:
+    ranks whose kernels wait for one another need a GPU each.)"""
+    import types
+    import torch
+    import torch.multiprocessing as mp
+    from paper_2511_21759_b200 import tp
+    engine()
+    ws = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    shared = tp.share_workspace(types.SimpleNamespace(ws=ws))
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    offset, n = 4096 + 256, 200
+    p = ctx.Process(target=_ipc_child, args=(shared, offset, n, q))
+    p.start()
+    status, detail = q.get(timeout=90)
+    p.join(timeout=60)
+    assert status == "ok", detail
+    assert p.exitcode == 0
+    torch.cuda.synchronize()
+    got = ws[offset:offset + n].cpu().numpy()
+    assert np.array_equal(got, np.arange(n, dtype=np.uint8))
+    assert int(ws[:offset].sum()) == 0 and int(ws[offset + n:].sum()) == 0
