@@ -340,7 +340,8 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
 
 /* ---- tensor parallelism (sessions of a model created with tp_world > 1) ----
  * odb_session_tp_buffers: device pointers (inside this session's workspace) of the three regions its peers
- * write into - receive slots for the partial sums, flag words, confidence statistics - and their sizes.  The
+ * write into - receive slots for the partial sums, flag words (followed by this rank's own arrival and sequence
+ * counters, which peers never touch), confidence statistics - and their sizes.  The
  * caller carries them to the other ranks (same process: as they are; other processes: as offsets into an
  * inter-process mapping of the workspace allocation) and hands every rank the R pointers of each kind with
  * odb_session_tp_attach (entry tp_rank is this session's own).  Until attached, refresh / step calls return
@@ -357,7 +358,7 @@ int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, 
  * is cut into odb_tp_segment_count segments at its exchange points (after a flag is raised, before it is waited
  * for).  With a range set, a refresh / step call launches only the kernels of segments [first, last) of the
  * forward; the caller issues segment k on every rank before segment k+1 on any, on one stream, so that every
- * flag is up before its wait kernel starts.  first = 0 begins a forward, later ranges continue it; the accept
+ * flag is up before the kernel that waits for it starts.  first = 0 begins a forward, later ranges continue it; the accept
  * follows the last segment.  first < 0 restores whole forwards. */
 int32_t odb_tp_segment_count(const odb_config* cfg);
 int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last);
@@ -366,8 +367,8 @@ int32_t odb_debug_tp_segments(odb_session* s, int32_t first, int32_t last);
  * absent ranks are whatever their blocks of the receive buffers hold (results are meaningless, device time is that
  * of one rank's kernels).  Attach the session to its own three regions for every rank first. */
 int32_t odb_debug_tp_alone(odb_session* s, int32_t enable);
-/* Test facility: one launch of the flag wait for exchange `kind` (0, 1: partial-sum slots, 2: statistics) with the
- * next sequence number and the given cycle limit; nothing raises the flags, so the wait expires and the status
+/* Test facility: one launch of the flag wait for exchange `kind` (0, 1: partial-sum slots, 2: statistics) for one exchange
+ * more than this rank has completed, with the given cycle limit; nothing raises the flags, so the wait expires and the status
  * word reports ODB_ERR_TIMEOUT (read and cleared by odb_session_status). */
 int32_t odb_debug_tp_expire_wait(odb_session* s, int32_t kind, int64_t limit_cycles);
 
