@@ -351,6 +351,9 @@ int32_t odb_session_profile_read(odb_session* s, double* ms_by_kind, int64_t* la
 int32_t odb_session_tp_buffers(odb_session* s, void** recv, size_t* recv_bytes, void** flags, size_t* flags_bytes,
                                void** conf, size_t* conf_bytes);
 int32_t odb_session_tp_attach(odb_session* s, void* const* peer_recv, void* const* peer_flags, void* const* peer_conf);
+/* Lets kernels on the calling thread's current device store into memory of `peer_device` (cudaDeviceEnablePeerAccess;
+ * already enabled, or peer_device being the current device, is success).  ODB_ERR_CUDA if the two cannot be peers. */
+int32_t odb_tp_enable_peer_access(int32_t peer_device);
 /* first and one-past-last vocabulary id of rank `rank`'s LM-head shard; ODB_ERR_ARG for a bad rank, the
  * configuration's own error for a configuration odb_model_create would refuse */
 int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, int32_t* last);

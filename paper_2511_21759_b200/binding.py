@@ -92,6 +92,7 @@ SIGNATURES = {
     "odb_session_tp_buffers": (C.c_int32, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_size_t), C.POINTER(C.c_void_p),
                                            C.POINTER(C.c_size_t), C.POINTER(C.c_void_p), C.POINTER(C.c_size_t)]),
     "odb_session_tp_attach": (C.c_int32, [C.c_void_p, C.POINTER(C.c_void_p), C.POINTER(C.c_void_p), C.POINTER(C.c_void_p)]),
+    "odb_tp_enable_peer_access": (C.c_int32, [C.c_int32]),
     "odb_tp_vocab_range": (C.c_int32, [C.POINTER(odb_config), C.c_int32, C.POINTER(C.c_int32), C.POINTER(C.c_int32)]),
     "odb_tp_segment_count": (C.c_int32, [C.POINTER(odb_config)]),
     "odb_debug_tp_segments": (C.c_int32, [C.c_void_p, C.c_int32, C.c_int32]),

@@ -1239,6 +1239,21 @@ int32_t odb_session_tp_attach(odb_session* s, void* const* peer_recv, void* cons
     return ODB_OK;
 }
 
+int32_t odb_tp_enable_peer_access(int32_t peer_device) {
+    int dev = 0, n = 0;
+    ODB_CUDA(cudaGetDevice(&dev));
+    ODB_CUDA(cudaGetDeviceCount(&n));
+    if (peer_device < 0 || peer_device >= n) return ODB_ERR_ARG;
+    if (peer_device == dev) return ODB_OK;
+    cudaError_t e = cudaDeviceEnablePeerAccess(peer_device, 0);
+    if (e == cudaErrorPeerAccessAlreadyEnabled) {
+        cudaGetLastError();   // clear the sticky-less error state
+        return ODB_OK;
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    return ODB_OK;
+}
+
 int32_t odb_tp_vocab_range(const odb_config* cfg, int32_t rank, int32_t* first, int32_t* last) {
     if (!first || !last) return ODB_ERR_ARG;
     const int32_t rc = check_config(cfg);

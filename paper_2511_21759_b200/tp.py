@@ -237,7 +237,13 @@ def attach_process_group(sess: E.Session, group=None):
     cfg = sess.model.cfg
     if cfg.tp_world != world or cfg.tp_rank != rank:
         raise ValueError(f"model shard is rank {cfg.tp_rank} of {cfg.tp_world}, process is rank {rank} of {world}")
-    everyone = gather_descriptors({"shared": share_workspace(sess), "bufs": tp_buffers(sess) + (sess.ws.data_ptr(),)}, group)
+    device = sess.ws.device.index
+    everyone = gather_descriptors({"shared": share_workspace(sess), "bufs": tp_buffers(sess) + (sess.ws.data_ptr(),),
+                                   "device": device}, group)
+    with torch.cuda.device(device):      # this rank's kernels store into every peer's memory
+        for r in range(world):
+            if r != rank:
+                B.check(B.lib().odb_tp_enable_peer_access(everyone[r]["device"]), "odb_tp_enable_peer_access")
     mapped = [None if r == rank else open_workspace(everyone[r]["shared"]) for r in range(world)]
     recv, flags, conf = peer_pointers(rank, [e["bufs"] for e in everyone],
                                       [None if m is None else m.data_ptr() for m in mapped], sess.ws.data_ptr())

@@ -143,6 +143,10 @@ def test_tp_state_errors():
         g.ranks[0].decode_block_resident(p)
     assert e.value.status == B.ODB_ERR_STATE
     g.close()
+    import torch
+    assert B.lib().odb_tp_enable_peer_access(torch.cuda.current_device()) == B.ODB_OK      # itself: nothing to enable
+    assert B.lib().odb_tp_enable_peer_access(torch.cuda.device_count()) == B.ODB_ERR_ARG   # no such device
+    assert B.lib().odb_tp_enable_peer_access(-1) == B.ODB_ERR_ARG
     with pytest.raises(B.OdbError) as e:                          # 688 FFN features do not divide into 2 x 64
         tp.model_shard_from_synth(synth.TINY, 0, 0, 2, max_batch=1, max_seq=64, max_block=16, max_copies=4)
     assert e.value.status == B.ODB_ERR_SHAPE
