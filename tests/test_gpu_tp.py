@@ -222,3 +222,31 @@ def test_tp_workspace_mapping_between_processes():
     got = ws[offset:offset + n].cpu().numpy()
     assert np.array_equal(got, np.arange(n, dtype=np.uint8))
     assert int(ws[:offset].sum()) == 0 and int(ws[offset + n:].sum()) == 0
+
+
+@requires_gpu
+@pytest.mark.parametrize("R,copies", [(2, 4), (4, 8)])
+def test_tp_ragged_batch_equals_independent_runs(R, copies):
+    """Three sequences of different prompt / response lengths in one tensor-parallel group: each must come out exactly as
+    when it runs alone through a group of the same size (sequences never see each other; the row tables, the
+    attention work items and the exchanges cover all sequences of a forward at once).  Free-running engine.generate
+    over the group object: refreshes of some sequences alternate with steps of the others."""
+    from paper_2511_21759_b200 import tp
+    E = engine()
+    shape = TP_PEAKY
+    lens = [(64, 64), (40, 48), (17, 30)]
+    params = E.DecodeParams(block_len=16, n_copies=copies)
+    xs = [synth.sequence(0, i, P, L, shape) for i, (P, L) in enumerate(lens)]
+    g = tp.TPGroupOneGPU(shape, 0, R, max_batch=3, max_seq=128, max_block=16, max_copies=8)
+    for i, (P, L) in enumerate(lens):
+        g.set_sequence(i, xs[i], P)
+    together, _ = E.generate(g, params)
+    assert g.status() == [0] * R
+    g.close()
+    for i, (P, L) in enumerate(lens):
+        g1 = tp.TPGroupOneGPU(shape, 0, R, max_batch=3, max_seq=128, max_block=16, max_copies=8)
+        g1.set_sequence(0, xs[i], P)
+        alone, _ = E.generate(g1, params)
+        g1.close()
+        assert np.array_equal(together[i], alone[0]), i
+        assert (together[i][P:] != shape.mask_id).all()
