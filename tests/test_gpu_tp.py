@@ -250,3 +250,27 @@ def test_tp_ragged_batch_equals_independent_runs(R, copies):
         g1.close()
         assert np.array_equal(together[i], alone[0]), i
         assert (together[i][P:] != shape.mask_id).all()
+
+
+@requires_gpu
+def test_tp_group_with_the_stochastic_reverse_step():
+    """The stochastic unmasking of Section 2.1, Eq. 1 as the accept rule under tensor parallelism: every rank gets the
+    caller's uniform deviates, so all ranks unmask the same positions as the oracle in every iteration."""
+    from paper_2511_21759_b200 import tp
+    E = engine()
+    shape, R = TP_TINY, 2
+    P, L, Bk, n = 40, 48, 16, 6
+    om = model_from_synth(shape, seed=4)
+    x0 = synth.sequence(4, 0, P, L, shape)
+    noise = lambda b, k: synth.uniform(9, 1000 * b + k, Bk)
+    kw = dict(block_len=Bk, n_copies=1, alp=False, sampling=True, sample_steps=n)
+    g = tp.TPGroupOneGPU(shape, 4, R, max_batch=1, max_seq=P + L, max_block=Bk, max_copies=4)
+    g.set_sequence(0, x0, P)
+    st = lockstep_generate(E, g, om, x0, P, E.DecodeParams(**kw), O.DecodeParams(**kw), noise=noise, check_logits=False)
+    assert g.status() == [0] * R and st["tokens"] == L and st["refreshes"] == L // Bk
+    _, otrace = O.generate(om, x0, P, O.DecodeParams(**kw), noise=noise)
+    g.set_sequence(0, x0, P)
+    gtok, gtrace = E.generate(g, E.DecodeParams(**kw), noise=lambda seq, b: np.stack([noise(b, k) for k in range(n)]))
+    assert [[p_ for p_, _ in t["seqs"][0]["accepted"]] for t in gtrace] == [[p_ for p_, _ in t["accepted"]] for t in otrace]
+    assert np.array_equal(gtok[0], st["tokens_final"])
+    g.close()
