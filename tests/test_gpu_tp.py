@@ -274,3 +274,30 @@ def test_tp_group_with_the_stochastic_reverse_step():
     assert [[p_ for p_, _ in t["seqs"][0]["accepted"]] for t in gtrace] == [[p_ for p_, _ in t["accepted"]] for t in otrace]
     assert np.array_equal(gtok[0], st["tokens_final"])
     g.close()
+
+
+@requires_gpu
+def test_tp_one_layer_without_lm_head():
+    """One-layer model without LM head over two ranks: each rank's K / V rows are exact functions of the embedding
+    (bit-equal to the oracle's columns of its heads except where fp32-vs-fp64 accumulation flips a bf16 rounding),
+    and the replicated residual stream after the last exchange matches the oracle's hidden state."""
+    from paper_2511_21759_b200 import tp
+    E = engine()
+    shape = TP_TINY.with_layers(1)
+    P, L, R = 40, 24, 2
+    om = model_from_synth(shape, seed=0, with_lm_head=False)
+    g = tp.TPGroupOneGPU(shape, 0, R, with_lm_head=False, max_batch=1, max_seq=P + L, max_block=16, max_copies=1)
+    x0 = synth.sequence(0, 0, P, L, shape)
+    g.set_sequence(0, x0, P)
+    g.refresh_prefill(E.DecodeParams(block_len=16), 0)
+    hid, fk, fv = O.forward_rows(om, x0.astype(np.int64), np.arange(P + L), None, None,
+                                 np.ones((P + L, P + L), bool), return_hidden=True)
+    hl = shape.n_heads // R
+    for r, sess in enumerate(g.ranks):
+        k = bf16_bits_to_f64(sess.debug_read("k")).reshape(P + L, hl, shape.head_dim)
+        v = bf16_bits_to_f64(sess.debug_read("v")).reshape(P + L, hl, shape.head_dim)
+        assert (k == fk[0][:, r * hl:(r + 1) * hl]).mean() > 0.99 and (v == fv[0][:, r * hl:(r + 1) * hl]).mean() > 0.99
+    h = g.debug_read("hidden")                                   # asserts the ranks hold the same bits
+    assert np.abs(h - hid).max() <= 2e-2 * np.sqrt((hid * hid).mean())
+    assert g.status() == [0] * R
+    g.close()
