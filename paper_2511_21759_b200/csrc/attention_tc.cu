@@ -10,13 +10,15 @@
 //            layout, the decoded rows of copy 0's tile.  Copies stay mutually invisible through this
 //            per-row key mask, no mask tensor exists.  Outputs are per-split (max, sum, unnormalised
 //            output) partials merged in split order by the merge kernel of attention.cu.
-// No causal mask.  Two passes over the key tiles of 64, both with S = Q K^T as one 128 x 64 x 128
-// tcgen05.mma group whose fp32 result lives in TMEM:
-//   pass 1  row maxima of S (thread r owns TMEM lane r = query row r: no cross-thread reduction);
-//   pass 2  P = exp2(S - max), row sums, P rounded to a two-term bf16 sum (value + remainder, as in the
-//           mma.sync kernel) and written to shared memory as the A operand of O += P V
-//           (128 x 128 x 64, V taken MN-major straight from its [key][dim] tile), O in TMEM.
-// Exact softmax, no rescaling of O.  Warp-specialised: warps 0..3 = softmax (one query row per thread),
+// No causal mask.  One pass over the key tiles of 64; per tile S = Q K^T is one 128 x 64 x 128 tcgen05.mma group
+// whose fp32 result lives in TMEM, and thread r owns TMEM lane r = query row r (no cross-thread reduction):
+//   the tile's largest visible score moves the row's shift M - an INTEGER in the log2 domain - only when it exceeds
+//   M by more than a slack of 4 (so P < 16); then O (in TMEM) and the row sum are multiplied by the exact power of two
+//   2^(M_old - M_new), once the previous P V has been added;
+//   P = exp2(S - M), row sums, P rounded to a two-term bf16 sum (value + remainder, as in the
+//   mma.sync kernel) and written to shared memory as the A operand of O += P V
+//   (128 x 128 x 64, V taken MN-major straight from its [key][dim] tile), O in TMEM.
+// Exact softmax (rescaling by powers of two changes no bit of a normal number).  Warp-specialised: warps 0..3 = softmax (one query row per thread),
 // warp 4 lane 0 = MMA issuer, warp 5 lane 0 = loader (TMA: boxes of 64 rows x 64 columns with the 128-byte
 // swizzle land in the canonical operand layout, two 64-column atoms per 128-wide row; rows past a buffer's
 // end read as zero, rows that are not keys of this work item are masked in the softmax and hold finite
@@ -130,6 +132,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
         : "r"(taddr)
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]),
+        "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]), "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]),
+        "r"(v[21]), "r"(v[22]), "r"(v[23]), "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]),
+        "r"(v[31])
+        : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 
 struct alignas(8) TcShared {
@@ -330,28 +345,11 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             tma_box(smem_u32(sQ) + 64 * 128, &tm_q, &sh->q_full, col0, q_row0 + 64);
             tma_box(smem_u32(sQ) + kTQ * 128, &tm_q, &sh->q_full, col0 + 64, q_row0);
             tma_box(smem_u32(sQ) + kTQ * 128 + 64 * 128, &tm_q, &sh->q_full, col0 + 64, q_row0 + 64);
-            // ---- pass 1 ----
             load_k(0);
+            load_v(0);
             load_k(1);
+            for (int t = 1; t < 1 + kAhead; ++t) hint_v(t);
             for (int t = 2; t < 2 + kAhead; ++t) hint_k(t);
-            for (int tile = 0; tile + 2 < ntiles && ok; ++tile) {
-                const int b = tile & 1;
-                ok = wait(&sh->k_empty[b], ph_ke[b]);            // S(tile) has read this buffer
-                if (ok) {
-                    load_k(tile + 2);
-                    hint_k(tile + 2 + kAhead);
-                }
-            }
-            // the last two S of pass 1 must have read their buffers before pass 2 refills them
-            for (int tile = ntiles > 2 ? ntiles - 2 : 0; tile < ntiles && ok; ++tile) ok = wait(&sh->k_empty[tile & 1], ph_ke[tile & 1]);
-            // ---- pass 2 ----
-            if (ok) {
-                load_k(0);
-                load_v(0);
-                load_k(1);
-                for (int t = 1; t < 1 + kAhead; ++t) hint_v(t);
-                for (int t = 2; t < 2 + kAhead; ++t) hint_k(t);
-            }
             // S(tile) completes long before P V(tile) (the softmax of the tile lies between them), and S(tile + 2) is
             // issued right behind P V(tile): the K buffer is refilled first, so that its load runs during that softmax
             for (int tile = 0; tile < ntiles && ok; ++tile) {
@@ -391,16 +389,6 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                 umma_commit(&sh->k_empty[b]);
                 umma_commit(&sh->s_full[b]);
             };
-            // ---- pass 1 ----
-            for (int tile = 0; tile < ntiles && ok; ++tile) {
-                const int b = tile & 1;
-                ok = wait(&sh->k_full[b], ph_kf[b]);
-                if (ok && tile >= 2) ok = wait(&sh->s_empty[b], ph_se[b]);   // S(tile - 2) has been read
-                if (!ok) break;
-                tc_fence_after();
-                issue_s(tile);
-            }
-            // ---- pass 2 ----
             auto issue_pv = [&](int tile, bool last) {
                 const uint32_t pa = smem_u32(sPh), pb = smem_u32(sPl), vb = smem_u32(sV);
 #pragma unroll
@@ -416,7 +404,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             for (int tile = 0; tile < ntiles && ok; ++tile) {
                 const int b = tile & 1;
                 ok = wait(&sh->k_full[b], ph_kf[b]);
-                if (ok) ok = wait(&sh->s_empty[b], ph_se[b]);        // the buffer's previous S has been read
+                if (ok && tile >= 2) ok = wait(&sh->s_empty[b], ph_se[b]);   // S(tile - 2) has been read
                 if (!ok) break;
                 tc_fence_after();
                 issue_s(tile);
@@ -465,8 +453,13 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             }
             return kt.copy == my_copy ? all : shared;
         };
-        // ---- pass 1: row maxima ----
-        float m_row = -INFINITY;
+        // ---- one pass over the key tiles: online softmax.  The row's shift M is an INTEGER in the log2 domain, so
+        // that moving it rescales O and the row sum by an exact power of two; it moves only when a tile's maximum
+        // exceeds it by more than kSlack (P then stays below 2^kSlack), which after the first tiles is rare. ----
+        constexpr float kSlack = 4.0f;
+        float M_row = -INFINITY;                                     // no visible key yet
+        float l_row = 0.f;
+        const uint32_t ph_base = smem_u32(sPh) + tid * 128, pl_base = smem_u32(sPl) + tid * 128;
         for (int tile = 0; tile < ntiles && ok; ++tile) {
             const int b = tile & 1;
             const KeyTile kt = key_tile(tile);
@@ -477,42 +470,37 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             // a whole tile of cached keys (or of a refresh) is seen by every row: no per-key test (the softmax
             // warps are bound by the instructions they issue per key)
             const bool full = kt.copy < 0 && kt.valid >= 64;
+            float m_t = -INFINITY;                                   // largest visible score of the tile
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
                 if (full) {
-                    float m0 = m_row, m1 = -INFINITY;
+                    float m0 = m_t, m1 = -INFINITY;
 #pragma unroll
                     for (int j = 0; j < 32; j += 4) {
                         m0 = fmaxf(m0, fmaxf(__uint_as_float(v[j]), __uint_as_float(v[j + 1])));
                         m1 = fmaxf(m1, fmaxf(__uint_as_float(v[j + 2]), __uint_as_float(v[j + 3])));
                     }
-                    m_row = fmaxf(m0, m1);
+                    m_t = fmaxf(m0, m1);
                 } else {
                     const unsigned m32 = static_cast<unsigned>(mask >> (half * 32));
 #pragma unroll
                     for (int j = 0; j < 32; ++j)
-                        if ((m32 >> j) & 1u) m_row = fmaxf(m_row, __uint_as_float(v[j]));
+                        if ((m32 >> j) & 1u) m_t = fmaxf(m_t, __uint_as_float(v[j]));
                 }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->s_empty[b]);
-        }
-        // ---- pass 2: P = exp2(S - max), row sums ----
-        const float m_log2 = m_row == -INFINITY ? 0.f : m_row * scale_log2;   // a row that sees no key of this split: every P is 0
-        float l_row = 0.f;
-        const uint32_t ph_base = smem_u32(sPh) + tid * 128, pl_base = smem_u32(sPl) + tid * 128;
-        for (int tile = 0; tile < ntiles && ok; ++tile) {
-            const int b = tile & 1;
-            const KeyTile kt = key_tile(tile);
-            const unsigned long long mask = tile_mask(kt);
-            ok = wait(&sh->s_full[b], ph_sf[b]);
-            if (!ok) break;
-            tc_fence_after();
+            float factor = 1.0f;                                     // what O and the row sum so far are multiplied by
+            const float mt_log2 = m_t * scale_log2;                  // -inf: the row sees no key of this tile
+            if (mt_log2 > M_row + kSlack) {                          // also the first visible key (M_row = -inf)
+                const float M_new = ceilf(mt_log2);
+                if (M_row != -INFINITY) factor = exp2f(M_row - M_new);   // an exact power of two
+                M_row = M_new;
+            }
+            const bool rescale = __any_sync(0xffffffffu, factor != 1.0f);
+            const float m_log2 = M_row == -INFINITY ? 0.f : M_row;   // a row that has seen no key: every P is masked to 0
             uint32_t hi[32], lo[32];                                 // row `tid` of P: 64 keys as bf16 pairs
-            const bool full = kt.copy < 0 && kt.valid >= 64;
+            float l_tile = 0.f;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
                 uint32_t v[32];
@@ -522,7 +510,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
 #pragma unroll
                 for (int u = 0; u < 16; ++u) {
                     const int j = 2 * u;
-                    // arguments are <= 0: the hardware exponential needs no range handling (far below zero it returns 0)
+                    // arguments are <= kSlack: the hardware exponential needs no range handling (far below zero it returns 0)
                     float p0 = ex2_approx(fmaf(__uint_as_float(v[j]), scale_log2, -m_log2));
                     float p1 = ex2_approx(fmaf(__uint_as_float(v[j + 1]), scale_log2, -m_log2));
                     if (!full) {
@@ -539,15 +527,28 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                     hi[half * 16 + u] = hb;
                     lo[half * 16 + u] = *reinterpret_cast<const uint32_t*>(&l);
                 }
-                l_row += l0 + l1;
+                l_tile += l0 + l1;
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->s_empty[b]);             // S(tile) is in registers
             if (tile > 0) {
-                ok = wait(&sh->p_empty, ph_pe);                      // P V(tile - 1) has read P
+                ok = wait(&sh->p_empty, ph_pe);                      // P V(tile - 1) has read P and has been added to O
                 if (!ok) break;
+                if (rescale) {                                       // warp-uniform; rows that keep their shift multiply by 1
+                    tc_fence_after();
+#pragma unroll 1
+                    for (int c = 0; c < kHD / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld32(tmem_o + lane_base + c * 32, v);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * factor);
+                        tmem_st32(tmem_o + lane_base + c * 32, v);
+                    }
+                    tc_fence_before();
+                }
             }
+            l_row = l_row * factor + l_tile;
 #pragma unroll
             for (int c = 0; c < 8; ++c) {                            // 8 keys = one 16-byte chunk
                 const uint32_t off = static_cast<uint32_t>((c ^ (tid & 7)) << 4);
@@ -562,6 +563,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(&sh->p_full);
         }
+        const float m_log2 = M_row == -INFINITY ? 0.f : M_row;      // the shift the row's sum and output carry
         if (ok && ntiles > 0) ok = wait(&sh->o_full, ph_of);
         if (ok) {
             tc_fence_after();
