@@ -471,9 +471,10 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             // warps are bound by the instructions they issue per key)
             const bool full = kt.copy < 0 && kt.valid >= 64;
             float m_t = -INFINITY;                                   // largest visible score of the tile
+            uint32_t sv[2][32];                                      // the row's 64 scores: read from TMEM once
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint32_t v[32];
+                uint32_t (&v)[32] = sv[half];
                 tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
                 if (full) {
                     float m0 = m_t, m1 = -INFINITY;
@@ -490,6 +491,9 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                         if ((m32 >> j) & 1u) m_t = fmaxf(m_t, __uint_as_float(v[j]));
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sh->s_empty[b]);             // S(tile) is in registers
             float factor = 1.0f;                                     // what O and the row sum so far are multiplied by
             const float mt_log2 = m_t * scale_log2;                  // -inf: the row sees no key of this tile
             if (mt_log2 > M_row + kSlack) {                          // also the first visible key (M_row = -inf)
@@ -503,8 +507,7 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
             float l_tile = 0.f;
 #pragma unroll
             for (int half = 0; half < 2; ++half) {
-                uint32_t v[32];
-                tmem_ld32((b ? tmem_s1 : tmem_s0) + lane_base + half * 32, v);
+                const uint32_t (&v)[32] = sv[half];
                 const unsigned m32 = full ? 0xffffffffu : static_cast<unsigned>(mask >> (half * 32));
                 float l0 = 0.f, l1 = 0.f;
 #pragma unroll
@@ -529,9 +532,6 @@ __global__ void __launch_bounds__(kThreads) attention_tc_kernel(const __grid_con
                 }
                 l_tile += l0 + l1;
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&sh->s_empty[b]);             // S(tile) is in registers
             if (tile > 0) {
                 ok = wait(&sh->p_empty, ph_pe);                      // P V(tile - 1) has read P and has been added to O
                 if (!ok) break;
