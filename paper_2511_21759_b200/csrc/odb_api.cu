@@ -768,10 +768,10 @@ int32_t forward(odb_session* s, int M, int n_lm, int n_tiles, bool write_cache, 
             if (sks < 2) sks = 2;
             sa.ksplit = sks;
             sa.pf = hint_of(m->p_gu[l], gu_bytes, 0);
-            // tensor-core work items when there are enough of them to fill the machine (batched steps: 33.5 -> 22.5 ms
-            // at 16 sequences x 256 rows); a single 128-row item per head is bound by its own dependency chain on
-            // either path (1.20 vs 1.12 ms at batch 1) and stays on the mma.sync kernel
-            static const int tc_step_min = getenv("ODB_ATTN_TC_STEP_MIN") ? atoi(getenv("ODB_ATTN_TC_STEP_MIN")) : 2 * 148;
+            // tensor-core work items for head dim 128 (batched steps: 33.5 -> 22.5 ms at 16 sequences x 256 rows with the
+            // first, two-pass version of that kernel, when a single 128-row item per head still lost to mma.sync, 1.20
+            // vs 1.12 ms per step at batch 1; in one pass it wins there too: 1.00 vs 1.13 ms, step 4.82 -> 4.63 ms)
+            static const int tc_step_min = getenv("ODB_ATTN_TC_STEP_MIN") ? atoi(getenv("ODB_ATTN_TC_STEP_MIN")) : 1;
             if (hd == 128 && tc_attention && n_step_tiles * H >= tc_step_min) {
                 const size_t cache_rows = static_cast<size_t>(c.max_batch) * c.n_layers * 2 * H * c.max_seq;
                 // with a work item for every CTA slot there is nothing to gain from key splits: one CTA per item takes

@@ -59,20 +59,20 @@ def test_edge_case_in_lockstep(name, shape_name, P, L, Bk, copies, max_iters):
 
 
 @requires_gpu
-def test_tensor_core_step_attention_on_small_batches():
-    """The decode-step attention on the tensor cores is selected only when a step has enough work items
-    to fill the machine (batched steps); an environment variable read once per process lowers that bar,
-    so the multi-copy head-dim-128 cases are run through it in a child process."""
+def test_step_attention_alternatives_for_head_dim_128():
+    """Multi-copy decode steps with head dim 128 run on the tensor-core attention with key splits.  The two other
+    configurations of that step are selected through environment variables read once per process, so the cases run
+    in child processes: the tensor-core kernel without key splits (one CTA per work item over cached and fresh keys,
+    final output: what batched steps with a work item for every CTA slot use), and the mma.sync multi-copy kernel
+    (the path of head dim 64, here at head dim 128)."""
     import os, subprocess, sys
     engine()
     names = ["hd128_ragged", "hd128_c8_stage2", "hd128_b64_c8", "hd128_c4_noprompt"]
     code = ("import sys; sys.path.insert(0, 'tests'); import test_gpu_edges as t\n"
             f"for c in t.CASES:\n    if c[0] in {names!r}: t.test_edge_case_in_lockstep(*c)\n")
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
-    # with key splits (the small-batch configuration) and without (one CTA per work item over cached and fresh
-    # keys, final output: what batched steps with a work item for every CTA slot use)
-    for extra in ({}, {"ODB_ATTN_KS": "1"}):
-        env = dict(os.environ, ODB_ATTN_TC_STEP_MIN="0", **extra)
+    for extra in ({"ODB_ATTN_KS": "1"}, {"ODB_ATTN_TC_STEP_MIN": "1000000"}):
+        env = dict(os.environ, **extra)
         r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True, timeout=900)
         assert r.returncode == 0, r.stdout[-2000:] + r.stderr[-2000:]
         assert r.stdout.count("iterations") == len(names), r.stdout[-2000:]
